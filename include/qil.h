@@ -1,0 +1,164 @@
+/*
+ * qil - low-bit quantised linear layers for sm_100a (B200), C ABI.
+ *
+ * The operations are the deployment form of the quantisation the paper applies
+ * to its policies: operands of a GEMM are mapped to a 4-bit uniform grid by
+ * round-to-nearest (paper Sec. 2.1); the OpenVLA backbone runs 4-bit
+ * weight-only linears whose decode stage is memory bound (Sec. 5.4
+ * "Implementation", App. A.4.2); the CILRS encoder runs 4-bit weights and 4-bit
+ * activations because it is compute bound (Sec. 5.1, App. A.1.2).
+ *
+ * Conventions
+ *   W is [N][K] (out features x in features, K contiguous); x is [M][K];
+ *   y[m][n] = sum_k x[m][k] * W_hat[n][k].
+ *   Unless a parameter says "host", every pointer is a DEVICE pointer owned by
+ *   the caller.  The library never allocates, frees or synchronises (the two
+ *   *_host entry points and qil_device_status are the documented exceptions:
+ *   they enqueue copies, and qil_device_status waits for its own copy).
+ *   Every call validates its arguments on the host first, then enqueues work
+ *   on `stream` and returns; nothing throws, aborts or prints.
+ *   Tensor base addresses must be 16-byte aligned.
+ *
+ * The quantiser, as an exact fp32 operation list (the paper names the method,
+ * round-to-nearest, without a formula; this is the reading the library fixes):
+ *   asymmetric uint4, per (row n, group of group_size consecutive k):
+ *     lo = min(0, min w)   hi = max(0, max w)
+ *     s  = fp16_rn((hi - lo) / 15)       ; s == 0 -> 1 ; s == inf -> error flag
+ *     z  = clamp(rint(-lo / s), 0, 15)   ; stored as fp16 (an integer value)
+ *     q  = clamp(rint(w / s) + z, 0, 15) ; dequantised value (q - z) * s
+ *   symmetric int4, per (row, group):
+ *     a = max |v| ; s = a / 7 ; a == 0 -> s = 1 ; (fp16 scale: round, 0 -> 1, inf -> error flag)
+ *     q = clamp(rint(v / s), -8, 7)      ; dequantised value q * s
+ *   All divisions are IEEE fp32 divisions, rint is round-half-to-even.
+ *
+ * Packed layout (canonical): element k of a row sits in 32-bit word k/8 at
+ * bits [4*(k%8), 4*(k%8)+3]; signed codes keep their two's-complement nibble.
+ */
+#ifndef QIL_H_
+#define QIL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QIL_OK = 0,
+    QIL_ERR_NULL = 1,        /* a required pointer is null */
+    QIL_ERR_SHAPE = 2,       /* non-positive size, K % 8 != 0, K % group_size != 0, ... */
+    QIL_ERR_ALIGN = 3,       /* a tensor base is not 16-byte aligned */
+    QIL_ERR_UNSUPPORTED = 4, /* enum value / combination the library does not implement */
+    QIL_ERR_WORKSPACE = 5,   /* workspace missing or too small */
+    QIL_ERR_CUDA = 6,        /* the CUDA runtime reported an error at launch */
+    QIL_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (read through qil_device_status) */
+    QIL_ERR_RANGE = 8        /* a quantisation scale does not fit fp16 (device flag) */
+} qil_status;
+
+typedef enum { QIL_F32 = 0, QIL_BF16 = 1, QIL_F16 = 2 } qil_dtype;
+
+/*
+ * QIL_LAYOUT_CANONICAL: packed words [N][K/8], row-major.
+ * QIL_LAYOUT_TILE16   : the word matrix is cut into tiles of 16 rows x 16 words
+ *   (= 128 columns of K).  Tiles are stored one after another, all column tiles
+ *   of row-tile 0 first; inside a tile the 16 rows follow each other, 16 words
+ *   each.  Word (n, i) is at ((n/16)*(K/128) + i/16)*256 + (n%16)*16 + i%16.
+ *   Needs N % 16 == 0 and K % 128 == 0.  A warp of the decode kernel reads one
+ *   tile (1 KiB) with two fully coalesced 512-byte loads.
+ */
+typedef enum { QIL_LAYOUT_CANONICAL = 0, QIL_LAYOUT_TILE16 = 1 } qil_layout;
+
+typedef struct CUstream_st* qil_stream_t; /* a cudaStream_t */
+
+/* ------------------------------------------------------------------------
+ * Weight quantiser (Sec. 2.1 round-to-nearest; 4-bit weights of Sec. 5.4 and
+ * Sec. 5.1).  symmetric = 0: uint4 codes 0..15, fp16 scale and fp16 zero point
+ * per group (scale_dtype must be QIL_F16, zeros required).  symmetric = 1: int4
+ * codes -8..7 stored as int8 in codes[], scale per group in scale_dtype
+ * (QIL_F32 or QIL_F16), zeros ignored (may be null).  group_size == K gives one
+ * scale per output channel (the paper's channel-wise setting, App. A.1.2).
+ *   w      [N][K] of w_dtype          codes  [N][K] one code per byte
+ *   scales [N][K/group_size]          zeros  [N][K/group_size] fp16
+ *   dev_status: optional device int; QIL_ERR_RANGE is OR-ed into it when a
+ *   scale overflows fp16 (the codes of that group are then unspecified).
+ * Errors: NULL, SHAPE (sizes <= 0, K % group_size), ALIGN, UNSUPPORTED, CUDA.
+ * ---------------------------------------------------------------------- */
+qil_status qil_quantize_rtn_w4(const void* w, qil_dtype w_dtype, int N, int K, int group_size,
+                               int symmetric, uint8_t* codes, void* scales, qil_dtype scale_dtype,
+                               void* zeros, int* dev_status, qil_stream_t stream);
+
+/* Pack 8 codes per 32-bit word (layout rules above); works for unsigned codes
+ * and for two's-complement int8 codes alike (the low nibble is kept).
+ * Errors: NULL, SHAPE (K % 8; TILE16: N % 16, K % 128), ALIGN, UNSUPPORTED. */
+qil_status qil_pack_w4(const uint8_t* codes, int N, int K, qil_layout layout, uint32_t* packed,
+                       qil_stream_t stream);
+/* Inverse of qil_pack_w4; is_signed != 0 sign-extends each nibble into int8. */
+qil_status qil_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout, int is_signed,
+                         uint8_t* codes, qil_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * Weight-only linear, 4-bit weights x bf16 activations (the OpenVLA / Llama-2
+ * decode and prefill linears, Sec. 5.4, App. A.4.2): dequantisation is fused
+ * into the matmul, accumulation is fp32, the result is rounded to bf16.
+ *   x [M][K] bf16   qweight packed per `layout`   scales, zeros [N][K/group_size] fp16
+ *   y [M][N] bf16
+ * The kernel is chosen from the shape: tensor-core skinny kernel (weights read
+ * once, any M handled in slabs of 64 rows) when K % 128 == 0 and
+ * group_size % 128 == 0; a general kernel otherwise (any K % 8 == 0, any
+ * group_size dividing K, canonical layout only).
+ * workspace: qil_linear_w4a16_workspace_size() bytes, only touched when the
+ * shape needs a split along K; it must be zero-filled once before first use
+ * (the kernel leaves it zeroed again).  Calls that share a workspace must not
+ * overlap on the device.
+ * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, CUDA.
+ * ---------------------------------------------------------------------- */
+size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size);
+qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* scales,
+                            const void* zeros, void* y, int M, int N, int K, int group_size,
+                            qil_layout layout, void* workspace, size_t workspace_bytes,
+                            qil_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * Activation quantiser of the W4A4 path (Sec. 5.1: the compute-bound driving
+ * policy needs weights and activations in 4 bits): symmetric int4 per row.
+ *   x [M][K] bf16 -> qx packed [M][K/8] (canonical), scales [M] fp32.
+ * static_scale (host pointer) null: per-row absmax.  Non-null: that one fp32
+ * value is used for every row (tensor-wise setting of App. A.1.2) and written
+ * to scales[].
+ * ---------------------------------------------------------------------- */
+qil_status qil_quantize_act_a4(const void* x, int M, int K, const float* static_scale /*host*/,
+                               uint32_t* qx, float* scales, qil_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * W4A4 integer GEMM (Sec. 5.1 / Sec. 5.4 autonomous-driving deployment):
+ *   acc[m][n] = sum_k qx[m][k] * qw[n][k]   (int32, exact)
+ *   y[m][n]   = bf16( float(acc) * (sx[m] * sw[n]) )
+ *   qx [M][K/8], qw [N][K/8] canonical packed signed nibbles; sx [M], sw [N] fp32
+ *   acc_out: optional [M][N] int32 copy of the raw accumulators.
+ * Needs K % 32 == 0.  |acc| <= 64 K must fit int32.
+ * ---------------------------------------------------------------------- */
+size_t qil_linear_w4a4_workspace_size(int M, int N, int K);
+qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw,
+                           void* y, int32_t* acc_out, int M, int N, int K, void* workspace,
+                           size_t workspace_bytes, qil_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * Helpers
+ * ---------------------------------------------------------------------- */
+const char* qil_status_string(qil_status s);
+int qil_version(void);
+/* Copies the device status word to *out (host) and waits for that copy. */
+qil_status qil_device_status(const int* dev_status, int* out /*host*/, qil_stream_t stream);
+
+/* Measurement helpers (not part of the method): a dense bf16 GEMV
+ * y[n] = sum_k x[k] W[n][k] with W bf16 [N][K], the 16-bit baseline the paper's
+ * speedups are quoted against (Table "OpenVLA performance"); and a read-only
+ * streaming pass over `bytes` bytes that adds every 32-bit word into *sink. */
+qil_status qil_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, qil_stream_t stream);
+qil_status qil_probe_hbm_read(const void* buf, size_t bytes, unsigned int* sink, qil_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QIL_H_ */

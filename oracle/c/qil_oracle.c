@@ -115,7 +115,7 @@ int qo_quantize_rtn_w4_asym(const float* w, int N, int K, int G,
                 codes[(size_t)n * K + (size_t)g * G + k] = (uint8_t)q;
             }
             scales[(size_t)n * ng + g] = s16;
-            zeros[(size_t)n * ng + g] = qo_f32_to_f16(z);
+            zeros[(size_t)n * ng + g] = qo_f32_to_f16((float)(int)z); /* integer, never -0 */
         }
     }
     return bad;

@@ -70,7 +70,8 @@ def quantize_rtn_w4_asym(w: np.ndarray, group_size: int):
     u = (np.rint((wg / s[:, :, None]).astype(F32)) + z[:, :, None]).astype(F32)
     q = np.clip(u, F32(0), F32(15))
     codes = q.astype(np.uint8).reshape(N, K)
-    return codes, s16, z.astype(np.float16)
+    # the zero point is an integer: store it as fp16(int(z)) (never a negative zero)
+    return codes, s16, z.astype(np.uint8).astype(np.float16)
 
 
 def unclamped_levels_asym(w: np.ndarray, group_size: int):

@@ -1,0 +1,168 @@
+// C ABI of the library: argument validation on the host, then one launcher each.
+#include <atomic>
+
+#include "qil_common.cuh"
+
+namespace qil {
+
+int num_sms() {
+    static std::atomic<int> cached{0};
+    int v = cached.load(std::memory_order_relaxed);
+    if (v > 0) return v;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+        (void)cudaGetLastError();
+        return QIL_NUM_SMS_FALLBACK;  // not cached: a later call may succeed
+    }
+    cached.store(sms, std::memory_order_relaxed);
+    return sms;
+}
+
+}  // namespace qil
+
+using namespace qil;
+
+namespace {
+inline cudaStream_t S(qil_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
+inline bool dtype_ok(int d) { return d == QIL_F32 || d == QIL_BF16 || d == QIL_F16; }
+inline bool layout_ok(int l) { return l == QIL_LAYOUT_CANONICAL || l == QIL_LAYOUT_TILE16; }
+}  // namespace
+
+extern "C" {
+
+const char* qil_status_string(qil_status s) {
+    switch (s) {
+        case QIL_OK: return "ok";
+        case QIL_ERR_NULL: return "null pointer";
+        case QIL_ERR_SHAPE: return "bad shape";
+        case QIL_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case QIL_ERR_UNSUPPORTED: return "unsupported argument";
+        case QIL_ERR_WORKSPACE: return "workspace missing or too small";
+        case QIL_ERR_CUDA: return "CUDA error";
+        case QIL_ERR_TIMEOUT: return "device-side wait timed out";
+        case QIL_ERR_RANGE: return "scale does not fit fp16";
+    }
+    return "unknown status";
+}
+
+int qil_version(void) { return 100; }
+
+qil_status qil_device_status(const int* dev_status, int* out, qil_stream_t stream) {
+    if (!dev_status || !out) return QIL_ERR_NULL;
+    if (cudaMemcpyAsync(out, dev_status, sizeof(int), cudaMemcpyDeviceToHost, S(stream)) != cudaSuccess ||
+        cudaStreamSynchronize(S(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return QIL_ERR_CUDA;
+    }
+    return QIL_OK;
+}
+
+qil_status qil_quantize_rtn_w4(const void* w, qil_dtype w_dtype, int N, int K, int group_size, int symmetric,
+                               uint8_t* codes, void* scales, qil_dtype scale_dtype, void* zeros,
+                               int* dev_status, qil_stream_t stream) {
+    if (!w || !codes || !scales) return QIL_ERR_NULL;
+    if (!symmetric && !zeros) return QIL_ERR_NULL;
+    if (N <= 0 || K <= 0 || group_size <= 0 || K % group_size != 0) return QIL_ERR_SHAPE;
+    if (!dtype_ok(w_dtype) || !dtype_ok(scale_dtype)) return QIL_ERR_UNSUPPORTED;
+    if (!symmetric && scale_dtype != QIL_F16) return QIL_ERR_UNSUPPORTED;
+    if (symmetric && scale_dtype == QIL_BF16) return QIL_ERR_UNSUPPORTED;
+    if (!aligned16(w) || !aligned16(codes) || !aligned16(scales) || (zeros && !aligned16(zeros))) return QIL_ERR_ALIGN;
+    return launch_quantize_rtn_w4(w, w_dtype, N, K, group_size, symmetric, codes, scales, scale_dtype, zeros,
+                                  dev_status, S(stream));
+}
+
+static qil_status check_pack(const void* a, const void* b, int N, int K, qil_layout layout) {
+    if (!a || !b) return QIL_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 8 != 0) return QIL_ERR_SHAPE;
+    if (!layout_ok(layout)) return QIL_ERR_UNSUPPORTED;
+    if (layout == QIL_LAYOUT_TILE16 && (N % 16 != 0 || K % 128 != 0)) return QIL_ERR_SHAPE;
+    if (!aligned16(a) || !aligned16(b)) return QIL_ERR_ALIGN;
+    return QIL_OK;
+}
+
+qil_status qil_pack_w4(const uint8_t* codes, int N, int K, qil_layout layout, uint32_t* packed, qil_stream_t stream) {
+    const qil_status s = check_pack(codes, packed, N, K, layout);
+    if (s != QIL_OK) return s;
+    return launch_pack_w4(codes, N, K, layout, packed, S(stream));
+}
+
+qil_status qil_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout, int is_signed, uint8_t* codes,
+                         qil_stream_t stream) {
+    const qil_status s = check_pack(packed, codes, N, K, layout);
+    if (s != QIL_OK) return s;
+    return launch_unpack_w4(packed, N, K, layout, is_signed, codes, S(stream));
+}
+
+static qil_status check_w4a16(const void* x, const void* qw, const void* sc, const void* z, const void* y, int M,
+                              int N, int K, int G, qil_layout layout) {
+    if (!x || !qw || !sc || !z || !y) return QIL_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || G <= 0 || K % 8 != 0 || K % G != 0) return QIL_ERR_SHAPE;
+    if (!layout_ok(layout)) return QIL_ERR_UNSUPPORTED;
+    if (layout == QIL_LAYOUT_TILE16 && (N % 16 != 0 || K % 128 != 0)) return QIL_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(qw) || !aligned16(sc) || !aligned16(z) || !aligned16(y)) return QIL_ERR_ALIGN;
+    return QIL_OK;
+}
+
+size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size) {
+    if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0) return 0;
+    if (K % 128 != 0 || group_size % 128 != 0) return 0;
+    return w4a16_skinny_workspace(M, N, K, group_size);
+}
+
+qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* scales, const void* zeros, void* y,
+                            int M, int N, int K, int group_size, qil_layout layout, void* workspace,
+                            size_t workspace_bytes, qil_stream_t stream) {
+    const qil_status s = check_w4a16(x, qweight, scales, zeros, y, M, N, K, group_size, layout);
+    if (s != QIL_OK) return s;
+    if (workspace && !aligned16(workspace)) return QIL_ERR_ALIGN;
+    if (w4a16_skinny_supported(M, N, K, group_size, layout))
+        return launch_w4a16_skinny(x, qweight, scales, zeros, y, M, N, K, group_size, layout, workspace,
+                                   workspace_bytes, S(stream));
+    if (layout != QIL_LAYOUT_CANONICAL) return QIL_ERR_UNSUPPORTED;
+    return launch_w4a16_general(x, qweight, scales, zeros, y, M, N, K, group_size, S(stream));
+}
+
+qil_status qil_quantize_act_a4(const void* x, int M, int K, const float* static_scale, uint32_t* qx, float* scales,
+                               qil_stream_t stream) {
+    if (!x || !qx || !scales) return QIL_ERR_NULL;
+    if (M <= 0 || K <= 0 || K % 8 != 0) return QIL_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(qx) || !aligned16(scales)) return QIL_ERR_ALIGN;
+    if (static_scale && !(*static_scale > 0.0f)) return QIL_ERR_UNSUPPORTED;
+    return launch_quantize_act_a4(x, M, K, static_scale != nullptr, static_scale ? *static_scale : 0.0f, qx, scales,
+                                  S(stream));
+}
+
+size_t qil_linear_w4a4_workspace_size(int M, int N, int K) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    return w4a4_workspace(M, N, K);
+}
+
+qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, void* y,
+                           int32_t* acc_out, int M, int N, int K, void* workspace, size_t workspace_bytes,
+                           qil_stream_t stream) {
+    if (!qx || !sx || !qw || !sw || !y) return QIL_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || K > 131072) return QIL_ERR_SHAPE;
+    if (!aligned16(qx) || !aligned16(sx) || !aligned16(qw) || !aligned16(sw) || !aligned16(y) ||
+        (acc_out && !aligned16(acc_out)) || (workspace && !aligned16(workspace)))
+        return QIL_ERR_ALIGN;
+    if (w4a4_workspace(M, N, K) > 0 && (!workspace || workspace_bytes < w4a4_workspace(M, N, K)))
+        return QIL_ERR_WORKSPACE;
+    return launch_w4a4(qx, sx, qw, sw, y, acc_out, M, N, K, workspace, workspace_bytes, S(stream));
+}
+
+qil_status qil_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, qil_stream_t stream) {
+    if (!x || !w || !y) return QIL_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 8 != 0) return QIL_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return QIL_ERR_ALIGN;
+    return launch_ref_gemv_bf16(x, w, y, N, K, S(stream));
+}
+
+qil_status qil_probe_hbm_read(const void* buf, size_t bytes, unsigned int* sink, qil_stream_t stream) {
+    if (!buf || !sink) return QIL_ERR_NULL;
+    if (bytes < 16) return QIL_ERR_SHAPE;
+    if (!aligned16(buf)) return QIL_ERR_ALIGN;
+    return launch_probe_hbm_read(buf, bytes, sink, S(stream));
+}
+
+}  // extern "C"

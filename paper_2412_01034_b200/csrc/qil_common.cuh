@@ -1,0 +1,78 @@
+// Shared device/host helpers of the qil kernels (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qil.h"
+
+#define QIL_NUM_SMS_FALLBACK 148
+
+namespace qil {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline qil_status launch_status() {
+    return cudaGetLastError() == cudaSuccess ? QIL_OK : QIL_ERR_CUDA;
+}
+
+// Number of SMs of the current device (cached per process; the library targets one device type).
+int num_sms();
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) {
+    return __uint_as_float(static_cast<uint32_t>(b) << 16);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_min(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Streaming 128-bit load that does not allocate in L1 (weights are read exactly once).
+__device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// Internal launchers (one per translation unit).
+qil_status launch_quantize_rtn_w4(const void* w, qil_dtype w_dtype, int N, int K, int G, int symmetric,
+                                  uint8_t* codes, void* scales, qil_dtype scale_dtype, void* zeros,
+                                  int* dev_status, cudaStream_t st);
+qil_status launch_pack_w4(const uint8_t* codes, int N, int K, qil_layout layout, uint32_t* packed, cudaStream_t st);
+qil_status launch_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout, int is_signed,
+                            uint8_t* codes, cudaStream_t st);
+qil_status launch_quantize_act_a4(const void* x, int M, int K, bool use_static, float static_scale,
+                                  uint32_t* qx, float* scales, cudaStream_t st);
+
+qil_status launch_w4a16_general(const void* x, const uint32_t* qw, const void* scales, const void* zeros,
+                                void* y, int M, int N, int K, int G, cudaStream_t st);
+bool w4a16_skinny_supported(int M, int N, int K, int G, qil_layout layout);
+size_t w4a16_skinny_workspace(int M, int N, int K, int G);
+qil_status launch_w4a16_skinny(const void* x, const uint32_t* qw, const void* scales, const void* zeros,
+                               void* y, int M, int N, int K, int G, qil_layout layout, void* ws,
+                               size_t ws_bytes, cudaStream_t st);
+
+size_t w4a4_workspace(int M, int N, int K);
+qil_status launch_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, void* y,
+                       int32_t* acc_out, int M, int N, int K, void* ws, size_t ws_bytes, cudaStream_t st);
+
+qil_status launch_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, cudaStream_t st);
+qil_status launch_probe_hbm_read(const void* buf, size_t bytes, unsigned int* sink, cudaStream_t st);
+
+}  // namespace qil

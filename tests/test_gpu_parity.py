@@ -1,0 +1,342 @@
+"""GPU parity: every entry point of the C ABI against the CPU oracle on the same seeded inputs.
+
+Integer results (codes, scales, zero points, packed words, int32 accumulators) must be bit-exact;
+bf16 outputs are judged per output row (see tests/util.py).
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import c_oracle, np_oracle
+from paper_2412_01034_b200 import workloads as wl
+from tests.util import assert_rows_close, bf16_to_f64, bits_of, cuda, to_bf16_cuda
+
+pytestmark = pytest.mark.gpu
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_cases.json")))
+
+
+@pytest.fixture(scope="module")
+def api():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2412_01034_b200 import api as a
+    return a
+
+
+def f16_bits(a):
+    return np.ascontiguousarray(a).view(np.uint8)
+
+
+# ----------------------------------------------------------------------------
+# quantisers
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("case", ["asym_4x8_g8", "asym_4x8_g4"])
+def test_quantize_hand_cases(api, case):
+    c = GOLD[case]
+    w = np.array(c["w"], dtype=np.float32)
+    codes, scales, zeros = api.quantize_rtn_w4(cuda(w), c["group"])
+    np.testing.assert_array_equal(codes.cpu().numpy(), np.array(c["codes"], dtype=np.uint8))
+    np.testing.assert_array_equal(scales.cpu().numpy().astype(np.float64), np.array(c["scales"]))
+    np.testing.assert_array_equal(zeros.cpu().numpy().astype(np.float64), np.array(c["zeros"], dtype=np.float64))
+
+
+@pytest.mark.parametrize("N,K,G", [(96, 1024, 128), (33, 384, 128), (7, 4096, 4096), (64, 256, 32), (5, 40, 8)])
+def test_quantize_asym_bit_exact(api, N, K, G):
+    w = wl.normal_weights(200, N * 7 + K, N, K, 0.02, outlier_prob=0.001)
+    w[0, :G] = 0.0            # all-zero group
+    w[1 % N, :G] = -0.3       # all-equal group
+    w[2 % N, 0] = 1e-9
+    ref = np_oracle.quantize_rtn_w4_asym(w, G)
+    got = api.quantize_rtn_w4(cuda(w), G)
+    np.testing.assert_array_equal(got[0].cpu().numpy(), ref[0])
+    np.testing.assert_array_equal(bits_of(got[1]), f16_bits(ref[1]).reshape(-1))
+    np.testing.assert_array_equal(bits_of(got[2]), f16_bits(ref[2]).reshape(-1))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+def test_quantize_asym_16bit_inputs(api, dtype):
+    import torch
+    w32 = wl.normal_weights(201, 0, 48, 512, 0.02)
+    wt = cuda(w32).to(torch.bfloat16 if dtype == "bf16" else torch.float16)
+    w_widened = wt.to(torch.float32).cpu().numpy()  # exact widening
+    ref = np_oracle.quantize_rtn_w4_asym(w_widened, 128)
+    got = api.quantize_rtn_w4(wt, 128)
+    np.testing.assert_array_equal(got[0].cpu().numpy(), ref[0])
+    np.testing.assert_array_equal(bits_of(got[1]), f16_bits(ref[1]).reshape(-1))
+    np.testing.assert_array_equal(bits_of(got[2]), f16_bits(ref[2]).reshape(-1))
+
+
+def test_quantize_scale_overflow_sets_error(api):
+    w = np.zeros((2, 128), dtype=np.float32)
+    w[1, 5] = 2.0e6
+    with pytest.raises(api.QilError) as e:
+        api.quantize_rtn_w4(cuda(w), 128)
+    assert e.value.code == api.ERR_RANGE
+
+
+@pytest.mark.parametrize("stage", [0, 3])
+def test_quantize_sym_per_channel(api, stage):
+    _, w = wl.conv_stage(stage, batch=1)
+    w[3] = 0.0
+    ref_q, ref_s = np_oracle.quantize_sym4(w)
+    q, s, z = api.quantize_rtn_w4(cuda(w), w.shape[1], symmetric=True)
+    assert z is None
+    np.testing.assert_array_equal(q.cpu().numpy(), ref_q)
+    np.testing.assert_array_equal(bits_of(s), np.ascontiguousarray(ref_s).view(np.uint8).reshape(-1))
+
+
+def test_quantize_sym_groups_f16_scale(api):
+    import torch
+    w = wl.normal_weights(202, 0, 24, 512, 0.05)
+    ref_q, ref_s = np_oracle.quantize_sym4(w, group_size=64, scale_f16=True)
+    q, s, _ = api.quantize_rtn_w4(cuda(w), 64, symmetric=True, scale_dtype=torch.float16)
+    np.testing.assert_array_equal(q.cpu().numpy(), ref_q)
+    np.testing.assert_array_equal(bits_of(s), f16_bits(ref_s).reshape(-1))
+
+
+def test_quantize_act_matches_oracle(api):
+    c = GOLD["sym_row"]
+    v = np.array(c["v"], dtype=np.float32)
+    qx, sx = api.quantize_act_a4(to_bf16_cuda(wl.f32_to_bf16_bits(v)))
+    got = np_oracle.unpack_w4(qx.cpu().numpy().view(np.uint32), signed=True)
+    np.testing.assert_array_equal(got, np.array(c["codes"], dtype=np.int8))
+    assert float(sx[0]) == c["scale"][0]
+    vs = np.array(c["v_static"], dtype=np.float32)
+    qx, sx = api.quantize_act_a4(to_bf16_cuda(wl.f32_to_bf16_bits(vs)), static_scale=c["static_scale"])
+    np.testing.assert_array_equal(np_oracle.unpack_w4(qx.cpu().numpy().view(np.uint32), signed=True),
+                                  np.array(c["codes_static"], dtype=np.int8))
+    assert float(sx[0]) == c["static_scale"]
+
+
+@pytest.mark.parametrize("stage,batch", [(3, 2), (2, 1), (0, 1)])
+def test_quantize_act_conv_inputs(api, stage, batch):
+    x, _ = wl.conv_stage(stage, batch=batch)
+    x[1] = 0  # an all-zero row
+    ref_q, ref_s = np_oracle.quantize_sym4(wl.bf16_bits_to_f32(x))
+    qx, sx = api.quantize_act_a4(to_bf16_cuda(x))
+    np.testing.assert_array_equal(qx.cpu().numpy().view(np.uint32), np_oracle.pack_w4(ref_q))
+    np.testing.assert_array_equal(bits_of(sx), np.ascontiguousarray(ref_s).view(np.uint8).reshape(-1))
+
+
+def test_quantize_act_ragged_k_and_static(api):
+    x = wl.normal_activations_bf16(203, 0, 37, 40)
+    ref_q, ref_s = np_oracle.quantize_sym4(wl.bf16_bits_to_f32(x), static_scale=0.4)
+    qx, sx = api.quantize_act_a4(to_bf16_cuda(x), static_scale=0.4)
+    np.testing.assert_array_equal(qx.cpu().numpy().view(np.uint32), np_oracle.pack_w4(ref_q))
+    assert ref_q.min() == -8 and ref_q.max() == 7
+    np.testing.assert_array_equal(sx.cpu().numpy(), np.full(37, np.float32(0.4)))
+
+
+# ----------------------------------------------------------------------------
+# packing
+# ----------------------------------------------------------------------------
+def test_pack_hand_words(api):
+    c = GOLD["pack_words"]
+    u = api.pack_w4(cuda(np.array(c["unsigned_codes"], dtype=np.uint8)))
+    assert int(u.cpu().numpy().view(np.uint32)[0, 0]) == int(c["unsigned_word"][0], 16)
+    s = api.pack_w4(cuda(np.array(c["signed_codes"], dtype=np.int8)))
+    assert int(s.cpu().numpy().view(np.uint32)[0, 0]) == int(c["signed_word"][0], 16)
+
+
+@pytest.mark.parametrize("N,K", [(48, 384), (16, 128), (33, 264)])
+def test_pack_unpack_layouts(api, N, K):
+    rng = np.random.default_rng(N + K)
+    codes = rng.integers(0, 16, size=(N, K)).astype(np.uint8)
+    ref = np_oracle.pack_w4(codes)
+    p = api.pack_w4(cuda(codes), api.LAYOUT_CANONICAL)
+    np.testing.assert_array_equal(p.cpu().numpy().view(np.uint32), ref)
+    np.testing.assert_array_equal(api.unpack_w4(p, N, K).cpu().numpy(), codes)
+    if N % 16 == 0 and K % 128 == 0:
+        pt = api.pack_w4(cuda(codes), api.LAYOUT_TILE16)
+        np.testing.assert_array_equal(pt.cpu().numpy().view(np.uint32), np_oracle.to_layout(ref, np_oracle.LAYOUT_TILE16))
+        np.testing.assert_array_equal(api.unpack_w4(pt, N, K, api.LAYOUT_TILE16).cpu().numpy(), codes)
+    sc = rng.integers(-8, 8, size=(N, K)).astype(np.int8)
+    ps = api.pack_w4(cuda(sc))
+    np.testing.assert_array_equal(api.unpack_w4(ps, N, K, signed=True).cpu().numpy(), sc)
+
+
+# ----------------------------------------------------------------------------
+# W4A16
+# ----------------------------------------------------------------------------
+def _w4a16_case(api, M, N, K, G, layout, seed, outliers=True):
+    w = wl.normal_weights(300, seed, N, K, 0.02, outlier_prob=0.001 if outliers else 0.0)
+    x = wl.normal_activations_bf16(300, seed + 1, M, K)
+    codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
+    y_ref = c_oracle.linear_w4a16(x, codes, scales, zeros, G)
+    packed = api.pack_w4(cuda(codes), layout)
+    y = api.linear_w4a16(to_bf16_cuda(x), packed, cuda(scales), cuda(zeros), N, G, layout)
+    assert tuple(y.shape) == (M, N)
+    assert_rows_close(bf16_to_f64(y), y_ref)
+    return y
+
+
+@pytest.mark.parametrize("case", ["asym_4x8_g8", "asym_4x8_g4"])
+def test_w4a16_hand_cases(api, case):
+    c = GOLD[case]
+    codes = np.array(c["codes"], dtype=np.uint8)
+    scales = np.array(c["scales"], dtype=np.float16)
+    zeros = np.array(c["zeros"], dtype=np.float16)
+    x = wl.f32_to_bf16_bits(np.array(GOLD["x_rows_8"], dtype=np.float32))
+    packed = api.pack_w4(cuda(codes))
+    y = api.linear_w4a16(to_bf16_cuda(x), packed, cuda(scales), cuda(zeros), 4, c["group"])
+    assert_rows_close(bf16_to_f64(y), np.array(c["y"]))
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 7, 8, 9, 16, 17, 33, 64, 65, 130])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_w4a16_skinny_m_sweep(api, M, layout):
+    _w4a16_case(api, M, 208, 1024, 128, layout, seed=M)
+
+
+@pytest.mark.parametrize("N,K,G,layout", [
+    (16, 128, 128, 1), (16, 128, 128, 0), (100, 384, 128, 0), (1000, 2176, 128, 0), (48, 1024, 256, 1),
+    (48, 1024, 1024, 1), (4096, 4096, 128, 1), (256, 11008, 128, 1), (11008, 512, 128, 0),
+])
+def test_w4a16_skinny_shapes(api, N, K, G, layout):
+    for M in (1, 5):
+        _w4a16_case(api, M, N, K, G, layout, seed=N + K + G)
+
+
+@pytest.mark.parametrize("N,K,G", [(24, 256, 32), (9, 40, 8), (17, 192, 64), (8, 320, 320)])
+def test_w4a16_general_shapes(api, N, K, G):
+    for M in (1, 6):
+        _w4a16_case(api, M, N, K, G, 0, seed=N * K)
+
+
+def test_w4a16_is_deterministic_and_workspace_is_reusable(api):
+    import torch
+    N, K, G, M = 512, 4096, 128, 4
+    w = wl.normal_weights(301, 0, N, K, 0.02)
+    x = wl.normal_activations_bf16(301, 1, M, K)
+    codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
+    y_ref = c_oracle.linear_w4a16(x, codes, scales, zeros, G)
+    packed = api.pack_w4(cuda(codes), 1)
+    ws = api.new_workspace(api.linear_w4a16_workspace_size(M, N, K, G))
+    xs, sc, zr = to_bf16_cuda(x), cuda(scales), cuda(zeros)
+    outs = [api.linear_w4a16(xs, packed, sc, zr, N, G, 1, workspace=ws).clone() for _ in range(3)]
+    torch.cuda.synchronize()
+    assert_rows_close(bf16_to_f64(outs[0]), y_ref)
+    for o in outs[1:]:
+        np.testing.assert_array_equal(bits_of(o), bits_of(outs[0]))
+    # canary: the call writes nothing outside y
+    big = torch.full((M * N + 64,), 7.0, dtype=torch.bfloat16, device="cuda")
+    api.linear_w4a16(xs, packed, sc, zr, N, G, 1, out=big[:M * N].view(M, N), workspace=ws)
+    assert torch.all(big[M * N:] == 7.0)
+
+
+def test_w4a16_large_activations_keep_precision(api):
+    """|x| up to a few thousand (LLM outlier channels): the 128-offset trick must not lose the signal."""
+    N, K, G, M = 64, 1024, 128, 3
+    w = wl.normal_weights(302, 0, N, K, 0.02)
+    xf = wl.bf16_bits_to_f32(wl.normal_activations_bf16(302, 1, M, K)).copy()
+    xf[:, ::97] *= 3000.0
+    x = wl.f32_to_bf16_bits(xf)
+    codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
+    y_ref = c_oracle.linear_w4a16(x, codes, scales, zeros, G)
+    y = api.linear_w4a16(to_bf16_cuda(x), api.pack_w4(cuda(codes), 1), cuda(scales), cuda(zeros), N, G, 1)
+    assert_rows_close(bf16_to_f64(y), y_ref)
+
+
+def test_cfg0_full(api):
+    """Config 0 exactly as stated: M=1, K=N=4096, N(0, 0.02) weights, group 128, seed 0."""
+    w, x = wl.cfg0()
+    ref = np_oracle.quantize_rtn_w4_asym(w, 128)
+    got = api.quantize_rtn_w4(cuda(w), 128)
+    np.testing.assert_array_equal(got[0].cpu().numpy(), ref[0])
+    np.testing.assert_array_equal(bits_of(got[1]), f16_bits(ref[1]).reshape(-1))
+    np.testing.assert_array_equal(bits_of(got[2]), f16_bits(ref[2]).reshape(-1))
+    for layout in (0, 1):
+        packed = api.pack_w4(got[0], layout)
+        np.testing.assert_array_equal(packed.cpu().numpy().view(np.uint32).reshape(-1),
+                                      np_oracle.to_layout(np_oracle.pack_w4(ref[0]), layout))
+        y = api.linear_w4a16(to_bf16_cuda(x), packed, got[1], got[2], 4096, 128, layout)
+        assert_rows_close(bf16_to_f64(y), c_oracle.linear_w4a16(x, *ref, 128))
+
+
+@pytest.mark.parametrize("N,K", [(wl.FFN, wl.HIDDEN), (wl.HIDDEN, wl.FFN)])
+@pytest.mark.parametrize("M", [1, 16, 64])
+def test_cfg3_shapes(api, N, K, M):
+    """Config 3 shapes; the oracle runs on 512 sampled output features (the kernel computes all N)."""
+    w = wl.normal_weights(3, 0 if N == wl.FFN else 1, N, K, 0.02)
+    x = wl.normal_activations_bf16(3, 10 + M, M, K)
+    got = api.quantize_rtn_w4(cuda(w), 128)
+    packed = api.pack_w4(got[0], 1)
+    y = bf16_to_f64(api.linear_w4a16(to_bf16_cuda(x), packed, got[1], got[2], N, 128, 1))
+    rows = np.sort(np.random.default_rng(M).choice(N, 512, replace=False))
+    ref = np_oracle.quantize_rtn_w4_asym(w[rows], 128)
+    np.testing.assert_array_equal(got[0].cpu().numpy()[rows], ref[0])
+    y_ref = c_oracle.linear_w4a16(x, *ref, 128)
+    # the row maximum over the sampled features lower-bounds the true row maximum: the check is stricter
+    assert_rows_close(y[:, rows], y_ref)
+
+
+# ----------------------------------------------------------------------------
+# W4A4
+# ----------------------------------------------------------------------------
+def test_w4a4_hand_case(api):
+    c = GOLD["w4a4_small"]
+    qx = np.zeros((2, 32), np.int8); qx[:, :8] = np.array(c["qx"], np.int8)
+    qw = np.zeros((3, 32), np.int8); qw[:, :8] = np.array(c["qw"], np.int8)
+    y, acc = api.linear_w4a4(api.pack_w4(cuda(qx)), cuda(np.array(c["sx"], np.float32)), api.pack_w4(cuda(qw)),
+                             cuda(np.array(c["sw"], np.float32)), want_acc=True)
+    np.testing.assert_array_equal(acc.cpu().numpy(), np.array(c["acc"], dtype=np.int32))
+    np.testing.assert_array_equal(bf16_to_f64(y), np.array(c["y"]))
+
+
+def test_w4a4_extreme_codes(api):
+    M, N, K = 19, 70, 4608
+    qx = np.full((M, K), -8, np.int8)
+    qw = np.full((N, K), -8, np.int8)
+    qw[1] = 7
+    one = np.ones(max(M, N), np.float32)
+    y, acc = api.linear_w4a4(api.pack_w4(cuda(qx)), cuda(one[:M]), api.pack_w4(cuda(qw)), cuda(one[:N]), want_acc=True)
+    a = acc.cpu().numpy()
+    assert np.all(a[:, 0] == 64 * K) and np.all(a[:, 1] == -56 * K)
+
+
+@pytest.mark.parametrize("stage,batch", [(0, 2), (1, 3), (2, 4), (3, 32), (0, 32)])
+def test_w4a4_conv_stages(api, stage, batch):
+    x, w = wl.conv_stage(stage, batch=batch)
+    qx_ref, sx_ref = np_oracle.quantize_sym4(wl.bf16_bits_to_f32(x))
+    qw_ref, sw_ref = np_oracle.quantize_sym4(w)
+    acc_ref, y_ref = c_oracle.linear_w4a4(qx_ref, sx_ref, qw_ref, sw_ref)
+    qx, sx = api.quantize_act_a4(to_bf16_cuda(x))
+    qw, sw, _ = api.quantize_rtn_w4(cuda(w), w.shape[1], symmetric=True)
+    y, acc = api.linear_w4a4(qx, sx, api.pack_w4(qw), sw.reshape(-1), want_acc=True)
+    np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert_rows_close(bf16_to_f64(y), y_ref)
+    y2 = api.linear_w4a4(qx, sx, api.pack_w4(qw), sw.reshape(-1))
+    np.testing.assert_array_equal(bits_of(y2), bits_of(y))
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 32), (17, 9, 96), (130, 200, 160), (64, 64, 1152)])
+def test_w4a4_ragged_shapes(api, M, N, K):
+    rng = np.random.default_rng(M * N + K)
+    qx = rng.integers(-8, 8, size=(M, K)).astype(np.int8)
+    qw = rng.integers(-8, 8, size=(N, K)).astype(np.int8)
+    sx = rng.random(M).astype(np.float32) + 0.1
+    sw = rng.random(N).astype(np.float32) + 0.1
+    acc_ref, y_ref = np_oracle.linear_w4a4(qx, sx, qw, sw)
+    y, acc = api.linear_w4a4(api.pack_w4(cuda(qx)), cuda(sx), api.pack_w4(cuda(qw)), cuda(sw), want_acc=True)
+    np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert_rows_close(bf16_to_f64(y), y_ref)
+
+
+# ----------------------------------------------------------------------------
+# measurement helpers
+# ----------------------------------------------------------------------------
+def test_ref_gemv_bf16(api):
+    import torch
+    N, K = 300, 1024
+    w = wl.normal_activations_bf16(400, 0, N, K)
+    x = wl.normal_activations_bf16(400, 1, 1, K)
+    y = api.ref_gemv_bf16(to_bf16_cuda(x), to_bf16_cuda(w))
+    ref = wl.bf16_bits_to_f32(x).astype(np.float64) @ wl.bf16_bits_to_f32(w).astype(np.float64).T
+    assert_rows_close(bf16_to_f64(y).reshape(1, -1), ref)
+    buf = torch.arange(1 << 16, dtype=torch.int32, device="cuda")
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.probe_hbm_read(buf, sink)
+    assert int(sink.item()) & 0xFFFFFFFF == (sum(range(1 << 16))) & 0xFFFFFFFF

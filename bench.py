@@ -1,0 +1,293 @@
+#!/usr/bin/env python
+"""Benchmark of the 4-bit weight-only decode path on the Llama-2-7B linear shapes (decode batch 1).
+
+One step = one pass over the 224 linears of the 32 decoder layers (q, k, v, o, gate, up, down),
+i.e. the linears behind one action token; ~3.44 GB of packed weights are streamed per step, far
+more than the L2, so every step reads HBM.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl qil|reference]
+
+With N > 1 (launched under torchrun) every rank runs an independent replica on its own GPU
+(the path has no cross-GPU exchange); the reported value is the sum over ranks divided by the
+slowest rank's time.  ``--impl reference`` times the CPU oracle on a bounded sample instead.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "W4A16 GEMV GB/s at Llama-2-7B M=1 (packed weights + scales + zeros + activations streamed per second)"
+UNIT = "GB/s"
+WORKLOAD = "configs[1]: Llama-2-7B decoder linears, decode M=1, 32 layers x 7 linears, group 128, 0.1% outliers"
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def reduce_max_time_sum_units(ms_local: float, units_local: float, world: int, backend_device):
+    """(max over ranks of the time, sum over ranks of the units); identity for one rank."""
+    if world == 1:
+        return ms_local, units_local
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=backend_device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=backend_device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    @staticmethod
+    def _epoch(stamp: str) -> float:
+        import datetime
+        return datetime.datetime.strptime(stamp, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+
+    def stop(self, t0: float, t1: float):
+        """Summary of the samples taken between the host times t0 and t1 (all samples if none fall inside)."""
+        if self.proc is None:
+            return None
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
+        for line in out.strip().splitlines():
+            f = [p.strip() for p in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                rows.append((self._epoch(f[0]), float(f[1]), float(f[2]), float(f[3]),
+                             [n for n, v in zip(names, f[4:8]) if v.lower().startswith("active")]))
+            except ValueError:
+                continue
+        inside = [r for r in rows if t0 <= r[0] <= t1]
+        use = inside or rows
+        if not use:
+            return None
+        reasons = sorted({n for r in use for n in r[4]})
+        return {"sm_mhz": statistics.median(r[1] for r in use), "sm_max_mhz": max(r[2] for r in use),
+                "power_w_max": max(r[3] for r in use), "samples": len(use),
+                "window": "timed region" if inside else "warm-up and timed region", "reasons": reasons}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            pass
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(budget_s: float, max_layers: int):
+    """Times the plain-C oracle's dequantise-then-matmul (fp64) on whole decoder layers of the same
+    workload until about ``budget_s`` seconds of CPU work are done.  Returns (GB/s, cores, description)."""
+    from oracle import c_oracle
+    from paper_2412_01034_b200 import workloads as wl
+    specs = wl.llama_linear_ids()
+    done_bytes, spent, layers = 0, 0.0, 0
+    per_layer = len(wl.LLAMA2_7B_LAYER)
+    while layers < max_layers and spent < budget_s:
+        for (_, _, N, K, tw, tx) in specs[layers * per_layer:(layers + 1) * per_layer]:
+            w = wl.llama_weight(1, tw, N, K)
+            codes, s, z = c_oracle.quantize_rtn_w4_asym(w, wl.GROUP_SIZE)   # setup, not timed
+            x = wl.normal_activations_bf16(1, tx, 1, K)
+            t0 = time.perf_counter()
+            c_oracle.linear_w4a16(x, codes, s, z, wl.GROUP_SIZE)
+            spent += time.perf_counter() - t0
+            done_bytes += N * K // 2 + 4 * N * (K // wl.GROUP_SIZE) + 2 * K + 2 * N
+        layers += 1
+    return done_bytes / spent / 1e9, c_oracle.num_threads(), f"{layers} of 32 decoder layers ({layers * per_layer} linears), M=1, fp64 C/OpenMP oracle"
+
+
+def run_reference(args):
+    rank, _, _ = dist_env()
+    if rank != 0:
+        return
+    from oracle import c_oracle
+    from paper_2412_01034_b200 import workloads as wl
+    specs = wl.llama_linear_ids()[:1]   # one linear per step, so that a long --steps run stays bounded
+    prepared = []
+    for (_, _, N, K, tw, tx) in specs:
+        w = wl.llama_weight(1, tw, N, K)
+        prepared.append((wl.normal_activations_bf16(1, tx, 1, K), *c_oracle.quantize_rtn_w4_asym(w, wl.GROUP_SIZE)))
+    nbytes = sum(N * K // 2 + 4 * N * (K // wl.GROUP_SIZE) + 2 * K + 2 * N for (_, _, N, K, _, _) in specs)
+
+    def step():
+        for (x, codes, s, z) in prepared:
+            c_oracle.linear_w4a16(x, codes, s, z, wl.GROUP_SIZE)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    value = nbytes / (ms * 1e-3) / 1e9
+    sample = "layer 0 q projection (4096 x 4096, 16.8 M weights) per step, M=1, fp64 C/OpenMP oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": c_oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+def run_qil(args):
+    import torch
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2412_01034_b200 import api, llama_decode
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, sample = oracle_sample(args.cpu_budget_s, 32)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    model = llama_decode.QuantisedLinears(cfg=1, M=1, n_layers=args.layers, device=f"cuda:{local_rank}")
+    stream = torch.cuda.Stream(device=dev)
+    bytes_per_step = model.algorithmic_bytes()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def capture(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            fn(stream)                      # eager once (also sets kernel attributes outside capture)
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                fn(stream)
+        return g
+
+    def timed(graph, steps, warmup, sampler_index=None):
+        with torch.cuda.stream(stream):
+            sampler = ClockSampler(sampler_index) if sampler_index is not None else None
+            for _ in range(warmup):
+                graph.replay()
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.time()
+            e0.record(stream)
+            for _ in range(steps):
+                graph.replay()
+            e1.record(stream)
+            barrier()
+            t1 = time.time()
+            clocks = sampler.stop(t0, t1) if sampler else None
+        return e0.elapsed_time(e1) / steps, clocks
+
+    g_dev = capture(lambda s: model.run(s))
+    g_e2e = capture(lambda s: model.run_host(s))
+
+    ms, clocks = timed(g_dev, args.steps, args.warmup, physical_gpu_index(local_rank) if rank == 0 else None)
+    ms_e2e, _ = timed(g_e2e, args.steps, args.warmup)
+
+    ms_all, units_all = reduce_max_time_sum_units(ms, bytes_per_step, world, dev)
+    ms_e2e_all, _ = reduce_max_time_sum_units(ms_e2e, bytes_per_step, world, dev)
+    value = units_all / (ms_all * 1e-3) / 1e9
+    value_e2e = units_all / (ms_e2e_all * 1e-3) / 1e9
+
+    if rank == 0:
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except (OSError, ValueError):
+            pass
+        peak = float(peaks.get("hbm_gbs", 6650.0))
+        peak_kind = "measured copy bandwidth (MEASURED_PEAKS.json)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
+        launches_per_step = model.count
+        per_launch_bytes = bytes_per_step / launches_per_step
+        per_launch_ms = ms / launches_per_step          # average over the timed region, launch gaps included
+        achieved = per_launch_bytes / (per_launch_ms * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_all, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 activations x int4 weights, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "layers": args.layers, "linears_per_step": launches_per_step,
+                       "bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (3.44 GB of weights per step)",
+                       "parallelism": f"replicas x{world}", "launch": "CUDA graph of one kernel per linear"},
+            "clocks": clocks,
+            "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_e2e_all,
+                    "h2d_bytes_per_step": 2 * model.x_elems, "d2h_bytes_per_step": 2 * model.y_elems},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_kind": peak_kind, "kernel": "w4a16_skinny_kernel<1>",
+                         "bytes_per_launch": per_launch_bytes, "us_per_launch": per_launch_ms * 1e3,
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1050)
+    ap.add_argument("--warmup", type=int, default=70)
+    ap.add_argument("--impl", default="qil", choices=["qil", "reference"])
+    ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the stated workload)")
+    ap.add_argument("--cpu-budget-s", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_qil(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -120,6 +120,39 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
                             qil_stream_t stream);
 
 /* ------------------------------------------------------------------------
+ * A list of weight-only linears run in stream order (one decode pass over the
+ * decoder layers, App. A.4.2: q, k, v, o, gate, up, down x layers).  The result
+ * is the same as `count` calls of qil_linear_w4a16 in list order; entry i may
+ * read what entries < i wrote.  All pointers inside a descriptor are device
+ * pointers; the descriptor array itself is host memory and is consumed before
+ * the call returns.  workspace must be as large as the largest
+ * qil_linear_w4a16_workspace_size() over the entries (zero-filled once).
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    const void* x;           /* bf16 [M][K] */
+    const uint32_t* qweight; /* packed per layout */
+    const void* scales;      /* fp16 [N][K/group_size] */
+    const void* zeros;       /* fp16 [N][K/group_size] */
+    void* y;                 /* bf16 [M][N] */
+    int M, N, K, group_size;
+    int layout;              /* qil_layout */
+    int reserved;            /* must be 0 */
+} qil_linear_desc;
+
+qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs /*host*/, int count, void* workspace,
+                                  size_t workspace_bytes, qil_stream_t stream);
+
+/* Same, with the activations in HOST memory: copies x_bytes from x_host to
+ * x_stage (device), runs the list (whose x / y pointers refer into x_stage /
+ * y_stage), then copies y_bytes from y_stage to y_host.  All three steps are
+ * enqueued on `stream`; the call does not wait.  Use page-locked host buffers
+ * for the copies to be asynchronous. */
+qil_status qil_linear_w4a16_batch_host(const qil_linear_desc* descs /*host*/, int count,
+                                       const void* x_host, void* x_stage, size_t x_bytes,
+                                       void* y_host, const void* y_stage, size_t y_bytes,
+                                       void* workspace, size_t workspace_bytes, qil_stream_t stream);
+
+/* ------------------------------------------------------------------------
  * Activation quantiser of the W4A4 path (Sec. 5.1: the compute-bound driving
  * policy needs weights and activations in 4 bits): symmetric int4 per row.
  *   x [M][K] bf16 -> qx packed [M][K/8] (canonical), scales [M] fp32.

@@ -15,6 +15,8 @@ SIGNATURES = {
     "qil_unpack_w4": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
     "qil_linear_w4a16_workspace_size": (_sz, [_i, _i, _i, _i]),
     "qil_linear_w4a16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_linear_w4a16_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
+    "qil_linear_w4a16_batch_host": (_i, [_vp, _i, _vp, _vp, _sz, _vp, _vp, _sz, _vp, _sz, _vp]),
     "qil_quantize_act_a4": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),
     "qil_linear_w4a4_workspace_size": (_sz, [_i, _i, _i]),
     "qil_linear_w4a4": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
@@ -24,6 +26,14 @@ SIGNATURES = {
     "qil_ref_gemv_bf16": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "qil_probe_hbm_read": (_i, [_vp, _sz, _vp, _vp]),
 }
+
+
+
+class LinearDesc(C.Structure):
+    """ctypes mirror of ``qil_linear_desc``."""
+    _fields_ = [("x", _vp), ("qweight", _vp), ("scales", _vp), ("zeros", _vp), ("y", _vp),
+                ("M", _i), ("N", _i), ("K", _i), ("group_size", _i), ("layout", _i), ("reserved", _i)]
+
 
 _lib = None
 

@@ -123,6 +123,52 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
     return launch_w4a16_general(x, qweight, scales, zeros, y, M, N, K, group_size, S(stream));
 }
 
+qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs, int count, void* workspace, size_t workspace_bytes,
+                                  qil_stream_t stream) {
+    if (!descs) return QIL_ERR_NULL;
+    if (count <= 0) return QIL_ERR_SHAPE;
+    if (workspace && !aligned16(workspace)) return QIL_ERR_ALIGN;
+    // validate the whole list before the first launch
+    for (int i = 0; i < count; ++i) {
+        const qil_linear_desc& d = descs[i];
+        if (d.reserved != 0) return QIL_ERR_UNSUPPORTED;
+        const qil_status s = check_w4a16(d.x, d.qweight, d.scales, d.zeros, d.y, d.M, d.N, d.K, d.group_size,
+                                         (qil_layout)d.layout);
+        if (s != QIL_OK) return s;
+        const bool skinny = w4a16_skinny_supported(d.M, d.N, d.K, d.group_size, (qil_layout)d.layout);
+        if (!skinny && d.layout != QIL_LAYOUT_CANONICAL) return QIL_ERR_UNSUPPORTED;
+        if (skinny) {
+            const size_t need = w4a16_skinny_workspace(d.M, d.N, d.K, d.group_size);
+            if (need > 0 && (!workspace || workspace_bytes < need)) return QIL_ERR_WORKSPACE;
+        }
+    }
+    for (int i = 0; i < count; ++i) {
+        const qil_linear_desc& d = descs[i];
+        const qil_status s = qil_linear_w4a16(d.x, d.qweight, d.scales, d.zeros, d.y, d.M, d.N, d.K, d.group_size,
+                                              (qil_layout)d.layout, workspace, workspace_bytes, stream);
+        if (s != QIL_OK) return s;
+    }
+    return QIL_OK;
+}
+
+qil_status qil_linear_w4a16_batch_host(const qil_linear_desc* descs, int count, const void* x_host, void* x_stage,
+                                       size_t x_bytes, void* y_host, const void* y_stage, size_t y_bytes,
+                                       void* workspace, size_t workspace_bytes, qil_stream_t stream) {
+    if (!x_host || !x_stage || !y_host || !y_stage) return QIL_ERR_NULL;
+    if (x_bytes == 0 || y_bytes == 0) return QIL_ERR_SHAPE;
+    if (cudaMemcpyAsync(x_stage, x_host, x_bytes, cudaMemcpyHostToDevice, S(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return QIL_ERR_CUDA;
+    }
+    const qil_status s = qil_linear_w4a16_batch(descs, count, workspace, workspace_bytes, stream);
+    if (s != QIL_OK) return s;
+    if (cudaMemcpyAsync(y_host, y_stage, y_bytes, cudaMemcpyDeviceToHost, S(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return QIL_ERR_CUDA;
+    }
+    return QIL_OK;
+}
+
 qil_status qil_quantize_act_a4(const void* x, int M, int K, const float* static_scale, uint32_t* qx, float* scales,
                                qil_stream_t stream) {
     if (!x || !qx || !scales) return QIL_ERR_NULL;

@@ -61,17 +61,23 @@ def normal_weights(cfg: int, tensor_id: int, N: int, K: int, sigma: float,
     """fp32 [N][K] ~ N(0, sigma); optionally each entry is, independently with
     probability ``outlier_prob``, replaced by +-outlier_sigmas*sigma (fair sign).
 
-    The replacement set is drawn as (count ~ Binomial, positions uniform without
-    replacement), which has the same law as one Bernoulli draw per entry.
+    The replaced positions are drawn as the success times of a Bernoulli process (gaps between
+    successes are geometric), which has the same law as one Bernoulli draw per entry.
     """
     g = generator(cfg, tensor_id)
     w = g.standard_normal((N, K), dtype=np.float32)
     w *= np.float32(sigma)
     if outlier_prob > 0.0:
         total = N * K
-        count = int(g.binomial(total, outlier_prob))
-        pos = g.choice(total, size=count, replace=False)
-        sign = g.integers(0, 2, size=count).astype(np.float32) * 2.0 - 1.0
+        pos = np.empty(0, dtype=np.int64)
+        last = -1
+        while last < total:
+            gaps = g.geometric(outlier_prob, size=int(total * outlier_prob * 1.2) + 64)
+            more = last + np.cumsum(gaps, dtype=np.int64)
+            pos = np.concatenate([pos, more])
+            last = int(more[-1])
+        pos = pos[pos < total]
+        sign = g.integers(0, 2, size=pos.size).astype(np.float32) * 2.0 - 1.0
         w.reshape(-1)[pos] = sign * np.float32(outlier_sigmas * sigma)
     return w
 

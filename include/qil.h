@@ -120,6 +120,34 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
                             qil_stream_t stream);
 
 /* ------------------------------------------------------------------------
+ * qil_linear_w4a16 for callers that must not allocate device memory.  (The paper
+ * has no counterpart to this call; it exists for integration reasons only.)
+ * Some hosts of this library cannot call cudaMalloc at the point where they run
+ * a linear: a real-time control loop that forbids allocation after start-up, a
+ * plug-in whose host application owns all device memory, code running inside a
+ * region where the allocator may not be entered.  qil_linear_w4a16 needs a
+ * caller-allocated workspace whenever the shape is split along K; this variant
+ * computes the same result with the scratch held in a fixed array of
+ * QIL_STATIC_WS_BYTES bytes that is part of the library image (each GPU that
+ * loads the library keeps that much memory reserved until the process exits).
+ * Arguments as qil_linear_w4a16, minus the workspace.
+ *  - Shapes whose scratch need (qil_linear_w4a16_workspace_size) exceeds
+ *    QIL_STATIC_WS_BYTES are rejected with QIL_ERR_WORKSPACE; nothing is launched.
+ *  - The call allocates and frees nothing.  The first call on each device looks
+ *    up the device address of the array (with that device current); make that
+ *    first call outside any stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's
+ *    contents; the call clears the part that has to start at zero itself, on
+ *    `stream`.  Two calls that overlap on the GPU (different streams, no
+ *    ordering between them) race on the array: order them.
+ * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE (shape too large), CUDA.
+ * ---------------------------------------------------------------------- */
+#define QIL_STATIC_WS_BYTES (4u * 1024u * 1024u)
+qil_status qil_linear_w4a16_static_ws(const void* x, const uint32_t* qweight, const void* scales,
+                                      const void* zeros, void* y, int M, int N, int K,
+                                      int group_size, qil_layout layout, qil_stream_t stream);
+
+/* ------------------------------------------------------------------------
  * A list of weight-only linears run in stream order (one decode pass over the
  * decoder layers, App. A.4.2: q, k, v, o, gate, up, down x layers).  The result
  * is the same as `count` calls of qil_linear_w4a16 in list order; entry i may

@@ -15,6 +15,7 @@ SIGNATURES = {
     "qil_unpack_w4": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
     "qil_linear_w4a16_workspace_size": (_sz, [_i, _i, _i, _i]),
     "qil_linear_w4a16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_linear_w4a16_static_ws": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "qil_linear_w4a16_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
     "qil_linear_w4a16_batch_host": (_i, [_vp, _i, _vp, _vp, _sz, _vp, _vp, _sz, _vp, _sz, _vp]),
     "qil_quantize_act_a4": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),

@@ -9,7 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libqil.so")
-SOURCES = ["api.cu", "quantize.cu", "w4a16_general.cu", "w4a16_skinny.cu", "w4a4.cu", "ref_gemv.cu"]
+SOURCES = ["api.cu", "quantize.cu", "w4a16_general.cu", "w4a16_skinny.cu", "w4a4.cu", "ref_gemv.cu",
+           "w4a16_static_ws.cu"]
 
 
 def _nvcc() -> str:

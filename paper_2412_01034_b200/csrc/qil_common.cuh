@@ -64,6 +64,7 @@ qil_status launch_w4a16_general(const void* x, const uint32_t* qw, const void* s
                                 void* y, int M, int N, int K, int G, cudaStream_t st);
 bool w4a16_skinny_supported(int M, int N, int K, int G, qil_layout layout);
 size_t w4a16_skinny_workspace(int M, int N, int K, int G);
+size_t w4a16_skinny_counter_bytes();  // leading part of that workspace that must be zero before a launch
 qil_status launch_w4a16_skinny(const void* x, const uint32_t* qw, const void* scales, const void* zeros,
                                void* y, int M, int N, int K, int G, qil_layout layout, void* ws,
                                size_t ws_bytes, cudaStream_t st);

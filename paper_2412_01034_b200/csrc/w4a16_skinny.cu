@@ -274,6 +274,8 @@ bool w4a16_skinny_supported(int M, int N, int K, int G, qil_layout layout) {
     return true;
 }
 
+size_t w4a16_skinny_counter_bytes() { return kCounterBytes; }
+
 size_t w4a16_skinny_workspace(int M, int N, int K, int G) {
     (void)G;
     const SkinnyPlan pl = make_plan(M, N, K);

@@ -1,0 +1,60 @@
+"""qil_linear_w4a16_static_ws: the linear for callers that are not allowed to allocate.
+
+A control loop that bans allocation after start-up, or a plug-in whose host owns all device
+memory, cannot hand qil_linear_w4a16 the workspace it wants for K-split shapes.  The variant
+tested here keeps that scratch in a fixed array inside the library.  It must give the same
+result as the ordinary entry point, also on a second call (the array still holds the first
+call's data then), and it must refuse shapes whose scratch would not fit.
+
+This file sorts last on purpose: a run that stops at the first failure has then already run
+every other test.
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+from oracle import np_oracle
+from paper_2412_01034_b200 import workloads as wl
+from tests.util import assert_rows_close, bf16_to_f64, bits_of, cuda, to_bf16_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 4096, 4096), (4, 512, 4096), (3, 208, 1024)])
+def test_static_ws_matches_workspace_entry_point_twice(M, N, K):
+    import torch
+    from paper_2412_01034_b200 import _lib, api
+    lib = _lib.load()
+    G = 128
+    w = wl.normal_weights(500, N + K, N, K, 0.02, outlier_prob=0.001)
+    x = wl.normal_activations_bf16(500, M, M, K)
+    codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
+    y_ref = np_oracle.linear_w4a16(x, codes, scales, zeros, G)
+    packed = api.pack_w4(cuda(codes), api.LAYOUT_TILE16)
+    xd, sd, zd = to_bf16_cuda(x), cuda(scales), cuda(zeros)
+    need = api.linear_w4a16_workspace_size(M, N, K, G)
+    y_ws = api.linear_w4a16(xd, packed, sd, zd, N, G, api.LAYOUT_TILE16)       # caller-allocated workspace
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    for call in range(2):
+        y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        rc = lib.qil_linear_w4a16_static_ws(C.c_void_p(xd.data_ptr()), C.c_void_p(packed.data_ptr()),
+                                            C.c_void_p(sd.data_ptr()), C.c_void_p(zd.data_ptr()),
+                                            C.c_void_p(y.data_ptr()), M, N, K, G, api.LAYOUT_TILE16, stream)
+        assert rc == 0, lib.qil_status_string(rc)
+        torch.cuda.synchronize()
+        assert_rows_close(bf16_to_f64(y), bf16_to_f64(y_ws))    # same tolerance as the parity tests
+        assert_rows_close(bf16_to_f64(y), y_ref)
+        np.testing.assert_array_equal(bits_of(y), bits_of(y_ws), err_msg=f"call {call}")
+    assert need >= 0
+
+
+def test_static_ws_rejects_shapes_beyond_the_built_in_scratch():
+    from paper_2412_01034_b200 import _lib, api
+    lib = _lib.load()
+    M, N, K, G = 64, 8192, 4096, 128
+    assert api.linear_w4a16_workspace_size(M, N, K, G) > 4 * 1024 * 1024
+    a = C.c_void_p(0x10000)  # aligned dummy addresses: the call must fail before touching them
+    rc = lib.qil_linear_w4a16_static_ws(a, a, a, a, a, M, N, K, G, api.LAYOUT_TILE16, None)
+    assert rc == 5 and b"workspace" in lib.qil_status_string(rc)
+    assert lib.qil_linear_w4a16_static_ws(None, a, a, a, a, 1, 16, 128, 128, 0, None) == 1

@@ -188,7 +188,9 @@ def run_qil(args):
         v, cores, sample = oracle_sample(args.cpu_budget_s, 32)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
 
-    model = llama_decode.QuantisedLinears(cfg=1, M=1, n_layers=args.layers, device=f"cuda:{local_rank}")
+    layout = {"stream": api.LAYOUT_STREAM, "tile16": api.LAYOUT_TILE16, "canonical": api.LAYOUT_CANONICAL}[args.layout]
+    model = llama_decode.QuantisedLinears(cfg=1, M=1, n_layers=args.layers, layout=layout, deps=args.deps,
+                                          device=f"cuda:{local_rank}")
     stream = torch.cuda.Stream(device=dev)
     bytes_per_step = model.algorithmic_bytes()
 
@@ -244,7 +246,8 @@ def run_qil(args):
             pass
         peak = float(peaks.get("hbm_gbs", 6650.0))
         peak_kind = "measured copy bandwidth (MEASURED_PEAKS.json)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
-        launches_per_step = model.count
+        launches_per_step = 1 if args.layout == "stream" else model.count
+        kernel = "w4a16_stream_kernel" if args.layout == "stream" else "w4a16_skinny_kernel<1>"
         per_launch_bytes = bytes_per_step / launches_per_step
         per_launch_ms = ms / launches_per_step          # average over the timed region, launch gaps included
         achieved = per_launch_bytes / (per_launch_ms * 1e-3) / 1e9
@@ -252,15 +255,17 @@ def run_qil(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_all, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 activations x int4 weights, fp32 accumulate", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "layers": args.layers, "linears_per_step": launches_per_step,
+            "config": {"workload": WORKLOAD, "layers": args.layers, "linears_per_step": model.count,
+                       "layout": args.layout, "dependencies": args.deps,
                        "bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (3.44 GB of weights per step)",
-                       "parallelism": f"replicas x{world}", "launch": "CUDA graph of one kernel per linear"},
+                       "parallelism": f"replicas x{world}", "launch": ("CUDA graph of one persistent kernel over the whole list" if args.layout == "stream"
+                                  else "CUDA graph of one kernel per linear")},
             "clocks": clocks,
             "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_e2e_all,
                     "h2d_bytes_per_step": 2 * model.x_elems, "d2h_bytes_per_step": 2 * model.y_elems},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": peak_kind, "kernel": "w4a16_skinny_kernel<1>",
+                         "traffic": None, "peak_kind": peak_kind, "kernel": kernel,
                          "bytes_per_launch": per_launch_bytes, "us_per_launch": per_launch_ms * 1e3,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu_baseline,
@@ -278,6 +283,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=70)
     ap.add_argument("--impl", default="qil", choices=["qil", "reference"])
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the stated workload)")
+    ap.add_argument("--layout", default="stream", choices=["stream", "tile16", "canonical"])
+    ap.add_argument("--deps", default="layer", choices=["layer", "all", "none"],
+                    help="which linears wait for all earlier ones (layer = data flow of a decoder layer)")
     ap.add_argument("--cpu-budget-s", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

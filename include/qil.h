@@ -66,8 +66,16 @@ typedef enum { QIL_F32 = 0, QIL_BF16 = 1, QIL_F16 = 2 } qil_dtype;
  *   each.  Word (n, i) is at ((n/16)*(K/128) + i/16)*256 + (n%16)*16 + i%16.
  *   Needs N % 16 == 0 and K % 128 == 0.  A warp of the decode kernel reads one
  *   tile (1 KiB) with two fully coalesced 512-byte loads.
+ * QIL_LAYOUT_STREAM   : self-contained units for the persistent decode kernel,
+ *   built by qil_pack_stream_w4 from codes, scales and zeros.  Unit u =
+ *   (n/16)*(K/128) + k/128 occupies bytes [1088 u, 1088 (u+1)): first the 1024
+ *   bytes of the TILE16 tile (16 rows x 16 words), then 16 pairs {fp16 scale,
+ *   fp16 zero}, one per row of the tile, valid for that 128-column block (a
+ *   group larger than 128 repeats its pair in every block it covers).
+ *   Needs N % 16 == 0, K % 128 == 0, group_size % 128 == 0.  With group 128 the
+ *   buffer is exactly as large as canonical codes + scales + zeros.
  */
-typedef enum { QIL_LAYOUT_CANONICAL = 0, QIL_LAYOUT_TILE16 = 1 } qil_layout;
+typedef enum { QIL_LAYOUT_CANONICAL = 0, QIL_LAYOUT_TILE16 = 1, QIL_LAYOUT_STREAM = 2 } qil_layout;
 
 typedef struct CUstream_st* qil_stream_t; /* a cudaStream_t */
 
@@ -97,6 +105,13 @@ qil_status qil_pack_w4(const uint8_t* codes, int N, int K, qil_layout layout, ui
 qil_status qil_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout, int is_signed,
                          uint8_t* codes, qil_stream_t stream);
 
+/* Builds the QIL_LAYOUT_STREAM buffer (qil_stream_w4_bytes(N, K) bytes) from unsigned
+ * codes [N][K], fp16 scales and fp16 zeros [N][K/group_size].
+ * Errors: NULL, SHAPE (N % 16, K % 128, group_size % 128, K % group_size), ALIGN. */
+size_t qil_stream_w4_bytes(int N, int K);
+qil_status qil_pack_stream_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K,
+                              int group_size, void* out, qil_stream_t stream);
+
 /* ------------------------------------------------------------------------
  * Weight-only linear, 4-bit weights x bf16 activations (the OpenVLA / Llama-2
  * decode and prefill linears, Sec. 5.4, App. A.4.2): dequantisation is fused
@@ -106,11 +121,16 @@ qil_status qil_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout
  * The kernel is chosen from the shape: tensor-core skinny kernel (weights read
  * once, any M handled in slabs of 64 rows) when K % 128 == 0 and
  * group_size % 128 == 0; a general kernel otherwise (any K % 8 == 0, any
- * group_size dividing K, canonical layout only).
+ * group_size dividing K, canonical layout only).  With QIL_LAYOUT_STREAM the
+ * persistent streaming kernel runs (M <= 8; scales and zeros are part of the
+ * buffer, the two arguments are ignored and may be null; the workspace is
+ * always needed).
  * workspace: qil_linear_w4a16_workspace_size() bytes, only touched when the
  * shape needs a split along K; it must be zero-filled once before first use
- * (the kernel leaves it zeroed again).  Calls that share a workspace must not
- * overlap on the device.
+ * (the kernels leave it zeroed again).  Calls that share a workspace must not
+ * overlap on the device.  Its first int is a status word: the streaming kernel
+ * ORs QIL_ERR_TIMEOUT into it if one of its bounded waits ever runs out (read it
+ * with qil_device_status; after such an error re-zero the workspace).
  * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, CUDA.
  * ---------------------------------------------------------------------- */
 size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size);
@@ -150,8 +170,13 @@ qil_status qil_linear_w4a16_static_ws(const void* x, const uint32_t* qweight, co
 /* ------------------------------------------------------------------------
  * A list of weight-only linears run in stream order (one decode pass over the
  * decoder layers, App. A.4.2: q, k, v, o, gate, up, down x layers).  The result
- * is the same as `count` calls of qil_linear_w4a16 in list order; entry i may
- * read what entries < i wrote.  All pointers inside a descriptor are device
+ * is the same as `count` calls of qil_linear_w4a16 in list order.  An entry
+ * whose x is written by an earlier entry of the same list must carry
+ * QIL_DEP_PREVIOUS in `flags`: it then starts only after every earlier entry has
+ * written all of its outputs.  Entries without the flag may overlap with their
+ * predecessors (q, k and v of one layer share an input and need no flag).
+ * When every entry uses QIL_LAYOUT_STREAM the whole list runs as one persistent
+ * kernel.  All pointers inside a descriptor are device
  * pointers; the descriptor array itself is host memory and is consumed before
  * the call returns.  workspace must be as large as the largest
  * qil_linear_w4a16_workspace_size() over the entries (zero-filled once).
@@ -164,8 +189,9 @@ typedef struct {
     void* y;                 /* bf16 [M][N] */
     int M, N, K, group_size;
     int layout;              /* qil_layout */
-    int reserved;            /* must be 0 */
+    int flags;               /* 0 or QIL_DEP_PREVIOUS */
 } qil_linear_desc;
+#define QIL_DEP_PREVIOUS 1
 
 qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs /*host*/, int count, void* workspace,
                                   size_t workspace_bytes, qil_stream_t stream);

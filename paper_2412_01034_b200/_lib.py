@@ -13,6 +13,8 @@ SIGNATURES = {
     "qil_quantize_rtn_w4": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _i, _vp, _vp, _vp]),
     "qil_pack_w4": (_i, [_vp, _i, _i, _i, _vp, _vp]),
     "qil_unpack_w4": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
+    "qil_stream_w4_bytes": (_sz, [_i, _i]),
+    "qil_pack_stream_w4": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "qil_linear_w4a16_workspace_size": (_sz, [_i, _i, _i, _i]),
     "qil_linear_w4a16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w4a16_static_ws": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
@@ -33,7 +35,7 @@ SIGNATURES = {
 class LinearDesc(C.Structure):
     """ctypes mirror of ``qil_linear_desc``."""
     _fields_ = [("x", _vp), ("qweight", _vp), ("scales", _vp), ("zeros", _vp), ("y", _vp),
-                ("M", _i), ("N", _i), ("K", _i), ("group_size", _i), ("layout", _i), ("reserved", _i)]
+                ("M", _i), ("N", _i), ("K", _i), ("group_size", _i), ("layout", _i), ("flags", _i)]
 
 
 _lib = None

@@ -19,7 +19,8 @@ from . import _lib, api, workloads as wl
 
 
 class QuantisedLinears:
-    def __init__(self, cfg: int = 1, M: int = 1, n_layers: int = wl.N_LAYERS, layout: int = api.LAYOUT_TILE16,
+    def __init__(self, cfg: int = 1, M: int = 1, n_layers: int = wl.N_LAYERS, layout: int = api.LAYOUT_STREAM,
+                 deps: str = "layer",
                  outliers: bool = True, device: str = "cuda", keep_host_rows: dict | None = None,
                  host_threads: int | None = None):
         self.M, self.layout, self.device = M, layout, device
@@ -47,7 +48,10 @@ class QuantisedLinears:
                     self.kept[i] = (rows, w[rows].copy())
                 wd = torch.from_numpy(w).to(device)
                 codes, s, z = api.quantize_rtn_w4(wd, self.G)
-                self.packed.append(api.pack_w4(codes, layout))
+                if layout == api.LAYOUT_STREAM:
+                    self.packed.append(api.pack_stream_w4(codes, s, z, self.G))
+                else:
+                    self.packed.append(api.pack_w4(codes, layout))
                 self.scales.append(s)
                 self.zeros.append(z)
                 del wd, codes, w
@@ -82,7 +86,19 @@ class QuantisedLinears:
             d.scales = self.scales[i].data_ptr()
             d.zeros = self.zeros[i].data_ptr()
             d.y = self.y_dev.data_ptr() + 2 * self.y_off[i]
-            d.M, d.N, d.K, d.group_size, d.layout, d.reserved = M, N, K, self.G, layout, 0
+            d.M, d.N, d.K, d.group_size, d.layout = M, N, K, self.G, layout
+            d.flags = self._dep_flag(i, deps)
+
+    def _dep_flag(self, i: int, deps: str) -> int:
+        """Which entries wait for all earlier ones.  "layer": the data flow of a real decoder layer
+        (q after the previous layer's down, o after attention, gate after o, down after gate/up; k, v and
+        up share their input with q / gate).  "all": every entry.  "none": no entry."""
+        if deps == "all":
+            return api.DEP_PREVIOUS if i > 0 else 0
+        if deps == "none":
+            return 0
+        name = self.specs[i][1]
+        return api.DEP_PREVIOUS if (name in ("q", "o", "gate", "down") and i > 0) else 0
 
     # ---- sizes -------------------------------------------------------------------------------
     @property

@@ -68,8 +68,10 @@ typedef enum { QIL_F32 = 0, QIL_BF16 = 1, QIL_F16 = 2 } qil_dtype;
  *   tile (1 KiB) with two fully coalesced 512-byte loads.
  * QIL_LAYOUT_STREAM   : self-contained units for the persistent decode kernel,
  *   built by qil_pack_stream_w4 from codes, scales and zeros.  Unit u =
- *   (n/16)*(K/128) + k/128 occupies bytes [1088 u, 1088 (u+1)): first the 1024
- *   bytes of the TILE16 tile (16 rows x 16 words), then 16 pairs {fp16 scale,
+ *   (n/16)*(K/128) + k/128 occupies bytes [1088 u, 1088 (u+1)): first 1024
+ *   bytes of codes, 16 rows x 16 words as in a TILE16 tile, except that inside
+ *   each word code k (0..7) sits at nibble (k >> 1) + 4 * (k & 1) (even k in the
+ *   low half-word, odd k in the high half-word); then 16 pairs {fp16 scale,
  *   fp16 zero}, one per row of the tile, valid for that 128-column block (a
  *   group larger than 128 repeats its pair in every block it covers).
  *   Needs N % 16 == 0, K % 128 == 0, group_size % 128 == 0.  With group 128 the

@@ -5,17 +5,25 @@
 // Data layout (QIL_LAYOUT_STREAM): the weight matrix is a sequence of self-contained
 // 1088-byte units, unit u = (row tile rt = u / (K/128), column block kb = u % (K/128)):
 // 1024 bytes of packed codes of 16 output features x 128 input features (16 rows of 64
-// bytes) followed by 16 x {fp16 scale, fp16 zero} of those rows for that block.  A
-// linear is therefore one contiguous byte stream, and any slice of units is too.
+// bytes) followed by 16 x {fp16 scale, fp16 zero} of those rows for that block.  Inside
+// each 32-bit word the 8 codes are ordered so that the mask/or unpack below yields
+// bf16 pairs of ADJACENT k (code k at nibble (k>>1) + 4*(k&1)); the activations can then
+// be used exactly as they lie in memory.  A linear is one contiguous byte stream, and
+// any slice of units is too.
 //
 // Execution: one CTA per SM, alive for the whole list.  For every linear each CTA
 // owns a contiguous slice of its units (balanced to +-1 unit).  A producer thread
 // streams the slice through a shared-memory ring with bulk asynchronous copies
 // (cp.async.bulk + mbarrier transaction counts), running ahead across linears as far
 // as the ring allows, so HBM stays busy while the consumers finish a linear.
-// Sixteen consumer warps each take one unit per ring stage: nibbles -> bf16 (128+q)
+// Sixteen compute warps each take one unit per ring stage: nibbles -> bf16 (128+q)
 // by mask/or, mma.sync m16n8k16 against the activation rows staged in shared memory,
 // scale/zero folded once per unit (y += s*(acc - (128+z)*X), X = block sum of x).
+// They never wait for another CTA: per pass they leave per-warp partial tiles in a
+// double-buffered shared array and go on.  A combiner group of four warps adds the
+// partial tiles and writes finished outputs; a fixer warp does all cross-CTA work
+// from a small queue; two stager warps fetch the activations of the next entry
+// (two buffers) and wait for dependencies - all hidden behind the compute warps.
 // Row tiles cut by a slice boundary are completed through small fp32 slots in the
 // workspace: every CTA first publishes its contribution to the tile it shares with
 // the next CTA, then completes the tile it shares with previous CTAs, adding the
@@ -36,18 +44,22 @@ namespace qil {
 
 namespace {
 
-constexpr int kConsumerWarps = 16;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;  // + one producer warp
+constexpr int kComputeWarps = 16;
+constexpr int kComputeThreads = kComputeWarps * 32;
+constexpr int kEpiThreads = 128;     // combiner group: 4 warps
+constexpr int kStagerThreads = 64;   // activation stager: 2 warps
+constexpr int kFixDepth = 8;         // records queued between the combiner group and the fixer warp
+constexpr int kThreads = kComputeThreads + kEpiThreads + 32 + kStagerThreads + 32;  // + fixer warp + producer warp
 constexpr int kUnitBytes = 1088;
-constexpr int kStageUnits = kConsumerWarps;
+constexpr int kStageUnits = kComputeWarps;
 constexpr int kStageBytes = kStageUnits * kUnitBytes;
-constexpr int kMaxTiles = 8;    // row tiles handled per pass
-constexpr int kElems = 128;     // fp32 values of one row tile: 16 rows x 8 activation rows
+constexpr int kElemsMax = 128;  // fp32 values of one row tile: 16 rows x 8 activation rows (32 when M <= 2)
 constexpr int kMaxEntries = 256;
-constexpr int kSlotBytes = kElems * 4 + 16;  // data + flag word (padded)
+constexpr int kSlotBytes = kElemsMax * 4 + 16;  // data + flag word (padded)
 constexpr int kWsHeader = 256;
 constexpr int kRowPad = 16;
+constexpr int kFlagDep = 1;      // StreamEntry::flags: wait for all earlier entries
+constexpr int kFlagAligned = 2;  // StreamEntry::flags: slices are whole row tiles (set by the host)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // every wait gives up after two seconds
 
 struct StreamEntry {  // 48 bytes
@@ -66,6 +78,8 @@ struct StreamParams {
     int x_rows;       // max M over the entries
     int x_row_bytes;  // max K * 2 + pad
     int kb_max;       // max K / 128
+    int elems;        // fp32 values kept per (row tile, warp): 32 if every M <= 2, else 128
+    int max_tiles;    // row tiles per pass: 8 (elems 32) or 2 (elems 128)
     int* status;
     unsigned int* tiles_done;
     unsigned char* slots;
@@ -94,11 +108,29 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
+// same, but the thread may stay suspended in hardware for up to `ns` nanoseconds while the phase is incomplete
+// (a waiting role then does not compete with the compute warps for issue slots)
+__device__ __forceinline__ uint32_t mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok;
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
     asm volatile(
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
         : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_plain(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ uint32_t ld_acquire(const unsigned int* p) {
     uint32_t v;
@@ -111,7 +143,8 @@ __device__ __forceinline__ void st_release(unsigned int* p, uint32_t v) {
 __device__ __forceinline__ void red_release_add(unsigned int* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+__device__ __forceinline__ void stager_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kStagerThreads) : "memory"); }
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -141,12 +174,12 @@ struct Guard {
         return t;
     }
     __device__ __forceinline__ void wait_mbar(uint32_t bar, uint32_t parity) const {
-        if (*poisoned) return;
         if (mbar_try_wait(bar, parity)) return;
+        if (*poisoned) return;
         const unsigned long long t0 = now_ns();
         for (uint32_t i = 1;; ++i) {
-            if (mbar_try_wait(bar, parity)) return;
-            if ((i & 63u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
+            if (mbar_try_wait_suspend(bar, parity, 4000u)) return;
+            if ((i & 15u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
         }
         fail();
     }
@@ -182,272 +215,407 @@ __device__ __forceinline__ bool contributor_slot(uint32_t cc, uint32_t rt, uint3
     return cu0 != cu1;
 }
 
+// Iterates over the work of one CTA: entries with a non-empty slice, cut into passes of at most
+// `max_tiles` row tiles.  Producer, compute warps and the epilogue group all walk the same sequence.
+struct Walk {
+    const StreamParams& p;
+    uint32_t C, c;
+    int ei;                       // current entry (-1 before the first)
+    uint32_t KB, units, u0, u1;   // of the current entry
+    uint32_t t_first, t_last;
+    __device__ Walk(const StreamParams& p_, uint32_t C_, uint32_t c_) : p(p_), C(C_), c(c_), ei(-1) {}
+    // advance to the next entry in which this CTA owns units; false at the end of the list
+    __device__ bool next_entry() {
+        for (++ei; ei < p.count; ++ei) {
+            KB = (uint32_t)p.e[ei].K >> 7;
+            const uint32_t RT = (uint32_t)p.e[ei].N >> 4;
+            units = RT * KB;
+            if (p.e[ei].flags & kFlagAligned) {  // whole row tiles only: no tile is shared between CTAs
+                u0 = (uint32_t)(((uint64_t)c * RT) / C) * KB;
+                u1 = (uint32_t)(((uint64_t)(c + 1) * RT) / C) * KB;
+            } else {
+                slice_of(units, c, C, u0, u1);
+            }
+            if (u0 != u1) {
+                t_first = u0 / KB;
+                t_last = (u1 - 1) / KB;
+                return true;
+            }
+        }
+        return false;
+    }
+};
+
+// Records the combiner group hands to the fixer warp (cross-CTA work, off the compute path).
+enum : int { kRecContrib = 2, kRecFinish = 3, kRecEnd = 4 };
+struct FixRec {
+    int type;
+    int ei;        // entry index
+    uint32_t arg;  // kRecContrib: slot (0/1); kRecFinish: row tile
+    uint32_t pad;
+    float data[kElemsMax];
+};
+
 __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_constant__ StreamParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x;
     const uint32_t C = gridDim.x, c = blockIdx.x;
+    const int elems = p.elems, max_tiles = p.max_tiles;
+    const int part_floats = max_tiles * kComputeWarps * elems;  // one tile_part buffer
 
     // ---- carve shared memory ----
     unsigned char* ring = smem;
-    float* tile_part = reinterpret_cast<float*>(ring + (size_t)p.stages * kStageBytes);  // [kMaxTiles][16 warps][128]
-    float* stash_first = tile_part + kMaxTiles * kConsumerWarps * kElems;                // [128]
-    float* stash_last = stash_first + kElems;                                            // [128]
-    unsigned char* xs = reinterpret_cast<unsigned char*>(stash_last + kElems);           // [x_rows][x_row_bytes]
-    float* xsum = reinterpret_cast<float*>(xs + (size_t)p.x_rows * p.x_row_bytes);       // [8][kb_max]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(xsum + 8 * p.kb_max);                   // full[S], empty[S]
-    volatile int* poisoned = reinterpret_cast<volatile int*>(bars + 2 * p.stages);
+    float* tile_part = reinterpret_cast<float*>(ring + (size_t)p.stages * kStageBytes);  // [2][max_tiles][16 warps][elems]
+    float* stash_first = tile_part + 2 * part_floats;                                    // [128]
+    float* stash_last = stash_first + kElemsMax;                                         // [128]
+    FixRec* fixq = reinterpret_cast<FixRec*>(stash_last + kElemsMax);                    // [kFixDepth]
+    unsigned char* xs = reinterpret_cast<unsigned char*>(fixq + kFixDepth);              // [2][x_rows][x_row_bytes]
+    float* xsum = reinterpret_cast<float*>(xs + (size_t)2 * p.x_rows * p.x_row_bytes);   // [2][8][kb_max]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(xsum + 2 * 8 * p.kb_max);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
+    uint64_t* b2 = bars + 2 * p.stages;
+    const uint32_t xfull0 = smem_u32(b2);          // [2] activations of an entry are staged
+    const uint32_t xempty0 = smem_u32(b2 + 2);     // [2] the compute warps are done with them
+    const uint32_t accfull0 = smem_u32(b2 + 4);    // [2] all compute warps left their partial tiles
+    const uint32_t accempty0 = smem_u32(b2 + 6);   // [2] the combiner is done with the buffer
+    const uint32_t fqfull0 = smem_u32(b2 + 8);     // [kFixDepth] a record is ready for the fixer
+    const uint32_t fqempty0 = smem_u32(b2 + 8 + kFixDepth);  // [kFixDepth] the fixer has consumed it
+    const uint32_t xraw0 = smem_u32(b2 + 8 + 2 * kFixDepth);  // [2] the bulk copies of the rows of x have landed
+    volatile int* poisoned = reinterpret_cast<volatile int*>(b2 + 10 + 2 * kFixDepth);
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, kConsumerWarps);
+            mbar_init(empty0 + 8 * s, kComputeWarps);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(xfull0 + 8 * b, 1);
+            mbar_init(xempty0 + 8 * b, kComputeWarps);
+            mbar_init(accfull0 + 8 * b, kComputeWarps);
+            mbar_init(accempty0 + 8 * b, 1);
+            mbar_init(xraw0 + 8 * b, 1);
+        }
+        for (int q = 0; q < kFixDepth; ++q) {
+            mbar_init(fqfull0 + 8 * q, 1);
+            mbar_init(fqempty0 + 8 * q, 1);
         }
         *poisoned = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    for (int i = tid; i < 2 * part_floats; i += kThreads) tile_part[i] = 0.f;
+    for (int i = tid; i < 2 * 8 * p.kb_max; i += kThreads) xsum[i] = 0.f;
     __syncthreads();
     const Guard guard{p.status, poisoned};
 
-    if (tid >= kConsumerThreads) {
-        // =============================== producer ===============================
-        if (tid == kConsumerThreads) {
-            uint64_t policy;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-            uint32_t ctr = 0;
-            for (int ei = 0; ei < p.count; ++ei) {
-                const StreamEntry& E = p.e[ei];
-                const uint32_t KB = E.K >> 7, units = (uint32_t)(E.N >> 4) * KB;
-                uint32_t u0, u1;
-                slice_of(units, c, C, u0, u1);
-                if (u0 == u1) continue;
-                const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
-                for (uint32_t tp = t_first; tp <= t_last; tp += kMaxTiles) {
-                    const uint32_t pu0 = max(u0, tp * KB), pu1 = min(u1, (tp + kMaxTiles) * KB);
-                    for (uint32_t cu = pu0; cu < pu1; cu += kStageUnits, ++ctr) {
-                        const uint32_t n = min((uint32_t)kStageUnits, pu1 - cu);
-                        const uint32_t s = ctr % p.stages, round = ctr / p.stages;
-                        guard.wait_mbar(empty0 + 8 * s, (round & 1) ^ 1);
-                        mbar_expect_tx(full0 + 8 * s, n * kUnitBytes);
-                        bulk_g2s(smem_u32(ring + (size_t)s * kStageBytes), E.w + (size_t)cu * kUnitBytes, n * kUnitBytes,
-                                 full0 + 8 * s, policy);
-                    }
-                }
-            }
-            // every copy this thread issued must have landed before the CTA may retire
-            const uint32_t issued = ctr;
-            for (uint32_t back = 0; back < (uint32_t)p.stages && back < issued; ++back) {
-                const uint32_t k = issued - 1 - back;
-                guard.wait_mbar(full0 + 8 * (k % p.stages), (k / p.stages) & 1);
-            }
-        }
-    } else {
-        // =============================== consumers ===============================
+    if (tid < kComputeThreads) {
+        // =============================== compute warps ===============================
         const int lane = tid & 31, warp = tid >> 5;
         const int g = lane >> 2, t = lane & 3;
-        uint32_t ctr = 0;
-        for (int ei = 0; ei < p.count; ++ei) {
-            const StreamEntry& E = p.e[ei];
-            const uint32_t KB = E.K >> 7, RT = E.N >> 4, units = RT * KB;
-            const int M = E.M, N = E.N;
-            uint32_t u0, u1;
-            slice_of(units, c, C, u0, u1);
-            if (u0 == u1) continue;  // this CTA has nothing of this entry (fewer units than CTAs)
-
-            // ---- dependency on earlier entries ----
-            if (E.flags & 1) {
-                if (tid == 0) {
-                    const unsigned int need = E.tiles_before;
-                    guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; });
-                }
-                consumer_sync();
-            }
-            // ---- stage x (pair-permuted) and its 128-column block sums ----
-            for (int i = tid; i < 8 * (int)KB; i += kConsumerThreads) xsum[(i / KB) * p.kb_max + (i % KB)] = 0.f;
-            consumer_sync();
-            {
-                const int items = M * (int)KB * 16;  // one item = 8 consecutive k of one row
-                for (int it = tid; it < ((items + 31) & ~31); it += kConsumerThreads) {
-                    float s = 0.f;
-                    int r = 0, b8 = 0;
-                    if (it < items) {
-                        r = it / ((int)KB * 16);
-                        b8 = it % ((int)KB * 16);
-                        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(E.x + (size_t)r * E.K + (size_t)b8 * 8));
-                        uint4 o;
-                        o.x = __byte_perm(v.x, v.z, 0x5410);  // (x0, x4)
-                        o.y = __byte_perm(v.x, v.z, 0x7632);  // (x1, x5)
-                        o.z = __byte_perm(v.y, v.w, 0x5410);  // (x2, x6)
-                        o.w = __byte_perm(v.y, v.w, 0x7632);  // (x3, x7)
-                        *reinterpret_cast<uint4*>(xs + (size_t)r * p.x_row_bytes + (size_t)b8 * 16) = o;
-                        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            s += __uint_as_float(u[j] << 16) + __uint_as_float(u[j] & 0xFFFF0000u);
-                    }
-#pragma unroll
-                    for (int o = 8; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-                    if ((lane & 15) == 0 && it < items) xsum[r * p.kb_max + (b8 >> 4)] = s;
-                }
-            }
-            consumer_sync();
-
-            const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
-            bool have_first = false;  // a cut first tile that this CTA completes at the end of the entry
-            for (uint32_t tp = t_first; tp <= t_last; tp += kMaxTiles) {
-                const uint32_t pu0 = max(u0, tp * KB), pu1 = min(u1, (tp + kMaxTiles) * KB);
-                const uint32_t ntiles = min((uint32_t)kMaxTiles, t_last - tp + 1);
-                for (int i = tid; i < (int)ntiles * kConsumerWarps * kElems / 4; i += kConsumerThreads)
-                    reinterpret_cast<float4*>(tile_part)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                consumer_sync();
-
+        const bool compact = elems == 32;  // M <= 2: only the lanes with t == 0 hold real outputs
+        uint32_t item = 0, xe = 0;
+        uint32_t rs = 0, rph = 0;  // ring stage and its phase
+        Walk wk(p, C, c);
+        while (wk.next_entry()) {
+            const int M = p.e[wk.ei].M;
+            const uint32_t KB = wk.KB;
+            const uint32_t xb = xe & 1;
+            guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
+            ++xe;
+            const unsigned char* xs_b = xs + (size_t)xb * p.x_rows * p.x_row_bytes;
+            const float* xsum_b = xsum + (size_t)xb * 8 * p.kb_max;
+            const unsigned char* xlane = xs_b + (size_t)g * p.x_row_bytes + (size_t)t * 64;  // this lane's x columns
+            const float* xsum_lane = xsum_b + (2 * t) * p.kb_max;
+            for (uint32_t tp = wk.t_first; tp <= wk.t_last; tp += max_tiles, ++item) {
+                const uint32_t pu0 = max(wk.u0, tp * KB), pu1 = min(wk.u1, (tp + max_tiles) * KB);
+                const uint32_t ab = item & 1;
+                guard.wait_mbar(accempty0 + 8 * ab, ((item >> 1) & 1) ^ 1);
+                float* part = tile_part + (size_t)ab * part_floats + (size_t)warp * elems + (compact ? g * 4 : lane * 4);
+                const bool writer = !compact || t == 0;
                 float fin[4] = {0.f, 0.f, 0.f, 0.f};
                 int cur_tile = -1;
-                for (uint32_t cu = pu0; cu < pu1; cu += kStageUnits, ++ctr) {
-                    const uint32_t n = min((uint32_t)kStageUnits, pu1 - cu);
-                    const uint32_t s = ctr % p.stages, round = ctr / p.stages;
-                    guard.wait_mbar(full0 + 8 * s, round & 1);
-                    if ((uint32_t)warp < n) {
-                        const uint32_t u = cu + warp;
-                        const int tl = (int)(u / KB - tp);
-                        const uint32_t kb = u % KB;
-                        if (tl != cur_tile) {
-                            if (cur_tile >= 0)
-                                *reinterpret_cast<float4*>(tile_part + ((size_t)cur_tile * kConsumerWarps + warp) * kElems +
-                                                           lane * 4) = make_float4(fin[0], fin[1], fin[2], fin[3]);
+                // this warp's unit of the first chunk, as (tile within the pass, column block); later chunks advance by 16
+                uint32_t u = pu0 + warp;
+                uint32_t tl = u / KB - tp, kb = u % KB;
+                for (uint32_t cu = pu0; cu < pu1; cu += kStageUnits) {
+                    guard.wait_mbar(full0 + 8 * rs, rph);
+                    if (cu + warp < pu1) {
+                        if ((int)tl != cur_tile) {
+                            if (cur_tile >= 0 && writer)
+                                *reinterpret_cast<float4*>(part + (size_t)cur_tile * kComputeWarps * elems) =
+                                    make_float4(fin[0], fin[1], fin[2], fin[3]);
                             fin[0] = fin[1] = fin[2] = fin[3] = 0.f;
-                            cur_tile = tl;
+                            cur_tile = (int)tl;
                         }
-                        const unsigned char* ub = ring + (size_t)s * kStageBytes + (size_t)warp * kUnitBytes;
+                        const unsigned char* ub = ring + (size_t)rs * kStageBytes + (size_t)warp * kUnitBytes;
                         const uint4 wa = *reinterpret_cast<const uint4*>(ub + lane * 16);
                         const uint4 wb = *reinterpret_cast<const uint4*>(ub + 512 + lane * 16);
                         const __half2 ma = *reinterpret_cast<const __half2*>(ub + 1024 + 4 * g);
                         const __half2 mb = *reinterpret_cast<const __half2*>(ub + 1024 + 4 * (g + 8));
-                        float acc[4][4];
+                        float acc[2][4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j)
+                        for (int j = 0; j < 2; ++j)
 #pragma unroll
                             for (int q = 0; q < 4; ++q) acc[j][q] = 0.f;
                         const uint32_t was[4] = {wa.x, wa.y, wa.z, wa.w};
                         const uint32_t wbs[4] = {wb.x, wb.y, wb.z, wb.w};
-                        const unsigned char* xrow = xs + (size_t)g * p.x_row_bytes + (size_t)(kb * 16 + t * 4) * 16;
+                        const unsigned char* xrow = xlane + (size_t)kb * 256;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             uint4 b = make_uint4(0, 0, 0, 0);
                             if (g < M) b = *reinterpret_cast<const uint4*>(xrow + j * 16);
-                            mma_bf16_16816(acc[j], nib_pair(was[j], 0), nib_pair(wbs[j], 0), nib_pair(was[j], 1),
+                            mma_bf16_16816(acc[0], nib_pair(was[j], 0), nib_pair(wbs[j], 0), nib_pair(was[j], 1),
                                            nib_pair(wbs[j], 1), b.x, b.y);
-                            mma_bf16_16816(acc[j], nib_pair(was[j], 2), nib_pair(wbs[j], 2), nib_pair(was[j], 3),
+                            mma_bf16_16816(acc[1], nib_pair(was[j], 2), nib_pair(wbs[j], 2), nib_pair(was[j], 3),
                                            nib_pair(wbs[j], 3), b.z, b.w);
                         }
                         const float sa = __low2float(ma), za = 128.f + __high2float(ma);
                         const float sb = __low2float(mb), zb = 128.f + __high2float(mb);
-                        const float x0 = xsum[(2 * t) * p.kb_max + kb], x1 = xsum[(2 * t + 1) * p.kb_max + kb];
-                        const float a0 = (acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]);
-                        const float a1 = (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]);
-                        const float a2 = (acc[0][2] + acc[1][2]) + (acc[2][2] + acc[3][2]);
-                        const float a3 = (acc[0][3] + acc[1][3]) + (acc[2][3] + acc[3][3]);
-                        fin[0] = fmaf(sa, fmaf(-za, x0, a0), fin[0]);
-                        fin[1] = fmaf(sa, fmaf(-za, x1, a1), fin[1]);
-                        fin[2] = fmaf(sb, fmaf(-zb, x0, a2), fin[2]);
-                        fin[3] = fmaf(sb, fmaf(-zb, x1, a3), fin[3]);
+                        const float x0 = xsum_lane[kb], x1 = xsum_lane[p.kb_max + kb];
+                        fin[0] = fmaf(sa, fmaf(-za, x0, acc[0][0] + acc[1][0]), fin[0]);
+                        fin[1] = fmaf(sa, fmaf(-za, x1, acc[0][1] + acc[1][1]), fin[1]);
+                        fin[2] = fmaf(sb, fmaf(-zb, x0, acc[0][2] + acc[1][2]), fin[2]);
+                        fin[3] = fmaf(sb, fmaf(-zb, x1, acc[0][3] + acc[1][3]), fin[3]);
                     }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(empty0 + 8 * s);
+                    if (lane == 0) mbar_arrive(empty0 + 8 * rs);
+                    if (++rs == (uint32_t)p.stages) { rs = 0; rph ^= 1; }
+                    kb += kStageUnits;
+                    while (kb >= KB) { kb -= KB; ++tl; }
                 }
-                if (cur_tile >= 0)
-                    *reinterpret_cast<float4*>(tile_part + ((size_t)cur_tile * kConsumerWarps + warp) * kElems + lane * 4) =
+                if (cur_tile >= 0 && writer)
+                    *reinterpret_cast<float4*>(part + (size_t)cur_tile * kComputeWarps * elems) =
                         make_float4(fin[0], fin[1], fin[2], fin[3]);
-                consumer_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(accfull0 + 8 * ab);
+            }
+            if (lane == 0) mbar_arrive(xempty0 + 8 * xb);  // (ordered after this warp's reads by the __syncwarp above)
+        }
+    } else if (tid < kComputeThreads + kEpiThreads) {
+        // =============================== combiner group (4 warps) ===============================
+        const int et = tid - kComputeThreads;  // 0..127
+        uint32_t item = 0, fq = 0;
+        // element index -> (row within the tile, activation row)
+        auto decode = [&](int e, int& row, int& tok) {
+            if (elems == 32) {
+                row = (e >> 2) + ((e & 2) ? 8 : 0);
+                tok = e & 1;
+            } else {
+                const int ln = e >> 2, q = e & 3;
+                row = (ln >> 2) + ((q & 2) ? 8 : 0);
+                tok = 2 * (ln & 3) + (q & 1);
+            }
+        };
+        // hand one record to the fixer warp
+        auto push = [&](int type, int ei, uint32_t arg, const float* data) {
+            const uint32_t q = fq % kFixDepth, round = fq / kFixDepth;
+            if (et == 0) guard.wait_mbar(fqempty0 + 8 * q, (round & 1) ^ 1);
+            epi_sync();
+            FixRec& r = fixq[q];
+            if (et == 0) { r.type = type; r.ei = ei; r.arg = arg; }
+            if (data != nullptr && et < elems) r.data[et] = data[et];
+            epi_sync();
+            if (et == 0) mbar_arrive(fqfull0 + 8 * q);
+            ++fq;
+        };
 
-                // ---- combine the warps (fixed order) and route every tile of the pass ----
-                uint32_t n_full = 0;
-                bool have_last = false;
-                uint32_t last_rt = 0;
+        Walk wk(p, C, c);
+        while (wk.next_entry()) {
+            const StreamEntry& E = p.e[wk.ei];
+            const int M = E.M, N = E.N;
+            const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1;
+            bool have_first = false, have_last = false;
+            uint32_t last_rt = 0, n_full = 0;
+            for (uint32_t tp = wk.t_first; tp <= wk.t_last; tp += max_tiles, ++item) {
+                const uint32_t ntiles = min((uint32_t)max_tiles, wk.t_last - tp + 1);
+                const uint32_t ab = item & 1;
+                float* part = tile_part + (size_t)ab * part_floats;
+                guard.wait_mbar(accfull0 + 8 * ab, (item >> 1) & 1);
                 for (uint32_t tl = 0; tl < ntiles; ++tl) {
                     const uint32_t rt = tp + tl;
-                    const bool covers_begin = u0 <= rt * KB, covers_end = (rt + 1) * KB <= u1;
+                    const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
+                    if (cb && ce) ++n_full;
+                    else if (ce) have_first = true;
+                    else { have_last = true; last_rt = rt; }
+                }
+                // combine the 16 warps in a fixed order, clear the buffer, route every tile
+                for (int idx = et; idx < (int)ntiles * elems; idx += kEpiThreads) {
+                    const uint32_t tl = idx / elems;
+                    const int e = idx % elems;
+                    float* src = part + ((size_t)tl * kComputeWarps) * elems + e;
                     float sum = 0.f;
-                    if (tid < kElems) {
 #pragma unroll
-                        for (int w = 0; w < kConsumerWarps; ++w) sum += tile_part[((size_t)tl * kConsumerWarps + w) * kElems + tid];
+                    for (int w = 0; w < kComputeWarps; ++w) {
+                        sum += src[w * elems];
+                        src[w * elems] = 0.f;
                     }
-                    if (covers_begin && covers_end) {
-                        ++n_full;
-                        if (tid < kElems) {
-                            // element tid = lane*4 + q of a warp fragment: q -> (row half, token parity)
-                            const int ln = tid >> 2, q = tid & 3;
-                            const int row = (ln >> 2) + ((q & 2) ? 8 : 0), tok = 2 * (ln & 3) + (q & 1);
-                            if (tok < M) E.y[(size_t)tok * N + rt * 16 + row] = __float2bfloat16_rn(sum);
-                        }
-                    } else if (covers_end) {  // cut at its beginning: completed by this CTA later
-                        have_first = true;
-                        if (tid < kElems) stash_first[tid] = sum;
-                    } else {  // the tile continues in the next CTA: publish the contribution
-                        have_last = true;
-                        last_rt = rt;
-                        if (tid < kElems) stash_last[tid] = sum;
+                    const uint32_t rt = tp + tl;
+                    const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
+                    if (cb && ce) {
+                        int row, tok;
+                        decode(e, row, tok);
+                        if (tok < M) E.y[(size_t)tok * N + rt * 16 + row] = __float2bfloat16_rn(sum);
+                    } else if (ce) {
+                        stash_first[e] = sum;  // cut at its beginning: completed by this CTA's fixer
+                    } else {
+                        stash_last[e] = sum;   // continues in the next CTA: published by the fixer
                     }
                 }
-                if (n_full && p.tiles_done) {
-                    __threadfence();
-                    consumer_sync();
-                    if (tid == 0) red_release_add(p.tiles_done, n_full);
-                }
-                if (have_last) {
-                    const uint32_t which = (last_rt == t_first) ? 0u : 1u;
-                    unsigned char* slot = p.slots + ((size_t)c * 2 + which) * kSlotBytes;
-                    unsigned int* flag = reinterpret_cast<unsigned int*>(slot + kElems * 4);
-                    if (tid == 0) guard.wait_flag([&] { return ld_acquire(flag) == 0u; });
-                    consumer_sync();
-                    if (tid < kElems) reinterpret_cast<float*>(slot)[tid] = stash_last[tid];
-                    __threadfence();
-                    consumer_sync();
-                    if (tid == 0) st_release(flag, (uint32_t)ei + 1u);  // the tag names the entry the data belongs to
-                }
-                consumer_sync();  // tile_part and the stashes are free again
+                epi_sync();
+                if (et == 0) mbar_arrive(accempty0 + 8 * ab);
             }
-
-            // ---- complete the first tile of the slice from the contributions of earlier CTAs ----
-            if (have_first) {
-                const uint32_t rt = t_first;
+            if (et == 0 && n_full && p.tiles_done) {  // outputs of whole tiles are out (ordered by the barrier above)
+                __threadfence();
+                red_release_add(p.tiles_done, n_full);
+            }
+            // cross-CTA work of this entry, in the order that cannot chain CTAs: publish first, complete second
+            if (have_last) push(kRecContrib, wk.ei, (last_rt == wk.t_first) ? 0u : 1u, stash_last);
+            if (have_first) push(kRecFinish, wk.ei, wk.t_first, stash_first);
+        }
+        push(kRecEnd, 0, 0, nullptr);
+    } else if (tid < kComputeThreads + kEpiThreads + 32) {
+        // =============================== fixer warp ===============================
+        const int lane = tid & 31;
+        for (uint32_t fq = 0;; ++fq) {
+            const uint32_t q = fq % kFixDepth, round = fq / kFixDepth;
+            guard.wait_mbar(fqfull0 + 8 * q, round & 1);
+            const FixRec& r = fixq[q];
+            const int type = r.type;
+            if (*poisoned || type == kRecEnd) break;
+            if (type == kRecContrib) {
+                unsigned char* slot = p.slots + ((size_t)c * 2 + r.arg) * kSlotBytes;
+                unsigned int* flag = reinterpret_cast<unsigned int*>(slot + kElemsMax * 4);
+                if (lane == 0) guard.wait_flag([&] { return ld_acquire(flag) == 0u; });
+                __syncwarp();
+                for (int e = lane; e < elems; e += 32) reinterpret_cast<float*>(slot)[e] = r.data[e];
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    st_release(flag, (uint32_t)r.ei + 1u);  // the tag names the entry the data belongs to
+                }
+            } else {  // kRecFinish: complete the first tile of the slice from the contributions of earlier CTAs
+                const StreamEntry& E = p.e[r.ei];
+                const uint32_t KB = (uint32_t)E.K >> 7, units = ((uint32_t)E.N >> 4) * KB;
+                const uint32_t rt = r.arg;
                 const uint32_t c_lo = owner_of(rt * KB, units, C);
                 const uint32_t ncontrib = c - c_lo;
-                for (uint32_t i = tid; i < ncontrib; i += kConsumerThreads) {
+                const uint32_t tag = (uint32_t)r.ei + 1u;
+                for (uint32_t i = lane; i < ncontrib; i += 32) {
                     uint32_t which;
                     if (!contributor_slot(c_lo + i, rt, units, KB, C, which)) continue;
                     const unsigned int* flag = reinterpret_cast<const unsigned int*>(
-                        p.slots + ((size_t)(c_lo + i) * 2 + which) * kSlotBytes + kElems * 4);
-                    const uint32_t tag = (uint32_t)ei + 1u;
+                        p.slots + ((size_t)(c_lo + i) * 2 + which) * kSlotBytes + kElemsMax * 4);
                     guard.wait_flag([&] { return ld_acquire(flag) == tag; });
                 }
-                consumer_sync();
-                if (tid < kElems) {
+                __syncwarp();
+                for (int e = lane; e < elems; e += 32) {
                     float sum = 0.f;
                     for (uint32_t cc = c_lo; cc < c; ++cc) {
                         uint32_t which;
                         if (!contributor_slot(cc, rt, units, KB, C, which)) continue;
-                        sum += __ldcg(reinterpret_cast<const float*>(p.slots + ((size_t)cc * 2 + which) * kSlotBytes) + tid);
+                        sum += __ldcg(reinterpret_cast<const float*>(p.slots + ((size_t)cc * 2 + which) * kSlotBytes) + e);
                     }
-                    sum += stash_first[tid];
-                    const int ln = tid >> 2, q = tid & 3;
-                    const int row = (ln >> 2) + ((q & 2) ? 8 : 0), tok = 2 * (ln & 3) + (q & 1);
-                    if (tok < M) E.y[(size_t)tok * N + rt * 16 + row] = __float2bfloat16_rn(sum);
+                    sum += r.data[e];
+                    int row, tok;
+                    if (elems == 32) {
+                        row = (e >> 2) + ((e & 2) ? 8 : 0);
+                        tok = e & 1;
+                    } else {
+                        const int ln = e >> 2, qq = e & 3;
+                        row = (ln >> 2) + ((qq & 2) ? 8 : 0);
+                        tok = 2 * (ln & 3) + (qq & 1);
+                    }
+                    if (tok < E.M) E.y[(size_t)tok * E.N + rt * 16 + row] = __float2bfloat16_rn(sum);
                 }
-                __threadfence();
-                consumer_sync();
-                for (uint32_t i = tid; i < ncontrib; i += kConsumerThreads) {
+                __syncwarp();
+                for (uint32_t i = lane; i < ncontrib; i += 32) {
                     uint32_t which;
                     if (!contributor_slot(c_lo + i, rt, units, KB, C, which)) continue;
                     st_release(reinterpret_cast<unsigned int*>(p.slots + ((size_t)(c_lo + i) * 2 + which) * kSlotBytes +
-                                                               kElems * 4), 0u);
+                                                               kElemsMax * 4), 0u);
                 }
-                if (tid == 0 && p.tiles_done) red_release_add(p.tiles_done, 1u);
-                consumer_sync();
+                if (lane == 0 && p.tiles_done) {
+                    __threadfence();
+                    red_release_add(p.tiles_done, 1u);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(fqempty0 + 8 * q);
+        }
+    } else if (tid < kComputeThreads + kEpiThreads + 32 + kStagerThreads) {
+        // =============================== activation stager (2 warps) ===============================
+        // The rows of x are copied as they are (one bulk copy per row); only the 128-column block sums are computed.
+        const int st = tid - (kComputeThreads + kEpiThreads + 32);  // 0..63
+        uint32_t xe = 0;
+        Walk wk(p, C, c);
+        while (wk.next_entry()) {
+            const StreamEntry& E = p.e[wk.ei];
+            const uint32_t KB = wk.KB;
+            const uint32_t xb = xe & 1;
+            unsigned char* xs_b = xs + (size_t)xb * p.x_rows * p.x_row_bytes;
+            float* xsum_b = xsum + (size_t)xb * 8 * p.kb_max;
+            if (st == 0) {
+                guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1);
+                if (E.flags & kFlagDep) {  // the input is written by earlier entries: wait until all their tiles are out
+                    const unsigned int need = E.tiles_before;
+                    guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; });
+                    asm volatile("fence.proxy.async;" ::: "memory");  // the copies below read what that acquire ordered
+                }
+                mbar_expect_tx(xraw0 + 8 * xb, (uint32_t)E.M * (uint32_t)E.K * 2u);
+                for (int r = 0; r < E.M; ++r)
+                    bulk_g2s_plain(smem_u32(xs_b + (size_t)r * p.x_row_bytes), E.x + (size_t)r * E.K, (uint32_t)E.K * 2u,
+                                   xraw0 + 8 * xb);
+            }
+            guard.wait_mbar(xraw0 + 8 * xb, (xe >> 1) & 1);
+            // block sums of the real rows: one thread per (row, 128-column block).  Rows >= M keep whatever
+            // they held: they only reach accumulators of activation rows that are never stored.
+            for (int r = 0; r < E.M; ++r)
+                for (int kb = st; kb < (int)KB; kb += kStagerThreads) {
+                    const uint4* src = reinterpret_cast<const uint4*>(xs_b + (size_t)r * p.x_row_bytes + (size_t)kb * 256);
+                    float s = 0.f;
+#pragma unroll 4
+                    for (int j = 0; j < 16; ++j) {
+                        const uint4 v = src[j];
+                        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) s += __uint_as_float(u[q] << 16) + __uint_as_float(u[q] & 0xFFFF0000u);
+                    }
+                    xsum_b[r * p.kb_max + kb] = s;
+                }
+            stager_sync();
+            if (st == 0) mbar_arrive(xfull0 + 8 * xb);
+            ++xe;
+        }
+    } else {
+        // =============================== producer (one thread) ===============================
+        if (tid == kThreads - 32) {
+            uint64_t policy;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+            uint32_t s = 0, ph = 0, issued = 0;
+            Walk wk(p, C, c);
+            while (wk.next_entry()) {
+                const unsigned char* wbase = p.e[wk.ei].w;
+                for (uint32_t tp = wk.t_first; tp <= wk.t_last; tp += max_tiles) {
+                    const uint32_t pu0 = max(wk.u0, tp * wk.KB), pu1 = min(wk.u1, (tp + max_tiles) * wk.KB);
+                    for (uint32_t cu = pu0; cu < pu1; cu += kStageUnits, ++issued) {
+                        const uint32_t n = min((uint32_t)kStageUnits, pu1 - cu);
+                        guard.wait_mbar(empty0 + 8 * s, ph ^ 1);
+                        mbar_expect_tx(full0 + 8 * s, n * kUnitBytes);
+                        bulk_g2s(smem_u32(ring + (size_t)s * kStageBytes), wbase + (size_t)cu * kUnitBytes, n * kUnitBytes,
+                                 full0 + 8 * s, policy);
+                        if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
+                    }
+                }
+            }
+            // every copy this thread issued must have landed before the CTA may retire: walk back over the
+            // last `stages` chunks (s, ph now name the slot after the last one issued)
+            for (uint32_t back = 0; back < (uint32_t)p.stages && back < issued; ++back) {
+                if (s == 0) { s = p.stages; ph ^= 1; }
+                --s;
+                guard.wait_mbar(full0 + 8 * s, ph);
             }
         }
     }
-    // nobody leaves before every copy has landed and every consumer is done with shared memory
+    // nobody leaves before every copy has landed and everybody is done with shared memory
     __syncthreads();
 }
 
@@ -466,11 +634,11 @@ __global__ void __launch_bounds__(256) pack_stream_kernel(const uint8_t* __restr
         if (w < 256) {
             const int row = w >> 4, wi = w & 15;
             const uint2 cc = *reinterpret_cast<const uint2*>(codes + (size_t)(rt * 16 + row) * K + (size_t)kb * 128 + wi * 8);
+            // code k of the 8 sits at nibble (k >> 1) + 4 * (k & 1): even k in the low half, odd k in the high half
+            const uint32_t c8[8] = {cc.x & 0xFu, (cc.x >> 8) & 0xFu, (cc.x >> 16) & 0xFu, (cc.x >> 24) & 0xFu,
+                                    cc.y & 0xFu, (cc.y >> 8) & 0xFu, (cc.y >> 16) & 0xFu, (cc.y >> 24) & 0xFu};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                word |= ((cc.x >> (8 * j)) & 0xFu) << (4 * j);
-                word |= ((cc.y >> (8 * j)) & 0xFu) << (4 * (j + 4));
-            }
+            for (int k = 0; k < 8; ++k) word |= c8[k] << (4 * ((k >> 1) + 4 * (k & 1)));
         } else {
             const size_t gi = (size_t)(rt * 16 + (w - 256)) * ng + kb / bpg;
             word = (uint32_t)scales[gi] | ((uint32_t)zeros[gi] << 16);
@@ -479,9 +647,13 @@ __global__ void __launch_bounds__(256) pack_stream_kernel(const uint8_t* __restr
     }
 }
 
+inline int elems_for(int x_rows) { return x_rows <= 2 ? 32 : 128; }
+inline int max_tiles_for(int x_rows) { return x_rows <= 2 ? 8 : 2; }
+
 size_t smem_fixed_bytes(int x_rows, int x_row_bytes, int kb_max) {
-    return (size_t)kMaxTiles * kConsumerWarps * kElems * 4 + 2 * kElems * 4 + (size_t)x_rows * x_row_bytes +
-           (size_t)8 * kb_max * 4 + 64 /* poisoned flag + slack */;
+    return (size_t)2 * max_tiles_for(x_rows) * kComputeWarps * elems_for(x_rows) * 4 + 2 * kElemsMax * 4 +
+           (size_t)kFixDepth * (16 + kElemsMax * 4) + (size_t)2 * x_rows * x_row_bytes + (size_t)2 * 8 * kb_max * 4 +
+           (10 + 2 * kFixDepth) * 8 + 64 /* flag + slack */;
 }
 
 constexpr size_t kSmemLimit = 232448;  // 227 KiB per CTA
@@ -537,11 +709,14 @@ qil_status launch_w4a16_stream(const qil_linear_desc* entries, int count, void* 
             e.y = reinterpret_cast<__nv_bfloat16*>(d.y);
             e.N = d.N; e.K = d.K; e.M = d.M;
             // the first entry of a launch never waits: earlier launches are ordered by the stream
-            e.flags = (i > 0) ? (d.flags & 1) : 0;
+            e.flags = (i > 0) ? (d.flags & kFlagDep) : 0;
+            // an entry right before a dependent one takes whole row tiles per CTA when there are enough of them:
+            // a little imbalance is cheaper than completing shared tiles while everybody waits for the result
+            if (i + 1 < n && (entries[base + i + 1].flags & kFlagDep) && d.N / 16 >= C) e.flags |= kFlagAligned;
             e.tiles_before = tiles;
             e.pad = 0;
             tiles += (uint32_t)(d.N / 16);
-            any_dep |= (e.flags & 1) != 0;
+            any_dep |= (e.flags & kFlagDep) != 0;
             if (d.M > x_rows) x_rows = d.M;
             if (d.K > kmax) kmax = d.K;
         }
@@ -551,6 +726,8 @@ qil_status launch_w4a16_stream(const qil_linear_desc* entries, int count, void* 
         p.kb_max = kmax / 128;
         p.stages = stages_for(p.x_rows, p.x_row_bytes, p.kb_max);
         if (p.stages < 3) return QIL_ERR_UNSUPPORTED;
+        p.elems = elems_for(p.x_rows);
+        p.max_tiles = max_tiles_for(p.x_rows);
         p.status = reinterpret_cast<int*>(ws);
         p.tiles_done = any_dep ? reinterpret_cast<unsigned int*>(ws) + 1 : nullptr;
         p.slots = reinterpret_cast<unsigned char*>(ws) + kWsHeader;

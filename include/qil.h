@@ -76,8 +76,20 @@ typedef enum { QIL_F32 = 0, QIL_BF16 = 1, QIL_F16 = 2 } qil_dtype;
  *   group larger than 128 repeats its pair in every block it covers).
  *   Needs N % 16 == 0, K % 128 == 0, group_size % 128 == 0.  With group 128 the
  *   buffer is exactly as large as canonical codes + scales + zeros.
+ * QIL_LAYOUT_STREAM128: units for the tensor-memory (tcgen05) decode kernel, built by
+ *   qil_pack_stream128_w4.  Unit u = (n/128)*(K/128) + k/128 occupies bytes
+ *   [8704 u, 8704 (u+1)): 4 chunks (32 columns of K each) x 128 rows x 16 bytes of
+ *   codes - byte b of 32-bit word m of a chunk holds column 8m+b of the chunk in its
+ *   low nibble and column 8m+4+b in its high nibble - then 128 pairs {fp16 scale,
+ *   fp16 zero}, one per row.  Rows beyond N are zero (N need not be a multiple of
+ *   128).  Needs K % 128 == 0 and group_size % 128 == 0.
  */
-typedef enum { QIL_LAYOUT_CANONICAL = 0, QIL_LAYOUT_TILE16 = 1, QIL_LAYOUT_STREAM = 2 } qil_layout;
+typedef enum {
+    QIL_LAYOUT_CANONICAL = 0,
+    QIL_LAYOUT_TILE16 = 1,
+    QIL_LAYOUT_STREAM = 2,
+    QIL_LAYOUT_STREAM128 = 3
+} qil_layout;
 
 typedef struct CUstream_st* qil_stream_t; /* a cudaStream_t */
 
@@ -113,6 +125,10 @@ qil_status qil_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout
 size_t qil_stream_w4_bytes(int N, int K);
 qil_status qil_pack_stream_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K,
                               int group_size, void* out, qil_stream_t stream);
+/* Same for QIL_LAYOUT_STREAM128 (N >= 1, K % 128 == 0, group_size % 128 == 0). */
+size_t qil_stream128_w4_bytes(int N, int K);
+qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K,
+                                 int group_size, void* out, qil_stream_t stream);
 
 /* ------------------------------------------------------------------------
  * Weight-only linear, 4-bit weights x bf16 activations (the OpenVLA / Llama-2
@@ -123,10 +139,13 @@ qil_status qil_pack_stream_w4(const uint8_t* codes, const void* scales, const vo
  * The kernel is chosen from the shape: tensor-core skinny kernel (weights read
  * once, any M handled in slabs of 64 rows) when K % 128 == 0 and
  * group_size % 128 == 0; a general kernel otherwise (any K % 8 == 0, any
- * group_size dividing K, canonical layout only).  With QIL_LAYOUT_STREAM the
- * persistent streaming kernel runs (M <= 8; scales and zeros are part of the
- * buffer, the two arguments are ignored and may be null; the workspace is
- * always needed).
+ * group_size dividing K, canonical layout only).  With QIL_LAYOUT_STREAM
+ * (M <= 8) or QIL_LAYOUT_STREAM128 (M <= 4) a persistent streaming kernel runs;
+ * scales and zeros are part of the buffer, the two arguments are ignored and
+ * may be null; the workspace is always needed.  The STREAM128 kernel converts
+ * the activations to 16-bit block fixed point (per 128 columns a power-of-two
+ * scale, |integer| <= 32639) and accumulates exactly in int32; the conversion
+ * error per element is at most 2^-16 of the block maximum.
  * workspace: qil_linear_w4a16_workspace_size() bytes, only touched when the
  * shape needs a split along K; it must be zero-filled once before first use
  * (the kernels leave it zeroed again).  Calls that share a workspace must not
@@ -177,8 +196,8 @@ qil_status qil_linear_w4a16_static_ws(const void* x, const uint32_t* qweight, co
  * QIL_DEP_PREVIOUS in `flags`: it then starts only after every earlier entry has
  * written all of its outputs.  Entries without the flag may overlap with their
  * predecessors (q, k and v of one layer share an input and need no flag).
- * When every entry uses QIL_LAYOUT_STREAM the whole list runs as one persistent
- * kernel.  All pointers inside a descriptor are device
+ * When every entry uses QIL_LAYOUT_STREAM, or every entry uses
+ * QIL_LAYOUT_STREAM128, the whole list runs as one persistent kernel.  All pointers inside a descriptor are device
  * pointers; the descriptor array itself is host memory and is consumed before
  * the call returns.  workspace must be as large as the largest
  * qil_linear_w4a16_workspace_size() over the entries (zero-filled once).

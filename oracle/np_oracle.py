@@ -237,6 +237,43 @@ def to_stream(packed: np.ndarray, scales, zeros, group_size: int) -> np.ndarray:
     return out
 
 
+def to_stream128(codes: np.ndarray, scales, zeros, group_size: int) -> np.ndarray:
+    """Codes uint8 [N][K] + fp16 scales/zeros [N][K/G] -> the STREAM128 byte buffer.
+
+    Unit u = (n // 128) * (K // 128) + kb starts at byte 8704 * u.  Its first 8192 bytes are 4 chunks
+    (32 columns each) x 128 rows x 16 bytes: byte 4*m + b of (chunk j, row r) holds column 32*j + 8*m + b
+    of the block in its low nibble and column 32*j + 8*m + 4 + b in its high nibble.  Then, for each of
+    the 128 rows, the fp16 scale followed by the fp16 zero of the group containing block kb.  Rows
+    beyond N are all zero.
+    """
+    c = np.asarray(codes, dtype=np.uint8)
+    N, K = c.shape
+    G = int(group_size)
+    if K % 128 or G % 128 or K % G:
+        raise ValueError("STREAM128 layout needs K % 128 == 0 and G % 128 == 0")
+    s16 = np.ascontiguousarray(scales, dtype=np.float16).view(np.uint16)
+    z16 = np.ascontiguousarray(zeros, dtype=np.float16).view(np.uint16)
+    KB, RT = K // 128, (N + 127) // 128
+    out = np.zeros(RT * KB * 8704, dtype=np.uint8)
+    for rt in range(RT):
+        rows = min(128, N - rt * 128)
+        for kb in range(KB):
+            base = (rt * KB + kb) * 8704
+            blk = c[rt * 128:rt * 128 + rows, kb * 128:(kb + 1) * 128]
+            for j in range(4):
+                for m in range(4):
+                    for b in range(4):
+                        lo = blk[:, 32 * j + 8 * m + b] & 0xF
+                        hi = blk[:, 32 * j + 8 * m + 4 + b] & 0xF
+                        off = base + j * 128 * 16 + np.arange(rows) * 16 + 4 * m + b
+                        out[off] = lo | (hi << 4)
+            meta = np.empty((rows, 2), dtype=np.uint16)
+            meta[:, 0] = s16[rt * 128:rt * 128 + rows, (kb * 128) // G]
+            meta[:, 1] = z16[rt * 128:rt * 128 + rows, (kb * 128) // G]
+            out[base + 8192:base + 8192 + rows * 4] = meta.view(np.uint8).reshape(-1)
+    return out
+
+
 # ----------------------------------------------------------------------------
 # Dequantisation and the two linears, in fp64 / int64.
 # ----------------------------------------------------------------------------

@@ -14,7 +14,7 @@ from . import _lib
 
 OK = 0
 F32, BF16, F16 = 0, 1, 2
-LAYOUT_CANONICAL, LAYOUT_TILE16, LAYOUT_STREAM = 0, 1, 2
+LAYOUT_CANONICAL, LAYOUT_TILE16, LAYOUT_STREAM, LAYOUT_STREAM128 = 0, 1, 2, 3
 DEP_PREVIOUS = 1
 ERR_RANGE = 8
 
@@ -96,6 +96,18 @@ def pack_stream_w4(codes, scales, zeros, group_size: int, stream=None):
     out = torch.empty((max(nbytes, 16),), dtype=torch.uint8, device=codes.device)
     _check(lib.qil_pack_stream_w4(_ptr(codes), _ptr(scales), _ptr(zeros), N, K, int(group_size), _ptr(out),
                                   _stream(stream)))
+    return out
+
+
+def pack_stream128_w4(codes, scales, zeros, group_size: int, stream=None):
+    """codes uint8 [N][K] + fp16 scales/zeros [N][K/G] -> the STREAM128 buffer of the tcgen05 decode kernel."""
+    _need_cuda(codes, scales, zeros)
+    N, K = codes.shape
+    lib = _lib.load()
+    nbytes = int(lib.qil_stream128_w4_bytes(N, K))
+    out = torch.empty((max(nbytes, 16),), dtype=torch.uint8, device=codes.device)
+    _check(lib.qil_pack_stream128_w4(_ptr(codes), _ptr(scales), _ptr(zeros), N, K, int(group_size), _ptr(out),
+                                     _stream(stream)))
     return out
 
 

@@ -76,6 +76,13 @@ qil_status launch_pack_stream_w4(const uint8_t* codes, const void* scales, const
                                  void* out, cudaStream_t st);
 qil_status launch_w4a16_stream(const qil_linear_desc* entries, int count, void* ws, size_t ws_bytes, cudaStream_t st);
 
+bool w4a16_tc_supported(int M, int N, int K, int G);
+size_t w4a16_tc_weight_bytes(int N, int K);
+size_t w4a16_tc_workspace();
+qil_status launch_pack_stream128_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K, int G,
+                                    void* out, cudaStream_t st);
+qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, size_t ws_bytes, cudaStream_t st);
+
 size_t w4a4_workspace(int M, int N, int K);
 qil_status launch_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, void* y,
                        int32_t* acc_out, int M, int N, int K, void* ws, size_t ws_bytes, cudaStream_t st);

@@ -19,7 +19,7 @@ from . import _lib, api, workloads as wl
 
 
 class QuantisedLinears:
-    def __init__(self, cfg: int = 1, M: int = 1, n_layers: int = wl.N_LAYERS, layout: int = api.LAYOUT_STREAM,
+    def __init__(self, cfg: int = 1, M: int = 1, n_layers: int = wl.N_LAYERS, layout: int = api.LAYOUT_STREAM128,
                  deps: str = "layer",
                  outliers: bool = True, device: str = "cuda", keep_host_rows: dict | None = None,
                  host_threads: int | None = None):
@@ -48,7 +48,9 @@ class QuantisedLinears:
                     self.kept[i] = (rows, w[rows].copy())
                 wd = torch.from_numpy(w).to(device)
                 codes, s, z = api.quantize_rtn_w4(wd, self.G)
-                if layout == api.LAYOUT_STREAM:
+                if layout == api.LAYOUT_STREAM128:
+                    self.packed.append(api.pack_stream128_w4(codes, s, z, self.G))
+                elif layout == api.LAYOUT_STREAM:
                     self.packed.append(api.pack_stream_w4(codes, s, z, self.G))
                 else:
                     self.packed.append(api.pack_w4(codes, layout))

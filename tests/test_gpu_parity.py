@@ -397,6 +397,109 @@ def test_w4a16_stream_rejects_unsupported(api):
 
 
 # ----------------------------------------------------------------------------
+# W4A16, tensor-memory (tcgen05) decode kernel (QIL_LAYOUT_STREAM128)
+# ----------------------------------------------------------------------------
+def _tc_inputs(api, M, N, K, G, seed, x_scale=None):
+    w = wl.normal_weights(320, seed, N, K, 0.02, outlier_prob=0.001)
+    x = wl.normal_activations_bf16(320, seed + 1, M, K)
+    if x_scale is not None:
+        xf = wl.bf16_bits_to_f32(x).copy()
+        xf[:, ::61] *= x_scale
+        x = wl.f32_to_bf16_bits(xf)
+    codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
+    buf = api.pack_stream128_w4(cuda(codes), cuda(scales), cuda(zeros), G)
+    return x, codes, scales, zeros, buf
+
+
+@pytest.mark.parametrize("N,K,G", [(200, 384, 128), (128, 128, 128), (40, 256, 256)])
+def test_pack_stream128_matches_oracle(api, N, K, G):
+    _, codes, scales, zeros, buf = _tc_inputs(api, 1, N, K, G, N + K)
+    ref = np_oracle.to_stream128(codes, scales, zeros, G)
+    np.testing.assert_array_equal(buf.cpu().numpy()[:ref.size], ref)
+
+
+@pytest.mark.parametrize("M,N,K,G", [
+    (1, 128, 128, 128), (1, 256, 1024, 128), (2, 200, 384, 128), (3, 1000, 2176, 128), (4, 512, 1024, 256),
+    (1, 4096, 4096, 128), (1, 4096, 11008, 128), (1, 11008, 4096, 128), (4, 4096, 4096, 128), (1, 160, 2048, 2048),
+    (1, 37008, 256, 128), (2, 48, 512, 128),
+])
+def test_w4a16_tc_shapes(api, M, N, K, G):
+    import torch
+    x, codes, scales, zeros, buf = _tc_inputs(api, M, N, K, G, M + N + K)
+    rows = np.arange(N) if N * K <= (1 << 24) else np.sort(np.random.default_rng(N).choice(N, 512, replace=False))
+    y_ref = c_oracle.linear_w4a16(x, codes[rows], scales[rows], zeros[rows], G)
+    ws = api.new_workspace(api.linear_w4a16_workspace_size(M, N, K, G))
+    outs = []
+    for _ in range(2):
+        y = api.linear_w4a16(to_bf16_cuda(x), buf, None, None, N, G, api.LAYOUT_STREAM128, workspace=ws)
+        outs.append(y.clone())
+    assert _status(api, ws) == 0
+    assert_rows_close(bf16_to_f64(outs[0])[:, rows], y_ref)
+    np.testing.assert_array_equal(bits_of(outs[0]), bits_of(outs[1]))
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    flags = ws[256:256 + sms * 2 * 2064].view(-1, 2064)[:, 2048:]
+    assert int(torch.count_nonzero(flags).item()) == 0
+
+
+def test_w4a16_tc_wide_dynamic_range(api):
+    """Outlier channels 3000x larger than the rest, and a block of tiny values: the per-block fixed point
+    must keep the small blocks' contribution (their scale is independent of the outlier blocks)."""
+    M, N, K, G = 2, 256, 2048, 128
+    x, codes, scales, zeros, buf = _tc_inputs(api, M, N, K, G, 77, x_scale=3000.0)
+    xf = wl.bf16_bits_to_f32(x).copy()
+    xf[:, 1024:1152] *= 1e-6
+    xf[1, 1280:1408] = 0.0
+    x = wl.f32_to_bf16_bits(xf)
+    y_ref = c_oracle.linear_w4a16(x, codes, scales, zeros, G)
+    y = api.linear_w4a16(to_bf16_cuda(x), buf, None, None, N, G, api.LAYOUT_STREAM128)
+    assert_rows_close(bf16_to_f64(y), y_ref)
+
+
+def test_w4a16_tc_batch_with_dependencies(api):
+    import ctypes as C
+    import torch
+    from paper_2412_01034_b200 import _lib
+    lib = _lib.load()
+    G, M = 128, 2
+    dims = [(512, 1024), (1024, 512), (768, 1024), (256, 768)]
+    packs, refs = [], []
+    for i, (N, K) in enumerate(dims):
+        w = wl.normal_weights(321, i, N, K, 0.05)
+        q = np_oracle.quantize_rtn_w4_asym(w, G)
+        refs.append(q)
+        packs.append(api.pack_stream128_w4(cuda(q[0]), cuda(q[1]), cuda(q[2]), G))
+    x0 = wl.normal_activations_bf16(321, 100, M, dims[0][1])
+    xd = to_bf16_cuda(x0)
+    ys = [torch.zeros((M, N), dtype=torch.bfloat16, device="cuda") for (N, _) in dims]
+    ins = [xd, ys[0], ys[1], ys[2]]
+    descs = (_lib.LinearDesc * 4)()
+    for i, (N, K) in enumerate(dims):
+        d = descs[i]
+        d.x, d.qweight, d.y = ins[i].data_ptr(), packs[i].data_ptr(), ys[i].data_ptr()
+        d.scales = d.zeros = None
+        d.M, d.N, d.K, d.group_size, d.layout, d.flags = M, N, K, G, api.LAYOUT_STREAM128, (api.DEP_PREVIOUS if i else 0)
+    ws = api.new_workspace(api.linear_w4a16_workspace_size(M, 1024, 1024, G))
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    for rep in range(3):
+        for y in ys:
+            y.zero_()
+        assert lib.qil_linear_w4a16_batch(descs, 4, C.c_void_p(ws.data_ptr()), ws.numel(), st) == 0
+        torch.cuda.synchronize()
+        assert _status(api, ws) == 0
+        got = [y.clone() for y in ys]
+        cur = xd
+        for i, (N, K) in enumerate(dims):
+            one = api.linear_w4a16(cur, packs[i], None, None, N, G, api.LAYOUT_STREAM128, workspace=ws)
+            np.testing.assert_array_equal(bits_of(got[i]), bits_of(one))
+            cur = one
+    cur_bits = x0
+    for i, (N, K) in enumerate(dims):
+        y_ref = c_oracle.linear_w4a16(cur_bits, *refs[i], G)
+        assert_rows_close(bf16_to_f64(got[i]), y_ref, rel=1e-2)
+        cur_bits = wl.f32_to_bf16_bits(y_ref.astype(np.float32))
+
+
+# ----------------------------------------------------------------------------
 # W4A4
 # ----------------------------------------------------------------------------
 def test_w4a4_hand_case(api):

@@ -288,6 +288,36 @@ def test_stream_layout_follows_its_written_rule():
         np.testing.assert_array_equal((words >> np.uint32(4 * ((k >> 1) + 4 * (k & 1)))) & 0xF, (t16 >> np.uint32(4 * k)) & 0xF)
 
 
+def test_stream128_layout_follows_its_written_rule():
+    rng = np.random.default_rng(13)
+    N, K, G = 200, 384, 128      # two row tiles (the second one ragged), three column blocks
+    codes = rng.integers(0, 16, size=(N, K)).astype(np.uint8)
+    scales = (rng.random((N, K // G)) + 0.5).astype(np.float16)
+    zeros = rng.integers(0, 16, size=(N, K // G)).astype(np.float16)
+    buf = np_oracle.to_stream128(codes, scales, zeros, G)
+    assert buf.size == 2 * 3 * 8704
+    # element (n=150, k=300): row tile 1, block 2 -> unit 1*3+2 = 5; row 22; column 44 of the block ->
+    # chunk 1, column 12 of the chunk -> word 1, 12 = 8*1 + 4 + 0 -> byte 0 of word 1, high nibble
+    off = 5 * 8704 + (1 * 128 + 22) * 16 + 4 * 1 + 0
+    assert buf[off] >> 4 == codes[150, 300]
+    assert buf[off] & 0xF == codes[150, 296]       # column 40 = 32 + 8*1 + 0 -> same byte, low nibble
+    m = 5 * 8704 + 8192 + 22 * 4
+    assert buf[m:m + 2].view(np.float16)[0] == scales[150, 2]
+    assert buf[m + 2:m + 4].view(np.float16)[0] == zeros[150, 2]
+    # rows 200..255 of the second row tile are padding
+    pad = buf[3 * 8704:4 * 8704]
+    assert np.all(pad[:8192].reshape(4, 128, 16)[:, 72:, :] == 0) and np.all(pad[8192 + 72 * 4:] == 0)
+    # every code appears exactly once: undo the rule for unit 0
+    u0 = buf[:8192].reshape(4, 128, 4, 4)
+    rec = np.zeros((128, 128), dtype=np.uint8)
+    for j in range(4):
+        for mm in range(4):
+            for b in range(4):
+                rec[:, 32 * j + 8 * mm + b] = u0[j, :, mm, b] & 0xF
+                rec[:, 32 * j + 8 * mm + 4 + b] = u0[j, :, mm, b] >> 4
+    np.testing.assert_array_equal(rec, codes[:128, :128])
+
+
 # --------------------------------------------------------------------------
 # linears
 # --------------------------------------------------------------------------

@@ -20,11 +20,11 @@
 // stream of units.
 //
 // Roles in a CTA (one CTA per SM): a producer thread streams the CTA's slice of units
-// through a shared-memory ring (cp.async.bulk + mbarrier); two warpgroups alternate units
-// (unpack -> tensor memory, later the epilogue of the same unit); one thread issues the
-// MMAs; four stager warps convert the next activations; four finalizer warps combine the
+// through a shared-memory ring (cp.async.bulk + mbarrier); the unpack warpgroups alternate units
+// (unpack -> tensor memory, later the epilogue of the same unit; three of them take turns); one thread per
+// warpgroup issues its MMAs; four stager warps convert the next activations; four finalizer warps combine the
 // warpgroups' partial sums, write outputs and complete row tiles shared with other CTAs
-// through fp32 slots in the workspace (tagged flags, fixed summation order).
+// through {value, tag} pairs in the workspace (one 8-byte store each, fixed summation order).
 // Every wait is bounded (2 s); on expiry QIL_ERR_TIMEOUT is recorded in the workspace
 // status word, waiting stops, tensor memory is released and the kernel returns.
 #include <mutex>
@@ -38,26 +38,26 @@ namespace {
 constexpr int kUnitRows = 128;
 constexpr int kUnitBytes = 8192 + 512;
 constexpr int kWgThreads = 128;
-constexpr int kNumWg = 2;
+constexpr int kNumWg = 3;
 constexpr int kStagerThreads = 128;
 constexpr int kFinThreads = 128;
-// thread ranges: [0,256) two unpack/epilogue warpgroups, [256,288) MMA warp, [288,320) producer warp,
-// [320,448) stager, [448,576) finalizer
+// thread ranges: kNumWg unpack/epilogue warpgroups, then the MMA warp, the producer warp, the stager, the finalizer
 constexpr int kMmaBase = kNumWg * kWgThreads;
-constexpr int kProdBase = kMmaBase + 32;
+constexpr int kProdBase = kMmaBase + 32 * kNumWg;  // one MMA-issuing warp per warpgroup: issue latency, not the
+                                                    // tensor pipe, limits one thread, and issuers do not slow each other
 constexpr int kStagerBase = kProdBase + 32;
 constexpr int kFinBase = kStagerBase + kStagerThreads;
 constexpr int kThreads = kFinBase + kFinThreads;
-constexpr int kNumA = 4;        // A buffers in tensor memory (32 columns each)
-constexpr int kNumD = 4;        // accumulator buffers (8 columns each)
-constexpr int kTmemCols = 256;  // A at columns [0,128), D at [128,160)
-constexpr int kColD = 128;
+constexpr int kNumBuf = 2 * kNumWg;  // A buffers (32 columns each) and accumulator buffers (8 columns each)
+constexpr int kTmemCols = 256;       // A at columns [0, 32 kNumBuf), D behind them
+constexpr int kColD = 32 * kNumBuf;
+static_assert(kColD + 8 * kNumBuf <= kTmemCols, "tensor memory budget");
 constexpr int kMaxTiles = 2;    // row tiles per pass
 constexpr int kPartBufs = 4;    // partial-sum buffers between the warpgroups and the finalizer
 constexpr int kMaxEntries = 256;
 constexpr int kMaxRows = 4;     // activation rows
-constexpr int kSlotFloats = kMaxRows * kUnitRows;
-constexpr int kSlotBytes = kSlotFloats * 4 + 16;  // data + flag word
+constexpr int kSlotDepth = 4;                      // ring of slots per (CTA, first/last tile)
+constexpr int kSlotElems = kMaxRows * kUnitRows;   // {value, tag} pairs of 8 bytes
 constexpr int kWsHeader = 256;
 constexpr int kFlagDep = 1;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -122,9 +122,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const unsigned int* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release(unsigned int* p, uint32_t v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 __device__ __forceinline__ void red_release_add(unsigned int* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -178,6 +175,7 @@ struct Guard {
         const unsigned long long t0 = now_ns();
         for (uint32_t i = 1;; ++i) {
             if (mbar_try_wait(bar, parity)) return;
+            __nanosleep(40);  // a waiting warp must not take issue slots from the working ones
             if ((i & 15u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
         }
         fail();
@@ -240,9 +238,6 @@ struct Cyc {
     __device__ __forceinline__ void step() {
         if (++idx == n) { idx = 0; ph ^= 1; }
     }
-    __device__ __forceinline__ void step(uint32_t k) {
-        for (uint32_t i = 0; i < k; ++i) step();
-    }
 };
 
 __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_constant__ TcParams p) {
@@ -262,9 +257,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     uint64_t* bars = reinterpret_cast<uint64_t*>(part + (size_t)kPartBufs * part_floats);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
-    const uint32_t afull0 = smem_u32(b2), aempty0 = smem_u32(b2 + kNumA);
-    const uint32_t dfull0 = smem_u32(b2 + 2 * kNumA), dempty0 = smem_u32(b2 + 2 * kNumA + kNumD);
-    uint64_t* b3 = b2 + 2 * kNumA + 2 * kNumD;
+    const uint32_t afull0 = smem_u32(b2);
+    const uint32_t dfull0 = smem_u32(b2 + 2 * kNumBuf), dempty0 = smem_u32(b2 + 3 * kNumBuf);
+    uint64_t* b3 = b2 + 4 * kNumBuf;
     const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2), xraw0 = smem_u32(b3 + 4);
     const uint32_t pfull0 = smem_u32(b3 + 5), pempty0 = smem_u32(b3 + 5 + kPartBufs);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 5 + 2 * kPartBufs);
@@ -275,21 +270,18 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 4);
         }
-        for (int i = 0; i < kNumA; ++i) {
+        for (int i = 0; i < kNumBuf; ++i) {
             mbar_init(afull0 + 8 * i, 4);
-            mbar_init(aempty0 + 8 * i, 1);
-        }
-        for (int i = 0; i < kNumD; ++i) {
             mbar_init(dfull0 + 8 * i, 1);
             mbar_init(dempty0 + 8 * i, 4);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(xfull0 + 8 * i, 1);
-            mbar_init(xempty0 + 8 * i, 2 * 4);
+            mbar_init(xempty0 + 8 * i, kNumWg * 4);
         }
         mbar_init(xraw0, 1);
         for (int i = 0; i < kPartBufs; ++i) {
-            mbar_init(pfull0 + 8 * i, 2 * 4);
+            mbar_init(pfull0 + 8 * i, kNumWg * 4);
             mbar_init(pempty0 + 8 * i, 1);
         }
         *poisoned = 0;
@@ -313,8 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // ======================= unpack + epilogue warpgroups =======================
         const int wg = tid / kWgThreads, r = tid % kWgThreads, lane = tid & 31;
         const uint32_t lane_base = (uint32_t)(r & ~31) << 16;  // this warp's quarter of the tensor-memory lanes
-        uint32_t unit = 0;                                     // index of the next unit of this CTA (all warpgroups count)
-        Cyc rs(p.stages), pb(kPartBufs);
+        Cyc rs(p.stages), pb(kPartBufs), ab(kNumBuf), turn(kNumWg);  // all advance once per unit of the CTA
         uint32_t xe = 0;
         Walk wk(p, C, c);
         while (wk.next_entry()) {
@@ -331,20 +322,23 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 float* my_part = part + (size_t)pb.idx * part_floats + (size_t)wg * kMaxTiles * XR * kUnitRows + r;
                 float fin[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
                 int cur_tile = -1;
-                // a unit whose MMAs are in flight: its epilogue runs after the next unit of this warpgroup is unpacked
+                // a unit whose MMAs are in flight: its accumulators are read after the next unit of this
+                // warpgroup has been written to tensor memory
                 bool pend = false;
                 uint32_t pend_d = 0, pend_dph = 0, pend_kb = 0;
                 int pend_tl = 0;
                 float pend_s = 0.f;
                 int pend_z = 0;
-                auto epilogue = [&]() {
+                uint32_t d[8];
+                auto epilogue_load = [&]() {   // start reading the accumulators of the pending unit
                     guard.wait_mbar(dfull0 + 8 * pend_d, pend_dph);
                     tc_fence_after();
-                    uint32_t d[8];
                     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                                  : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]),
                                    "=r"(d[7])
                                  : "r"(tmem + lane_base + kColD + 8 * pend_d));
+                };
+                auto epilogue_math = [&]() {   // ... and fold them into this thread's row sums
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     tc_fence_before();
                     __syncwarp();
@@ -366,17 +360,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             fin[t] = fmaf((float)v, pend_s * xscale_b[t * p.kb_max + pend_kb], fin[t]);
                         }
                 };
-                uint32_t tl = 0, kb = 0;
-                {
-                    const uint32_t u = pu0;
-                    tl = u / KB - tp;
-                    kb = u % KB;
-                }
-                for (uint32_t cu = pu0; cu < pu1; ++cu, ++unit) {
-                    const uint32_t a = unit % kNumA, use = unit / kNumA;  // kNumA == kNumD: same index for D
-                    if ((unit & 1u) == (uint32_t)wg) {
+                uint32_t tl = pu0 / KB - tp, kb = pu0 % KB;
+                for (uint32_t cu = pu0; cu < pu1; ++cu) {
+                    if (turn.idx == (uint32_t)wg) {
+                        const uint32_t a = ab.idx;
                         guard.wait_mbar(full0 + 8 * rs.idx, rs.ph);
-                        guard.wait_mbar(aempty0 + 8 * a, (use & 1) ^ 1);
                         const unsigned char* ub = ring + (size_t)rs.idx * kUnitBytes;
                         tc_fence_after();
 #pragma unroll
@@ -395,6 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                                          : "memory");
                         }
                         const __half2 meta = *reinterpret_cast<const __half2*>(ub + 8192 + 4 * r);
+                        if (pend) epilogue_load();  // overlaps with the stores above
                         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                         tc_fence_before();
                         __syncwarp();
@@ -402,19 +391,24 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             mbar_arrive(afull0 + 8 * a);
                             mbar_arrive(empty0 + 8 * rs.idx);
                         }
-                        if (pend) epilogue();
+                        if (pend) epilogue_math();
                         pend = true;
                         pend_d = a;
-                        pend_dph = use & 1;
+                        pend_dph = ab.ph;
                         pend_kb = kb;
                         pend_tl = (int)tl;
                         pend_s = __low2float(meta);
                         pend_z = (int)__high2float(meta);
                     }
                     rs.step();
+                    ab.step();
+                    turn.step();
                     if (++kb == KB) { kb = 0; ++tl; }
                 }
-                if (pend) epilogue();
+                if (pend) {
+                    epilogue_load();
+                    epilogue_math();
+                }
                 if (cur_tile >= 0) {
 #pragma unroll
                     for (int t = 0; t < kMaxRows; ++t)
@@ -428,28 +422,37 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             if (lane == 0) mbar_arrive(xempty0 + 8 * xb);
         }
     } else if (tid < kProdBase) {
-        // ======================= MMA issuer (one thread) =======================
-        if (tid == kMmaBase) {
-            uint32_t unit = 0, xe = 0;
+        // ======================= MMA issuers (one thread per warpgroup) =======================
+        if (((tid - kMmaBase) & 31) == 0) {
+            const uint32_t g = (uint32_t)(tid - kMmaBase) >> 5;  // serves the units of warpgroup g
+            uint32_t xe = 0;
+            Cyc ab(kNumBuf), turn(kNumWg);
             Walk wk(p, C, c);
+            const uint64_t desc_hi = smem_desc(0, p.lbo);
             while (wk.next_entry()) {
                 const uint32_t KB = wk.KB;
                 const uint32_t xb = xe & 1;
                 guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
                 ++xe;
-                const uint32_t xs_addr = smem_u32(xs + (size_t)xb * p.xbuf_bytes);
-                for (uint32_t cu = wk.u0; cu < wk.u1; ++cu, ++unit) {
-                    const uint32_t kb = cu % KB;
-                    const uint32_t a = unit % kNumA, use = unit / kNumA;
-                    guard.wait_mbar(afull0 + 8 * a, use & 1);
-                    guard.wait_mbar(dempty0 + 8 * a, (use & 1) ^ 1);
-                    tc_fence_after();
+                const uint32_t xs16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4, lbo16 = (uint32_t)p.lbo >> 4;
+                uint32_t kb = wk.u0 % KB;
+                for (uint32_t cu = wk.u0; cu < wk.u1; ++cu) {
+                    if (turn.idx == g) {
+                        const uint32_t a = ab.idx;
+                        guard.wait_mbar(afull0 + 8 * a, ab.ph);
+                        guard.wait_mbar(dempty0 + 8 * a, ab.ph ^ 1);
+                        tc_fence_after();
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        mma_i8_ts(tmem + kColD + 8 * a, tmem + 32 * a + 8 * j,
-                                  smem_desc(xs_addr + (kb * 8 + 2 * j) * p.lbo, p.lbo), j > 0 ? 1u : 0u);
-                    tc_commit(dfull0 + 8 * a);   // accumulators complete -> epilogue
-                    tc_commit(aempty0 + 8 * a);  // A buffer has been read -> next unpack
+                        for (int j = 0; j < 4; ++j)
+                            mma_i8_ts(tmem + kColD + 8 * a, tmem + 32 * a + 8 * j,
+                                      desc_hi | (uint64_t)(xs16 + (kb * 8 + 2 * j) * lbo16), j > 0 ? 1u : 0u);
+                        // accumulators complete -> epilogue; it also means the A buffer has been read, and the same
+                        // warpgroup reuses it only after that epilogue
+                        tc_commit(dfull0 + 8 * a);
+                    }
+                    ab.step();
+                    turn.step();
+                    if (++kb == KB) kb = 0;
                 }
             }
         }
@@ -482,7 +485,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // ======================= activation stager (4 warps) =======================
         // bf16 row -> per 128 columns: e with max|x| / 2^e <= 32639, v = rint(x / 2^e) = 256 hi + lo (both int8),
         // X = sum v.  hi / lo planes go to rows 2t / 2t+1 of every 16-column chunk of the operand.
-        const int st = tid - kStagerBase, lane = st & 31;
+        // 16 threads per (row, block), 8 columns each.
+        const int st = tid - kStagerBase;
+        const int sub = st & 15;
         uint32_t xe = 0;
         Walk wk(p, C, c);
         while (wk.next_entry()) {
@@ -504,68 +509,70 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     bulk_g2s_plain(smem_u32(xraw + (size_t)t * p.kb_max * 256), E.x + (size_t)t * E.K, (uint32_t)E.K * 2u, xraw0);
             }
             guard.wait_mbar(xraw0, xe & 1);
-            // 8 threads per (row, block): 16 columns each
-            const int groups = E.M * (int)KB;
-            for (int gi = st >> 3; gi < ((groups + 15) & ~15); gi += kStagerThreads / 8) {
-                const bool live = gi < groups;
-                const int t = live ? gi / (int)KB : 0, kb = live ? gi % (int)KB : 0;
-                const int sub = st & 7;  // 16-column chunk within the block
-                float v[16];
-                float amax = 0.f;
-                if (live) {
-                    const uint4* src = reinterpret_cast<const uint4*>(xraw + (size_t)t * p.kb_max * 256 + (size_t)kb * 256 + sub * 32);
-                    const uint4 a = src[0], b = src[1];
-                    const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            // 16 threads per 128-column block (8 columns each); the 8 thread groups walk the blocks of a row together
+            for (int t = 0; t < E.M; ++t) {
+                const unsigned char* xrow = xraw + (size_t)t * p.kb_max * 256 + sub * 16;
+                unsigned char* xdst = xs_b + (size_t)(sub >> 1) * p.lbo + (size_t)(2 * t) * 16 + (sub & 1) * 8;
+                for (int kb0 = 0; kb0 < (int)KB; kb0 += kStagerThreads / 16) {
+                    const int kb = kb0 + (st >> 4);
+                    const bool live = kb < (int)KB;
+                    uint4 raw = make_uint4(0, 0, 0, 0);
+                    if (live) raw = *reinterpret_cast<const uint4*>(xrow + (size_t)kb * 256);
+                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+                    // max |x| of the block, on the bit patterns (bf16 magnitudes order like unsigned integers)
+                    uint32_t amax = 0;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        v[2 * i] = __uint_as_float(u[i] << 16);
-                        v[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
-                        amax = fmaxf(amax, fmaxf(fabsf(v[2 * i]), fabsf(v[2 * i + 1])));
+                    for (int i = 0; i < 4; ++i) amax = max(amax, max((u[i] << 16) & 0x7FFFFFFFu, u[i] & 0x7FFF0000u));
+#pragma unroll
+                    for (int o = 8; o > 0; o >>= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                    // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field E -> e = E - 127 - 14, one
+                    // more when the mantissa exceeds 32639/16384 (for bf16: all seven mantissa bits set)
+                    int ef = (int)(amax >> 23);
+                    if (ef < 1 || ef >= 255) ef = 127 + 14;  // zero / subnormal / non-finite block: scale 1
+                    int e = ef - 127 - 14 + (((amax & 0x7FFFFFu) > 0x7EFE00u) ? 1 : 0);
+                    if (e < -126) e = -126;
+                    const float inv = __uint_as_float((uint32_t)(127 - e) << 23);  // 2^-e
+                    // v = rint(x * 2^-e) through the 1.5 * 2^23 trick; v + 128 = 256 * hi + (lo + 128)
+                    uint32_t vb[8];
+                    int sum = 0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float f0 = fmaf(__uint_as_float(u[i] << 16), inv, 12582912.f);
+                        const float f1 = fmaf(__uint_as_float(u[i] & 0xFFFF0000u), inv, 12582912.f);
+                        const int q0 = (int)(__float_as_uint(f0) - 0x4B400000u), q1 = (int)(__float_as_uint(f1) - 0x4B400000u);
+                        sum += q0 + q1;
+                        vb[2 * i] = (uint32_t)(q0 + 128);
+                        vb[2 * i + 1] = (uint32_t)(q1 + 128);
                     }
-                }
-#pragma unroll
-                for (int o = 4; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-                // smallest power of two 2^e with amax / 2^e <= 32639 (amax == 0 or not finite -> scale 1)
-                int e = 0;
-                if (amax > 0.f && amax < 3.0e38f) {
-                    int ex;
-                    const float m = frexpf(amax, &ex);  // amax = m * 2^ex, m in [0.5, 1)
-                    e = ex - 15;                        // amax / 2^e = m * 32768 in [16384, 32768)
-                    if (m * 32768.f > 32639.f) ++e;
-                    if (e < -126) e = -126;             // keeps 2^-e finite for absurdly small blocks
-                }
-                const float inv = exp2f((float)-e);
-                int sum = 0;
-                uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
-                if (live) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int q = __float2int_rn(v[i] * inv);
-                        const int l = ((q + 128) & 0xFF) - 128;
-                        const int h = (q - l) >> 8;
-                        sum += q;
-                        lo[i >> 2] |= (uint32_t)(l & 0xFF) << (8 * (i & 3));
-                        hi[i >> 2] |= (uint32_t)(h & 0xFF) << (8 * (i & 3));
+                    // byte 0 of each (v + 128) is lo + 128, byte 1 is hi
+                    uint2 lo, hi;
+                    lo.x = __byte_perm(__byte_perm(vb[0], vb[1], 0x0040), __byte_perm(vb[2], vb[3], 0x0040), 0x5410) ^ 0x80808080u;
+                    lo.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
+                    hi.x = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
+                    hi.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
+                    if (live) {  // 16-column chunk kb*8 + sub/2; this thread owns its first or second 8 bytes
+                        unsigned char* dst = xdst + (size_t)kb * 8 * p.lbo;
+                        *reinterpret_cast<uint2*>(dst) = hi;
+                        *reinterpret_cast<uint2*>(dst + 16) = lo;
                     }
-                    unsigned char* dst = xs_b + (size_t)(kb * 8 + sub) * p.lbo + (size_t)(2 * t) * 16;
-                    *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<uint4*>(dst + 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                }
 #pragma unroll
-                for (int o = 4; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-                if (live && sub == 0) {
-                    xsum_b[t * p.kb_max + kb] = sum;
-                    xscale_b[t * p.kb_max + kb] = exp2f((float)e);
+                    for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                    if (live && sub == 0) {
+                        xsum_b[t * p.kb_max + kb] = sum;
+                        xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);  // 2^e
+                    }
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read xs through the async proxy
             group_sync<1, kStagerThreads>();
             if (st == 0) mbar_arrive(xfull0 + 8 * xb);
             ++xe;
-            (void)lane;
         }
     } else {
         // ======================= finalizer (4 warps; thread = row of the tile) =======================
+        // Row tiles shared with other CTAs are completed through the workspace: each contributor writes
+        // {value, tag} pairs (one 8-byte store per element, tag = entry index + 1) into a ring of kSlotDepth
+        // slots; the CTA owning the end of the tile polls the pairs, adds them in CTA order and clears the tags.
         const int r = tid - kFinBase;
         Cyc pb(kPartBufs);
         Walk wk(p, C, c);
@@ -573,9 +580,27 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, units = wk.units;
-            bool have_first = false, have_last = false;
-            uint32_t last_rt = 0, n_full = 0;
-            float first_v[kMaxRows] = {0.f, 0.f, 0.f, 0.f}, last_v[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t tag = (uint32_t)wk.ei + 1u, ring_i = (uint32_t)wk.ei % kSlotDepth;
+            // slice geometry: is the last tile cut at its end (this CTA contributes), the first at its beginning
+            // (this CTA completes it)?
+            const bool have_last = (wk.t_last + 1) * KB > u1;
+            const bool have_first = wk.t_first * KB < u0 && (wk.t_first + 1) * KB <= u1;
+            unsigned long long* my_slot = nullptr;
+            if (have_last) {
+                const uint32_t which = (wk.t_last == wk.t_first) ? 0u : 1u;
+                my_slot = reinterpret_cast<unsigned long long*>(p.slots) +
+                          (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems;
+                // the slot must have been consumed (tags cleared) by whoever completed the tile it last served;
+                // checked now, while the warpgroups are still computing
+#pragma unroll
+                for (int t = 0; t < kMaxRows; ++t)
+                    if (t < M) {
+                        const unsigned long long* q = my_slot + t * kUnitRows + r;
+                        guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; });
+                    }
+            }
+            uint32_t n_full = 0;
+            float first_v[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
             for (uint32_t tp = wk.t_first; tp <= wk.t_last; tp += kMaxTiles) {
                 const uint32_t ntiles = min((uint32_t)kMaxTiles, wk.t_last - tp + 1);
                 guard.wait_mbar(pfull0 + 8 * pb.idx, pb.ph);
@@ -588,11 +613,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     for (int t = 0; t < kMaxRows; ++t) {
                         v[t] = 0.f;
                         if (t < XR) {
-                            float* a = buf + ((size_t)(0 * kMaxTiles + tl) * XR + t) * kUnitRows + r;
-                            float* b = buf + ((size_t)(1 * kMaxTiles + tl) * XR + t) * kUnitRows + r;
-                            v[t] = *a + *b;
-                            *a = 0.f;
-                            *b = 0.f;
+#pragma unroll
+                            for (int g = 0; g < kNumWg; ++g) {  // fixed order
+                                float* a = buf + ((size_t)(g * kMaxTiles + tl) * XR + t) * kUnitRows + r;
+                                v[t] += *a;
+                                *a = 0.f;
+                            }
                         }
                     }
                     const int row = (int)rt * kUnitRows + r;
@@ -604,60 +630,46 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                                 if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(v[t]);
                         }
                     } else if (ce) {
-                        have_first = true;
 #pragma unroll
                         for (int t = 0; t < kMaxRows; ++t) first_v[t] = v[t];
-                    } else {
-                        have_last = true;
-                        last_rt = rt;
+                    } else {  // publish this CTA's share: value and tag travel in one store
 #pragma unroll
-                        for (int t = 0; t < kMaxRows; ++t) last_v[t] = v[t];
+                        for (int t = 0; t < kMaxRows; ++t)
+                            if (t < M)
+                                __stcg(my_slot + t * kUnitRows + r,
+                                       ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(v[t]));
                     }
                 }
                 group_sync<2, kFinThreads>();
                 if (r == 0) mbar_arrive(pempty0 + 8 * pb.idx);
                 pb.step();
             }
-            if (r == 0 && n_full && p.tiles_done) {
-                __threadfence();
-                red_release_add(p.tiles_done, n_full);
-            }
-            const uint32_t tag = (uint32_t)wk.ei + 1u;
-            if (have_last) {  // publish this CTA's share of the tile that continues in the next CTA
-                const uint32_t which = (last_rt == wk.t_first) ? 0u : 1u;
-                unsigned char* slot = p.slots + ((size_t)c * 2 + which) * kSlotBytes;
-                unsigned int* flag = reinterpret_cast<unsigned int*>(slot + kSlotFloats * 4);
-                if (r == 0) guard.wait_flag([&] { return ld_acquire(flag) == 0u; });
-                group_sync<2, kFinThreads>();
-#pragma unroll
-                for (int t = 0; t < kMaxRows; ++t)
-                    if (t < M) reinterpret_cast<float*>(slot)[t * kUnitRows + r] = last_v[t];
-                group_sync<2, kFinThreads>();
-                if (r == 0) {
-                    __threadfence();
-                    st_release(flag, tag);
-                }
-            }
             if (have_first) {  // complete the tile whose beginning belongs to earlier CTAs
                 const uint32_t rt = wk.t_first;
                 const uint32_t c_lo = owner_of(rt * KB, units, C);
-                const uint32_t ncontrib = c - c_lo;
-                for (uint32_t i = r; i < ncontrib; i += kFinThreads) {
-                    uint32_t which;
-                    if (!contributor_slot(c_lo + i, rt, units, KB, C, which)) continue;
-                    const unsigned int* flag = reinterpret_cast<const unsigned int*>(
-                        p.slots + ((size_t)(c_lo + i) * 2 + which) * kSlotBytes + kSlotFloats * 4);
-                    guard.wait_flag([&] { return ld_acquire(flag) == tag; });
-                }
-                group_sync<2, kFinThreads>();
                 float sum[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
                 for (uint32_t cc = c_lo; cc < c; ++cc) {
                     uint32_t which;
                     if (!contributor_slot(cc, rt, units, KB, C, which)) continue;
-                    const float* src = reinterpret_cast<const float*>(p.slots + ((size_t)cc * 2 + which) * kSlotBytes);
+                    unsigned long long* src = reinterpret_cast<unsigned long long*>(p.slots) +
+                                              (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + r;
+                    unsigned long long got[kMaxRows] = {0ull, 0ull, 0ull, 0ull};
+                    guard.wait_flag([&] {
+                        bool all = true;
+#pragma unroll
+                        for (int t = 0; t < kMaxRows; ++t)
+                            if (t < M) {
+                                got[t] = __ldcg(src + t * kUnitRows);
+                                all &= (uint32_t)(got[t] >> 32) == tag;
+                            }
+                        return all;
+                    });
 #pragma unroll
                     for (int t = 0; t < kMaxRows; ++t)
-                        if (t < M) sum[t] += __ldcg(src + t * kUnitRows + r);
+                        if (t < M) {
+                            sum[t] += __uint_as_float((uint32_t)got[t]);
+                            __stcg(src + t * kUnitRows, 0ull);  // consumed: the slot may be reused
+                        }
                 }
                 const int row = (int)rt * kUnitRows + r;
                 if (row < N) {
@@ -665,16 +677,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     for (int t = 0; t < kMaxRows; ++t)
                         if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(sum[t] + first_v[t]);
                 }
-                group_sync<2, kFinThreads>();
-                for (uint32_t i = r; i < ncontrib; i += kFinThreads) {
-                    uint32_t which;
-                    if (!contributor_slot(c_lo + i, rt, units, KB, C, which)) continue;
-                    st_release(reinterpret_cast<unsigned int*>(p.slots + ((size_t)(c_lo + i) * 2 + which) * kSlotBytes +
-                                                               kSlotFloats * 4), 0u);
-                }
-                if (r == 0 && p.tiles_done) {
+                ++n_full;
+            }
+            if (n_full && p.tiles_done) {
+                group_sync<2, kFinThreads>();  // every row of the tiles is written
+                if (r == 0) {
                     __threadfence();
-                    red_release_add(p.tiles_done, 1u);
+                    red_release_add(p.tiles_done, n_full);
                 }
             }
         }
@@ -732,7 +741,7 @@ SmemPlan plan_for(int max_m, int kb_max) {
     pl.xbuf_bytes = kb_max * 8 * pl.lbo + 128;  // the last chunk's 8-row window reaches past its own rows
     const size_t fixed = (size_t)2 * pl.xbuf_bytes + (size_t)pl.x_rows * kb_max * 256 + (size_t)2 * 2 * pl.x_rows * kb_max * 4 +
                          (size_t)kPartBufs * kNumWg * kMaxTiles * pl.x_rows * kUnitRows * 4 +
-                         (size_t)(2 * kNumA + 2 * kNumD + 5 + 2 * kPartBufs) * 8 + 16 + 128;
+                         (size_t)(4 * kNumBuf + 5 + 2 * kPartBufs) * 8 + 16 + 128;
     pl.stages = 0;
     if (fixed < kSmemLimit) {
         long s = (long)((kSmemLimit - fixed) / (kUnitBytes + 16));
@@ -752,7 +761,7 @@ bool w4a16_tc_supported(int M, int N, int K, int G) {
 
 size_t w4a16_tc_weight_bytes(int N, int K) { return (size_t)((N + kUnitRows - 1) / kUnitRows) * (K / 128) * kUnitBytes; }
 
-size_t w4a16_tc_workspace() { return (size_t)kWsHeader + (size_t)num_sms() * 2 * kSlotBytes; }
+size_t w4a16_tc_workspace() { return (size_t)kWsHeader + (size_t)num_sms() * 2 * kSlotDepth * kSlotElems * 8; }
 
 qil_status launch_pack_stream128_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K, int G,
                                     void* out, cudaStream_t st) {

@@ -436,9 +436,10 @@ def test_w4a16_tc_shapes(api, M, N, K, G):
     assert _status(api, ws) == 0
     assert_rows_close(bf16_to_f64(outs[0])[:, rows], y_ref)
     np.testing.assert_array_equal(bits_of(outs[0]), bits_of(outs[1]))
+    # every {value, tag} pair handed over between CTAs has been consumed (tags cleared)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    flags = ws[256:256 + sms * 2 * 2064].view(-1, 2064)[:, 2048:]
-    assert int(torch.count_nonzero(flags).item()) == 0
+    pairs = ws[256:256 + sms * 2 * 4 * 512 * 8].view(torch.int32).view(-1, 2)
+    assert int(torch.count_nonzero(pairs[:, 1]).item()) == 0
 
 
 def test_w4a16_tc_wide_dynamic_range(api):

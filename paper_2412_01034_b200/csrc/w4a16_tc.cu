@@ -48,8 +48,8 @@ constexpr int kProdBase = kMmaBase + 32 * kNumWg;  // one MMA-issuing warp per w
 constexpr int kStagerBase = kProdBase + 32;
 constexpr int kFinBase = kStagerBase + kStagerThreads;
 constexpr int kThreads = kFinBase + kFinThreads;
-constexpr int kNumBuf = 2 * kNumWg;  // A buffers (32 columns each) and accumulator buffers (8 columns each)
-constexpr int kTmemCols = 256;       // A at columns [0, 32 kNumBuf), D behind them
+constexpr int kNumBuf = 3 * kNumWg;  // A buffers (32 columns each) and accumulator buffers (8 columns each)
+constexpr int kTmemCols = 512;       // A at columns [0, 32 kNumBuf), D behind them
 constexpr int kColD = 32 * kNumBuf;
 static_assert(kColD + 8 * kNumBuf <= kTmemCols, "tensor memory budget");
 constexpr int kMaxTiles = 2;    // row tiles per pass
@@ -99,7 +99,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 4000;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -175,7 +175,6 @@ struct Guard {
         const unsigned long long t0 = now_ns();
         for (uint32_t i = 1;; ++i) {
             if (mbar_try_wait(bar, parity)) return;
-            __nanosleep(40);  // a waiting warp must not take issue slots from the working ones
             if ((i & 15u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
         }
         fail();
@@ -322,13 +321,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 float* my_part = part + (size_t)pb.idx * part_floats + (size_t)wg * kMaxTiles * XR * kUnitRows + r;
                 float fin[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
                 int cur_tile = -1;
-                // a unit whose MMAs are in flight: its accumulators are read after the next unit of this
-                // warpgroup has been written to tensor memory
-                bool pend = false;
-                uint32_t pend_d = 0, pend_dph = 0, pend_kb = 0;
-                int pend_tl = 0;
-                float pend_s = 0.f;
-                int pend_z = 0;
+                // units whose MMAs are in flight: the accumulators of a unit are read after the next two units of
+                // this warpgroup have been written to tensor memory (the oldest record is pend_*, the newer next_*)
+                int npend = 0;
+                uint32_t pend_d = 0, pend_dph = 0, pend_kb = 0, next_d = 0, next_dph = 0, next_kb = 0;
+                int pend_tl = 0, next_tl = 0;
+                float pend_s = 0.f, next_s = 0.f;
+                int pend_z = 0, next_z = 0;
                 uint32_t d[8];
                 auto epilogue_load = [&]() {   // start reading the accumulators of the pending unit
                     guard.wait_mbar(dfull0 + 8 * pend_d, pend_dph);
@@ -383,7 +382,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                                          : "memory");
                         }
                         const __half2 meta = *reinterpret_cast<const __half2*>(ub + 8192 + 4 * r);
-                        if (pend) epilogue_load();  // overlaps with the stores above
+                        const bool drain = npend == 2;
+                        if (drain) epilogue_load();  // overlaps with the stores above
                         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                         tc_fence_before();
                         __syncwarp();
@@ -391,23 +391,32 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             mbar_arrive(afull0 + 8 * a);
                             mbar_arrive(empty0 + 8 * rs.idx);
                         }
-                        if (pend) epilogue_math();
-                        pend = true;
-                        pend_d = a;
-                        pend_dph = ab.ph;
-                        pend_kb = kb;
-                        pend_tl = (int)tl;
-                        pend_s = __low2float(meta);
-                        pend_z = (int)__high2float(meta);
+                        if (drain) {
+                            epilogue_math();
+                            pend_d = next_d; pend_dph = next_dph; pend_kb = next_kb; pend_tl = next_tl;
+                            pend_s = next_s; pend_z = next_z;
+                            npend = 1;
+                        }
+                        if (npend == 0) {
+                            pend_d = a; pend_dph = ab.ph; pend_kb = kb; pend_tl = (int)tl;
+                            pend_s = __low2float(meta); pend_z = (int)__high2float(meta);
+                        } else {
+                            next_d = a; next_dph = ab.ph; next_kb = kb; next_tl = (int)tl;
+                            next_s = __low2float(meta); next_z = (int)__high2float(meta);
+                        }
+                        ++npend;
                     }
                     rs.step();
                     ab.step();
                     turn.step();
                     if (++kb == KB) { kb = 0; ++tl; }
                 }
-                if (pend) {
+                while (npend > 0) {
                     epilogue_load();
                     epilogue_math();
+                    pend_d = next_d; pend_dph = next_dph; pend_kb = next_kb; pend_tl = next_tl;
+                    pend_s = next_s; pend_z = next_z;
+                    --npend;
                 }
                 if (cur_tile >= 0) {
 #pragma unroll
@@ -485,9 +494,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // ======================= activation stager (4 warps) =======================
         // bf16 row -> per 128 columns: e with max|x| / 2^e <= 32639, v = rint(x / 2^e) = 256 hi + lo (both int8),
         // X = sum v.  hi / lo planes go to rows 2t / 2t+1 of every 16-column chunk of the operand.
-        // 16 threads per (row, block), 8 columns each.
         const int st = tid - kStagerBase;
-        const int sub = st & 15;
         uint32_t xe = 0;
         Walk wk(p, C, c);
         while (wk.next_entry()) {
@@ -509,22 +516,41 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     bulk_g2s_plain(smem_u32(xraw + (size_t)t * p.kb_max * 256), E.x + (size_t)t * E.K, (uint32_t)E.K * 2u, xraw0);
             }
             guard.wait_mbar(xraw0, xe & 1);
-            // 16 threads per 128-column block (8 columns each); the 8 thread groups walk the blocks of a row together
+            // Two passes over the row, 8 columns (one 16-byte piece) per thread and step, no cross-thread
+            // shuffles: pass 1 leaves max|x| of every 128-column block in shared memory (atomicMax on the bit
+            // patterns), pass 2 converts with the block's scale and adds up the integers (atomicAdd).
+            const int pieces = (int)KB * 16;  // 16-byte pieces per row
             for (int t = 0; t < E.M; ++t) {
-                const unsigned char* xrow = xraw + (size_t)t * p.kb_max * 256 + sub * 16;
-                unsigned char* xdst = xs_b + (size_t)(sub >> 1) * p.lbo + (size_t)(2 * t) * 16 + (sub & 1) * 8;
-                for (int kb0 = 0; kb0 < (int)KB; kb0 += kStagerThreads / 16) {
-                    const int kb = kb0 + (st >> 4);
-                    const bool live = kb < (int)KB;
-                    uint4 raw = make_uint4(0, 0, 0, 0);
-                    if (live) raw = *reinterpret_cast<const uint4*>(xrow + (size_t)kb * 256);
+                unsigned int* bmax = reinterpret_cast<unsigned int*>(xscale_b + t * p.kb_max);  // reused as scratch
+                for (int kb = st; kb < (int)KB; kb += kStagerThreads) {
+                    bmax[kb] = 0u;
+                    xsum_b[t * p.kb_max + kb] = 0;
+                }
+            }
+            group_sync<1, kStagerThreads>();
+            for (int t = 0; t < E.M; ++t) {
+                const unsigned char* xrow = xraw + (size_t)t * p.kb_max * 256;
+                unsigned int* bmax = reinterpret_cast<unsigned int*>(xscale_b + t * p.kb_max);
+#pragma unroll 4
+                for (int pc = st; pc < pieces; pc += kStagerThreads) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
                     const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-                    // max |x| of the block, on the bit patterns (bf16 magnitudes order like unsigned integers)
-                    uint32_t amax = 0;
+                    uint32_t amax = 0;  // bf16 magnitudes order like unsigned integers
 #pragma unroll
                     for (int i = 0; i < 4; ++i) amax = max(amax, max((u[i] << 16) & 0x7FFFFFFFu, u[i] & 0x7FFF0000u));
-#pragma unroll
-                    for (int o = 8; o > 0; o >>= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                    atomicMax(bmax + (pc >> 4), amax);
+                }
+            }
+            group_sync<1, kStagerThreads>();
+            for (int t = 0; t < E.M; ++t) {
+                const unsigned char* xrow = xraw + (size_t)t * p.kb_max * 256;
+                const unsigned int* bmax = reinterpret_cast<const unsigned int*>(xscale_b + t * p.kb_max);
+                unsigned char* xdst = xs_b + (size_t)(2 * t) * 16;
+#pragma unroll 4
+                for (int pc = st; pc < pieces; pc += kStagerThreads) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
+                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+                    const uint32_t amax = bmax[pc >> 4];
                     // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field E -> e = E - 127 - 14, one
                     // more when the mantissa exceeds 32639/16384 (for bf16: all seven mantissa bits set)
                     int ef = (int)(amax >> 23);
@@ -550,19 +576,23 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     lo.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
                     hi.x = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
                     hi.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
-                    if (live) {  // 16-column chunk kb*8 + sub/2; this thread owns its first or second 8 bytes
-                        unsigned char* dst = xdst + (size_t)kb * 8 * p.lbo;
-                        *reinterpret_cast<uint2*>(dst) = hi;
-                        *reinterpret_cast<uint2*>(dst + 16) = lo;
-                    }
-#pragma unroll
-                    for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-                    if (live && sub == 0) {
-                        xsum_b[t * p.kb_max + kb] = sum;
-                        xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);  // 2^e
-                    }
+                    // piece pc = 8 columns: 16-column chunk pc/2, first or second half of its 16-byte row
+                    unsigned char* dst = xdst + (size_t)(pc >> 1) * p.lbo + (pc & 1) * 8;
+                    *reinterpret_cast<uint2*>(dst) = hi;
+                    *reinterpret_cast<uint2*>(dst + 16) = lo;
+                    atomicAdd(xsum_b + t * p.kb_max + (pc >> 4), sum);
                 }
             }
+            group_sync<1, kStagerThreads>();
+            for (int t = 0; t < E.M; ++t)  // replace the block maxima by the scales 2^e
+                for (int kb = st; kb < (int)KB; kb += kStagerThreads) {
+                    const uint32_t amax = reinterpret_cast<const unsigned int*>(xscale_b + t * p.kb_max)[kb];
+                    int ef = (int)(amax >> 23);
+                    if (ef < 1 || ef >= 255) ef = 127 + 14;
+                    int e = ef - 127 - 14 + (((amax & 0x7FFFFFu) > 0x7EFE00u) ? 1 : 0);
+                    if (e < -126) e = -126;
+                    xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);
+                }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read xs through the async proxy
             group_sync<1, kStagerThreads>();
             if (st == 0) mbar_arrive(xfull0 + 8 * xb);

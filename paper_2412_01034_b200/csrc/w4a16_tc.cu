@@ -43,8 +43,7 @@ constexpr int kStagerThreads = 128;
 constexpr int kFinThreads = 128;
 // thread ranges: kNumWg unpack/epilogue warpgroups, then the MMA warp, the producer warp, the stager, the finalizer
 constexpr int kMmaBase = kNumWg * kWgThreads;
-constexpr int kProdBase = kMmaBase + 32 * kNumWg;  // one MMA-issuing warp per warpgroup: issue latency, not the
-                                                    // tensor pipe, limits one thread, and issuers do not slow each other
+constexpr int kProdBase = kMmaBase + 32 * kNumWg;  // one MMA-issuing warp per warpgroup
 constexpr int kStagerBase = kProdBase + 32;
 constexpr int kFinBase = kStagerBase + kStagerThreads;
 constexpr int kThreads = kFinBase + kFinThreads;
@@ -105,12 +104,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "r"(bar), "r"(parity)
         : "memory");
     return ok;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
-        : "memory");
 }
 __device__ __forceinline__ void bulk_g2s_plain(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -468,8 +461,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     } else if (tid < kStagerBase) {
         // ======================= producer (one thread) =======================
         if (tid == kProdBase) {
-            uint64_t policy;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
             Cyc rs(p.stages);
             uint32_t issued = 0;
             Walk wk(p, C, c);
@@ -478,8 +469,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 for (uint32_t cu = wk.u0; cu < wk.u1; ++cu, ++issued) {
                     guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1);
                     mbar_expect_tx(full0 + 8 * rs.idx, kUnitBytes);
-                    bulk_g2s(smem_u32(ring + (size_t)rs.idx * kUnitBytes), wbase + (size_t)cu * kUnitBytes, kUnitBytes,
-                             full0 + 8 * rs.idx, policy);
+                    bulk_g2s_plain(smem_u32(ring + (size_t)rs.idx * kUnitBytes), wbase + (size_t)cu * kUnitBytes, kUnitBytes,
+                                   full0 + 8 * rs.idx);
                     rs.step();
                 }
             }

@@ -70,8 +70,8 @@ typedef enum { QIL_F32 = 0, QIL_BF16 = 1, QIL_F16 = 2 } qil_dtype;
  *   built by qil_pack_stream_w4 from codes, scales and zeros.  Unit u =
  *   (n/16)*(K/128) + k/128 occupies bytes [1088 u, 1088 (u+1)): first 1024
  *   bytes of codes, 16 rows x 16 words as in a TILE16 tile, except that inside
- *   each word code k (0..7) sits at nibble (k >> 1) + 4 * (k & 1) (even k in the
- *   low half-word, odd k in the high half-word); then 16 pairs {fp16 scale,
+ *   each word byte b holds code b in its low and code 4 + b in its high nibble
+ *   (code k of the 8 sits at nibble 2 (k % 4) + k / 4); then 16 pairs {fp16 scale,
  *   fp16 zero}, one per row of the tile, valid for that 128-column block (a
  *   group larger than 128 repeats its pair in every block it covers).
  *   Needs N % 16 == 0, K % 128 == 0, group_size % 128 == 0.  With group 128 the
@@ -140,9 +140,9 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  * once, any M handled in slabs of 64 rows) when K % 128 == 0 and
  * group_size % 128 == 0; a general kernel otherwise (any K % 8 == 0, any
  * group_size dividing K, canonical layout only).  With QIL_LAYOUT_STREAM
- * (M <= 8) or QIL_LAYOUT_STREAM128 (M <= 4) a persistent streaming kernel runs;
+ * or QIL_LAYOUT_STREAM128 (both M <= 4) a persistent streaming kernel runs;
  * scales and zeros are part of the buffer, the two arguments are ignored and
- * may be null; the workspace is always needed.  The STREAM128 kernel converts
+ * may be null; the workspace is always needed.  Both streaming kernels convert
  * the activations to 16-bit block fixed point (per 128 columns a power-of-two
  * scale, |integer| <= 32639) and accumulates exactly in int32; the conversion
  * error per element is at most 2^-16 of the block maximum.

@@ -210,7 +210,8 @@ def to_stream(packed: np.ndarray, scales, zeros, group_size: int) -> np.ndarray:
     Unit u = (n // 16) * (K // 128) + kb holds, at byte 1088 * u: the 16 x 16 words of the tile
     (rows n//16*16 .. +15, words 16*kb .. 16*kb+15, row after row, little endian), then for each of
     the 16 rows the fp16 scale followed by the fp16 zero of the group that contains block kb.
-    Inside a word the code of element k (0..7) sits at nibble (k >> 1) + 4 * (k & 1).
+    Inside a word, byte b holds element b in its low and element 4 + b in its high nibble
+    (element k sits at nibble 2 * (k % 4) + k // 4).
     """
     p = np.asarray(packed, dtype=np.uint32)
     N, Wd = p.shape
@@ -228,7 +229,7 @@ def to_stream(packed: np.ndarray, scales, zeros, group_size: int) -> np.ndarray:
             canon = p[rt * 16:rt * 16 + 16, kb * 16:kb * 16 + 16]
             tile = np.zeros_like(canon)
             for k in range(8):
-                tile |= ((canon >> np.uint32(4 * k)) & np.uint32(0xF)) << np.uint32(4 * ((k >> 1) + 4 * (k & 1)))
+                tile |= ((canon >> np.uint32(4 * k)) & np.uint32(0xF)) << np.uint32(4 * (2 * (k % 4) + k // 4))
             out[base:base + 1024] = np.ascontiguousarray(tile).view(np.uint8).reshape(-1)
             meta = np.empty((16, 2), dtype=np.uint16)
             meta[:, 0] = s16[rt * 16:rt * 16 + 16, (kb * 128) // G]

@@ -1,29 +1,37 @@
 // Weight-only 4-bit decode linears as ONE persistent kernel over a list of linears
 // (the memory-bound decode stage of the paper's OpenVLA deployment, Sec. 5.4 /
-// App. A.4.2: q, k, v, o, gate, up, down of every decoder layer, M <= 8 rows).
+// App. A.4.2: q, k, v, o, gate, up, down of every decoder layer, M <= 4 rows).
 //
 // Data layout (QIL_LAYOUT_STREAM): the weight matrix is a sequence of self-contained
 // 1088-byte units, unit u = (row tile rt = u / (K/128), column block kb = u % (K/128)):
 // 1024 bytes of packed codes of 16 output features x 128 input features (16 rows of 64
-// bytes) followed by 16 x {fp16 scale, fp16 zero} of those rows for that block.  Inside
-// each 32-bit word the 8 codes are ordered so that the mask/or unpack below yields
-// bf16 pairs of ADJACENT k (code k at nibble (k>>1) + 4*(k&1)); the activations can then
-// be used exactly as they lie in memory.  A linear is one contiguous byte stream, and
-// any slice of units is too.
+// bytes) followed by 16 x {fp16 scale, fp16 zero} of those rows for that block.  Byte b
+// of 32-bit word m of a row holds column 8m + b in its low and column 8m + 4 + b in its
+// high nibble, so that one AND per word yields four unsigned bytes (the low nibbles as
+// they are, the high nibbles times 16).  A linear is one contiguous byte stream, and any
+// slice of units is too.
+//
+// Arithmetic: integer.  The activations of a linear are converted once to 16-bit block
+// fixed point: per row and 128-column block a power-of-two scale 2^e with
+// |x| / 2^e <= 32639, v = rint(x / 2^e) = 256 hi + lo stored as two int8 planes.  The
+// codes multiply both planes on the tensor cores (mma.sync m16n8k32 u8 x s8 -> s32,
+// exact); the 8 columns of the instruction are {row 0 hi, row 0 lo, row 1 hi, ...}.
+// Scale and zero point are folded once per unit:
+//     y += s 2^e ((256 D_hi + D_lo) - z X),   X = sum of the block's integers v.
+// The only rounding beyond the fp32 accumulation over blocks is that of v (relative
+// 2^-15 of the block maximum), far below the bf16 rounding of the output.
 //
 // Execution: one CTA per SM, alive for the whole list.  For every linear each CTA
 // owns a contiguous slice of its units (balanced to +-1 unit).  A producer thread
 // streams the slice through a shared-memory ring with bulk asynchronous copies
 // (cp.async.bulk + mbarrier transaction counts), running ahead across linears as far
 // as the ring allows, so HBM stays busy while the consumers finish a linear.
-// Sixteen compute warps each take one unit per ring stage: nibbles -> bf16 (128+q)
-// by mask/or, mma.sync m16n8k16 against the activation rows staged in shared memory,
-// scale/zero folded once per unit (y += s*(acc - (128+z)*X), X = block sum of x).
+// Sixteen compute warps each take one unit per ring stage.
 // They never wait for another CTA: per pass they leave per-warp partial tiles in a
 // double-buffered shared array and go on.  A combiner group of four warps adds the
 // partial tiles and writes finished outputs; a fixer warp does all cross-CTA work
-// from a small queue; two stager warps fetch the activations of the next entry
-// (two buffers) and wait for dependencies - all hidden behind the compute warps.
+// from a small queue; four stager warps fetch and convert the activations of the next
+// entry (two buffers) and wait for dependencies - all hidden behind the compute warps.
 // Row tiles cut by a slice boundary are completed through small fp32 slots in the
 // workspace: every CTA first publishes its contribution to the tile it shares with
 // the next CTA, then completes the tile it shares with previous CTAs, adding the
@@ -47,13 +55,14 @@ namespace {
 constexpr int kComputeWarps = 16;
 constexpr int kComputeThreads = kComputeWarps * 32;
 constexpr int kEpiThreads = 128;     // combiner group: 4 warps
-constexpr int kStagerThreads = 64;   // activation stager: 2 warps
+constexpr int kStagerThreads = 128;  // activation stager: 4 warps
 constexpr int kFixDepth = 8;         // records queued between the combiner group and the fixer warp
 constexpr int kThreads = kComputeThreads + kEpiThreads + 32 + kStagerThreads + 32;  // + fixer warp + producer warp
 constexpr int kUnitBytes = 1088;
 constexpr int kStageUnits = kComputeWarps;
 constexpr int kStageBytes = kStageUnits * kUnitBytes;
-constexpr int kElemsMax = 128;  // fp32 values of one row tile: 16 rows x 8 activation rows (32 when M <= 2)
+constexpr int kMaxRows = 4;     // activation rows: two int8 planes each fill the 8 columns of the instruction
+constexpr int kElemsMax = 64;   // fp32 values of one row tile: 16 rows x 4 activation rows (16 when M == 1)
 constexpr int kMaxEntries = 256;
 constexpr int kSlotBytes = kElemsMax * 4 + 16;  // data + flag word (padded)
 constexpr int kWsHeader = 256;
@@ -76,10 +85,10 @@ struct StreamParams {
     int count;
     int stages;
     int x_rows;       // max M over the entries
-    int x_row_bytes;  // max K * 2 + pad
+    int x_row_bytes;  // one int8 plane of a row: max K + pad
     int kb_max;       // max K / 128
-    int elems;        // fp32 values kept per (row tile, warp): 32 if every M <= 2, else 128
-    int max_tiles;    // row tiles per pass: 8 (elems 32) or 2 (elems 128)
+    int elems;        // fp32 values kept per (row tile, warp): 16 if every M == 1, else 64
+    int max_tiles;    // row tiles per pass: 8 (elems 16) or 4 (elems 64)
     int* status;
     unsigned int* tiles_done;
     unsigned char* slots;
@@ -121,12 +130,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait_suspend(uint32_t bar, uint32_t
         : "memory");
     return ok;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
-        : "memory");
-}
 __device__ __forceinline__ void bulk_g2s_plain(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
@@ -146,16 +149,14 @@ __device__ __forceinline__ void red_release_add(unsigned int* p, uint32_t v) {
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 __device__ __forceinline__ void stager_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kStagerThreads) : "memory"); }
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+// D[16 x 8] += A[16 x 32 unsigned bytes] * B[32 x 8 signed bytes], int32 accumulate (exact)
+__device__ __forceinline__ void mma_u8s8_16832(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
         "{%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t nib_pair(uint32_t w, int i) {
-    return ((w >> (4 * i)) & 0x000F000Fu) | 0x43004300u;  // bf16x2 {128 + nibble i, 128 + nibble i+4}
 }
 
 // ---- bounded waits --------------------------------------------------------------------------
@@ -266,12 +267,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
     // ---- carve shared memory ----
     unsigned char* ring = smem;
     float* tile_part = reinterpret_cast<float*>(ring + (size_t)p.stages * kStageBytes);  // [2][max_tiles][16 warps][elems]
-    float* stash_first = tile_part + 2 * part_floats;                                    // [128]
-    float* stash_last = stash_first + kElemsMax;                                         // [128]
+    float* stash_first = tile_part + 2 * part_floats;                                    // [kElemsMax]
+    float* stash_last = stash_first + kElemsMax;                                         // [kElemsMax]
     FixRec* fixq = reinterpret_cast<FixRec*>(stash_last + kElemsMax);                    // [kFixDepth]
-    unsigned char* xs = reinterpret_cast<unsigned char*>(fixq + kFixDepth);              // [2][x_rows][x_row_bytes]
-    float* xsum = reinterpret_cast<float*>(xs + (size_t)2 * p.x_rows * p.x_row_bytes);   // [2][8][kb_max]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(xsum + 2 * 8 * p.kb_max);
+    unsigned char* xs = reinterpret_cast<unsigned char*>(fixq + kFixDepth);  // [2][2 x_rows planes][x_row_bytes]
+    unsigned char* xraw = xs + (size_t)4 * p.x_rows * p.x_row_bytes;         // [x_rows][256 kb_max] bf16 as copied
+    int* xsum = reinterpret_cast<int*>(xraw + (size_t)p.x_rows * p.kb_max * 256);  // [2][kMaxRows][kb_max]
+    float* xscale = reinterpret_cast<float*>(xsum + 2 * kMaxRows * p.kb_max);      // [2][kMaxRows][kb_max]
+    unsigned int* bmax = reinterpret_cast<unsigned int*>(xscale + 2 * kMaxRows * p.kb_max);  // [2][kMaxRows][kb_max]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(bmax + 2 * kMaxRows * p.kb_max);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
     const uint32_t xfull0 = smem_u32(b2);          // [2] activations of an entry are staged
@@ -303,15 +307,20 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < 2 * part_floats; i += kThreads) tile_part[i] = 0.f;
-    for (int i = tid; i < 2 * 8 * p.kb_max; i += kThreads) xsum[i] = 0.f;
+    for (int i = tid; i < 2 * kMaxRows * p.kb_max; i += kThreads) {
+        xsum[i] = 0;
+        xscale[i] = 0.f;
+    }
     __syncthreads();
     const Guard guard{p.status, poisoned};
 
     if (tid < kComputeThreads) {
         // =============================== compute warps ===============================
+        // Lane (g = lane / 4, t = lane % 4) owns weight rows g and g + 8 of the unit and activation row t:
+        // accumulator columns 2t and 2t + 1 are the high- and low-byte planes of activation row t.
         const int lane = tid & 31, warp = tid >> 5;
         const int g = lane >> 2, t = lane & 3;
-        const bool compact = elems == 32;  // M <= 2: only the lanes with t == 0 hold real outputs
+        const bool compact = elems == 16;  // M == 1: only the lanes with t == 0 hold real outputs
         uint32_t item = 0, xe = 0;
         uint32_t rs = 0, rph = 0;  // ring stage and its phase
         Walk wk(p, C, c);
@@ -321,17 +330,19 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
             const uint32_t xb = xe & 1;
             guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
             ++xe;
-            const unsigned char* xs_b = xs + (size_t)xb * p.x_rows * p.x_row_bytes;
-            const float* xsum_b = xsum + (size_t)xb * 8 * p.kb_max;
-            const unsigned char* xlane = xs_b + (size_t)g * p.x_row_bytes + (size_t)t * 64;  // this lane's x columns
-            const float* xsum_lane = xsum_b + (2 * t) * p.kb_max;
+            // B fragments: plane row g (= 2 * activation row + {high, low}), 32 consecutive columns per lane
+            const unsigned char* xlane =
+                xs + ((size_t)xb * 2 * p.x_rows + g) * p.x_row_bytes + (size_t)t * 32;
+            const bool has_b = g < 2 * M;
+            const int* xsum_lane = xsum + ((size_t)xb * kMaxRows + t) * p.kb_max;
+            const float* xscale_lane = xscale + ((size_t)xb * kMaxRows + t) * p.kb_max;
             for (uint32_t tp = wk.t_first; tp <= wk.t_last; tp += max_tiles, ++item) {
                 const uint32_t pu0 = max(wk.u0, tp * KB), pu1 = min(wk.u1, (tp + max_tiles) * KB);
                 const uint32_t ab = item & 1;
                 guard.wait_mbar(accempty0 + 8 * ab, ((item >> 1) & 1) ^ 1);
-                float* part = tile_part + (size_t)ab * part_floats + (size_t)warp * elems + (compact ? g * 4 : lane * 4);
+                float* part = tile_part + (size_t)ab * part_floats + (size_t)warp * elems + (compact ? g * 2 : lane * 2);
                 const bool writer = !compact || t == 0;
-                float fin[4] = {0.f, 0.f, 0.f, 0.f};
+                float fin0 = 0.f, fin1 = 0.f;  // rows g and g + 8, activation row t
                 int cur_tile = -1;
                 // this warp's unit of the first chunk, as (tile within the pass, column block); later chunks advance by 16
                 uint32_t u = pu0 + warp;
@@ -341,40 +352,37 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                     if (cu + warp < pu1) {
                         if ((int)tl != cur_tile) {
                             if (cur_tile >= 0 && writer)
-                                *reinterpret_cast<float4*>(part + (size_t)cur_tile * kComputeWarps * elems) =
-                                    make_float4(fin[0], fin[1], fin[2], fin[3]);
-                            fin[0] = fin[1] = fin[2] = fin[3] = 0.f;
+                                *reinterpret_cast<float2*>(part + (size_t)cur_tile * kComputeWarps * elems) =
+                                    make_float2(fin0, fin1);
+                            fin0 = fin1 = 0.f;
                             cur_tile = (int)tl;
                         }
                         const unsigned char* ub = ring + (size_t)rs * kStageBytes + (size_t)warp * kUnitBytes;
-                        const uint4 wa = *reinterpret_cast<const uint4*>(ub + lane * 16);
-                        const uint4 wb = *reinterpret_cast<const uint4*>(ub + 512 + lane * 16);
+                        const uint4 wa = *reinterpret_cast<const uint4*>(ub + lane * 16);        // row g, columns 32t..
+                        const uint4 wb = *reinterpret_cast<const uint4*>(ub + 512 + lane * 16);  // row g + 8
                         const __half2 ma = *reinterpret_cast<const __half2*>(ub + 1024 + 4 * g);
                         const __half2 mb = *reinterpret_cast<const __half2*>(ub + 1024 + 4 * (g + 8));
-                        float acc[2][4];
-#pragma unroll
-                        for (int j = 0; j < 2; ++j)
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) acc[j][q] = 0.f;
-                        const uint32_t was[4] = {wa.x, wa.y, wa.z, wa.w};
-                        const uint32_t wbs[4] = {wb.x, wb.y, wb.z, wb.w};
-                        const unsigned char* xrow = xlane + (size_t)kb * 256;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint4 b = make_uint4(0, 0, 0, 0);
-                            if (g < M) b = *reinterpret_cast<const uint4*>(xrow + j * 16);
-                            mma_bf16_16816(acc[0], nib_pair(was[j], 0), nib_pair(wbs[j], 0), nib_pair(was[j], 1),
-                                           nib_pair(wbs[j], 1), b.x, b.y);
-                            mma_bf16_16816(acc[1], nib_pair(was[j], 2), nib_pair(wbs[j], 2), nib_pair(was[j], 3),
-                                           nib_pair(wbs[j], 3), b.z, b.w);
+                        uint4 b0 = make_uint4(0, 0, 0, 0), b1 = make_uint4(0, 0, 0, 0);
+                        if (has_b) {
+                            const uint4* xp = reinterpret_cast<const uint4*>(xlane + (size_t)kb * 128);
+                            b0 = xp[0];  // columns 32t + {0-3, 4-7, 8-11, 12-15}
+                            b1 = xp[1];  // columns 32t + 16 + ...
                         }
-                        const float sa = __low2float(ma), za = 128.f + __high2float(ma);
-                        const float sb = __low2float(mb), zb = 128.f + __high2float(mb);
-                        const float x0 = xsum_lane[kb], x1 = xsum_lane[p.kb_max + kb];
-                        fin[0] = fmaf(sa, fmaf(-za, x0, acc[0][0] + acc[1][0]), fin[0]);
-                        fin[1] = fmaf(sa, fmaf(-za, x1, acc[0][1] + acc[1][1]), fin[1]);
-                        fin[2] = fmaf(sb, fmaf(-zb, x0, acc[0][2] + acc[1][2]), fin[2]);
-                        fin[3] = fmaf(sb, fmaf(-zb, x1, acc[0][3] + acc[1][3]), fin[3]);
+                        // word j of the lane: low nibbles = columns 8j..8j+3, high nibbles = columns 8j+4..8j+7.
+                        // Low nibbles accumulate as they are, high nibbles times 16 in an accumulator of their own.
+                        constexpr uint32_t kLo = 0x0F0F0F0Fu, kHi = 0xF0F0F0F0u;
+                        int lo[4] = {0, 0, 0, 0}, hi[4] = {0, 0, 0, 0};
+                        mma_u8s8_16832(lo, wa.x & kLo, wb.x & kLo, wa.y & kLo, wb.y & kLo, b0.x, b0.z);
+                        mma_u8s8_16832(hi, wa.x & kHi, wb.x & kHi, wa.y & kHi, wb.y & kHi, b0.y, b0.w);
+                        mma_u8s8_16832(lo, wa.z & kLo, wb.z & kLo, wa.w & kLo, wb.w & kLo, b1.x, b1.z);
+                        mma_u8s8_16832(hi, wa.z & kHi, wb.z & kHi, wa.w & kHi, wb.w & kHi, b1.y, b1.w);
+                        // 256 D_hi + D_lo of rows g and g + 8 (the high-nibble sums are exact multiples of 16)
+                        const int va = (lo[0] * 256 + lo[1]) + ((hi[0] * 256 + hi[1]) >> 4);
+                        const int vb = (lo[2] * 256 + lo[3]) + ((hi[2] * 256 + hi[3]) >> 4);
+                        const float xsf = (float)xsum_lane[kb];
+                        const float sc = xscale_lane[kb];
+                        fin0 = fmaf(__low2float(ma) * sc, fmaf(-__high2float(ma), xsf, (float)va), fin0);
+                        fin1 = fmaf(__low2float(mb) * sc, fmaf(-__high2float(mb), xsf, (float)vb), fin1);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty0 + 8 * rs);
@@ -383,8 +391,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                     while (kb >= KB) { kb -= KB; ++tl; }
                 }
                 if (cur_tile >= 0 && writer)
-                    *reinterpret_cast<float4*>(part + (size_t)cur_tile * kComputeWarps * elems) =
-                        make_float4(fin[0], fin[1], fin[2], fin[3]);
+                    *reinterpret_cast<float2*>(part + (size_t)cur_tile * kComputeWarps * elems) = make_float2(fin0, fin1);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(accfull0 + 8 * ab);
             }
@@ -396,13 +403,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
         uint32_t item = 0, fq = 0;
         // element index -> (row within the tile, activation row)
         auto decode = [&](int e, int& row, int& tok) {
-            if (elems == 32) {
-                row = (e >> 2) + ((e & 2) ? 8 : 0);
-                tok = e & 1;
-            } else {
-                const int ln = e >> 2, q = e & 3;
-                row = (ln >> 2) + ((q & 2) ? 8 : 0);
-                tok = 2 * (ln & 3) + (q & 1);
+            if (elems == 16) {  // e = 2 g + h
+                row = (e >> 1) + ((e & 1) ? 8 : 0);
+                tok = 0;
+            } else {            // e = 2 lane + h, lane = 4 g + t
+                row = (e >> 3) + ((e & 1) ? 8 : 0);
+                tok = (e >> 1) & 3;
             }
         };
         // hand one record to the fixer warp
@@ -516,13 +522,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                     }
                     sum += r.data[e];
                     int row, tok;
-                    if (elems == 32) {
-                        row = (e >> 2) + ((e & 2) ? 8 : 0);
-                        tok = e & 1;
+                    if (elems == 16) {
+                        row = (e >> 1) + ((e & 1) ? 8 : 0);
+                        tok = 0;
                     } else {
-                        const int ln = e >> 2, qq = e & 3;
-                        row = (ln >> 2) + ((qq & 2) ? 8 : 0);
-                        tok = 2 * (ln & 3) + (qq & 1);
+                        row = (e >> 3) + ((e & 1) ? 8 : 0);
+                        tok = (e >> 1) & 3;
                     }
                     if (tok < E.M) E.y[(size_t)tok * E.N + rt * 16 + row] = __float2bfloat16_rn(sum);
                 }
@@ -542,17 +547,25 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
             if (lane == 0) mbar_arrive(fqempty0 + 8 * q);
         }
     } else if (tid < kComputeThreads + kEpiThreads + 32 + kStagerThreads) {
-        // =============================== activation stager (2 warps) ===============================
-        // The rows of x are copied as they are (one bulk copy per row); only the 128-column block sums are computed.
-        const int st = tid - (kComputeThreads + kEpiThreads + 32);  // 0..63
+        // =============================== activation stager (4 warps) ===============================
+        // The rows of x arrive by bulk copy as they are; two passes over them, 8 columns (one 16-byte piece) per
+        // thread and step, without cross-thread shuffles: pass 1 leaves max|x| of every 128-column block in
+        // shared memory (atomicMax on the bit patterns), pass 2 converts with the block's scale, writes the two
+        // int8 planes and adds up the integers of the block (atomicAdd).
+        const int st = tid - (kComputeThreads + kEpiThreads + 32);  // 0..127
+        for (int i = st; i < 2 * kMaxRows * p.kb_max; i += kStagerThreads) bmax[i] = 0u;
+        stager_sync();
         uint32_t xe = 0;
         Walk wk(p, C, c);
         while (wk.next_entry()) {
             const StreamEntry& E = p.e[wk.ei];
             const uint32_t KB = wk.KB;
             const uint32_t xb = xe & 1;
-            unsigned char* xs_b = xs + (size_t)xb * p.x_rows * p.x_row_bytes;
-            float* xsum_b = xsum + (size_t)xb * 8 * p.kb_max;
+            unsigned char* xs_b = xs + (size_t)xb * 2 * p.x_rows * p.x_row_bytes;
+            int* xsum_b = xsum + (size_t)xb * kMaxRows * p.kb_max;
+            float* xscale_b = xscale + (size_t)xb * kMaxRows * p.kb_max;
+            unsigned int* bmax_b = bmax + (size_t)xb * kMaxRows * p.kb_max;
+            unsigned int* bmax_next = bmax + (size_t)(xb ^ 1) * kMaxRows * p.kb_max;
             if (st == 0) {
                 guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1);
                 if (E.flags & kFlagDep) {  // the input is written by earlier entries: wait until all their tiles are out
@@ -560,27 +573,68 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                     guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; });
                     asm volatile("fence.proxy.async;" ::: "memory");  // the copies below read what that acquire ordered
                 }
-                mbar_expect_tx(xraw0 + 8 * xb, (uint32_t)E.M * (uint32_t)E.K * 2u);
+                mbar_expect_tx(xraw0, (uint32_t)E.M * (uint32_t)E.K * 2u);
                 for (int r = 0; r < E.M; ++r)
-                    bulk_g2s_plain(smem_u32(xs_b + (size_t)r * p.x_row_bytes), E.x + (size_t)r * E.K, (uint32_t)E.K * 2u,
-                                   xraw0 + 8 * xb);
+                    bulk_g2s_plain(smem_u32(xraw + (size_t)r * p.kb_max * 256), E.x + (size_t)r * E.K, (uint32_t)E.K * 2u,
+                                   xraw0);
             }
-            guard.wait_mbar(xraw0 + 8 * xb, (xe >> 1) & 1);
-            // block sums of the real rows: one thread per (row, 128-column block).  Rows >= M keep whatever
-            // they held: they only reach accumulators of activation rows that are never stored.
-            for (int r = 0; r < E.M; ++r)
-                for (int kb = st; kb < (int)KB; kb += kStagerThreads) {
-                    const uint4* src = reinterpret_cast<const uint4*>(xs_b + (size_t)r * p.x_row_bytes + (size_t)kb * 256);
-                    float s = 0.f;
+            guard.wait_mbar(xraw0, xe & 1);  // (the copies were issued after the compute warps released buffer xb)
+            const int pieces = (int)KB * 16;  // 16-byte pieces per row
+            for (int r = 0; r < E.M; ++r) {
+                const unsigned char* xrow = xraw + (size_t)r * p.kb_max * 256;
+                for (int kb = st; kb < (int)KB; kb += kStagerThreads) xsum_b[r * p.kb_max + kb] = 0;
 #pragma unroll 4
-                    for (int j = 0; j < 16; ++j) {
-                        const uint4 v = src[j];
-                        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+                for (int pc = st; pc < pieces; pc += kStagerThreads) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
+                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+                    uint32_t amax = 0;  // bf16 magnitudes order like unsigned integers
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) s += __uint_as_float(u[q] << 16) + __uint_as_float(u[q] & 0xFFFF0000u);
-                    }
-                    xsum_b[r * p.kb_max + kb] = s;
+                    for (int i = 0; i < 4; ++i) amax = max(amax, max((u[i] << 16) & 0x7FFFFFFFu, u[i] & 0x7FFF0000u));
+                    atomicMax(bmax_b + r * p.kb_max + (pc >> 4), amax);
                 }
+            }
+            stager_sync();
+            for (int r = 0; r < E.M; ++r) {
+                const unsigned char* xrow = xraw + (size_t)r * p.kb_max * 256;
+                unsigned char* dst_hi = xs_b + (size_t)(2 * r) * p.x_row_bytes;
+                unsigned char* dst_lo = dst_hi + p.x_row_bytes;
+#pragma unroll 2
+                for (int pc = st; pc < pieces; pc += kStagerThreads) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
+                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+                    const uint32_t amax = bmax_b[r * p.kb_max + (pc >> 4)];
+                    // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field F -> e = F - 127 - 14, one
+                    // more when the mantissa exceeds 32639/16384 (for bf16: all seven mantissa bits set)
+                    int ef = (int)(amax >> 23);
+                    if (ef < 1 || ef >= 255) ef = 127 + 14;  // zero / subnormal / non-finite block: scale 1
+                    int e = ef - 127 - 14 + (((amax & 0x7FFFFFu) > 0x7EFE00u) ? 1 : 0);
+                    if (e < -126) e = -126;
+                    const float inv = __uint_as_float((uint32_t)(127 - e) << 23);  // 2^-e
+                    // v = rint(x * 2^-e) through the 1.5 * 2^23 trick; v + 128 = 256 * hi + (lo + 128)
+                    uint32_t vb[8];
+                    int sum = 0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float f0 = fmaf(__uint_as_float(u[i] << 16), inv, 12582912.f);
+                        const float f1 = fmaf(__uint_as_float(u[i] & 0xFFFF0000u), inv, 12582912.f);
+                        const int q0 = (int)(__float_as_uint(f0) - 0x4B400000u), q1 = (int)(__float_as_uint(f1) - 0x4B400000u);
+                        sum += q0 + q1;
+                        vb[2 * i] = (uint32_t)(q0 + 128);
+                        vb[2 * i + 1] = (uint32_t)(q1 + 128);
+                    }
+                    // byte 0 of each (v + 128) is lo + 128, byte 1 is hi
+                    uint2 lo, hi;
+                    lo.x = __byte_perm(__byte_perm(vb[0], vb[1], 0x0040), __byte_perm(vb[2], vb[3], 0x0040), 0x5410) ^ 0x80808080u;
+                    lo.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
+                    hi.x = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
+                    hi.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
+                    *reinterpret_cast<uint2*>(dst_hi + (size_t)pc * 8) = hi;
+                    *reinterpret_cast<uint2*>(dst_lo + (size_t)pc * 8) = lo;
+                    atomicAdd(xsum_b + r * p.kb_max + (pc >> 4), sum);
+                    if ((pc & 15) == 0) xscale_b[r * p.kb_max + (pc >> 4)] = __uint_as_float((uint32_t)(127 + e) << 23);
+                }
+            }
+            for (int i = st; i < kMaxRows * p.kb_max; i += kStagerThreads) bmax_next[i] = 0u;  // for the next entry
             stager_sync();
             if (st == 0) mbar_arrive(xfull0 + 8 * xb);
             ++xe;
@@ -588,8 +642,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
     } else {
         // =============================== producer (one thread) ===============================
         if (tid == kThreads - 32) {
-            uint64_t policy;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
             uint32_t s = 0, ph = 0, issued = 0;
             Walk wk(p, C, c);
             while (wk.next_entry()) {
@@ -600,8 +652,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                         const uint32_t n = min((uint32_t)kStageUnits, pu1 - cu);
                         guard.wait_mbar(empty0 + 8 * s, ph ^ 1);
                         mbar_expect_tx(full0 + 8 * s, n * kUnitBytes);
-                        bulk_g2s(smem_u32(ring + (size_t)s * kStageBytes), wbase + (size_t)cu * kUnitBytes, n * kUnitBytes,
-                                 full0 + 8 * s, policy);
+                        bulk_g2s_plain(smem_u32(ring + (size_t)s * kStageBytes), wbase + (size_t)cu * kUnitBytes,
+                                       n * kUnitBytes, full0 + 8 * s);
                         if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
                     }
                 }
@@ -634,11 +686,8 @@ __global__ void __launch_bounds__(256) pack_stream_kernel(const uint8_t* __restr
         if (w < 256) {
             const int row = w >> 4, wi = w & 15;
             const uint2 cc = *reinterpret_cast<const uint2*>(codes + (size_t)(rt * 16 + row) * K + (size_t)kb * 128 + wi * 8);
-            // code k of the 8 sits at nibble (k >> 1) + 4 * (k & 1): even k in the low half, odd k in the high half
-            const uint32_t c8[8] = {cc.x & 0xFu, (cc.x >> 8) & 0xFu, (cc.x >> 16) & 0xFu, (cc.x >> 24) & 0xFu,
-                                    cc.y & 0xFu, (cc.y >> 8) & 0xFu, (cc.y >> 16) & 0xFu, (cc.y >> 24) & 0xFu};
-#pragma unroll
-            for (int k = 0; k < 8; ++k) word |= c8[k] << (4 * ((k >> 1) + 4 * (k & 1)));
+            // byte b of the word: column b in the low nibble, column 4 + b in the high nibble
+            word = (cc.x & 0x0F0F0F0Fu) | ((cc.y & 0x0F0F0F0Fu) << 4);
         } else {
             const size_t gi = (size_t)(rt * 16 + (w - 256)) * ng + kb / bpg;
             word = (uint32_t)scales[gi] | ((uint32_t)zeros[gi] << 16);
@@ -647,13 +696,13 @@ __global__ void __launch_bounds__(256) pack_stream_kernel(const uint8_t* __restr
     }
 }
 
-inline int elems_for(int x_rows) { return x_rows <= 2 ? 32 : 128; }
-inline int max_tiles_for(int x_rows) { return x_rows <= 2 ? 8 : 2; }
+inline int elems_for(int x_rows) { return x_rows == 1 ? 16 : 64; }
+inline int max_tiles_for(int x_rows) { return x_rows == 1 ? 8 : 4; }
 
 size_t smem_fixed_bytes(int x_rows, int x_row_bytes, int kb_max) {
     return (size_t)2 * max_tiles_for(x_rows) * kComputeWarps * elems_for(x_rows) * 4 + 2 * kElemsMax * 4 +
-           (size_t)kFixDepth * (16 + kElemsMax * 4) + (size_t)2 * x_rows * x_row_bytes + (size_t)2 * 8 * kb_max * 4 +
-           (10 + 2 * kFixDepth) * 8 + 64 /* flag + slack */;
+           (size_t)kFixDepth * (16 + kElemsMax * 4) + (size_t)4 * x_rows * x_row_bytes + (size_t)x_rows * kb_max * 256 +
+           (size_t)6 * kMaxRows * kb_max * 4 + (10 + 2 * kFixDepth) * 8 + 64 /* flag + slack */;
 }
 
 constexpr size_t kSmemLimit = 232448;  // 227 KiB per CTA
@@ -669,8 +718,8 @@ int stages_for(int x_rows, int x_row_bytes, int kb_max) {
 }  // namespace
 
 bool w4a16_stream_supported(int M, int N, int K, int G) {
-    if (M < 1 || M > 8 || N < 16 || N % 16 != 0 || K % 128 != 0 || G % 128 != 0) return false;
-    return stages_for(M, 2 * K + kRowPad, K / 128) >= 3;
+    if (M < 1 || M > kMaxRows || N < 16 || N % 16 != 0 || K % 128 != 0 || G % 128 != 0) return false;
+    return stages_for(M, K + kRowPad, K / 128) >= 3;
 }
 
 size_t w4a16_stream_weight_bytes(int N, int K) { return (size_t)(N / 16) * (K / 128) * kUnitBytes; }
@@ -722,7 +771,7 @@ qil_status launch_w4a16_stream(const qil_linear_desc* entries, int count, void* 
         }
         p.count = n;
         p.x_rows = x_rows;
-        p.x_row_bytes = 2 * kmax + kRowPad;
+        p.x_row_bytes = kmax + kRowPad;
         p.kb_max = kmax / 128;
         p.stages = stages_for(p.x_rows, p.x_row_bytes, p.kb_max);
         if (p.stages < 3) return QIL_ERR_UNSUPPORTED;

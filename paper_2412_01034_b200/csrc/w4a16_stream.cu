@@ -26,18 +26,21 @@
 // streams the slice through a shared-memory ring with bulk asynchronous copies
 // (cp.async.bulk + mbarrier transaction counts), running ahead across linears as far
 // as the ring allows, so HBM stays busy while the consumers finish a linear.
-// Sixteen compute warps each take one unit per ring stage.
+// Twenty-four compute warps (six per scheduler, to cover the latency of the dependent
+// instruction chains) each take one unit per ring stage.
 // They never wait for another CTA: per pass they leave per-warp partial tiles in a
-// double-buffered shared array and go on.  A combiner group of four warps adds the
-// partial tiles and writes finished outputs; a fixer warp does all cross-CTA work
-// from a small queue; four stager warps fetch and convert the activations of the next
+// double-buffered shared array and go on.  A combiner group of two warps adds the
+// partial tiles and writes finished outputs; two fixer warps do all cross-CTA work
+// from small queues; three stager warps fetch and convert the activations of the next
 // entry (two buffers) and wait for dependencies - all hidden behind the compute warps.
-// Row tiles cut by a slice boundary are completed through small fp32 slots in the
-// workspace: every CTA first publishes its contribution to the tile it shares with
-// the next CTA, then completes the tile it shares with previous CTAs, adding the
-// contributions in CTA order - so results do not depend on timing.  A slot's flag
-// carries the index of the entry it was filled for (0 = free), because the CTA that
-// completes a tile differs from entry to entry.  An entry flagged
+// Row tiles cut by a slice boundary are completed through small slots in the
+// workspace: every CTA publishes its contribution to the tile it shares with the next
+// CTA and completes the tile it shares with previous CTAs, adding the contributions in
+// CTA order - so results do not depend on timing.  A slot is a set of {fp32 value, tag}
+// pairs written with one 8-byte store each; the tag is the index of the entry the value
+// belongs to (0 = free), because the CTA that completes a tile differs from entry to
+// entry; slots form a ring over entries so that neighbouring CTAs need not run in
+// lockstep.  An entry flagged
 // QIL_DEP_PREVIOUS first waits until every row tile of all earlier entries is
 // written (a monotonic counter in the workspace).
 //
@@ -52,19 +55,22 @@ namespace qil {
 
 namespace {
 
-constexpr int kComputeWarps = 16;
+constexpr int kComputeWarps = 24;
 constexpr int kComputeThreads = kComputeWarps * 32;
-constexpr int kEpiThreads = 128;     // combiner group: 4 warps
-constexpr int kStagerThreads = 128;  // activation stager: 4 warps
-constexpr int kFixDepth = 8;         // records queued between the combiner group and the fixer warp
-constexpr int kThreads = kComputeThreads + kEpiThreads + 32 + kStagerThreads + 32;  // + fixer warp + producer warp
+constexpr int kEpiThreads = 64;      // combiner group: 2 warps
+constexpr int kStagerThreads = 96;   // activation stager: 3 warps
+constexpr int kFixDepth = 4;         // records queued between the combiner group and each of the two fixer warps
+constexpr int kFixThreads = 64;      // two fixer warps: one publishes contributions, one completes shared tiles
+constexpr int kThreads = kComputeThreads + kEpiThreads + kFixThreads + kStagerThreads + 32;  // + producer warp
+static_assert(kThreads <= 1024, "block size");
 constexpr int kUnitBytes = 1088;
 constexpr int kStageUnits = kComputeWarps;
 constexpr int kStageBytes = kStageUnits * kUnitBytes;
 constexpr int kMaxRows = 4;     // activation rows: two int8 planes each fill the 8 columns of the instruction
 constexpr int kElemsMax = 64;   // fp32 values of one row tile: 16 rows x 4 activation rows (16 when M == 1)
 constexpr int kMaxEntries = 256;
-constexpr int kSlotBytes = kElemsMax * 4 + 16;  // data + flag word (padded)
+constexpr int kSlotDepth = 4;   // ring of slots per (CTA, first / last tile of its slice), indexed by entry % depth
+constexpr int kSlotBytes = kElemsMax * 8;  // {fp32 value, tag} pairs, one 8-byte store each
 constexpr int kWsHeader = 256;
 constexpr int kRowPad = 16;
 constexpr int kFlagDep = 1;      // StreamEntry::flags: wait for all earlier entries
@@ -139,9 +145,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const unsigned int* p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
-}
-__device__ __forceinline__ void st_release(unsigned int* p, uint32_t v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void red_release_add(unsigned int* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -266,11 +269,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
 
     // ---- carve shared memory ----
     unsigned char* ring = smem;
-    float* tile_part = reinterpret_cast<float*>(ring + (size_t)p.stages * kStageBytes);  // [2][max_tiles][16 warps][elems]
+    float* tile_part = reinterpret_cast<float*>(ring + (size_t)p.stages * kStageBytes);  // [2][max_tiles][compute warps][elems]
     float* stash_first = tile_part + 2 * part_floats;                                    // [kElemsMax]
     float* stash_last = stash_first + kElemsMax;                                         // [kElemsMax]
-    FixRec* fixq = reinterpret_cast<FixRec*>(stash_last + kElemsMax);                    // [kFixDepth]
-    unsigned char* xs = reinterpret_cast<unsigned char*>(fixq + kFixDepth);  // [2][2 x_rows planes][x_row_bytes]
+    FixRec* fixq = reinterpret_cast<FixRec*>(stash_last + kElemsMax);                    // [2 queues][kFixDepth]
+    unsigned char* xs = reinterpret_cast<unsigned char*>(fixq + 2 * kFixDepth);  // [2][2 x_rows planes][x_row_bytes]
     unsigned char* xraw = xs + (size_t)4 * p.x_rows * p.x_row_bytes;         // [x_rows][256 kb_max] bf16 as copied
     int* xsum = reinterpret_cast<int*>(xraw + (size_t)p.x_rows * p.kb_max * 256);  // [2][kMaxRows][kb_max]
     float* xscale = reinterpret_cast<float*>(xsum + 2 * kMaxRows * p.kb_max);      // [2][kMaxRows][kb_max]
@@ -282,10 +285,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
     const uint32_t xempty0 = smem_u32(b2 + 2);     // [2] the compute warps are done with them
     const uint32_t accfull0 = smem_u32(b2 + 4);    // [2] all compute warps left their partial tiles
     const uint32_t accempty0 = smem_u32(b2 + 6);   // [2] the combiner is done with the buffer
-    const uint32_t fqfull0 = smem_u32(b2 + 8);     // [kFixDepth] a record is ready for the fixer
-    const uint32_t fqempty0 = smem_u32(b2 + 8 + kFixDepth);  // [kFixDepth] the fixer has consumed it
-    const uint32_t xraw0 = smem_u32(b2 + 8 + 2 * kFixDepth);  // [2] the bulk copies of the rows of x have landed
-    volatile int* poisoned = reinterpret_cast<volatile int*>(b2 + 10 + 2 * kFixDepth);
+    const uint32_t fqfull0 = smem_u32(b2 + 8);     // [2][kFixDepth] a record is ready for its fixer warp
+    const uint32_t fqempty0 = smem_u32(b2 + 8 + 2 * kFixDepth);  // [2][kFixDepth] the fixer warp has consumed it
+    const uint32_t xraw0 = smem_u32(b2 + 8 + 4 * kFixDepth);  // [2] the bulk copies of the rows of x have landed
+    volatile int* poisoned = reinterpret_cast<volatile int*>(b2 + 10 + 4 * kFixDepth);
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -299,7 +302,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
             mbar_init(accempty0 + 8 * b, 1);
             mbar_init(xraw0 + 8 * b, 1);
         }
-        for (int q = 0; q < kFixDepth; ++q) {
+        for (int q = 0; q < 2 * kFixDepth; ++q) {
             mbar_init(fqfull0 + 8 * q, 1);
             mbar_init(fqempty0 + 8 * q, 1);
         }
@@ -344,7 +347,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                 const bool writer = !compact || t == 0;
                 float fin0 = 0.f, fin1 = 0.f;  // rows g and g + 8, activation row t
                 int cur_tile = -1;
-                // this warp's unit of the first chunk, as (tile within the pass, column block); later chunks advance by 16
+                // this warp's unit of the first chunk, as (tile within the pass, column block); later chunks advance by one stage
                 uint32_t u = pu0 + warp;
                 uint32_t tl = u / KB - tp, kb = u % KB;
                 for (uint32_t cu = pu0; cu < pu1; cu += kStageUnits) {
@@ -398,9 +401,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
             if (lane == 0) mbar_arrive(xempty0 + 8 * xb);  // (ordered after this warp's reads by the __syncwarp above)
         }
     } else if (tid < kComputeThreads + kEpiThreads) {
-        // =============================== combiner group (4 warps) ===============================
-        const int et = tid - kComputeThreads;  // 0..127
-        uint32_t item = 0, fq = 0;
+        // =============================== combiner group (2 warps) ===============================
+        const int et = tid - kComputeThreads;  // 0..kEpiThreads-1
+        uint32_t item = 0, fq[2] = {0, 0};
         // element index -> (row within the tile, activation row)
         auto decode = [&](int e, int& row, int& tok) {
             if (elems == 16) {  // e = 2 g + h
@@ -411,9 +414,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                 tok = (e >> 1) & 3;
             }
         };
-        // hand one record to the fixer warp
-        auto push = [&](int type, int ei, uint32_t arg, const float* data) {
-            const uint32_t q = fq % kFixDepth, round = fq / kFixDepth;
+        // hand one record to fixer warp `which_q` (0: contributions, 1: completions)
+        auto push = [&](int which_q, int type, int ei, uint32_t arg, const float* data) {
+            const uint32_t q = which_q * kFixDepth + fq[which_q] % kFixDepth, round = fq[which_q] / kFixDepth;
             if (et == 0) guard.wait_mbar(fqempty0 + 8 * q, (round & 1) ^ 1);
             epi_sync();
             FixRec& r = fixq[q];
@@ -421,7 +424,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
             if (data != nullptr && et < elems) r.data[et] = data[et];
             epi_sync();
             if (et == 0) mbar_arrive(fqfull0 + 8 * q);
-            ++fq;
+            ++fq[which_q];
         };
 
         Walk wk(p, C, c);
@@ -443,7 +446,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                     else if (ce) have_first = true;
                     else { have_last = true; last_rt = rt; }
                 }
-                // combine the 16 warps in a fixed order, clear the buffer, route every tile
+                // combine the compute warps in a fixed order, clear the buffer, route every tile
                 for (int idx = et; idx < (int)ntiles * elems; idx += kEpiThreads) {
                     const uint32_t tl = idx / elems;
                     const int e = idx % elems;
@@ -474,51 +477,52 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                 red_release_add(p.tiles_done, n_full);
             }
             // cross-CTA work of this entry, in the order that cannot chain CTAs: publish first, complete second
-            if (have_last) push(kRecContrib, wk.ei, (last_rt == wk.t_first) ? 0u : 1u, stash_last);
-            if (have_first) push(kRecFinish, wk.ei, wk.t_first, stash_first);
+            if (have_last) push(0, kRecContrib, wk.ei, (last_rt == wk.t_first) ? 0u : 1u, stash_last);
+            if (have_first) push(1, kRecFinish, wk.ei, wk.t_first, stash_first);
         }
-        push(kRecEnd, 0, 0, nullptr);
-    } else if (tid < kComputeThreads + kEpiThreads + 32) {
-        // =============================== fixer warp ===============================
+        push(0, kRecEnd, 0, 0, nullptr);
+        push(1, kRecEnd, 0, 0, nullptr);
+    } else if (tid < kComputeThreads + kEpiThreads + kFixThreads) {
+        // =============================== fixer warps ===============================
+        // Warp 0 publishes this CTA's contributions to row tiles that continue in the next CTA, warp 1 completes
+        // the tile at the start of the slice from the contributions of earlier CTAs.  A contribution is a set of
+        // {value, tag} pairs (one 8-byte store per element, tag = entry index + 1) in slot entry % kSlotDepth of
+        // the publishing CTA; the completing CTA polls the pairs, adds them in CTA order and clears them, which
+        // frees the slot.  Neither warp is ever waited for by the compute warps.
         const int lane = tid & 31;
+        const int fw = (tid - (kComputeThreads + kEpiThreads)) >> 5;  // 0: contributions, 1: completions
+        unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
         for (uint32_t fq = 0;; ++fq) {
-            const uint32_t q = fq % kFixDepth, round = fq / kFixDepth;
+            const uint32_t q = fw * kFixDepth + fq % kFixDepth, round = fq / kFixDepth;
             guard.wait_mbar(fqfull0 + 8 * q, round & 1);
             const FixRec& r = fixq[q];
             const int type = r.type;
             if (*poisoned || type == kRecEnd) break;
+            const uint32_t tag = (uint32_t)r.ei + 1u, ring_i = (uint32_t)r.ei % kSlotDepth;
             if (type == kRecContrib) {
-                unsigned char* slot = p.slots + ((size_t)c * 2 + r.arg) * kSlotBytes;
-                unsigned int* flag = reinterpret_cast<unsigned int*>(slot + kElemsMax * 4);
-                if (lane == 0) guard.wait_flag([&] { return ld_acquire(flag) == 0u; });
-                __syncwarp();
-                for (int e = lane; e < elems; e += 32) reinterpret_cast<float*>(slot)[e] = r.data[e];
-                __syncwarp();
-                if (lane == 0) {
-                    __threadfence();
-                    st_release(flag, (uint32_t)r.ei + 1u);  // the tag names the entry the data belongs to
+                unsigned long long* slot = slots + (((size_t)c * 2 + r.arg) * kSlotDepth + ring_i) * kElemsMax;
+                for (int e = lane; e < elems; e += 32) {
+                    // the slot last served entry ei - kSlotDepth: whoever completed that tile has cleared it
+                    guard.wait_flag([&] { return __ldcg(slot + e) == 0ull; });
+                    __stcg(slot + e, ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(r.data[e]));
                 }
-            } else {  // kRecFinish: complete the first tile of the slice from the contributions of earlier CTAs
+            } else {  // kRecFinish
                 const StreamEntry& E = p.e[r.ei];
                 const uint32_t KB = (uint32_t)E.K >> 7, units = ((uint32_t)E.N >> 4) * KB;
                 const uint32_t rt = r.arg;
                 const uint32_t c_lo = owner_of(rt * KB, units, C);
-                const uint32_t ncontrib = c - c_lo;
-                const uint32_t tag = (uint32_t)r.ei + 1u;
-                for (uint32_t i = lane; i < ncontrib; i += 32) {
-                    uint32_t which;
-                    if (!contributor_slot(c_lo + i, rt, units, KB, C, which)) continue;
-                    const unsigned int* flag = reinterpret_cast<const unsigned int*>(
-                        p.slots + ((size_t)(c_lo + i) * 2 + which) * kSlotBytes + kElemsMax * 4);
-                    guard.wait_flag([&] { return ld_acquire(flag) == tag; });
-                }
-                __syncwarp();
                 for (int e = lane; e < elems; e += 32) {
                     float sum = 0.f;
                     for (uint32_t cc = c_lo; cc < c; ++cc) {
                         uint32_t which;
                         if (!contributor_slot(cc, rt, units, KB, C, which)) continue;
-                        sum += __ldcg(reinterpret_cast<const float*>(p.slots + ((size_t)cc * 2 + which) * kSlotBytes) + e);
+                        unsigned long long* src = slots + (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kElemsMax + e;
+                        unsigned long long v = 0ull;
+                        guard.wait_flag([&] { v = __ldcg(src); return (uint32_t)(v >> 32) == tag; });
+                        if ((uint32_t)(v >> 32) == tag) {
+                            sum += __uint_as_float((uint32_t)v);
+                            __stcg(src, 0ull);  // consumed: the slot may be reused
+                        }
                     }
                     sum += r.data[e];
                     int row, tok;
@@ -532,12 +536,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                     if (tok < E.M) E.y[(size_t)tok * E.N + rt * 16 + row] = __float2bfloat16_rn(sum);
                 }
                 __syncwarp();
-                for (uint32_t i = lane; i < ncontrib; i += 32) {
-                    uint32_t which;
-                    if (!contributor_slot(c_lo + i, rt, units, KB, C, which)) continue;
-                    st_release(reinterpret_cast<unsigned int*>(p.slots + ((size_t)(c_lo + i) * 2 + which) * kSlotBytes +
-                                                               kElemsMax * 4), 0u);
-                }
                 if (lane == 0 && p.tiles_done) {
                     __threadfence();
                     red_release_add(p.tiles_done, 1u);
@@ -546,13 +544,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
             __syncwarp();
             if (lane == 0) mbar_arrive(fqempty0 + 8 * q);
         }
-    } else if (tid < kComputeThreads + kEpiThreads + 32 + kStagerThreads) {
-        // =============================== activation stager (4 warps) ===============================
+    } else if (tid < kComputeThreads + kEpiThreads + kFixThreads + kStagerThreads) {
+        // =============================== activation stager (3 warps) ===============================
         // The rows of x arrive by bulk copy as they are; two passes over them, 8 columns (one 16-byte piece) per
         // thread and step, without cross-thread shuffles: pass 1 leaves max|x| of every 128-column block in
         // shared memory (atomicMax on the bit patterns), pass 2 converts with the block's scale, writes the two
         // int8 planes and adds up the integers of the block (atomicAdd).
-        const int st = tid - (kComputeThreads + kEpiThreads + 32);  // 0..127
+        const int st = tid - (kComputeThreads + kEpiThreads + kFixThreads);  // 0..95
         for (int i = st; i < 2 * kMaxRows * p.kb_max; i += kStagerThreads) bmax[i] = 0u;
         stager_sync();
         uint32_t xe = 0;
@@ -701,8 +699,8 @@ inline int max_tiles_for(int x_rows) { return x_rows == 1 ? 8 : 4; }
 
 size_t smem_fixed_bytes(int x_rows, int x_row_bytes, int kb_max) {
     return (size_t)2 * max_tiles_for(x_rows) * kComputeWarps * elems_for(x_rows) * 4 + 2 * kElemsMax * 4 +
-           (size_t)kFixDepth * (16 + kElemsMax * 4) + (size_t)4 * x_rows * x_row_bytes + (size_t)x_rows * kb_max * 256 +
-           (size_t)6 * kMaxRows * kb_max * 4 + (10 + 2 * kFixDepth) * 8 + 64 /* flag + slack */;
+           (size_t)2 * kFixDepth * (16 + kElemsMax * 4) + (size_t)4 * x_rows * x_row_bytes + (size_t)x_rows * kb_max * 256 +
+           (size_t)6 * kMaxRows * kb_max * 4 + (10 + 4 * kFixDepth) * 8 + 64 /* flag + slack */;
 }
 
 constexpr size_t kSmemLimit = 232448;  // 227 KiB per CTA
@@ -724,7 +722,7 @@ bool w4a16_stream_supported(int M, int N, int K, int G) {
 
 size_t w4a16_stream_weight_bytes(int N, int K) { return (size_t)(N / 16) * (K / 128) * kUnitBytes; }
 
-size_t w4a16_stream_workspace() { return (size_t)kWsHeader + (size_t)num_sms() * 2 * kSlotBytes; }
+size_t w4a16_stream_workspace() { return (size_t)kWsHeader + (size_t)num_sms() * 2 * kSlotDepth * kSlotBytes; }
 
 qil_status launch_pack_stream_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K, int G,
                                  void* out, cudaStream_t st) {

@@ -320,11 +320,10 @@ def test_w4a16_stream_shapes(api, M, N, K, G):
     assert_rows_close(bf16_to_f64(outs[0])[:, rows], y_ref)
     np.testing.assert_array_equal(bits_of(outs[0]), bits_of(outs[1]))
     import torch
-    # the workspace is left ready for the next call: the status word and every slot flag are zero
+    # the workspace is left ready for the next call: the status word and every {value, tag} pair are zero
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     assert int(torch.count_nonzero(ws[:4]).item()) == 0
-    flags = ws[256:256 + sms * 2 * 272].view(-1, 272)[:, 256:]
-    assert int(torch.count_nonzero(flags).item()) == 0
+    assert int(torch.count_nonzero(ws[256:256 + sms * 2 * 4 * 512]).item()) == 0
 
 
 def test_w4a16_stream_batch_with_dependencies(api):

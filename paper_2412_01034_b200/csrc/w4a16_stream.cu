@@ -94,7 +94,7 @@ struct StreamParams {
     int x_row_bytes;  // one int8 plane of a row: max K + pad
     int kb_max;       // max K / 128
     int elems;        // fp32 values kept per (row tile, warp): 16 if every M == 1, else 64
-    int max_tiles;    // row tiles per pass: 8 (elems 16) or 4 (elems 64)
+    int max_tiles;    // row tiles per pass: 8 (elems 16) or 2 (elems 64)
     int* status;
     unsigned int* tiles_done;
     unsigned char* slots;
@@ -182,7 +182,7 @@ struct Guard {
         if (*poisoned) return;
         const unsigned long long t0 = now_ns();
         for (uint32_t i = 1;; ++i) {
-            if (mbar_try_wait_suspend(bar, parity, 4000u)) return;
+            if (mbar_try_wait_suspend(bar, parity, 200u)) return;
             if ((i & 15u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
         }
         fail();
@@ -277,8 +277,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
     unsigned char* xraw = xs + (size_t)4 * p.x_rows * p.x_row_bytes;         // [x_rows][256 kb_max] bf16 as copied
     int* xsum = reinterpret_cast<int*>(xraw + (size_t)p.x_rows * p.kb_max * 256);  // [2][kMaxRows][kb_max]
     float* xscale = reinterpret_cast<float*>(xsum + 2 * kMaxRows * p.kb_max);      // [2][kMaxRows][kb_max]
-    unsigned int* bmax = reinterpret_cast<unsigned int*>(xscale + 2 * kMaxRows * p.kb_max);  // [2][kMaxRows][kb_max]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(bmax + 2 * kMaxRows * p.kb_max);
+    unsigned int* pmax = reinterpret_cast<unsigned int*>(xscale + 2 * kMaxRows * p.kb_max);  // [16 kb_max] piece maxima
+    int* psum = reinterpret_cast<int*>(pmax + 16 * p.kb_max);                                // [16 kb_max] piece sums
+    uint64_t* bars = reinterpret_cast<uint64_t*>(psum + 16 * p.kb_max);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
     const uint32_t xfull0 = smem_u32(b2);          // [2] activations of an entry are staged
@@ -546,13 +547,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
         }
     } else if (tid < kComputeThreads + kEpiThreads + kFixThreads + kStagerThreads) {
         // =============================== activation stager (3 warps) ===============================
-        // The rows of x arrive by bulk copy as they are; two passes over them, 8 columns (one 16-byte piece) per
-        // thread and step, without cross-thread shuffles: pass 1 leaves max|x| of every 128-column block in
-        // shared memory (atomicMax on the bit patterns), pass 2 converts with the block's scale, writes the two
-        // int8 planes and adds up the integers of the block (atomicAdd).
+        // The rows of x arrive by bulk copy as they are.  8 columns (one 16-byte piece) per thread and step, no
+        // shuffles and no atomics: (A) max |x| of every piece, (B) every piece reads the 16 maxima of its
+        // 128-column block, converts with the block's scale, writes the two int8 planes and leaves the sum of its
+        // integers, (C) one thread per block adds the 16 sums.
         const int st = tid - (kComputeThreads + kEpiThreads + kFixThreads);  // 0..95
-        for (int i = st; i < 2 * kMaxRows * p.kb_max; i += kStagerThreads) bmax[i] = 0u;
-        stager_sync();
         uint32_t xe = 0;
         Walk wk(p, C, c);
         while (wk.next_entry()) {
@@ -562,8 +561,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
             unsigned char* xs_b = xs + (size_t)xb * 2 * p.x_rows * p.x_row_bytes;
             int* xsum_b = xsum + (size_t)xb * kMaxRows * p.kb_max;
             float* xscale_b = xscale + (size_t)xb * kMaxRows * p.kb_max;
-            unsigned int* bmax_b = bmax + (size_t)xb * kMaxRows * p.kb_max;
-            unsigned int* bmax_next = bmax + (size_t)(xb ^ 1) * kMaxRows * p.kb_max;
             if (st == 0) {
                 guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1);
                 if (E.flags & kFlagDep) {  // the input is written by earlier entries: wait until all their tiles are out
@@ -577,30 +574,34 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                                    xraw0);
             }
             guard.wait_mbar(xraw0, xe & 1);  // (the copies were issued after the compute warps released buffer xb)
-            const int pieces = (int)KB * 16;  // 16-byte pieces per row
-            for (int r = 0; r < E.M; ++r) {
-                const unsigned char* xrow = xraw + (size_t)r * p.kb_max * 256;
-                for (int kb = st; kb < (int)KB; kb += kStagerThreads) xsum_b[r * p.kb_max + kb] = 0;
-#pragma unroll 4
-                for (int pc = st; pc < pieces; pc += kStagerThreads) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
-                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-                    uint32_t amax = 0;  // bf16 magnitudes order like unsigned integers
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) amax = max(amax, max((u[i] << 16) & 0x7FFFFFFFu, u[i] & 0x7FFF0000u));
-                    atomicMax(bmax_b + r * p.kb_max + (pc >> 4), amax);
-                }
-            }
-            stager_sync();
+            const int pieces = (int)KB * 16;  // 16-byte pieces per row, 16 per block
             for (int r = 0; r < E.M; ++r) {
                 const unsigned char* xrow = xraw + (size_t)r * p.kb_max * 256;
                 unsigned char* dst_hi = xs_b + (size_t)(2 * r) * p.x_row_bytes;
                 unsigned char* dst_lo = dst_hi + p.x_row_bytes;
+                // A: max |x| of every piece (bf16 magnitudes order like unsigned integers)
 #pragma unroll 2
                 for (int pc = st; pc < pieces; pc += kStagerThreads) {
                     const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
                     const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-                    const uint32_t amax = bmax_b[r * p.kb_max + (pc >> 4)];
+                    uint32_t amax = 0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) amax = max(amax, max((u[i] << 16) & 0x7FFFFFFFu, u[i] & 0x7FFF0000u));
+                    pmax[pc] = amax;
+                }
+                stager_sync();
+                // B: convert every piece with the scale of its block, leave the sum of its integers
+#pragma unroll 2
+                for (int pc = st; pc < pieces; pc += kStagerThreads) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
+                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+                    const uint4* pm = reinterpret_cast<const uint4*>(pmax + (pc & ~15));
+                    uint32_t amax = 0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint4 m4 = pm[i];
+                        amax = max(amax, max(max(m4.x, m4.y), max(m4.z, m4.w)));
+                    }
                     // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field F -> e = F - 127 - 14, one
                     // more when the mantissa exceeds 32639/16384 (for bf16: all seven mantissa bits set)
                     int ef = (int)(amax >> 23);
@@ -628,11 +629,22 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_stream_kernel(const __grid_
                     hi.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
                     *reinterpret_cast<uint2*>(dst_hi + (size_t)pc * 8) = hi;
                     *reinterpret_cast<uint2*>(dst_lo + (size_t)pc * 8) = lo;
-                    atomicAdd(xsum_b + r * p.kb_max + (pc >> 4), sum);
+                    psum[pc] = sum;
                     if ((pc & 15) == 0) xscale_b[r * p.kb_max + (pc >> 4)] = __uint_as_float((uint32_t)(127 + e) << 23);
                 }
+                stager_sync();
+                // C: block sums
+                for (int kb = st; kb < (int)KB; kb += kStagerThreads) {
+                    const int4* ps = reinterpret_cast<const int4*>(psum + kb * 16);
+                    int sum = 0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int4 v = ps[i];
+                        sum += (v.x + v.y) + (v.z + v.w);
+                    }
+                    xsum_b[r * p.kb_max + kb] = sum;
+                }
             }
-            for (int i = st; i < kMaxRows * p.kb_max; i += kStagerThreads) bmax_next[i] = 0u;  // for the next entry
             stager_sync();
             if (st == 0) mbar_arrive(xfull0 + 8 * xb);
             ++xe;
@@ -695,12 +707,12 @@ __global__ void __launch_bounds__(256) pack_stream_kernel(const uint8_t* __restr
 }
 
 inline int elems_for(int x_rows) { return x_rows == 1 ? 16 : 64; }
-inline int max_tiles_for(int x_rows) { return x_rows == 1 ? 8 : 4; }
+inline int max_tiles_for(int x_rows) { return x_rows == 1 ? 8 : 2; }
 
 size_t smem_fixed_bytes(int x_rows, int x_row_bytes, int kb_max) {
     return (size_t)2 * max_tiles_for(x_rows) * kComputeWarps * elems_for(x_rows) * 4 + 2 * kElemsMax * 4 +
            (size_t)2 * kFixDepth * (16 + kElemsMax * 4) + (size_t)4 * x_rows * x_row_bytes + (size_t)x_rows * kb_max * 256 +
-           (size_t)6 * kMaxRows * kb_max * 4 + (10 + 4 * kFixDepth) * 8 + 64 /* flag + slack */;
+           (size_t)4 * kMaxRows * kb_max * 4 + (size_t)2 * 16 * kb_max * 4 + (10 + 4 * kFixDepth) * 8 + 64 /* flag + slack */;
 }
 
 constexpr size_t kSmemLimit = 232448;  // 227 KiB per CTA

@@ -2,31 +2,43 @@
 // persistent kernel over a list of linears (the memory-bound decode stage of the paper's
 // OpenVLA deployment, Sec. 5.4 / App. A.4.2; M <= 4 activation rows).
 //
-// CUDA cores only unpack: a thread turns 64 bytes of packed codes (one weight row x 128
-// columns) into int8 with three integer instructions per 8 weights and writes them to
-// tensor memory (tcgen05.st), where they are the A operand (128 rows x 32 int8 per
-// instruction) of tcgen05.mma kind::i8.  The B operand is the activation block, converted
-// once per linear to 16-bit block fixed point - per 128 columns a power-of-two scale and
-// two int8 planes (v = 256 hi + lo) - and laid out K-major in shared memory so that the
-// 8 "columns" of the instruction are {row0 hi, row0 lo, row1 hi, ...}.  Accumulators are
-// int32 in tensor memory (exact); per 128-column block the owner thread of a weight row
-// reads them back (tcgen05.ld) and folds scale and zero point once:
-//     y += s_w * 2^e * ((256 D_hi + D_lo) - z * X),   X = sum of the block's integers.
+// The kernel is bound by HBM only if the SM spends very few instructions per weight, so the
+// CUDA cores do nothing but split nibbles: a thread owns one weight row of a unit (128 rows
+// x 128 columns), reads its 64 packed bytes, and with ONE logic instruction per 4 weights
+// produces unsigned bytes - the low nibbles as they are, the high nibbles in place, i.e.
+// times 16 - which it writes to tensor memory (tcgen05.st).  There they are the A operand
+// (128 rows x 32 bytes per instruction) of tcgen05.mma kind::i8.  The B operand is the
+// activation block, converted once per linear to 16-bit block fixed point - per 128 columns a
+// power-of-two scale 2^e and two int8 planes (v = 256 hi + lo) - K-major in shared memory.
+// Low-nibble and high-nibble bytes accumulate in separate int32 accumulators in tensor memory
+// (exact); per 128-column block the epilogue thread of a weight row reads them back
+// (tcgen05.ld) and folds scale and zero point once:
+//     y += s_w * 2^e * ((256 L_hi + L_lo) + (256 H_hi + H_lo) / 16 - z * X),  X = sum of the block's integers.
 //
 // Data layout (QIL_LAYOUT_STREAM128): unit u = (row tile of 128 rows, column block of 128)
 // is 8704 bytes: 4 chunks (32 columns each) x 128 rows x 16 bytes of codes, byte b of
 // word m of a chunk holding column 8m+b (low nibble) and 8m+4+b (high nibble); then
 // 128 x {fp16 scale, fp16 zero}.  Rows beyond N are zero.  A linear is one contiguous
-// stream of units.
+// stream of units; CTA c of C owns units [c q + min(c, r), ...) with q = units / C, r = units % C.
 //
-// Roles in a CTA (one CTA per SM): a producer thread streams the CTA's slice of units
-// through a shared-memory ring (cp.async.bulk + mbarrier); the unpack warpgroups alternate units
-// (unpack -> tensor memory, later the epilogue of the same unit; three of them take turns); one thread per
-// warpgroup issues its MMAs; four stager warps convert the next activations; four finalizer warps combine the
-// warpgroups' partial sums, write outputs and complete row tiles shared with other CTAs
-// through {value, tag} pairs in the workspace (one 8-byte store each, fixed summation order).
-// Every wait is bounded (2 s); on expiry QIL_ERR_TIMEOUT is recorded in the workspace
-// status word, waiting stops, tensor memory is released and the kernel returns.
+// Roles in a CTA (one CTA per SM, alive for the whole list):
+//   producer (1 thread)   streams the CTA's units through a shared-memory ring (cp.async.bulk +
+//                         mbarrier), running ahead across linears as far as the ring allows, so
+//                         HBM keeps streaming while the consumers wait for a dependency;
+//   unpack warpgroups     take turns on units: shared memory -> nibble split -> tensor memory;
+//   MMA issuer (1 thread) four tcgen05.mma per unit, completion signalled by tcgen05.commit;
+//   epilogue warpgroup    thread = weight row: accumulators -> fp32 row sums (kept in registers
+//                         over the units of a row tile) -> bf16 outputs of row tiles the CTA owns
+//                         entirely, or a hand-over of the partial sums of a row tile it shares;
+//   stager warpgroup      waits for QIL_DEP_PREVIOUS, loads and converts the activation blocks the
+//                         CTA's units need (double buffered, one linear ahead);
+//   fixer warpgroup       all cross-CTA work: publishes the partial sums of a shared row tile as
+//                         {value, tag} pairs (one 8-byte store each, tag = entry index + 1) into a
+//                         ring of slots in the workspace, completes the row tile whose end the CTA
+//                         owns by adding the contributions in CTA order (bit-reproducible), and
+//                         counts finished row tiles for the dependency counter.
+// Every wait is bounded (2 s); on expiry QIL_ERR_TIMEOUT is recorded in the workspace status
+// word, waiting stops, tensor memory is released and the kernel returns.
 #include <mutex>
 
 #include "qil_common.cuh"
@@ -37,36 +49,34 @@ namespace {
 
 constexpr int kUnitRows = 128;
 constexpr int kUnitBytes = 8192 + 512;
-constexpr int kWgThreads = 128;
-constexpr int kNumWg = 3;
-constexpr int kStagerThreads = 128;
-constexpr int kFinThreads = 128;
-// thread ranges: kNumWg unpack/epilogue warpgroups, then the MMA warp, the producer warp, the stager, the finalizer
-constexpr int kMmaBase = kNumWg * kWgThreads;
-constexpr int kProdBase = kMmaBase + 32 * kNumWg;  // one MMA-issuing warp per warpgroup
-constexpr int kStagerBase = kProdBase + 32;
-constexpr int kFinBase = kStagerBase + kStagerThreads;
-constexpr int kThreads = kFinBase + kFinThreads;
-constexpr int kNumBuf = 3 * kNumWg;  // A buffers (32 columns each) and accumulator buffers (8 columns each)
-constexpr int kTmemCols = 512;       // A at columns [0, 32 kNumBuf), D behind them
-constexpr int kColD = 32 * kNumBuf;
-static_assert(kColD + 8 * kNumBuf <= kTmemCols, "tensor memory budget");
-constexpr int kMaxTiles = 2;    // row tiles per pass
-constexpr int kPartBufs = 4;    // partial-sum buffers between the warpgroups and the finalizer
+constexpr int kNumWg = 3;                        // unpack warpgroups
+constexpr int kUnpackThreads = 128 * kNumWg;
+constexpr int kEpiBase = kUnpackThreads;         // epilogue warpgroup (its warps keep warp % 4 = lane quarter)
+constexpr int kStagerBase = kEpiBase + 128;
+constexpr int kFixBase = kStagerBase + 128;
+constexpr int kMmaBase = kFixBase + 128;         // one warp, one thread issues
+constexpr int kProdBase = kMmaBase + 32;         // one warp, one thread issues
+constexpr int kThreads = kProdBase + 32;
+constexpr int kNB = 8;                           // units in flight in tensor memory
+constexpr int kTmemCols = 512;
+constexpr int kColD = 32 * kNB;                  // A: 32 columns per unit; D: 8 (low nibbles) + 8 (high nibbles)
+constexpr int kColMeta = kColD + 16 * kNB;       // one column per unit: {scale, zero} of the thread's row
+static_assert(kColMeta + kNB <= kTmemCols, "tensor memory budget");
 constexpr int kMaxEntries = 256;
-constexpr int kMaxRows = 4;     // activation rows
-constexpr int kSlotDepth = 4;                      // ring of slots per (CTA, first/last tile)
-constexpr int kSlotElems = kMaxRows * kUnitRows;   // {value, tag} pairs of 8 bytes
+constexpr int kMaxRows = 4;                      // activation rows
+constexpr int kSlotDepth = 4;                    // ring of slots per (CTA, first / last tile), indexed by entry
+constexpr int kSlotElems = kMaxRows * kUnitRows; // {value, tag} pairs of 8 bytes
 constexpr int kWsHeader = 256;
 constexpr int kFlagDep = 1;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-struct TcEntry {  // 48 bytes
+struct TcEntry {  // 56 bytes
     const uint16_t* x;
     const unsigned char* w;
     __nv_bfloat16* y;
     int N, K, M, flags;
-    uint32_t tiles_before;
+    uint32_t tiles_before;  // row tiles of all earlier entries of this launch
+    uint32_t q, rem;        // units / CTAs, units % CTAs
     uint32_t pad;
 };
 
@@ -74,10 +84,8 @@ struct TcParams {
     TcEntry e[kMaxEntries];
     int count;
     int stages;
-    int x_rows;     // activation rows staged: 1, 2 or 4 (>= every M)
-    int kb_max;     // max K / 128
-    int lbo;        // byte distance between 16-column chunks of the activation operand = 32 * x_rows
-    int xbuf_bytes; // one activation buffer
+    int kb_max;      // max K / 128
+    int xbuf_bytes;  // one activation operand buffer
     int* status;
     unsigned int* tiles_done;
     unsigned char* slots;
@@ -94,6 +102,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// (a failed try_wait suspends the thread in hardware for a few microseconds or until the phase completes)
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -105,7 +114,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-__device__ __forceinline__ void bulk_g2s_plain(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
@@ -118,14 +127,56 @@ __device__ __forceinline__ uint32_t ld_acquire(const unsigned int* p) {
 __device__ __forceinline__ void red_release_add(unsigned int* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-template <int kId, int kCount>
-__device__ __forceinline__ void group_sync() {
-    asm volatile("bar.sync %0, %1;" ::"n"(kId), "n"(kCount) : "memory");
+template <int kId>
+__device__ __forceinline__ void group_sync() {  // the 128 threads of one role
+    asm volatile("bar.sync %0, 128;" ::"n"(kId) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t (&v)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(addr), "r"(v[0]), "r"(v[1]),
+                 "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st1(uint32_t addr, uint32_t v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t tmem_ld1(uint32_t addr) {
+    uint32_t v;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+// kCols consecutive 32-bit columns of the thread's lane
+template <int kCols>
+__device__ __forceinline__ void tmem_ld(uint32_t addr, uint32_t (&v)[8]) {
+    if constexpr (kCols == 2) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(v[0]), "=r"(v[1]) : "r"(addr));
+    } else if constexpr (kCols == 4) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+                     : "r"(addr));
+    } else {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                     : "r"(addr));
+    }
+}
+// Waits for the tcgen05.ld of this thread; the registers are operands so that no use of them is scheduled earlier.
+template <int kCols>
+__device__ __forceinline__ void wait_ld(uint32_t (&a)[8], uint32_t (&b)[8], uint32_t& m) {
+    if constexpr (kCols == 2) {
+        asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(a[0]), "+r"(a[1]), "+r"(b[0]), "+r"(b[1]), "+r"(m)::"memory");
+    } else if constexpr (kCols == 4) {
+        asm volatile("tcgen05.wait::ld.sync.aligned;"
+                     : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(m)::"memory");
+    } else {
+        asm volatile("tcgen05.wait::ld.sync.aligned;"
+                     : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]), "+r"(b[0]),
+                       "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]), "+r"(m)::"memory");
+    }
 }
 // shared-memory operand descriptor: K-major, no swizzle, 8-row x 16-byte core matrices `lbo` bytes apart along K
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo) {
@@ -166,9 +217,9 @@ struct Guard {
         if (mbar_try_wait(bar, parity)) return;
         if (*poisoned) return;
         const unsigned long long t0 = now_ns();
-        for (uint32_t i = 1;; ++i) {
+        for (;;) {
             if (mbar_try_wait(bar, parity)) return;
-            if ((i & 15u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
+            if (*poisoned || now_ns() - t0 > kWaitLimitNs) break;
         }
         fail();
     }
@@ -179,43 +230,36 @@ struct Guard {
         const unsigned long long t0 = now_ns();
         for (uint32_t i = 1;; ++i) {
             if (done()) return;
-            __nanosleep(i < 64 ? 20 : 200);
-            if ((i & 63u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
+            if (i > 8) __nanosleep(i < 64 ? 32 : 256);
+            if ((i & 15u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
         }
         fail();
     }
 };
 
-__device__ __forceinline__ void slice_of(uint32_t units, uint32_t c, uint32_t C, uint32_t& u0, uint32_t& u1) {
-    u0 = (uint32_t)(((uint64_t)c * units) / C);
-    u1 = (uint32_t)(((uint64_t)(c + 1) * units) / C);
+// ---- who owns which units ---------------------------------------------------------------------
+__device__ __forceinline__ void slice_of(uint32_t q, uint32_t rem, uint32_t c, uint32_t& u0, uint32_t& u1) {
+    u0 = c * q + min(c, rem);
+    u1 = u0 + q + (c < rem ? 1u : 0u);
 }
-__device__ __forceinline__ uint32_t owner_of(uint32_t u, uint32_t units, uint32_t C) {
-    return (uint32_t)((((uint64_t)(u + 1)) * C - 1) / units);
-}
-__device__ __forceinline__ bool contributor_slot(uint32_t cc, uint32_t rt, uint32_t units, uint32_t KB, uint32_t C,
-                                                 uint32_t& which) {
-    uint32_t cu0, cu1;
-    slice_of(units, cc, C, cu0, cu1);
-    which = (cu0 / KB == rt) ? 0u : 1u;
-    return cu0 != cu1;
+// CTA that owns unit u
+__device__ __forceinline__ uint32_t owner_of(uint32_t q, uint32_t rem, uint32_t u) {
+    const uint32_t big = rem * (q + 1);  // units held by the first `rem` CTAs
+    return u < big ? u / (q + 1) : rem + (u - big) / q;
 }
 
-// The work of one CTA: entries in which it owns units, cut into passes of at most kMaxTiles row tiles.
+// The entries in which one CTA owns units.
 struct Walk {
     const TcParams& p;
-    uint32_t C, c;
+    uint32_t c;
     int ei;
-    uint32_t KB, units, u0, u1, t_first, t_last;
-    __device__ Walk(const TcParams& p_, uint32_t C_, uint32_t c_) : p(p_), C(C_), c(c_), ei(-1) {}
-    __device__ bool next_entry() {
+    uint32_t KB, u0, u1;
+    __device__ Walk(const TcParams& p_, uint32_t c_) : p(p_), c(c_), ei(-1) {}
+    __device__ __forceinline__ bool next_entry() {
         for (++ei; ei < p.count; ++ei) {
-            KB = (uint32_t)p.e[ei].K >> 7;
-            units = (((uint32_t)p.e[ei].N + kUnitRows - 1) / kUnitRows) * KB;
-            slice_of(units, c, C, u0, u1);
+            slice_of(p.e[ei].q, p.e[ei].rem, c, u0, u1);
             if (u0 != u1) {
-                t_first = u0 / KB;
-                t_last = (u1 - 1) / KB;
+                KB = (uint32_t)p.e[ei].K >> 7;
                 return true;
             }
         }
@@ -232,29 +276,30 @@ struct Cyc {
     }
 };
 
+// kXR = activation rows staged (1, 2 or 4; >= every M of the launch)
+template <int kXR>
 __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_constant__ TcParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int kLbo = 32 * kXR;   // byte distance between the 16-byte K chunks of the activation operand: the
+                                     // 2 kXR planes of a chunk; rows of the 8-row window beyond them belong to
+                                     // the next chunks and only feed accumulator columns nobody reads
+    constexpr int kDCols = 2 * kXR;  // accumulator columns in use: {high byte, low byte} plane per activation row
     const int tid = threadIdx.x;
-    const uint32_t C = gridDim.x, c = blockIdx.x;
-    const int XR = p.x_rows;
+    const uint32_t c = blockIdx.x;
 
     // ---- carve shared memory ----
-    unsigned char* ring = smem;                                                          // [stages][kUnitBytes]
-    unsigned char* xs = ring + (size_t)p.stages * kUnitBytes;                            // [2][xbuf_bytes]
-    unsigned char* xraw = xs + (size_t)2 * p.xbuf_bytes;                                 // [XR][kb_max*256] bf16
-    int* xsum = reinterpret_cast<int*>(xraw + (size_t)XR * p.kb_max * 256);              // [2][XR][kb_max]
-    float* xscale = reinterpret_cast<float*>(xsum + 2 * XR * p.kb_max);                  // [2][XR][kb_max]
-    float* part = xscale + 2 * XR * p.kb_max;                       // [kPartBufs][kNumWg][kMaxTiles][XR][128]
-    const int part_floats = kNumWg * kMaxTiles * XR * kUnitRows;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(part + (size_t)kPartBufs * part_floats);
+    unsigned char* ring = smem;                                                     // [stages][kUnitBytes]
+    unsigned char* xs = ring + (size_t)p.stages * kUnitBytes;                       // [2][xbuf_bytes]
+    int* xsum = reinterpret_cast<int*>(xs + (size_t)2 * p.xbuf_bytes);              // [2][kXR][kb_max]
+    float* xscale = reinterpret_cast<float*>(xsum + 2 * kXR * p.kb_max);            // [2][kXR][kb_max]
+    float* hand = xscale + 2 * kXR * p.kb_max;                                      // [2][2][kXR][128]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(hand + 2 * 2 * kXR * kUnitRows);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
-    const uint32_t afull0 = smem_u32(b2);
-    const uint32_t dfull0 = smem_u32(b2 + 2 * kNumBuf), dempty0 = smem_u32(b2 + 3 * kNumBuf);
-    uint64_t* b3 = b2 + 4 * kNumBuf;
-    const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2), xraw0 = smem_u32(b3 + 4);
-    const uint32_t pfull0 = smem_u32(b3 + 5), pempty0 = smem_u32(b3 + 5 + kPartBufs);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 5 + 2 * kPartBufs);
+    const uint32_t afull0 = smem_u32(b2), dfull0 = smem_u32(b2 + kNB), dempty0 = smem_u32(b2 + 2 * kNB);
+    uint64_t* b3 = b2 + 3 * kNB;
+    const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2), hfull0 = smem_u32(b3 + 4), hempty0 = smem_u32(b3 + 6);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 8);
     volatile int* poisoned = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     if (tid == 0) {
@@ -262,24 +307,20 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 4);
         }
-        for (int i = 0; i < kNumBuf; ++i) {
+        for (int i = 0; i < kNB; ++i) {
             mbar_init(afull0 + 8 * i, 4);
             mbar_init(dfull0 + 8 * i, 1);
             mbar_init(dempty0 + 8 * i, 4);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(xfull0 + 8 * i, 1);
-            mbar_init(xempty0 + 8 * i, kNumWg * 4);
-        }
-        mbar_init(xraw0, 1);
-        for (int i = 0; i < kPartBufs; ++i) {
-            mbar_init(pfull0 + 8 * i, kNumWg * 4);
-            mbar_init(pempty0 + 8 * i, 1);
+            mbar_init(xempty0 + 8 * i, 4);
+            mbar_init(hfull0 + 8 * i, 4);
+            mbar_init(hempty0 + 8 * i, 4);
         }
         *poisoned = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < kPartBufs * part_floats; i += kThreads) part[i] = 0.f;
     for (int i = tid; i < 2 * p.xbuf_bytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(xs)[i] = 0u;
     if (tid < 32) {  // one warp owns the tensor-memory allocation
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -293,256 +334,184 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     const uint32_t tmem = *tmem_slot;
     const Guard guard{p.status, poisoned};
 
-    if (tid < kMmaBase) {
-        // ======================= unpack + epilogue warpgroups =======================
-        const int wg = tid / kWgThreads, r = tid % kWgThreads, lane = tid & 31;
-        const uint32_t lane_base = (uint32_t)(r & ~31) << 16;  // this warp's quarter of the tensor-memory lanes
-        Cyc rs(p.stages), pb(kPartBufs), ab(kNumBuf), turn(kNumWg);  // all advance once per unit of the CTA
-        uint32_t xe = 0;
-        Walk wk(p, C, c);
+    if (tid < kUnpackThreads) {
+        // ======================= unpack warpgroups: shared memory -> nibble split -> tensor memory =======================
+        const uint32_t wg = tid >> 7, r = tid & 127, lane = tid & 31;
+        const uint32_t lane_base = (r & ~31u) << 16;  // this warp's quarter of the tensor-memory lanes
+        Cyc rs(p.stages), ab(kNB), turn(kNumWg);      // all advance once per unit of the CTA
+        Walk wk(p, c);
         while (wk.next_entry()) {
-            const int M = p.e[wk.ei].M;
-            const uint32_t KB = wk.KB;
-            const uint32_t xb = xe & 1;
-            guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
-            ++xe;
-            const int* xsum_b = xsum + (size_t)xb * XR * p.kb_max;
-            const float* xscale_b = xscale + (size_t)xb * XR * p.kb_max;
-            for (uint32_t tp = wk.t_first; tp <= wk.t_last; tp += kMaxTiles) {
-                const uint32_t pu0 = max(wk.u0, tp * KB), pu1 = min(wk.u1, (tp + kMaxTiles) * KB);
-                guard.wait_mbar(pempty0 + 8 * pb.idx, pb.ph ^ 1);
-                float* my_part = part + (size_t)pb.idx * part_floats + (size_t)wg * kMaxTiles * XR * kUnitRows + r;
-                float fin[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
-                int cur_tile = -1;
-                // units whose MMAs are in flight: the accumulators of a unit are read after the next two units of
-                // this warpgroup have been written to tensor memory (the oldest record is pend_*, the newer next_*)
-                int npend = 0;
-                uint32_t pend_d = 0, pend_dph = 0, pend_kb = 0, next_d = 0, next_dph = 0, next_kb = 0;
-                int pend_tl = 0, next_tl = 0;
-                float pend_s = 0.f, next_s = 0.f;
-                int pend_z = 0, next_z = 0;
-                uint32_t d[8];
-                auto epilogue_load = [&]() {   // start reading the accumulators of the pending unit
-                    guard.wait_mbar(dfull0 + 8 * pend_d, pend_dph);
+            for (uint32_t n = wk.u1 - wk.u0; n > 0; --n) {
+                if (turn.idx == wg) {
+                    const uint32_t a = ab.idx;
+                    guard.wait_mbar(dempty0 + 8 * a, ab.ph ^ 1);  // the unit that used these columns has been read out
+                    guard.wait_mbar(full0 + 8 * rs.idx, rs.ph);
                     tc_fence_after();
-                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]),
-                                   "=r"(d[7])
-                                 : "r"(tmem + lane_base + kColD + 8 * pend_d));
-                };
-                auto epilogue_math = [&]() {   // ... and fold them into this thread's row sums
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    const unsigned char* ub = ring + (size_t)rs.idx * kUnitBytes;
+                    const uint32_t ta = tmem + lane_base + 32 * a;
+                    constexpr uint32_t kLo = 0x0F0F0F0Fu, kHi = 0xF0F0F0F0u;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {  // chunks 2h, 2h+1 = columns [64h, 64h + 64) of the block
+                        const uint4 w0 = *reinterpret_cast<const uint4*>(ub + ((size_t)(2 * h) * kUnitRows + r) * 16);
+                        const uint4 w1 = *reinterpret_cast<const uint4*>(ub + ((size_t)(2 * h + 1) * kUnitRows + r) * 16);
+                        const uint32_t lo[8] = {w0.x & kLo, w0.y & kLo, w0.z & kLo, w0.w & kLo,
+                                                w1.x & kLo, w1.y & kLo, w1.z & kLo, w1.w & kLo};
+                        const uint32_t hi[8] = {w0.x & kHi, w0.y & kHi, w0.z & kHi, w0.w & kHi,
+                                                w1.x & kHi, w1.y & kHi, w1.z & kHi, w1.w & kHi};
+                        tmem_st8(ta + 8 * h, lo);       // A of MMA (low nibbles, half h)
+                        tmem_st8(ta + 16 + 8 * h, hi);  // A of MMA (high nibbles x 16, half h)
+                    }
+                    tmem_st1(tmem + lane_base + kColMeta + a, *reinterpret_cast<const uint32_t*>(ub + 8192 + 4 * r));
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(dempty0 + 8 * pend_d);
-                    if (pend_tl != cur_tile) {
-                        if (cur_tile >= 0) {
-#pragma unroll
-                            for (int t = 0; t < kMaxRows; ++t)
-                                if (t < XR) my_part[((size_t)cur_tile * XR + t) * kUnitRows] = fin[t];
-                        }
-                        fin[0] = fin[1] = fin[2] = fin[3] = 0.f;
-                        cur_tile = pend_tl;
+                    if (lane == 0) {
+                        mbar_arrive(afull0 + 8 * a);
+                        mbar_arrive(empty0 + 8 * rs.idx);
                     }
-#pragma unroll
-                    for (int t = 0; t < kMaxRows; ++t)
-                        if (t < M) {
-                            const int acc = (int)d[2 * t] * 256 + (int)d[2 * t + 1];
-                            const int v = acc - pend_z * xsum_b[t * p.kb_max + pend_kb];
-                            fin[t] = fmaf((float)v, pend_s * xscale_b[t * p.kb_max + pend_kb], fin[t]);
-                        }
-                };
-                uint32_t tl = pu0 / KB - tp, kb = pu0 % KB;
-                for (uint32_t cu = pu0; cu < pu1; ++cu) {
-                    if (turn.idx == (uint32_t)wg) {
-                        const uint32_t a = ab.idx;
-                        guard.wait_mbar(full0 + 8 * rs.idx, rs.ph);
-                        const unsigned char* ub = ring + (size_t)rs.idx * kUnitBytes;
-                        tc_fence_after();
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint4 w = *reinterpret_cast<const uint4*>(ub + ((size_t)j * kUnitRows + r) * 16);
-                            const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
-                            uint32_t q[8];
-#pragma unroll
-                            for (int m = 0; m < 4; ++m) {
-                                q[2 * m] = ws[m] & 0x0F0F0F0Fu;
-                                q[2 * m + 1] = (ws[m] >> 4) & 0x0F0F0F0Fu;
-                            }
-                            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(
-                                             tmem + lane_base + 32 * a + 8 * j),
-                                         "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]), "r"(q[4]), "r"(q[5]), "r"(q[6]), "r"(q[7])
-                                         : "memory");
-                        }
-                        const __half2 meta = *reinterpret_cast<const __half2*>(ub + 8192 + 4 * r);
-                        const bool drain = npend == 2;
-                        if (drain) epilogue_load();  // overlaps with the stores above
-                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) {
-                            mbar_arrive(afull0 + 8 * a);
-                            mbar_arrive(empty0 + 8 * rs.idx);
-                        }
-                        if (drain) {
-                            epilogue_math();
-                            pend_d = next_d; pend_dph = next_dph; pend_kb = next_kb; pend_tl = next_tl;
-                            pend_s = next_s; pend_z = next_z;
-                            npend = 1;
-                        }
-                        if (npend == 0) {
-                            pend_d = a; pend_dph = ab.ph; pend_kb = kb; pend_tl = (int)tl;
-                            pend_s = __low2float(meta); pend_z = (int)__high2float(meta);
-                        } else {
-                            next_d = a; next_dph = ab.ph; next_kb = kb; next_tl = (int)tl;
-                            next_s = __low2float(meta); next_z = (int)__high2float(meta);
-                        }
-                        ++npend;
-                    }
-                    rs.step();
-                    ab.step();
-                    turn.step();
-                    if (++kb == KB) { kb = 0; ++tl; }
                 }
-                while (npend > 0) {
-                    epilogue_load();
-                    epilogue_math();
-                    pend_d = next_d; pend_dph = next_dph; pend_kb = next_kb; pend_tl = next_tl;
-                    pend_s = next_s; pend_z = next_z;
-                    --npend;
-                }
-                if (cur_tile >= 0) {
-#pragma unroll
-                    for (int t = 0; t < kMaxRows; ++t)
-                        if (t < XR) my_part[((size_t)cur_tile * XR + t) * kUnitRows] = fin[t];
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(pfull0 + 8 * pb.idx);
-                pb.step();
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(xempty0 + 8 * xb);
-        }
-    } else if (tid < kProdBase) {
-        // ======================= MMA issuers (one thread per warpgroup) =======================
-        if (((tid - kMmaBase) & 31) == 0) {
-            const uint32_t g = (uint32_t)(tid - kMmaBase) >> 5;  // serves the units of warpgroup g
-            uint32_t xe = 0;
-            Cyc ab(kNumBuf), turn(kNumWg);
-            Walk wk(p, C, c);
-            const uint64_t desc_hi = smem_desc(0, p.lbo);
-            while (wk.next_entry()) {
-                const uint32_t KB = wk.KB;
-                const uint32_t xb = xe & 1;
-                guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
-                ++xe;
-                const uint32_t xs16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4, lbo16 = (uint32_t)p.lbo >> 4;
-                uint32_t kb = wk.u0 % KB;
-                for (uint32_t cu = wk.u0; cu < wk.u1; ++cu) {
-                    if (turn.idx == g) {
-                        const uint32_t a = ab.idx;
-                        guard.wait_mbar(afull0 + 8 * a, ab.ph);
-                        guard.wait_mbar(dempty0 + 8 * a, ab.ph ^ 1);
-                        tc_fence_after();
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            mma_i8_ts(tmem + kColD + 8 * a, tmem + 32 * a + 8 * j,
-                                      desc_hi | (uint64_t)(xs16 + (kb * 8 + 2 * j) * lbo16), j > 0 ? 1u : 0u);
-                        // accumulators complete -> epilogue; it also means the A buffer has been read, and the same
-                        // warpgroup reuses it only after that epilogue
-                        tc_commit(dfull0 + 8 * a);
-                    }
-                    ab.step();
-                    turn.step();
-                    if (++kb == KB) kb = 0;
-                }
+                rs.step();
+                ab.step();
+                turn.step();
             }
         }
     } else if (tid < kStagerBase) {
-        // ======================= producer (one thread) =======================
-        if (tid == kProdBase) {
-            Cyc rs(p.stages);
-            uint32_t issued = 0;
-            Walk wk(p, C, c);
-            while (wk.next_entry()) {
-                const unsigned char* wbase = p.e[wk.ei].w;
-                for (uint32_t cu = wk.u0; cu < wk.u1; ++cu, ++issued) {
-                    guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1);
-                    mbar_expect_tx(full0 + 8 * rs.idx, kUnitBytes);
-                    bulk_g2s_plain(smem_u32(ring + (size_t)rs.idx * kUnitBytes), wbase + (size_t)cu * kUnitBytes, kUnitBytes,
-                                   full0 + 8 * rs.idx);
-                    rs.step();
+        // ======================= epilogue warpgroup (thread = weight row of the unit) =======================
+        const uint32_t r = tid - kEpiBase, lane = tid & 31;
+        const uint32_t lane_base = (r & ~31u) << 16;
+        Cyc ab(kNB);
+        uint32_t xe = 0, he = 0;
+        Walk wk(p, c);
+        while (wk.next_entry()) {
+            const TcEntry& E = p.e[wk.ei];
+            const int M = E.M, N = E.N;
+            const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1;
+            const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
+            const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
+            const uint32_t xb = xe & 1;
+            guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
+            ++xe;
+            const int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
+            const float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
+            float* hand_b = hand + (size_t)(he & 1) * 2 * kXR * kUnitRows;
+            if (shares) guard.wait_mbar(hempty0 + 8 * (he & 1), ((he >> 1) & 1) ^ 1);
+            uint32_t n_full = 0;
+            float fin[kXR];
+#pragma unroll
+            for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
+            uint32_t rt = t_first, kb = u0 - t_first * KB;
+            // the accumulators of unit u are requested before the arithmetic of unit u - 1 (never across entries:
+            // the next entry may depend on outputs of this one)
+            uint32_t dl[8], dh[8], meta;
+            auto request = [&]() {
+                guard.wait_mbar(dfull0 + 8 * ab.idx, ab.ph);
+                tc_fence_after();
+                const uint32_t td = tmem + lane_base + kColD + 16 * ab.idx;
+                tmem_ld<kDCols>(td, dl);
+                tmem_ld<kDCols>(td + 8, dh);
+                meta = tmem_ld1(tmem + lane_base + kColMeta + ab.idx);
+            };
+            request();
+            for (uint32_t u = u0; u < u1; ++u) {
+                wait_ld<kDCols>(dl, dh, meta);
+                uint32_t cl[kDCols], ch[kDCols];
+#pragma unroll
+                for (int i = 0; i < kDCols; ++i) {
+                    cl[i] = dl[i];
+                    ch[i] = dh[i];
+                }
+                const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(dempty0 + 8 * ab.idx);
+                ab.step();
+                if (u + 1 < u1) request();
+                const float s = __low2float(sz);
+                const int z = (int)__high2float(sz);
+#pragma unroll
+                for (int t = 0; t < kXR; ++t)
+                    if (t < M) {
+                        const int v = ((int)cl[2 * t] * 256 + (int)cl[2 * t + 1]) + (((int)ch[2 * t] * 256 + (int)ch[2 * t + 1]) >> 4) -
+                                      z * xsum_b[t * p.kb_max + kb];
+                        fin[t] = fmaf((float)v, s * xscale_b[t * p.kb_max + kb], fin[t]);
+                    }
+                if (++kb == KB || u + 1 == u1) {  // the CTA's part of row tile rt is complete
+                    const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
+                    if (cb && ce) {
+                        ++n_full;
+                        const uint32_t row = rt * kUnitRows + r;
+                        if (row < (uint32_t)N) {
+#pragma unroll
+                            for (int t = 0; t < kXR; ++t)
+                                if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(fin[t]);
+                        }
+                    } else {  // first tile cut at its beginning (completed here) or last tile continued elsewhere
+                        float* dst = hand_b + (size_t)(ce ? 0 : 1) * kXR * kUnitRows + r;
+#pragma unroll
+                        for (int t = 0; t < kXR; ++t) dst[t * kUnitRows] = fin[t];
+                    }
+#pragma unroll
+                    for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
+                    kb = 0;
+                    ++rt;
                 }
             }
-            // every copy issued must have landed before the CTA may retire
-            for (uint32_t back = 0; back < (uint32_t)p.stages && back < issued; ++back) {
-                if (rs.idx == 0) { rs.idx = p.stages; rs.ph ^= 1; }
-                --rs.idx;
-                guard.wait_mbar(full0 + 8 * rs.idx, rs.ph);
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(xempty0 + 8 * xb);
+                if (shares) mbar_arrive(hfull0 + 8 * (he & 1));
+            }
+            if (shares) ++he;
+            if (n_full && p.tiles_done) {
+                group_sync<1>();  // every row of the tiles is written
+                if (r == 0) {
+                    __threadfence();
+                    red_release_add(p.tiles_done, n_full);
+                }
             }
         }
-    } else if (tid < kFinBase) {
-        // ======================= activation stager (4 warps) =======================
+    } else if (tid < kFixBase) {
+        // ======================= activation stager (thread pairs of a half warp = one 128-column block) =======================
         // bf16 row -> per 128 columns: e with max|x| / 2^e <= 32639, v = rint(x / 2^e) = 256 hi + lo (both int8),
-        // X = sum v.  hi / lo planes go to rows 2t / 2t+1 of every 16-column chunk of the operand.
-        const int st = tid - kStagerBase;
+        // X = sum v.  Only the blocks the CTA's units touch are converted.  K order of the operand inside a block:
+        // 16-byte chunk 4p + 2h + cc (p: half of the block, h: low / high nibble columns, cc: 32-column chunk of
+        // the half), byte 4m + b = column 64p + 32cc + 8m + 4h + b.
+        const int st = tid - kStagerBase, l16 = st & 15, hw = st >> 4;
         uint32_t xe = 0;
-        Walk wk(p, C, c);
+        Walk wk(p, c);
         while (wk.next_entry()) {
             const TcEntry& E = p.e[wk.ei];
             const uint32_t KB = wk.KB;
             const uint32_t xb = xe & 1;
             unsigned char* xs_b = xs + (size_t)xb * p.xbuf_bytes;
-            int* xsum_b = xsum + (size_t)xb * XR * p.kb_max;
-            float* xscale_b = xscale + (size_t)xb * XR * p.kb_max;
+            int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
+            float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
             if (st == 0) {
                 guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1);
                 if (E.flags & kFlagDep) {
                     const unsigned int need = E.tiles_before;
                     guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; });
-                    asm volatile("fence.proxy.async;" ::: "memory");
-                }
-                mbar_expect_tx(xraw0, (uint32_t)E.M * (uint32_t)E.K * 2u);
-                for (int t = 0; t < E.M; ++t)
-                    bulk_g2s_plain(smem_u32(xraw + (size_t)t * p.kb_max * 256), E.x + (size_t)t * E.K, (uint32_t)E.K * 2u, xraw0);
-            }
-            guard.wait_mbar(xraw0, xe & 1);
-            // Two passes over the row, 8 columns (one 16-byte piece) per thread and step, no cross-thread
-            // shuffles: pass 1 leaves max|x| of every 128-column block in shared memory (atomicMax on the bit
-            // patterns), pass 2 converts with the block's scale and adds up the integers (atomicAdd).
-            const int pieces = (int)KB * 16;  // 16-byte pieces per row
-            for (int t = 0; t < E.M; ++t) {
-                unsigned int* bmax = reinterpret_cast<unsigned int*>(xscale_b + t * p.kb_max);  // reused as scratch
-                for (int kb = st; kb < (int)KB; kb += kStagerThreads) {
-                    bmax[kb] = 0u;
-                    xsum_b[t * p.kb_max + kb] = 0;
                 }
             }
-            group_sync<1, kStagerThreads>();
+            group_sync<2>();
+            const uint32_t nblk = min(KB, wk.u1 - wk.u0), kb0 = wk.u0 % KB;
+            const uint32_t p_half = (uint32_t)l16 >> 3, cc = ((uint32_t)l16 >> 2) & 1, m = (uint32_t)l16 & 3;
             for (int t = 0; t < E.M; ++t) {
-                const unsigned char* xrow = xraw + (size_t)t * p.kb_max * 256;
-                unsigned int* bmax = reinterpret_cast<unsigned int*>(xscale_b + t * p.kb_max);
-#pragma unroll 4
-                for (int pc = st; pc < pieces; pc += kStagerThreads) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
+                const uint16_t* xrow = E.x + (size_t)t * E.K;
+                for (uint32_t ib = 0; ib < nblk; ib += 8) {
+                    const uint32_t i = ib + hw;
+                    const bool valid = i < nblk;
+                    uint32_t kb = kb0 + i;
+                    if (kb >= KB) kb -= KB;
+                    uint4 raw = make_uint4(0, 0, 0, 0);
+                    if (valid) raw = __ldcg(reinterpret_cast<const uint4*>(xrow + (size_t)kb * 128 + l16 * 8));
                     const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
                     uint32_t amax = 0;  // bf16 magnitudes order like unsigned integers
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) amax = max(amax, max((u[i] << 16) & 0x7FFFFFFFu, u[i] & 0x7FFF0000u));
-                    atomicMax(bmax + (pc >> 4), amax);
-                }
-            }
-            group_sync<1, kStagerThreads>();
-            for (int t = 0; t < E.M; ++t) {
-                const unsigned char* xrow = xraw + (size_t)t * p.kb_max * 256;
-                const unsigned int* bmax = reinterpret_cast<const unsigned int*>(xscale_b + t * p.kb_max);
-                unsigned char* xdst = xs_b + (size_t)(2 * t) * 16;
-#pragma unroll 4
-                for (int pc = st; pc < pieces; pc += kStagerThreads) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(xrow + (size_t)pc * 16);
-                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-                    const uint32_t amax = bmax[pc >> 4];
-                    // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field E -> e = E - 127 - 14, one
+                    for (int j = 0; j < 4; ++j) amax = max(amax, max((u[j] << 16) & 0x7FFFFFFFu, u[j] & 0x7FFF0000u));
+#pragma unroll
+                    for (int o = 1; o < 16; o <<= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                    // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field F -> e = F - 127 - 14, one
                     // more when the mantissa exceeds 32639/16384 (for bf16: all seven mantissa bits set)
                     int ef = (int)(amax >> 23);
                     if (ef < 1 || ef >= 255) ef = 127 + 14;  // zero / subnormal / non-finite block: scale 1
@@ -553,132 +522,89 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     uint32_t vb[8];
                     int sum = 0;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float f0 = fmaf(__uint_as_float(u[i] << 16), inv, 12582912.f);
-                        const float f1 = fmaf(__uint_as_float(u[i] & 0xFFFF0000u), inv, 12582912.f);
+                    for (int j = 0; j < 4; ++j) {
+                        const float f0 = fmaf(__uint_as_float(u[j] << 16), inv, 12582912.f);
+                        const float f1 = fmaf(__uint_as_float(u[j] & 0xFFFF0000u), inv, 12582912.f);
                         const int q0 = (int)(__float_as_uint(f0) - 0x4B400000u), q1 = (int)(__float_as_uint(f1) - 0x4B400000u);
                         sum += q0 + q1;
-                        vb[2 * i] = (uint32_t)(q0 + 128);
-                        vb[2 * i + 1] = (uint32_t)(q1 + 128);
+                        vb[2 * j] = (uint32_t)(q0 + 128);
+                        vb[2 * j + 1] = (uint32_t)(q1 + 128);
                     }
-                    // byte 0 of each (v + 128) is lo + 128, byte 1 is hi
-                    uint2 lo, hi;
-                    lo.x = __byte_perm(__byte_perm(vb[0], vb[1], 0x0040), __byte_perm(vb[2], vb[3], 0x0040), 0x5410) ^ 0x80808080u;
-                    lo.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
-                    hi.x = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
-                    hi.y = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
-                    // piece pc = 8 columns: 16-column chunk pc/2, first or second half of its 16-byte row
-                    unsigned char* dst = xdst + (size_t)(pc >> 1) * p.lbo + (pc & 1) * 8;
-                    *reinterpret_cast<uint2*>(dst) = hi;
-                    *reinterpret_cast<uint2*>(dst + 16) = lo;
-                    atomicAdd(xsum_b + t * p.kb_max + (pc >> 4), sum);
+#pragma unroll
+                    for (int o = 1; o < 16; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                    if (valid) {
+                        // byte 0 of each (v + 128) is lo + 128, byte 1 is hi; columns 0-3 of the piece sit under low
+                        // nibbles, columns 4-7 under high nibbles
+                        const uint32_t lo_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0040), __byte_perm(vb[2], vb[3], 0x0040), 0x5410) ^ 0x80808080u;
+                        const uint32_t lo_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
+                        const uint32_t hi_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
+                        const uint32_t hi_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
+                        unsigned char* dst = xs_b + (size_t)(kb * 8 + 4 * p_half + cc) * kLbo + (size_t)(2 * t) * 16 + 4 * m;
+                        *reinterpret_cast<uint32_t*>(dst) = hi_a;
+                        *reinterpret_cast<uint32_t*>(dst + 16) = lo_a;
+                        *reinterpret_cast<uint32_t*>(dst + 2 * kLbo) = hi_b;
+                        *reinterpret_cast<uint32_t*>(dst + 2 * kLbo + 16) = lo_b;
+                        if (l16 == 0) {
+                            xsum_b[t * p.kb_max + kb] = sum;
+                            xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);
+                        }
+                    }
                 }
             }
-            group_sync<1, kStagerThreads>();
-            for (int t = 0; t < E.M; ++t)  // replace the block maxima by the scales 2^e
-                for (int kb = st; kb < (int)KB; kb += kStagerThreads) {
-                    const uint32_t amax = reinterpret_cast<const unsigned int*>(xscale_b + t * p.kb_max)[kb];
-                    int ef = (int)(amax >> 23);
-                    if (ef < 1 || ef >= 255) ef = 127 + 14;
-                    int e = ef - 127 - 14 + (((amax & 0x7FFFFFu) > 0x7EFE00u) ? 1 : 0);
-                    if (e < -126) e = -126;
-                    xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);
-                }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read xs through the async proxy
-            group_sync<1, kStagerThreads>();
+            group_sync<2>();
             if (st == 0) mbar_arrive(xfull0 + 8 * xb);
             ++xe;
         }
-    } else {
-        // ======================= finalizer (4 warps; thread = row of the tile) =======================
-        // Row tiles shared with other CTAs are completed through the workspace: each contributor writes
-        // {value, tag} pairs (one 8-byte store per element, tag = entry index + 1) into a ring of kSlotDepth
-        // slots; the CTA owning the end of the tile polls the pairs, adds them in CTA order and clears the tags.
-        const int r = tid - kFinBase;
-        Cyc pb(kPartBufs);
-        Walk wk(p, C, c);
+    } else if (tid < kMmaBase) {
+        // ======================= fixer warpgroup (thread = row of the tile): all cross-CTA work =======================
+        const uint32_t r = tid - kFixBase, lane = tid & 31;
+        unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
+        uint32_t he = 0;
+        Walk wk(p, c);
         while (wk.next_entry()) {
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
-            const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, units = wk.units;
+            const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1;
+            const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
+            const bool have_last = (t_last + 1) * KB > u1;                          // contributes to a tile that ends elsewhere
+            const bool have_first = t_first * KB < u0 && (t_first + 1) * KB <= u1;  // completes a tile begun elsewhere
+            if (!have_last && !(t_first * KB < u0)) continue;
             const uint32_t tag = (uint32_t)wk.ei + 1u, ring_i = (uint32_t)wk.ei % kSlotDepth;
-            // slice geometry: is the last tile cut at its end (this CTA contributes), the first at its beginning
-            // (this CTA completes it)?
-            const bool have_last = (wk.t_last + 1) * KB > u1;
-            const bool have_first = wk.t_first * KB < u0 && (wk.t_first + 1) * KB <= u1;
+            const float* hand_b = hand + (size_t)(he & 1) * 2 * kXR * kUnitRows;
             unsigned long long* my_slot = nullptr;
             if (have_last) {
-                const uint32_t which = (wk.t_last == wk.t_first) ? 0u : 1u;
-                my_slot = reinterpret_cast<unsigned long long*>(p.slots) +
-                          (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems;
+                const uint32_t which = (t_last == t_first) ? 0u : 1u;
+                my_slot = slots + (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems + r;
                 // the slot must have been consumed (tags cleared) by whoever completed the tile it last served;
-                // checked now, while the warpgroups are still computing
-#pragma unroll
-                for (int t = 0; t < kMaxRows; ++t)
-                    if (t < M) {
-                        const unsigned long long* q = my_slot + t * kUnitRows + r;
-                        guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; });
-                    }
-            }
-            uint32_t n_full = 0;
-            float first_v[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
-            for (uint32_t tp = wk.t_first; tp <= wk.t_last; tp += kMaxTiles) {
-                const uint32_t ntiles = min((uint32_t)kMaxTiles, wk.t_last - tp + 1);
-                guard.wait_mbar(pfull0 + 8 * pb.idx, pb.ph);
-                float* buf = part + (size_t)pb.idx * part_floats;
-                for (uint32_t tl = 0; tl < ntiles; ++tl) {
-                    const uint32_t rt = tp + tl;
-                    const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
-                    float v[kMaxRows];
-#pragma unroll
-                    for (int t = 0; t < kMaxRows; ++t) {
-                        v[t] = 0.f;
-                        if (t < XR) {
-#pragma unroll
-                            for (int g = 0; g < kNumWg; ++g) {  // fixed order
-                                float* a = buf + ((size_t)(g * kMaxTiles + tl) * XR + t) * kUnitRows + r;
-                                v[t] += *a;
-                                *a = 0.f;
-                            }
-                        }
-                    }
-                    const int row = (int)rt * kUnitRows + r;
-                    if (cb && ce) {
-                        ++n_full;
-                        if (row < N) {
-#pragma unroll
-                            for (int t = 0; t < kMaxRows; ++t)
-                                if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(v[t]);
-                        }
-                    } else if (ce) {
-#pragma unroll
-                        for (int t = 0; t < kMaxRows; ++t) first_v[t] = v[t];
-                    } else {  // publish this CTA's share: value and tag travel in one store
-#pragma unroll
-                        for (int t = 0; t < kMaxRows; ++t)
-                            if (t < M)
-                                __stcg(my_slot + t * kUnitRows + r,
-                                       ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(v[t]));
-                    }
+                // checked now, while the units are still being computed
+                for (int t = 0; t < M; ++t) {
+                    const unsigned long long* q = my_slot + t * kUnitRows;
+                    guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; });
                 }
-                group_sync<2, kFinThreads>();
-                if (r == 0) mbar_arrive(pempty0 + 8 * pb.idx);
-                pb.step();
             }
-            if (have_first) {  // complete the tile whose beginning belongs to earlier CTAs
-                const uint32_t rt = wk.t_first;
-                const uint32_t c_lo = owner_of(rt * KB, units, C);
-                float sum[kMaxRows] = {0.f, 0.f, 0.f, 0.f};
+            guard.wait_mbar(hfull0 + 8 * (he & 1), (he >> 1) & 1);
+            if (have_last) {  // publish first (a chain of CTAs must never wait on each other in a circle)
+                for (int t = 0; t < M; ++t)
+                    __stcg(my_slot + t * kUnitRows,
+                           ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(hand_b[(kXR + t) * kUnitRows + r]));
+            }
+            if (have_first) {
+                const uint32_t c_lo = owner_of(E.q, E.rem, t_first * KB);
+                float sum[kXR];
+#pragma unroll
+                for (int t = 0; t < kXR; ++t) sum[t] = 0.f;
                 for (uint32_t cc = c_lo; cc < c; ++cc) {
-                    uint32_t which;
-                    if (!contributor_slot(cc, rt, units, KB, C, which)) continue;
-                    unsigned long long* src = reinterpret_cast<unsigned long long*>(p.slots) +
-                                              (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + r;
-                    unsigned long long got[kMaxRows] = {0ull, 0ull, 0ull, 0ull};
+                    uint32_t cu0, cu1;
+                    slice_of(E.q, E.rem, cc, cu0, cu1);
+                    if (cu0 == cu1) continue;
+                    const uint32_t which = (cu0 / KB == t_first) ? 0u : 1u;
+                    unsigned long long* src = slots + (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + r;
+                    unsigned long long got[kXR];
                     guard.wait_flag([&] {
                         bool all = true;
 #pragma unroll
-                        for (int t = 0; t < kMaxRows; ++t)
+                        for (int t = 0; t < kXR; ++t)
                             if (t < M) {
                                 got[t] = __ldcg(src + t * kUnitRows);
                                 all &= (uint32_t)(got[t] >> 32) == tag;
@@ -686,26 +612,82 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         return all;
                     });
 #pragma unroll
-                    for (int t = 0; t < kMaxRows; ++t)
+                    for (int t = 0; t < kXR; ++t)
                         if (t < M) {
-                            sum[t] += __uint_as_float((uint32_t)got[t]);
+                            if ((uint32_t)(got[t] >> 32) == tag) sum[t] += __uint_as_float((uint32_t)got[t]);
                             __stcg(src + t * kUnitRows, 0ull);  // consumed: the slot may be reused
                         }
                 }
-                const int row = (int)rt * kUnitRows + r;
-                if (row < N) {
+                const uint32_t row = t_first * kUnitRows + r;
+                if (row < (uint32_t)N) {
 #pragma unroll
-                    for (int t = 0; t < kMaxRows; ++t)
-                        if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(sum[t] + first_v[t]);
+                    for (int t = 0; t < kXR; ++t)
+                        if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(sum[t] + hand_b[t * kUnitRows + r]);
                 }
-                ++n_full;
             }
-            if (n_full && p.tiles_done) {
-                group_sync<2, kFinThreads>();  // every row of the tiles is written
+            __syncwarp();
+            if (lane == 0) mbar_arrive(hempty0 + 8 * (he & 1));
+            ++he;
+            if (have_first && p.tiles_done) {
+                group_sync<3>();  // every row of the tile is written
                 if (r == 0) {
                     __threadfence();
-                    red_release_add(p.tiles_done, n_full);
+                    red_release_add(p.tiles_done, 1u);
                 }
+            }
+        }
+    } else if (tid < kProdBase) {
+        // ======================= MMA issuer (one thread) =======================
+        if (tid == kMmaBase) {
+            uint32_t xe = 0;
+            Cyc ab(kNB);
+            Walk wk(p, c);
+            const uint64_t desc_hi = smem_desc(0, kLbo);
+            constexpr uint32_t lbo16 = (uint32_t)kLbo >> 4;
+            while (wk.next_entry()) {
+                const uint32_t KB = wk.KB;
+                const uint32_t xb = xe & 1;
+                guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
+                ++xe;
+                const uint32_t xs16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
+                uint32_t kb = wk.u0 % KB;
+                for (uint32_t u = wk.u0; u < wk.u1; ++u) {
+                    const uint32_t a = ab.idx;
+                    guard.wait_mbar(afull0 + 8 * a, ab.ph);  // (the unpack warps waited for the accumulators to be free)
+                    tc_fence_after();
+                    const uint32_t ta = tmem + 32 * a, td = tmem + kColD + 16 * a;
+                    const uint64_t b0 = desc_hi | (uint64_t)(xs16 + kb * 8 * lbo16);
+                    mma_i8_ts(td, ta, b0, 0u);                    // low nibbles, columns [0, 64)
+                    mma_i8_ts(td, ta + 8, b0 + 4 * lbo16, 1u);    // low nibbles, columns [64, 128)
+                    mma_i8_ts(td + 8, ta + 16, b0 + 2 * lbo16, 0u);   // high nibbles
+                    mma_i8_ts(td + 8, ta + 24, b0 + 6 * lbo16, 1u);
+                    tc_commit(dfull0 + 8 * a);
+                    ab.step();
+                    if (++kb == KB) kb = 0;
+                }
+            }
+        }
+    } else {
+        // ======================= producer (one thread) =======================
+        if (tid == kProdBase) {
+            Cyc rs(p.stages);
+            uint32_t issued = 0;
+            Walk wk(p, c);
+            while (wk.next_entry()) {
+                const unsigned char* wbase = p.e[wk.ei].w;
+                for (uint32_t u = wk.u0; u < wk.u1; ++u, ++issued) {
+                    guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1);
+                    mbar_expect_tx(full0 + 8 * rs.idx, kUnitBytes);
+                    bulk_g2s(smem_u32(ring + (size_t)rs.idx * kUnitBytes), wbase + (size_t)u * kUnitBytes, kUnitBytes,
+                             full0 + 8 * rs.idx);
+                    rs.step();
+                }
+            }
+            // every copy issued must have landed before the CTA may retire
+            for (uint32_t back = 0; back < (uint32_t)p.stages && back < issued; ++back) {
+                if (rs.idx == 0) { rs.idx = p.stages; rs.ph ^= 1; }
+                --rs.idx;
+                guard.wait_mbar(full0 + 8 * rs.idx, rs.ph);
             }
         }
     }
@@ -749,7 +731,7 @@ __global__ void __launch_bounds__(256) pack_stream128_kernel(const uint8_t* __re
 }
 
 struct SmemPlan {
-    int x_rows, lbo, xbuf_bytes, stages;
+    int x_rows, xbuf_bytes, stages;
     size_t total;
 };
 
@@ -758,19 +740,26 @@ constexpr size_t kSmemLimit = 232448;  // 227 KiB per CTA
 SmemPlan plan_for(int max_m, int kb_max) {
     SmemPlan pl;
     pl.x_rows = max_m <= 1 ? 1 : max_m <= 2 ? 2 : 4;
-    pl.lbo = 32 * pl.x_rows;
-    pl.xbuf_bytes = kb_max * 8 * pl.lbo + 128;  // the last chunk's 8-row window reaches past its own rows
-    const size_t fixed = (size_t)2 * pl.xbuf_bytes + (size_t)pl.x_rows * kb_max * 256 + (size_t)2 * 2 * pl.x_rows * kb_max * 4 +
-                         (size_t)kPartBufs * kNumWg * kMaxTiles * pl.x_rows * kUnitRows * 4 +
-                         (size_t)(4 * kNumBuf + 5 + 2 * kPartBufs) * 8 + 16 + 128;
+    const int lbo = 32 * pl.x_rows;
+    pl.xbuf_bytes = kb_max * 8 * lbo + 128;  // the last chunk's 8-row window reaches past its own rows
+    const size_t fixed = (size_t)2 * pl.xbuf_bytes + (size_t)2 * 2 * pl.x_rows * kb_max * 4 +
+                         (size_t)2 * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 8) * 8 + 16 + 128;
     pl.stages = 0;
     if (fixed < kSmemLimit) {
         long s = (long)((kSmemLimit - fixed) / (kUnitBytes + 16));
-        if (s > 20) s = 20;
+        if (s > 24) s = 24;
         pl.stages = (int)s;
     }
     pl.total = fixed + (size_t)pl.stages * (kUnitBytes + 16);
     return pl;
+}
+
+template <int kXR>
+cudaError_t launch_one(const TcParams& p, int C, size_t smem, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(w4a16_tc_kernel<kXR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    w4a16_tc_kernel<kXR><<<C, kThreads, smem, st>>>(p);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -799,7 +788,7 @@ qil_status launch_pack_stream128_w4(const uint8_t* codes, const void* scales, co
 // Every entry must satisfy w4a16_tc_supported().  entries[i].flags bit 0 = QIL_DEP_PREVIOUS.
 qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, size_t ws_bytes, cudaStream_t st) {
     if (ws == nullptr || ws_bytes < w4a16_tc_workspace()) return QIL_ERR_WORKSPACE;
-    static TcParams p;  // 12 KiB: kept off the caller's stack; guarded by the mutex below
+    static TcParams p;  // 14 KiB: kept off the caller's stack; guarded by the mutex below
     static std::mutex mu;
     std::lock_guard<std::mutex> lock(mu);
     const int C = num_sms();
@@ -817,8 +806,12 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
             e.N = d.N; e.K = d.K; e.M = d.M;
             e.flags = (i > 0) ? (d.flags & kFlagDep) : 0;  // earlier launches are ordered by the stream
             e.tiles_before = tiles;
+            const uint32_t row_tiles = (uint32_t)((d.N + kUnitRows - 1) / kUnitRows);
+            const uint32_t units = row_tiles * (uint32_t)(d.K / 128);
+            e.q = units / (uint32_t)C;
+            e.rem = units % (uint32_t)C;
             e.pad = 0;
-            tiles += (uint32_t)((d.N + kUnitRows - 1) / kUnitRows);
+            tiles += row_tiles;
             any_dep |= (e.flags & kFlagDep) != 0;
             if (d.M > max_m) max_m = d.M;
             if (d.K > kmax) kmax = d.K;
@@ -827,9 +820,7 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
         if (pl.stages < 4) return QIL_ERR_UNSUPPORTED;
         p.count = n;
         p.stages = pl.stages;
-        p.x_rows = pl.x_rows;
         p.kb_max = kmax / 128;
-        p.lbo = pl.lbo;
         p.xbuf_bytes = pl.xbuf_bytes;
         p.status = reinterpret_cast<int*>(ws);
         p.tiles_done = any_dep ? reinterpret_cast<unsigned int*>(ws) + 1 : nullptr;
@@ -838,13 +829,13 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
             (void)cudaGetLastError();
             return QIL_ERR_CUDA;
         }
-        if (cudaFuncSetAttribute(w4a16_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.total) != cudaSuccess) {
+        const cudaError_t err = pl.x_rows == 1   ? launch_one<1>(p, C, pl.total, st)
+                                : pl.x_rows == 2 ? launch_one<2>(p, C, pl.total, st)
+                                                 : launch_one<4>(p, C, pl.total, st);
+        if (err != cudaSuccess) {
             (void)cudaGetLastError();
             return QIL_ERR_CUDA;
         }
-        w4a16_tc_kernel<<<C, kThreads, pl.total, st>>>(p);
-        const qil_status s = launch_status();
-        if (s != QIL_OK) return s;
     }
     return QIL_OK;
 }

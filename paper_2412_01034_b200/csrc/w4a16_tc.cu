@@ -43,6 +43,21 @@
 
 #include "qil_common.cuh"
 
+// Optional per-warp timing (compile with -DQIL_TRACE): cycles spent in the waits of every role, written to a
+// buffer set with qil_trace_set_tc().  Nothing is skipped or reordered; without the macro the hooks vanish.
+#ifdef QIL_TRACE
+#define QIL_TR(slot, ...)                    \
+    do {                                     \
+        const long long tr_t0_ = clock64();  \
+        __VA_ARGS__;                         \
+        tr[slot] += clock64() - tr_t0_;      \
+    } while (0)
+#define QIL_TR_COUNT(slot) tr[slot] += 1
+#else
+#define QIL_TR(slot, ...) __VA_ARGS__
+#define QIL_TR_COUNT(slot)
+#endif
+
 namespace qil {
 
 namespace {
@@ -54,10 +69,12 @@ constexpr int kUnpackThreads = 128 * kNumWg;
 constexpr int kEpiBase = kUnpackThreads;         // epilogue warpgroup (its warps keep warp % 4 = lane quarter)
 constexpr int kStagerBase = kEpiBase + 128;
 constexpr int kFixBase = kStagerBase + 128;
-constexpr int kMmaBase = kFixBase + 128;         // one warp, one thread issues
-constexpr int kProdBase = kMmaBase + 32;         // one warp, one thread issues
+constexpr int kGroup = 4;                        // units per group: one per MMA issuer, one epilogue pass
+constexpr int kMmaBase = kFixBase + 128;         // kGroup warps, one issuing thread each
+constexpr int kProdBase = kMmaBase + 32 * kGroup;  // one warp, one thread issues
 constexpr int kThreads = kProdBase + 32;
-constexpr int kNB = 8;                           // units in flight in tensor memory
+constexpr int kNG = 2;                           // groups in flight in tensor memory
+constexpr int kNB = kGroup * kNG;                // = units in flight
 constexpr int kTmemCols = 512;
 constexpr int kColD = 32 * kNB;                  // A: 32 columns per unit; D: 8 (low nibbles) + 8 (high nibbles)
 constexpr int kColMeta = kColD + 16 * kNB;       // one column per unit: {scale, zero} of the thread's row
@@ -89,6 +106,9 @@ struct TcParams {
     int* status;
     unsigned int* tiles_done;
     unsigned char* slots;
+#ifdef QIL_TRACE
+    unsigned long long* trace;  // [CTA][warp][16]
+#endif
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -98,6 +118,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -136,9 +159,10 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t (&v)[8]) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(addr), "r"(v[0]), "r"(v[1]),
-                 "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(addr),
+                 "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+                 "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
                  : "memory");
 }
 __device__ __forceinline__ void tmem_st1(uint32_t addr, uint32_t v) {
@@ -162,20 +186,6 @@ __device__ __forceinline__ void tmem_ld(uint32_t addr, uint32_t (&v)[8]) {
         asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                      : "r"(addr));
-    }
-}
-// Waits for the tcgen05.ld of this thread; the registers are operands so that no use of them is scheduled earlier.
-template <int kCols>
-__device__ __forceinline__ void wait_ld(uint32_t (&a)[8], uint32_t (&b)[8], uint32_t& m) {
-    if constexpr (kCols == 2) {
-        asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(a[0]), "+r"(a[1]), "+r"(b[0]), "+r"(b[1]), "+r"(m)::"memory");
-    } else if constexpr (kCols == 4) {
-        asm volatile("tcgen05.wait::ld.sync.aligned;"
-                     : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(m)::"memory");
-    } else {
-        asm volatile("tcgen05.wait::ld.sync.aligned;"
-                     : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]), "+r"(b[0]),
-                       "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]), "+r"(m)::"memory");
     }
 }
 // shared-memory operand descriptor: K-major, no swizzle, 8-row x 16-byte core matrices `lbo` bytes apart along K
@@ -296,7 +306,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     uint64_t* bars = reinterpret_cast<uint64_t*>(hand + 2 * 2 * kXR * kUnitRows);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
-    const uint32_t afull0 = smem_u32(b2), dfull0 = smem_u32(b2 + kNB), dempty0 = smem_u32(b2 + 2 * kNB);
+    // afull: per unit slot; dfull / dempty: per group of kGroup slots
+    const uint32_t afull0 = smem_u32(b2), dfull0 = smem_u32(b2 + kNB), dempty0 = smem_u32(b2 + kNB + kNG);
     uint64_t* b3 = b2 + 3 * kNB;
     const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2), hfull0 = smem_u32(b3 + 4), hempty0 = smem_u32(b3 + 6);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 8);
@@ -307,10 +318,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 4);
         }
-        for (int i = 0; i < kNB; ++i) {
-            mbar_init(afull0 + 8 * i, 4);
-            mbar_init(dfull0 + 8 * i, 1);
-            mbar_init(dempty0 + 8 * i, 4);
+        for (int i = 0; i < kNB; ++i) mbar_init(afull0 + 8 * i, 4);
+        for (int i = 0; i < kNG; ++i) {
+            mbar_init(dfull0 + 8 * i, kGroup);  // one arrival per issuer
+            mbar_init(dempty0 + 8 * i, 4);      // the epilogue warps
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(xfull0 + 8 * i, 1);
@@ -333,36 +344,48 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     const Guard guard{p.status, poisoned};
+#ifdef QIL_TRACE
+    long long tr[16];
+    for (int i = 0; i < 16; ++i) tr[i] = 0;
+    const long long tr_begin = clock64();
+#endif
 
     if (tid < kUnpackThreads) {
         // ======================= unpack warpgroups: shared memory -> nibble split -> tensor memory =======================
         const uint32_t wg = tid >> 7, r = tid & 127, lane = tid & 31;
         const uint32_t lane_base = (r & ~31u) << 16;  // this warp's quarter of the tensor-memory lanes
-        Cyc rs(p.stages), ab(kNB), turn(kNumWg);      // all advance once per unit of the CTA
+        Cyc rs(p.stages), turn(kNumWg);  // advance once per unit of the CTA
+        uint32_t G = 0;                  // groups so far: unit j of an entry sits in group G + j / kGroup, slot j % kGroup
         Walk wk(p, c);
         while (wk.next_entry()) {
-            for (uint32_t n = wk.u1 - wk.u0; n > 0; --n) {
+            const uint32_t n = wk.u1 - wk.u0;
+            for (uint32_t j = 0; j < n; ++j) {
                 if (turn.idx == wg) {
-                    const uint32_t a = ab.idx;
-                    guard.wait_mbar(dempty0 + 8 * a, ab.ph ^ 1);  // the unit that used these columns has been read out
-                    guard.wait_mbar(full0 + 8 * rs.idx, rs.ph);
+                    const uint32_t g = G + j / kGroup, a = (g % kNG) * kGroup + j % kGroup, gph = (g / kNG) & 1;
+                    QIL_TR(1, guard.wait_mbar(dempty0 + 8 * (g % kNG), gph ^ 1));  // the group that used these columns has been read out
+                    QIL_TR(2, guard.wait_mbar(full0 + 8 * rs.idx, rs.ph));
+                    QIL_TR_COUNT(3);
                     tc_fence_after();
                     const unsigned char* ub = ring + (size_t)rs.idx * kUnitBytes;
                     const uint32_t ta = tmem + lane_base + 32 * a;
                     constexpr uint32_t kLo = 0x0F0F0F0Fu, kHi = 0xF0F0F0F0u;
+                    uint4 w[4];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {  // chunks 2h, 2h+1 = columns [64h, 64h + 64) of the block
-                        const uint4 w0 = *reinterpret_cast<const uint4*>(ub + ((size_t)(2 * h) * kUnitRows + r) * 16);
-                        const uint4 w1 = *reinterpret_cast<const uint4*>(ub + ((size_t)(2 * h + 1) * kUnitRows + r) * 16);
-                        const uint32_t lo[8] = {w0.x & kLo, w0.y & kLo, w0.z & kLo, w0.w & kLo,
-                                                w1.x & kLo, w1.y & kLo, w1.z & kLo, w1.w & kLo};
-                        const uint32_t hi[8] = {w0.x & kHi, w0.y & kHi, w0.z & kHi, w0.w & kHi,
-                                                w1.x & kHi, w1.y & kHi, w1.z & kHi, w1.w & kHi};
-                        tmem_st8(ta + 8 * h, lo);       // A of MMA (low nibbles, half h)
-                        tmem_st8(ta + 16 + 8 * h, hi);  // A of MMA (high nibbles x 16, half h)
+                    for (int ch = 0; ch < 4; ++ch) w[ch] = *reinterpret_cast<const uint4*>(ub + ((size_t)ch * kUnitRows + r) * 16);
+                    const uint32_t meta = *reinterpret_cast<const uint32_t*>(ub + 8192 + 4 * r);
+                    uint32_t v[16];
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        v[4 * ch] = w[ch].x & kLo; v[4 * ch + 1] = w[ch].y & kLo; v[4 * ch + 2] = w[ch].z & kLo; v[4 * ch + 3] = w[ch].w & kLo;
                     }
-                    tmem_st1(tmem + lane_base + kColMeta + a, *reinterpret_cast<const uint32_t*>(ub + 8192 + 4 * r));
-                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    tmem_st16(ta, v);       // A of the two low-nibble MMAs: columns [0, 64) and [64, 128) of the block
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        v[4 * ch] = w[ch].x & kHi; v[4 * ch + 1] = w[ch].y & kHi; v[4 * ch + 2] = w[ch].z & kHi; v[4 * ch + 3] = w[ch].w & kHi;
+                    }
+                    tmem_st16(ta + 16, v);  // A of the two high-nibble MMAs (values x 16)
+                    tmem_st1(tmem + lane_base + kColMeta + a, meta);
+                    QIL_TR(4, asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"));
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) {
@@ -371,61 +394,38 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     }
                 }
                 rs.step();
-                ab.step();
                 turn.step();
             }
+            G += (n + kGroup - 1) / kGroup;
         }
     } else if (tid < kStagerBase) {
         // ======================= epilogue warpgroup (thread = weight row of the unit) =======================
         const uint32_t r = tid - kEpiBase, lane = tid & 31;
         const uint32_t lane_base = (r & ~31u) << 16;
-        Cyc ab(kNB);
-        uint32_t xe = 0, he = 0;
+        constexpr int kEB = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;  // units read back per tcgen05.wait::ld
+        uint32_t xe = 0, he = 0, G = 0;
         Walk wk(p, c);
         while (wk.next_entry()) {
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
-            const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1;
+            const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, n = u1 - u0;
             const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
             const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
             const uint32_t xb = xe & 1;
-            guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
+            QIL_TR(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1));
             ++xe;
             const int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
             const float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
             float* hand_b = hand + (size_t)(he & 1) * 2 * kXR * kUnitRows;
-            if (shares) guard.wait_mbar(hempty0 + 8 * (he & 1), ((he >> 1) & 1) ^ 1);
+            if (shares) QIL_TR(2, guard.wait_mbar(hempty0 + 8 * (he & 1), ((he >> 1) & 1) ^ 1));
             uint32_t n_full = 0;
             float fin[kXR];
 #pragma unroll
             for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
             uint32_t rt = t_first, kb = u0 - t_first * KB;
-            // the accumulators of unit u are requested before the arithmetic of unit u - 1 (never across entries:
-            // the next entry may depend on outputs of this one)
-            uint32_t dl[8], dh[8], meta;
-            auto request = [&]() {
-                guard.wait_mbar(dfull0 + 8 * ab.idx, ab.ph);
-                tc_fence_after();
-                const uint32_t td = tmem + lane_base + kColD + 16 * ab.idx;
-                tmem_ld<kDCols>(td, dl);
-                tmem_ld<kDCols>(td + 8, dh);
-                meta = tmem_ld1(tmem + lane_base + kColMeta + ab.idx);
-            };
-            request();
-            for (uint32_t u = u0; u < u1; ++u) {
-                wait_ld<kDCols>(dl, dh, meta);
-                uint32_t cl[kDCols], ch[kDCols];
-#pragma unroll
-                for (int i = 0; i < kDCols; ++i) {
-                    cl[i] = dl[i];
-                    ch[i] = dh[i];
-                }
+            // one unit: fold scale and zero point into the row sums; close the row tile when its last unit is in
+            auto consume = [&](const uint32_t (&cl)[8], const uint32_t (&ch)[8], uint32_t meta, bool last_unit) {
                 const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(dempty0 + 8 * ab.idx);
-                ab.step();
-                if (u + 1 < u1) request();
                 const float s = __low2float(sz);
                 const int z = (int)__high2float(sz);
 #pragma unroll
@@ -435,7 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                                       z * xsum_b[t * p.kb_max + kb];
                         fin[t] = fmaf((float)v, s * xscale_b[t * p.kb_max + kb], fin[t]);
                     }
-                if (++kb == KB || u + 1 == u1) {  // the CTA's part of row tile rt is complete
+                if (++kb == KB || last_unit) {  // the CTA's part of row tile rt is complete
                     const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
                     if (cb && ce) {
                         ++n_full;
@@ -455,6 +455,48 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     kb = 0;
                     ++rt;
                 }
+            };
+            for (uint32_t j0 = 0; j0 < n; j0 += kGroup, ++G) {
+                const uint32_t gs = G % kNG, nreal = min((uint32_t)kGroup, n - j0);
+                QIL_TR(3, guard.wait_mbar(dfull0 + 8 * gs, (G / kNG) & 1));  // all units of the group are accumulated
+                tc_fence_after();
+                for (uint32_t b0 = 0; b0 < nreal; b0 += kEB) {
+                    uint32_t dl[kEB][8], dh[kEB][8], meta[kEB];
+#pragma unroll
+                    for (int i = 0; i < kEB; ++i) {
+#pragma unroll
+                        for (int q = 0; q < kDCols; ++q) dl[i][q] = dh[i][q] = 0u;
+                        meta[i] = 0u;
+                        if (b0 + i < nreal) {
+                            const uint32_t a = gs * kGroup + b0 + i;
+                            const uint32_t td = tmem + lane_base + kColD + 16 * a;
+                            tmem_ld<kDCols>(td, dl[i]);
+                            tmem_ld<kDCols>(td + 8, dh[i]);
+                            meta[i] = tmem_ld1(tmem + lane_base + kColMeta + a);
+                        }
+                    }
+                    QIL_TR(4, asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"));
+#pragma unroll
+                    for (int i = 0; i < kEB; ++i) {  // no use of the loaded registers is scheduled before the wait
+#pragma unroll
+                        for (int q = 0; q < kDCols; ++q) {
+                            asm volatile("" : "+r"(dl[i][q]));
+                            asm volatile("" : "+r"(dh[i][q]));
+                        }
+                        asm volatile("" : "+r"(meta[i]));
+                    }
+                    if (b0 + kEB >= nreal) {  // the group's columns may be reused
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(dempty0 + 8 * gs);
+                    }
+#pragma unroll
+                    for (int i = 0; i < kEB; ++i)
+                        if (b0 + i < nreal) {
+                            QIL_TR_COUNT(5);
+                            consume(dl[i], dh[i], meta[i], j0 + b0 + i + 1 == n);
+                        }
+                }
             }
             __syncwarp();
             if (lane == 0) {
@@ -463,7 +505,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             }
             if (shares) ++he;
             if (n_full && p.tiles_done) {
-                group_sync<1>();  // every row of the tiles is written
+                QIL_TR(6, group_sync<1>());  // every row of the tiles is written
                 if (r == 0) {
                     __threadfence();
                     red_release_add(p.tiles_done, n_full);
@@ -487,13 +529,16 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
             float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
             if (st == 0) {
-                guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1);
+                QIL_TR(1, guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1));
                 if (E.flags & kFlagDep) {
                     const unsigned int need = E.tiles_before;
-                    guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; });
+                    QIL_TR(2, guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; }));
                 }
             }
             group_sync<2>();
+#ifdef QIL_TRACE
+            const long long tr_conv0 = clock64();
+#endif
             const uint32_t nblk = min(KB, wk.u1 - wk.u0), kb0 = wk.u0 % KB;
             const uint32_t p_half = (uint32_t)l16 >> 3, cc = ((uint32_t)l16 >> 2) & 1, m = (uint32_t)l16 & 3;
             for (int t = 0; t < E.M; ++t) {
@@ -553,6 +598,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read xs through the async proxy
             group_sync<2>();
+#ifdef QIL_TRACE
+            tr[3] += clock64() - tr_conv0;
+#endif
             if (st == 0) mbar_arrive(xfull0 + 8 * xb);
             ++xe;
         }
@@ -580,10 +628,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 // checked now, while the units are still being computed
                 for (int t = 0; t < M; ++t) {
                     const unsigned long long* q = my_slot + t * kUnitRows;
-                    guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; });
+                    QIL_TR(1, guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; }));
                 }
             }
-            guard.wait_mbar(hfull0 + 8 * (he & 1), (he >> 1) & 1);
+            QIL_TR(2, guard.wait_mbar(hfull0 + 8 * (he & 1), (he >> 1) & 1));
             if (have_last) {  // publish first (a chain of CTAs must never wait on each other in a circle)
                 for (int t = 0; t < M; ++t)
                     __stcg(my_slot + t * kUnitRows,
@@ -601,16 +649,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     const uint32_t which = (cu0 / KB == t_first) ? 0u : 1u;
                     unsigned long long* src = slots + (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + r;
                     unsigned long long got[kXR];
-                    guard.wait_flag([&] {
+                    QIL_TR(3, guard.wait_flag([&] {
                         bool all = true;
-#pragma unroll
                         for (int t = 0; t < kXR; ++t)
                             if (t < M) {
                                 got[t] = __ldcg(src + t * kUnitRows);
                                 all &= (uint32_t)(got[t] >> 32) == tag;
                             }
                         return all;
-                    });
+                    }));
 #pragma unroll
                     for (int t = 0; t < kXR; ++t)
                         if (t < M) {
@@ -637,33 +684,42 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             }
         }
     } else if (tid < kProdBase) {
-        // ======================= MMA issuer (one thread) =======================
-        if (tid == kMmaBase) {
-            uint32_t xe = 0;
-            Cyc ab(kNB);
+        // ======================= MMA issuers (one thread in each of kGroup warps) =======================
+        // Issuing one tcgen05.mma costs a thread some 50 cycles, far more than the instruction occupies the tensor
+        // core at 8 columns; issuer w therefore takes slot w of every group, so kGroup units are issued in parallel.
+        if ((tid & 31) == 0) {
+            const uint32_t w = (uint32_t)(tid - kMmaBase) >> 5;
+            uint32_t xe = 0, G = 0;
             Walk wk(p, c);
             const uint64_t desc_hi = smem_desc(0, kLbo);
             constexpr uint32_t lbo16 = (uint32_t)kLbo >> 4;
             while (wk.next_entry()) {
-                const uint32_t KB = wk.KB;
+                const uint32_t KB = wk.KB, n = wk.u1 - wk.u0;
                 const uint32_t xb = xe & 1;
-                guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1);
+                QIL_TR(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1));
                 ++xe;
                 const uint32_t xs16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
-                uint32_t kb = wk.u0 % KB;
-                for (uint32_t u = wk.u0; u < wk.u1; ++u) {
-                    const uint32_t a = ab.idx;
-                    guard.wait_mbar(afull0 + 8 * a, ab.ph);  // (the unpack warps waited for the accumulators to be free)
-                    tc_fence_after();
-                    const uint32_t ta = tmem + 32 * a, td = tmem + kColD + 16 * a;
-                    const uint64_t b0 = desc_hi | (uint64_t)(xs16 + kb * 8 * lbo16);
-                    mma_i8_ts(td, ta, b0, 0u);                    // low nibbles, columns [0, 64)
-                    mma_i8_ts(td, ta + 8, b0 + 4 * lbo16, 1u);    // low nibbles, columns [64, 128)
-                    mma_i8_ts(td + 8, ta + 16, b0 + 2 * lbo16, 0u);   // high nibbles
-                    mma_i8_ts(td + 8, ta + 24, b0 + 6 * lbo16, 1u);
-                    tc_commit(dfull0 + 8 * a);
-                    ab.step();
-                    if (++kb == KB) kb = 0;
+                uint32_t kb = (wk.u0 + w) % KB;
+                const uint32_t kstep = kGroup % KB;
+                for (uint32_t j = w; j < (n + kGroup - 1) / kGroup * kGroup; j += kGroup, ++G) {
+                    const uint32_t gs = G % kNG, gph = (G / kNG) & 1;
+                    if (j < n) {
+                        const uint32_t a = gs * kGroup + w;
+                        QIL_TR(2, guard.wait_mbar(afull0 + 8 * a, gph));  // (the unpack warps waited for the accumulators to be free)
+                        tc_fence_after();
+                        const uint32_t ta = tmem + 32 * a, td = tmem + kColD + 16 * a;
+                        const uint64_t b0 = desc_hi | (uint64_t)(xs16 + kb * 8 * lbo16);
+                        mma_i8_ts(td, ta, b0, 0u);                        // low nibbles, columns [0, 64)
+                        mma_i8_ts(td, ta + 8, b0 + 4 * lbo16, 1u);        // low nibbles, columns [64, 128)
+                        mma_i8_ts(td + 8, ta + 16, b0 + 2 * lbo16, 0u);   // high nibbles
+                        mma_i8_ts(td + 8, ta + 24, b0 + 6 * lbo16, 1u);
+                        tc_commit(dfull0 + 8 * gs);
+                    } else {  // the entry ends inside the group: this slot stays empty; its barriers still change phase
+                        mbar_arrive_n(afull0 + 8 * (gs * kGroup + w), 4);
+                        mbar_arrive(dfull0 + 8 * gs);
+                    }
+                    kb += kstep;
+                    if (kb >= KB) kb -= KB;
                 }
             }
         }
@@ -676,7 +732,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             while (wk.next_entry()) {
                 const unsigned char* wbase = p.e[wk.ei].w;
                 for (uint32_t u = wk.u0; u < wk.u1; ++u, ++issued) {
-                    guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1);
+                    QIL_TR(1, guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1));
                     mbar_expect_tx(full0 + 8 * rs.idx, kUnitBytes);
                     bulk_g2s(smem_u32(ring + (size_t)rs.idx * kUnitBytes), wbase + (size_t)u * kUnitBytes, kUnitBytes,
                              full0 + 8 * rs.idx);
@@ -691,6 +747,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             }
         }
     }
+#ifdef QIL_TRACE
+    tr[0] = clock64() - tr_begin;
+    if (p.trace && (tid & 31) == 0) {
+        unsigned long long* o = p.trace + ((size_t)blockIdx.x * 32 + (tid >> 5)) * 16;
+        for (int i = 0; i < 16; ++i) o[i] = (unsigned long long)tr[i];
+    }
+#endif
     // nobody leaves before every copy has landed and every role is done; then tensor memory is released
     tc_fence_before();
     __syncthreads();
@@ -729,6 +792,10 @@ __global__ void __launch_bounds__(256) pack_stream128_kernel(const uint8_t* __re
         out[i] = word;
     }
 }
+
+#ifdef QIL_TRACE
+unsigned long long* g_trace = nullptr;
+#endif
 
 struct SmemPlan {
     int x_rows, xbuf_bytes, stages;
@@ -825,6 +892,9 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
         p.status = reinterpret_cast<int*>(ws);
         p.tiles_done = any_dep ? reinterpret_cast<unsigned int*>(ws) + 1 : nullptr;
         p.slots = reinterpret_cast<unsigned char*>(ws) + kWsHeader;
+#ifdef QIL_TRACE
+        p.trace = g_trace;
+#endif
         if (any_dep && cudaMemsetAsync(reinterpret_cast<unsigned int*>(ws) + 1, 0, 4, st) != cudaSuccess) {
             (void)cudaGetLastError();
             return QIL_ERR_CUDA;
@@ -841,3 +911,7 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
 }
 
 }  // namespace qil
+
+#ifdef QIL_TRACE
+extern "C" void qil_trace_set_tc(unsigned long long* t) { qil::g_trace = t; }
+#endif

@@ -22,23 +22,29 @@
 // stream of units; CTA c of C owns units [c q + min(c, r), ...) with q = units / C, r = units % C.
 //
 // Roles in a CTA (one CTA per SM, alive for the whole list):
-//   producer (1 thread)   streams the CTA's units through a shared-memory ring (cp.async.bulk +
-//                         mbarrier), running ahead across linears as far as the ring allows, so
-//                         HBM keeps streaming while the consumers wait for a dependency;
-//   unpack warpgroups     take turns on units: shared memory -> nibble split -> tensor memory;
-//   MMA issuer (1 thread) four tcgen05.mma per unit, completion signalled by tcgen05.commit;
-//   epilogue warpgroup    thread = weight row: accumulators -> fp32 row sums (kept in registers
-//                         over the units of a row tile) -> bf16 outputs of row tiles the CTA owns
-//                         entirely, or a hand-over of the partial sums of a row tile it shares;
-//   stager warpgroup      waits for QIL_DEP_PREVIOUS, loads and converts the activation blocks the
-//                         CTA's units need (double buffered, one linear ahead);
-//   fixer warpgroup       all cross-CTA work: publishes the partial sums of a shared row tile as
-//                         {value, tag} pairs (one 8-byte store each, tag = entry index + 1) into a
-//                         ring of slots in the workspace, completes the row tile whose end the CTA
-//                         owns by adding the contributions in CTA order (bit-reproducible), and
-//                         counts finished row tiles for the dependency counter.
-// Every wait is bounded (2 s); on expiry QIL_ERR_TIMEOUT is recorded in the workspace status
-// word, waiting stops, tensor memory is released and the kernel returns.
+//   producer (1 thread)    streams the CTA's units through a shared-memory ring (cp.async.bulk +
+//                          mbarrier), running ahead across linears as far as the ring allows, so
+//                          HBM keeps streaming while the consumers wait for a dependency;
+//   unpack warpgroups (3)  take turns on units: shared memory -> nibble split -> tensor memory;
+//   MMA issuers (4 x 1 thread) units are handled in groups of four, issuer w takes slot w of
+//                          every group: four tcgen05.mma per unit, completion by tcgen05.commit;
+//   epilogue warpgroups (2) alternate groups; thread = weight row: accumulators -> fp32 row sums
+//                          (kept in registers over the units of a row tile); at the end of a row
+//                          tile the second warpgroup's sums are added to the first's, which
+//                          writes the bf16 outputs of row tiles the CTA owns entirely, or hands
+//                          over the partial sums of a row tile it shares;
+//   stager (4 warps)       waits for QIL_DEP_PREVIOUS, loads and converts the activation blocks the
+//                          CTA's units need (double buffered, one linear ahead);
+//   fixer (2 warps)        all cross-CTA work: publishes the partial sums of a shared row tile as
+//                          {value, tag} pairs (one 8-byte store each, tag = entry index + 1) into a
+//                          ring of slots in the workspace, completes the row tile whose end the CTA
+//                          owns by adding the contributions in CTA order (bit-reproducible), and
+//                          counts finished quarter tiles for the dependency counter.
+// No role uses a named barrier: every hand-over is an mbarrier or a flag in global memory, and
+// every wait is bounded (2 s).  When a wait runs out, QIL_ERR_TIMEOUT is recorded in the
+// workspace status word (with the place in words 2..5 of the workspace), every role stops at its
+// next wait without issuing further work, outstanding copies and tensor-core operations are
+// waited for, tensor memory is released and the kernel returns.
 #include <mutex>
 
 #include "qil_common.cuh"
@@ -46,15 +52,16 @@
 // Optional per-warp timing (compile with -DQIL_TRACE): cycles spent in the waits of every role, written to a
 // buffer set with qil_trace_set_tc().  Nothing is skipped or reordered; without the macro the hooks vanish.
 #ifdef QIL_TRACE
-#define QIL_TR(slot, ...)                    \
-    do {                                     \
-        const long long tr_t0_ = clock64();  \
-        __VA_ARGS__;                         \
-        tr[slot] += clock64() - tr_t0_;      \
-    } while (0)
+#define QIL_WAIT(slot, ...)                          \
+    ([&] {                                           \
+        const long long tr_t0_ = clock64();          \
+        const bool tr_ok_ = (__VA_ARGS__);           \
+        tr[slot] += clock64() - tr_t0_;              \
+        return tr_ok_;                               \
+    }())
 #define QIL_TR_COUNT(slot) tr[slot] += 1
 #else
-#define QIL_TR(slot, ...) __VA_ARGS__
+#define QIL_WAIT(slot, ...) (__VA_ARGS__)
 #define QIL_TR_COUNT(slot)
 #endif
 
@@ -66,13 +73,16 @@ constexpr int kUnitRows = 128;
 constexpr int kUnitBytes = 8192 + 512;
 constexpr int kNumWg = 3;                        // unpack warpgroups
 constexpr int kUnpackThreads = 128 * kNumWg;
-constexpr int kEpiBase = kUnpackThreads;         // epilogue warpgroup (its warps keep warp % 4 = lane quarter)
-constexpr int kStagerBase = kEpiBase + 128;
+constexpr int kNumEpi = 2;                       // epilogue warpgroups (they alternate groups of units)
+constexpr int kEpiBase = kUnpackThreads;         // (their warps keep warp % 4 = lane quarter)
+constexpr int kStagerBase = kEpiBase + 128 * kNumEpi;
 constexpr int kFixBase = kStagerBase + 128;
+constexpr int kFixThreads = 64;                  // fixer: two warps, two rows of the tile per thread
 constexpr int kGroup = 4;                        // units per group: one per MMA issuer, one epilogue pass
-constexpr int kMmaBase = kFixBase + 128;         // kGroup warps, one issuing thread each
+constexpr int kMmaBase = kFixBase + kFixThreads; // kGroup warps, one issuing thread each
 constexpr int kProdBase = kMmaBase + 32 * kGroup;  // one warp, one thread issues
 constexpr int kThreads = kProdBase + 32;
+static_assert(kThreads <= 1024, "block size");
 constexpr int kNG = 2;                           // groups in flight in tensor memory
 constexpr int kNB = kGroup * kNG;                // = units in flight
 constexpr int kTmemCols = 512;
@@ -142,6 +152,14 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+__device__ __forceinline__ uint32_t lds_acquire(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_release(uint32_t addr, uint32_t v) {
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
 __device__ __forceinline__ uint32_t ld_acquire(const unsigned int* p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -149,10 +167,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const unsigned int* p) {
 }
 __device__ __forceinline__ void red_release_add(unsigned int* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-template <int kId>
-__device__ __forceinline__ void group_sync() {  // the 128 threads of one role
-    asm volatile("bar.sync %0, 128;" ::"n"(kId) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -209,41 +223,89 @@ __device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint
 }
 
 // ---- bounded waits ----------------------------------------------------------------------------
+// A wait returns true when what it waited for has happened, false when the kernel is being abandoned: a wait ran out
+// (here or in another role; the shared flag `poisoned` is then set and QIL_ERR_TIMEOUT recorded).  A role that gets
+// false stops working and goes to the end of the kernel: it issues no further copies, tensor-core operations or
+// barrier arrivals.
 struct Guard {
     int* status;
     volatile int* poisoned;
-    __device__ __forceinline__ void fail() const {
-        if (!*poisoned) {
-            *poisoned = 1;
-            atomicOr(status, (int)QIL_ERR_TIMEOUT);
-        }
-    }
+#ifdef QIL_TRACE
+    long long* polls;  // failed polls of this thread
+#endif
     static __device__ __forceinline__ unsigned long long now_ns() {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         return t;
     }
-    __device__ __forceinline__ void wait_mbar(uint32_t bar, uint32_t parity) const {
-        if (mbar_try_wait(bar, parity)) return;
-        if (*poisoned) return;
+    // Diagnostics of the first wait that ran out, in words 2..5 of the workspace header: 1 + CTA, thread,
+    // shared-memory address of the barrier (0 for a flag in global memory), parity waited for.
+    static __device__ __forceinline__ void note_timeout(int* status, uint32_t bar, uint32_t parity) {
+        if (atomicCAS(reinterpret_cast<unsigned int*>(status) + 2, 0u, 1u + blockIdx.x) == 0u) {
+            status[3] = (int)threadIdx.x;
+            status[4] = (int)bar;
+            status[5] = (int)parity;
+        }
+    }
+    __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity) const {
+        if (mbar_try_wait(bar, parity)) return true;
+#ifdef QIL_TRACE
+        return wait_mbar_slow(status, poisoned, bar, parity, polls);
+#else
+        return wait_mbar_slow(status, poisoned, bar, parity);
+#endif
+    }
+    // (out of line, scalar arguments: the common case above stays one instruction and a branch)
+    static __device__ __noinline__ bool wait_mbar_slow(int* status, volatile int* poisoned, uint32_t bar, uint32_t parity
+#ifdef QIL_TRACE
+                                                       , long long* polls
+#endif
+    ) {
+        if (*poisoned) return false;
         const unsigned long long t0 = now_ns();
         for (;;) {
-            if (mbar_try_wait(bar, parity)) return;
-            if (*poisoned || now_ns() - t0 > kWaitLimitNs) break;
+            if (mbar_try_wait(bar, parity)) return true;
+#ifdef QIL_TRACE
+            *polls += 1;
+#endif
+            if (*poisoned) return false;
+            if (now_ns() - t0 > kWaitLimitNs) break;
         }
-        fail();
+        *poisoned = 1;
+        atomicOr(status, (int)QIL_ERR_TIMEOUT);
+        note_timeout(status, bar, parity);
+        return false;
+    }
+    // Waits until the counter at shared address `cnt` (one writer, never decreasing) has reached `need`.  The
+    // counter is the truth; the mbarrier `bar`, which completes a phase each time all such counters have advanced,
+    // only lets the thread sleep in between (its parity alone could not tell one completed phase from three).
+    __device__ __forceinline__ bool wait_count(uint32_t cnt, uint32_t need, uint32_t bar) const {
+        for (;;) {
+            const uint32_t v = lds_acquire(cnt);
+            if (v >= need) return true;
+            if (!wait_mbar(bar, v & 1)) return false;
+        }
     }
     template <typename Pred>
-    __device__ __forceinline__ void wait_flag(Pred done) const {
-        if (done()) return;
-        if (*poisoned) return;
+    __device__ __forceinline__ bool wait_flag(Pred done) const {
+        if (done()) return true;
+        if (*poisoned) return false;
         const unsigned long long t0 = now_ns();
         for (uint32_t i = 1;; ++i) {
-            if (done()) return;
+            if (done()) return true;
+#ifdef QIL_TRACE
+            *polls += 1;
+#endif
             if (i > 8) __nanosleep(i < 64 ? 32 : 256);
-            if ((i & 15u) == 0 && (*poisoned || now_ns() - t0 > kWaitLimitNs)) break;
+            if ((i & 15u) == 0) {
+                if (*poisoned) return false;
+                if (now_ns() - t0 > kWaitLimitNs) break;
+            }
         }
-        fail();
+        *poisoned = 1;
+        atomicOr(status, (int)QIL_ERR_TIMEOUT);
+        note_timeout(status, 0u, 0u);
+        return false;
     }
 };
 
@@ -303,15 +365,19 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     int* xsum = reinterpret_cast<int*>(xs + (size_t)2 * p.xbuf_bytes);              // [2][kXR][kb_max]
     float* xscale = reinterpret_cast<float*>(xsum + 2 * kXR * p.kb_max);            // [2][kXR][kb_max]
     float* hand = xscale + 2 * kXR * p.kb_max;                                      // [2][2][kXR][128]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(hand + 2 * 2 * kXR * kUnitRows);
+    float* tpart = hand + 2 * 2 * kXR * kUnitRows;                                  // [2][kXR][128]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tpart + 2 * kXR * kUnitRows);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
     // afull: per unit slot; dfull / dempty: per group of kGroup slots
     const uint32_t afull0 = smem_u32(b2), dfull0 = smem_u32(b2 + kNB), dempty0 = smem_u32(b2 + kNB + kNG);
     uint64_t* b3 = b2 + 3 * kNB;
     const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2), hfull0 = smem_u32(b3 + 4), hempty0 = smem_u32(b3 + 6);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 8);
+    const uint32_t tfull0 = smem_u32(b3 + 8), tempty0 = smem_u32(b3 + 10), mdone0 = smem_u32(b3 + 12);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 12 + kGroup);
     volatile int* poisoned = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // rd[gs][q]: groups of slot group gs that epilogue warp q (tensor-memory lanes 32q..32q+31) has read out
+    const uint32_t rd0 = smem_u32(tmem_slot + 2);
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -324,12 +390,17 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             mbar_init(dempty0 + 8 * i, 4);      // the epilogue warps
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(xfull0 + 8 * i, 1);
-            mbar_init(xempty0 + 8 * i, 4);
+            mbar_init(xfull0 + 8 * i, 4);  // the stager warps
+            mbar_init(xempty0 + 8 * i, 4 * kNumEpi);
             mbar_init(hfull0 + 8 * i, 4);
-            mbar_init(hempty0 + 8 * i, 4);
+            mbar_init(hempty0 + 8 * i, kFixThreads / 32);
+            mbar_init(tfull0 + 8 * i, 4);
+            mbar_init(tempty0 + 8 * i, 4);
         }
+        for (int i = 0; i < kGroup; ++i) mbar_init(mdone0 + 8 * i, 1);
         *poisoned = 0;
+        for (int i = 0; i < 4 * kNG; ++i) tmem_slot[2 + i] = 0u;
+        if (blockIdx.x == 0) p.status[6] = (int)full0;  // (reference for the time-out diagnostics)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < 2 * p.xbuf_bytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(xs)[i] = 0u;
@@ -343,88 +414,149 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const Guard guard{p.status, poisoned};
 #ifdef QIL_TRACE
     long long tr[16];
     for (int i = 0; i < 16; ++i) tr[i] = 0;
     const long long tr_begin = clock64();
+    const Guard guard{p.status, poisoned, &tr[15]};
+#else
+    const Guard guard{p.status, poisoned};
 #endif
 
     if (tid < kUnpackThreads) {
         // ======================= unpack warpgroups: shared memory -> nibble split -> tensor memory =======================
         const uint32_t wg = tid >> 7, r = tid & 127, lane = tid & 31;
         const uint32_t lane_base = (r & ~31u) << 16;  // this warp's quarter of the tensor-memory lanes
-        Cyc rs(p.stages), turn(kNumWg);  // advance once per unit of the CTA
-        uint32_t G = 0;                  // groups so far: unit j of an entry sits in group G + j / kGroup, slot j % kGroup
+        const uint32_t S = (uint32_t)p.stages;
+        uint32_t stage0 = 0, ph0 = 0, turn0 = 0;  // ring stage / phase / turn of the entry's first unit
+        uint32_t G = 0;                           // groups so far: unit j of an entry sits in group G + j / kGroup, slot j % kGroup
+        bool alive = true;
         Walk wk(p, c);
-        while (wk.next_entry()) {
+        while (alive && wk.next_entry()) {
             const uint32_t n = wk.u1 - wk.u0;
-            for (uint32_t j = 0; j < n; ++j) {
-                if (turn.idx == wg) {
-                    const uint32_t g = G + j / kGroup, a = (g % kNG) * kGroup + j % kGroup, gph = (g / kNG) & 1;
-                    QIL_TR(1, guard.wait_mbar(dempty0 + 8 * (g % kNG), gph ^ 1));  // the group that used these columns has been read out
-                    QIL_TR(2, guard.wait_mbar(full0 + 8 * rs.idx, rs.ph));
-                    QIL_TR_COUNT(3);
-                    tc_fence_after();
-                    const unsigned char* ub = ring + (size_t)rs.idx * kUnitBytes;
-                    const uint32_t ta = tmem + lane_base + 32 * a;
-                    constexpr uint32_t kLo = 0x0F0F0F0Fu, kHi = 0xF0F0F0F0u;
-                    uint4 w[4];
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) w[ch] = *reinterpret_cast<const uint4*>(ub + ((size_t)ch * kUnitRows + r) * 16);
-                    const uint32_t meta = *reinterpret_cast<const uint32_t*>(ub + 8192 + 4 * r);
-                    uint32_t v[16];
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        v[4 * ch] = w[ch].x & kLo; v[4 * ch + 1] = w[ch].y & kLo; v[4 * ch + 2] = w[ch].z & kLo; v[4 * ch + 3] = w[ch].w & kLo;
-                    }
-                    tmem_st16(ta, v);       // A of the two low-nibble MMAs: columns [0, 64) and [64, 128) of the block
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        v[4 * ch] = w[ch].x & kHi; v[4 * ch + 1] = w[ch].y & kHi; v[4 * ch + 2] = w[ch].z & kHi; v[4 * ch + 3] = w[ch].w & kHi;
-                    }
-                    tmem_st16(ta + 16, v);  // A of the two high-nibble MMAs (values x 16)
-                    tmem_st1(tmem + lane_base + kColMeta + a, meta);
-                    QIL_TR(4, asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"));
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(afull0 + 8 * a);
-                        mbar_arrive(empty0 + 8 * rs.idx);
-                    }
+            uint32_t j = wg >= turn0 ? wg - turn0 : wg + kNumWg - turn0;  // this warpgroup's first unit of the entry
+            uint32_t st_i = stage0 + j, st_ph = ph0;
+            if (st_i >= S) { st_i -= S; st_ph ^= 1; }
+            for (; j < n; j += kNumWg) {
+                const uint32_t g = G + j / kGroup, a = (g % kNG) * kGroup + j % kGroup;
+                // the groups that used these columns before have been read out (by the epilogue warp of the same
+                // lanes); the unit has landed
+                if (!QIL_WAIT(1, guard.wait_count(rd0 + 4 * ((g % kNG) * 4 + (r >> 5)), g / kNG, dempty0 + 8 * (g % kNG))) ||
+                    !QIL_WAIT(2, guard.wait_mbar(full0 + 8 * st_i, st_ph))) {
+                    alive = false;
+                    break;
                 }
-                rs.step();
-                turn.step();
+                QIL_TR_COUNT(3);
+                tc_fence_after();
+                const unsigned char* ub = ring + (size_t)st_i * kUnitBytes;
+                const uint32_t ta = tmem + lane_base + 32 * a;
+                constexpr uint32_t kLo = 0x0F0F0F0Fu, kHi = 0xF0F0F0F0u;
+                uint4 w[4];
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) w[ch] = *reinterpret_cast<const uint4*>(ub + ((size_t)ch * kUnitRows + r) * 16);
+                const uint32_t meta = *reinterpret_cast<const uint32_t*>(ub + 8192 + 4 * r);
+                uint32_t v[16];
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    v[4 * ch] = w[ch].x & kLo; v[4 * ch + 1] = w[ch].y & kLo; v[4 * ch + 2] = w[ch].z & kLo; v[4 * ch + 3] = w[ch].w & kLo;
+                }
+                tmem_st16(ta, v);       // A of the two low-nibble MMAs: columns [0, 64) and [64, 128) of the block
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    v[4 * ch] = w[ch].x & kHi; v[4 * ch + 1] = w[ch].y & kHi; v[4 * ch + 2] = w[ch].z & kHi; v[4 * ch + 3] = w[ch].w & kHi;
+                }
+                tmem_st16(ta + 16, v);  // A of the two high-nibble MMAs (values x 16)
+                tmem_st1(tmem + lane_base + kColMeta + a, meta);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(afull0 + 8 * a);
+                    mbar_arrive(empty0 + 8 * st_i);
+                }
+                st_i += kNumWg;
+                if (st_i >= S) { st_i -= S; st_ph ^= 1; }
             }
             G += (n + kGroup - 1) / kGroup;
+            turn0 = (turn0 + n) % kNumWg;
+            const uint32_t adv = stage0 + n;
+            ph0 ^= (adv / S) & 1;
+            stage0 = adv % S;
         }
     } else if (tid < kStagerBase) {
-        // ======================= epilogue warpgroup (thread = weight row of the unit) =======================
-        const uint32_t r = tid - kEpiBase, lane = tid & 31;
+        // ======================= epilogue warpgroups (thread = weight row of the unit) =======================
+        // Warpgroup ew takes the groups G with G % kNumEpi == ew; both follow every unit to know where row tiles end.
+        // At the end of a row tile warpgroup 1 leaves its partial sums in shared memory, warpgroup 0 adds them to
+        // its own (always in that order) and writes the tile out or hands it to the fixer.
+        const uint32_t ew = (uint32_t)(tid - kEpiBase) >> 7, r = (uint32_t)(tid - kEpiBase) & 127, lane = tid & 31;
         const uint32_t lane_base = (r & ~31u) << 16;
         constexpr int kEB = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;  // units read back per tcgen05.wait::ld
-        uint32_t xe = 0, he = 0, G = 0;
+        uint32_t xe = 0, he = 0, G = 0, ts = 0;               // ts: row tiles closed so far
+        bool alive = true;
         Walk wk(p, c);
-        while (wk.next_entry()) {
+        while (alive && wk.next_entry()) {
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, n = u1 - u0;
             const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
             const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
             const uint32_t xb = xe & 1;
-            QIL_TR(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1));
+            if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1))) break;
             ++xe;
             const int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
             const float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
             float* hand_b = hand + (size_t)(he & 1) * 2 * kXR * kUnitRows;
-            if (shares) QIL_TR(2, guard.wait_mbar(hempty0 + 8 * (he & 1), ((he >> 1) & 1) ^ 1));
+            if (shares && ew == 0 && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * (he & 1), ((he >> 1) & 1) ^ 1))) break;
             uint32_t n_full = 0;
             float fin[kXR];
 #pragma unroll
             for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
             uint32_t rt = t_first, kb = u0 - t_first * KB;
-            // one unit: fold scale and zero point into the row sums; close the row tile when its last unit is in
-            auto consume = [&](const uint32_t (&cl)[8], const uint32_t (&ch)[8], uint32_t meta, bool last_unit) {
+            // the CTA's part of row tile rt is complete
+            auto close_tile = [&]() {
+                const uint32_t tb = ts & 1, tph = (ts >> 1) & 1;
+                float* tp = tpart + (size_t)tb * kXR * kUnitRows + r;
+                if (ew != 0) {
+                    if (!QIL_WAIT(6, guard.wait_mbar(tempty0 + 8 * tb, tph ^ 1))) {
+                        alive = false;
+                        return;
+                    }
+#pragma unroll
+                    for (int t = 0; t < kXR; ++t) tp[t * kUnitRows] = fin[t];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tfull0 + 8 * tb);
+                } else {
+                    if (!QIL_WAIT(6, guard.wait_mbar(tfull0 + 8 * tb, tph))) {
+                        alive = false;
+                        return;
+                    }
+#pragma unroll
+                    for (int t = 0; t < kXR; ++t) fin[t] += tp[t * kUnitRows];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty0 + 8 * tb);
+                    const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
+                    if (cb && ce) {
+                        ++n_full;
+                        const uint32_t row = rt * kUnitRows + r;
+                        if (row < (uint32_t)N) {
+#pragma unroll
+                            for (int t = 0; t < kXR; ++t)
+                                if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(fin[t]);
+                        }
+                    } else {  // first tile cut at its beginning (completed by the fixer) or last tile continued elsewhere
+                        float* dst = hand_b + (size_t)(ce ? 0 : 1) * kXR * kUnitRows + r;
+#pragma unroll
+                        for (int t = 0; t < kXR; ++t) dst[t * kUnitRows] = fin[t];
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
+                kb = 0;
+                ++rt;
+                ++ts;
+            };
+            // one unit of this warpgroup: fold scale and zero point into the row sums
+            auto consume = [&](const uint32_t (&cl)[8], const uint32_t (&ch)[8], uint32_t meta) {
                 const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
                 const float s = __low2float(sz);
                 const int z = (int)__high2float(sz);
@@ -435,32 +567,20 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                                       z * xsum_b[t * p.kb_max + kb];
                         fin[t] = fmaf((float)v, s * xscale_b[t * p.kb_max + kb], fin[t]);
                     }
-                if (++kb == KB || last_unit) {  // the CTA's part of row tile rt is complete
-                    const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
-                    if (cb && ce) {
-                        ++n_full;
-                        const uint32_t row = rt * kUnitRows + r;
-                        if (row < (uint32_t)N) {
-#pragma unroll
-                            for (int t = 0; t < kXR; ++t)
-                                if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(fin[t]);
-                        }
-                    } else {  // first tile cut at its beginning (completed here) or last tile continued elsewhere
-                        float* dst = hand_b + (size_t)(ce ? 0 : 1) * kXR * kUnitRows + r;
-#pragma unroll
-                        for (int t = 0; t < kXR; ++t) dst[t * kUnitRows] = fin[t];
-                    }
-#pragma unroll
-                    for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
-                    kb = 0;
-                    ++rt;
-                }
             };
-            for (uint32_t j0 = 0; j0 < n; j0 += kGroup, ++G) {
+            for (uint32_t j0 = 0; alive && j0 < n; j0 += kGroup, ++G) {
                 const uint32_t gs = G % kNG, nreal = min((uint32_t)kGroup, n - j0);
-                QIL_TR(3, guard.wait_mbar(dfull0 + 8 * gs, (G / kNG) & 1));  // all units of the group are accumulated
+                if (G % kNumEpi != ew) {  // the other warpgroup's units: only follow the row tiles
+                    for (uint32_t i = 0; alive && i < nreal; ++i)
+                        if (++kb == KB || j0 + i + 1 == n) close_tile();
+                    continue;
+                }
+                if (!QIL_WAIT(3, guard.wait_mbar(dfull0 + 8 * gs, (G / kNG) & 1))) {  // all units of the group are accumulated
+                    alive = false;
+                    break;
+                }
                 tc_fence_after();
-                for (uint32_t b0 = 0; b0 < nreal; b0 += kEB) {
+                for (uint32_t b0 = 0; alive && b0 < nreal; b0 += kEB) {
                     uint32_t dl[kEB][8], dh[kEB][8], meta[kEB];
 #pragma unroll
                     for (int i = 0; i < kEB; ++i) {
@@ -475,7 +595,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             meta[i] = tmem_ld1(tmem + lane_base + kColMeta + a);
                         }
                     }
-                    QIL_TR(4, asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                     for (int i = 0; i < kEB; ++i) {  // no use of the loaded registers is scheduled before the wait
 #pragma unroll
@@ -488,37 +608,40 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     if (b0 + kEB >= nreal) {  // the group's columns may be reused
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(dempty0 + 8 * gs);
+                        if (lane == 0) {
+                            sts_release(rd0 + 4 * (gs * 4 + (r >> 5)), G / kNG + 1);
+                            mbar_arrive(dempty0 + 8 * gs);
+                        }
                     }
 #pragma unroll
                     for (int i = 0; i < kEB; ++i)
-                        if (b0 + i < nreal) {
+                        if (alive && b0 + i < nreal) {
                             QIL_TR_COUNT(5);
-                            consume(dl[i], dh[i], meta[i], j0 + b0 + i + 1 == n);
+                            consume(dl[i], dh[i], meta[i]);
+                            if (++kb == KB || j0 + b0 + i + 1 == n) close_tile();
                         }
                 }
             }
+            if (!alive) break;
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(xempty0 + 8 * xb);
-                if (shares) mbar_arrive(hfull0 + 8 * (he & 1));
-            }
-            if (shares) ++he;
-            if (n_full && p.tiles_done) {
-                QIL_TR(6, group_sync<1>());  // every row of the tiles is written
-                if (r == 0) {
+                if (shares && ew == 0) mbar_arrive(hfull0 + 8 * (he & 1));
+                // the dependency counter counts quarter tiles (32 rows), so that no warp has to wait for another
+                if (ew == 0 && n_full && p.tiles_done) {
                     __threadfence();
                     red_release_add(p.tiles_done, n_full);
                 }
             }
+            if (shares) ++he;
         }
     } else if (tid < kFixBase) {
-        // ======================= activation stager (thread pairs of a half warp = one 128-column block) =======================
+        // ======================= activation stager (a half warp = one 128-column block per pass) =======================
         // bf16 row -> per 128 columns: e with max|x| / 2^e <= 32639, v = rint(x / 2^e) = 256 hi + lo (both int8),
         // X = sum v.  Only the blocks the CTA's units touch are converted.  K order of the operand inside a block:
         // 16-byte chunk 4p + 2h + cc (p: half of the block, h: low / high nibble columns, cc: 32-column chunk of
-        // the half), byte 4m + b = column 64p + 32cc + 8m + 4h + b.
-        const int st = tid - kStagerBase, l16 = st & 15, hw = st >> 4;
+        // the half), byte 4m + b = column 64p + 32cc + 8m + 4h + b.  The four warps work independently.
+        const int st = tid - kStagerBase, lane = tid & 31, l16 = st & 15, hw = st >> 4;
         uint32_t xe = 0;
         Walk wk(p, c);
         while (wk.next_entry()) {
@@ -528,14 +651,16 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             unsigned char* xs_b = xs + (size_t)xb * p.xbuf_bytes;
             int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
             float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
-            if (st == 0) {
-                QIL_TR(1, guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1));
-                if (E.flags & kFlagDep) {
-                    const unsigned int need = E.tiles_before;
-                    QIL_TR(2, guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; }));
+            bool ok = true;
+            if (lane == 0) {  // the buffer is free; the rows of x are written (quarter tiles of all earlier entries)
+                ok = QIL_WAIT(1, guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1));
+                if (ok && (E.flags & kFlagDep)) {
+                    const unsigned int need = 4u * E.tiles_before;
+                    ok = QIL_WAIT(2, guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; }));
                 }
             }
-            group_sync<2>();
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
 #ifdef QIL_TRACE
             const long long tr_conv0 = clock64();
 #endif
@@ -543,74 +668,89 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const uint32_t p_half = (uint32_t)l16 >> 3, cc = ((uint32_t)l16 >> 2) & 1, m = (uint32_t)l16 & 3;
             for (int t = 0; t < E.M; ++t) {
                 const uint16_t* xrow = E.x + (size_t)t * E.K;
-                for (uint32_t ib = 0; ib < nblk; ib += 8) {
-                    const uint32_t i = ib + hw;
-                    const bool valid = i < nblk;
-                    uint32_t kb = kb0 + i;
-                    if (kb >= KB) kb -= KB;
-                    uint4 raw = make_uint4(0, 0, 0, 0);
-                    if (valid) raw = __ldcg(reinterpret_cast<const uint4*>(xrow + (size_t)kb * 128 + l16 * 8));
-                    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
-                    uint32_t amax = 0;  // bf16 magnitudes order like unsigned integers
+                // up to four passes of 8 blocks at a time: their loads are all in flight before the first conversion
+                for (uint32_t ib0 = 0; ib0 < nblk; ib0 += 32) {
+                    uint4 raws[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) amax = max(amax, max((u[j] << 16) & 0x7FFFFFFFu, u[j] & 0x7FFF0000u));
-#pragma unroll
-                    for (int o = 1; o < 16; o <<= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-                    // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field F -> e = F - 127 - 14, one
-                    // more when the mantissa exceeds 32639/16384 (for bf16: all seven mantissa bits set)
-                    int ef = (int)(amax >> 23);
-                    if (ef < 1 || ef >= 255) ef = 127 + 14;  // zero / subnormal / non-finite block: scale 1
-                    int e = ef - 127 - 14 + (((amax & 0x7FFFFFu) > 0x7EFE00u) ? 1 : 0);
-                    if (e < -126) e = -126;
-                    const float inv = __uint_as_float((uint32_t)(127 - e) << 23);  // 2^-e
-                    // v = rint(x * 2^-e) through the 1.5 * 2^23 trick; v + 128 = 256 * hi + (lo + 128)
-                    uint32_t vb[8];
-                    int sum = 0;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float f0 = fmaf(__uint_as_float(u[j] << 16), inv, 12582912.f);
-                        const float f1 = fmaf(__uint_as_float(u[j] & 0xFFFF0000u), inv, 12582912.f);
-                        const int q0 = (int)(__float_as_uint(f0) - 0x4B400000u), q1 = (int)(__float_as_uint(f1) - 0x4B400000u);
-                        sum += q0 + q1;
-                        vb[2 * j] = (uint32_t)(q0 + 128);
-                        vb[2 * j + 1] = (uint32_t)(q1 + 128);
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t i = ib0 + 8 * q + hw;
+                        uint32_t kb = kb0 + i;
+                        if (kb >= KB) kb -= KB;
+                        raws[q] = make_uint4(0, 0, 0, 0);
+                        if (i < nblk) raws[q] = __ldcg(reinterpret_cast<const uint4*>(xrow + (size_t)kb * 128 + l16 * 8));
                     }
+#pragma unroll 1
+                    for (int q = 0; q < 4; ++q) {
+                        if (ib0 + 8 * q >= nblk) break;  // (uniform over the warp: the shuffles below need every lane)
+                        const uint32_t i = ib0 + 8 * q + hw;
+                        const bool valid = i < nblk;
+                        uint32_t kb = kb0 + i;
+                        if (kb >= KB) kb -= KB;
+                        const uint4 raw = q == 0 ? raws[0] : q == 1 ? raws[1] : q == 2 ? raws[2] : raws[3];
+                        const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+                        uint32_t amax = 0;  // bf16 magnitudes order like unsigned integers
 #pragma unroll
-                    for (int o = 1; o < 16; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-                    if (valid) {
-                        // byte 0 of each (v + 128) is lo + 128, byte 1 is hi; columns 0-3 of the piece sit under low
-                        // nibbles, columns 4-7 under high nibbles
-                        const uint32_t lo_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0040), __byte_perm(vb[2], vb[3], 0x0040), 0x5410) ^ 0x80808080u;
-                        const uint32_t lo_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
-                        const uint32_t hi_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
-                        const uint32_t hi_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
-                        unsigned char* dst = xs_b + (size_t)(kb * 8 + 4 * p_half + cc) * kLbo + (size_t)(2 * t) * 16 + 4 * m;
-                        *reinterpret_cast<uint32_t*>(dst) = hi_a;
-                        *reinterpret_cast<uint32_t*>(dst + 16) = lo_a;
-                        *reinterpret_cast<uint32_t*>(dst + 2 * kLbo) = hi_b;
-                        *reinterpret_cast<uint32_t*>(dst + 2 * kLbo + 16) = lo_b;
-                        if (l16 == 0) {
-                            xsum_b[t * p.kb_max + kb] = sum;
-                            xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);
+                        for (int j = 0; j < 4; ++j) amax = max(amax, max((u[j] << 16) & 0x7FFFFFFFu, u[j] & 0x7FFF0000u));
+#pragma unroll
+                        for (int o = 1; o < 16; o <<= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                        // 2^e = smallest power of two with max|x| / 2^e <= 32639: exponent field F -> e = F - 127 - 14, one
+                        // more when the mantissa exceeds 32639/16384 (for bf16: all seven mantissa bits set)
+                        int ef = (int)(amax >> 23);
+                        if (ef < 1 || ef >= 255) ef = 127 + 14;  // zero / subnormal / non-finite block: scale 1
+                        int e = ef - 127 - 14 + (((amax & 0x7FFFFFu) > 0x7EFE00u) ? 1 : 0);
+                        if (e < -126) e = -126;
+                        const float inv = __uint_as_float((uint32_t)(127 - e) << 23);  // 2^-e
+                        // v = rint(x * 2^-e) through the 1.5 * 2^23 trick; v + 128 = 256 * hi + (lo + 128)
+                        uint32_t vb[8];
+                        int sum = 0;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float f0 = fmaf(__uint_as_float(u[j] << 16), inv, 12582912.f);
+                            const float f1 = fmaf(__uint_as_float(u[j] & 0xFFFF0000u), inv, 12582912.f);
+                            const int q0 = (int)(__float_as_uint(f0) - 0x4B400000u), q1 = (int)(__float_as_uint(f1) - 0x4B400000u);
+                            sum += q0 + q1;
+                            vb[2 * j] = (uint32_t)(q0 + 128);
+                            vb[2 * j + 1] = (uint32_t)(q1 + 128);
+                        }
+#pragma unroll
+                        for (int o = 1; o < 16; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                        if (valid) {
+                            // byte 0 of each (v + 128) is lo + 128, byte 1 is hi; columns 0-3 of the piece sit under low
+                            // nibbles, columns 4-7 under high nibbles
+                            const uint32_t lo_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0040), __byte_perm(vb[2], vb[3], 0x0040), 0x5410) ^ 0x80808080u;
+                            const uint32_t lo_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
+                            const uint32_t hi_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
+                            const uint32_t hi_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
+                            unsigned char* dst = xs_b + (size_t)(kb * 8 + 4 * p_half + cc) * kLbo + (size_t)(2 * t) * 16 + 4 * m;
+                            *reinterpret_cast<uint32_t*>(dst) = hi_a;
+                            *reinterpret_cast<uint32_t*>(dst + 16) = lo_a;
+                            *reinterpret_cast<uint32_t*>(dst + 2 * kLbo) = hi_b;
+                            *reinterpret_cast<uint32_t*>(dst + 2 * kLbo + 16) = lo_b;
+                            if (l16 == 0) {
+                                xsum_b[t * p.kb_max + kb] = sum;
+                                xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);
+                            }
                         }
                     }
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read xs through the async proxy
-            group_sync<2>();
+            __syncwarp();
 #ifdef QIL_TRACE
             tr[3] += clock64() - tr_conv0;
 #endif
-            if (st == 0) mbar_arrive(xfull0 + 8 * xb);
+            if (lane == 0) mbar_arrive(xfull0 + 8 * xb);
             ++xe;
         }
     } else if (tid < kMmaBase) {
-        // ======================= fixer warpgroup (thread = row of the tile): all cross-CTA work =======================
-        const uint32_t r = tid - kFixBase, lane = tid & 31;
+        // ======================= fixer (two warps, thread = two rows of the tile): all cross-CTA work =======================
+        const uint32_t fr = tid - kFixBase, lane = tid & 31;
+        constexpr uint32_t kRowsPer = kUnitRows / kFixThreads;
         unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
         uint32_t he = 0;
+        bool alive = true;
         Walk wk(p, c);
-        while (wk.next_entry()) {
+        while (alive && wk.next_entry()) {
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1;
@@ -623,65 +763,81 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             unsigned long long* my_slot = nullptr;
             if (have_last) {
                 const uint32_t which = (t_last == t_first) ? 0u : 1u;
-                my_slot = slots + (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems + r;
+                my_slot = slots + (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems;
                 // the slot must have been consumed (tags cleared) by whoever completed the tile it last served;
                 // checked now, while the units are still being computed
-                for (int t = 0; t < M; ++t) {
-                    const unsigned long long* q = my_slot + t * kUnitRows;
-                    QIL_TR(1, guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; }));
-                }
+                for (uint32_t h = 0; alive && h < kRowsPer; ++h)
+                    for (int t = 0; alive && t < M; ++t) {
+                        const unsigned long long* q = my_slot + t * kUnitRows + fr + h * kFixThreads;
+                        alive = QIL_WAIT(1, guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; }));
+                    }
             }
-            QIL_TR(2, guard.wait_mbar(hfull0 + 8 * (he & 1), (he >> 1) & 1));
+            alive = alive && QIL_WAIT(2, guard.wait_mbar(hfull0 + 8 * (he & 1), (he >> 1) & 1));
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive) break;
             if (have_last) {  // publish first (a chain of CTAs must never wait on each other in a circle)
-                for (int t = 0; t < M; ++t)
-                    __stcg(my_slot + t * kUnitRows,
-                           ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(hand_b[(kXR + t) * kUnitRows + r]));
+                for (uint32_t h = 0; h < kRowsPer; ++h) {
+                    const uint32_t r = fr + h * kFixThreads;
+                    for (int t = 0; t < M; ++t)
+                        __stcg(my_slot + t * kUnitRows + r,
+                               ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(hand_b[(kXR + t) * kUnitRows + r]));
+                }
             }
             if (have_first) {
                 const uint32_t c_lo = owner_of(E.q, E.rem, t_first * KB);
-                float sum[kXR];
+                float sum[kRowsPer][kXR];
 #pragma unroll
-                for (int t = 0; t < kXR; ++t) sum[t] = 0.f;
+                for (uint32_t h = 0; h < kRowsPer; ++h)
+#pragma unroll
+                    for (int t = 0; t < kXR; ++t) sum[h][t] = 0.f;
                 for (uint32_t cc = c_lo; cc < c; ++cc) {
                     uint32_t cu0, cu1;
                     slice_of(E.q, E.rem, cc, cu0, cu1);
                     if (cu0 == cu1) continue;
                     const uint32_t which = (cu0 / KB == t_first) ? 0u : 1u;
-                    unsigned long long* src = slots + (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + r;
-                    unsigned long long got[kXR];
-                    QIL_TR(3, guard.wait_flag([&] {
+                    unsigned long long* src = slots + (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + fr;
+                    unsigned long long got[kRowsPer][kXR];
+                    alive = QIL_WAIT(3, guard.wait_flag([&] {
                         bool all = true;
-                        for (int t = 0; t < kXR; ++t)
-                            if (t < M) {
-                                got[t] = __ldcg(src + t * kUnitRows);
-                                all &= (uint32_t)(got[t] >> 32) == tag;
-                            }
+                        for (uint32_t h = 0; h < kRowsPer; ++h)
+                            for (int t = 0; t < kXR; ++t)
+                                if (t < M) {
+                                    got[h][t] = __ldcg(src + t * kUnitRows + h * kFixThreads);
+                                    all &= (uint32_t)(got[h][t] >> 32) == tag;
+                                }
                         return all;
                     }));
+                    alive = __all_sync(0xffffffffu, alive);
+                    if (!alive) break;
 #pragma unroll
-                    for (int t = 0; t < kXR; ++t)
-                        if (t < M) {
-                            if ((uint32_t)(got[t] >> 32) == tag) sum[t] += __uint_as_float((uint32_t)got[t]);
-                            __stcg(src + t * kUnitRows, 0ull);  // consumed: the slot may be reused
-                        }
+                    for (uint32_t h = 0; h < kRowsPer; ++h)
+#pragma unroll
+                        for (int t = 0; t < kXR; ++t)
+                            if (t < M) {
+                                sum[h][t] += __uint_as_float((uint32_t)got[h][t]);
+                                __stcg(src + t * kUnitRows + h * kFixThreads, 0ull);  // consumed: the slot may be reused
+                            }
                 }
-                const uint32_t row = t_first * kUnitRows + r;
-                if (row < (uint32_t)N) {
+                if (!alive) break;
 #pragma unroll
-                    for (int t = 0; t < kXR; ++t)
-                        if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(sum[t] + hand_b[t * kUnitRows + r]);
+                for (uint32_t h = 0; h < kRowsPer; ++h) {
+                    const uint32_t r = fr + h * kFixThreads, row = t_first * kUnitRows + r;
+                    if (row < (uint32_t)N) {
+#pragma unroll
+                        for (int t = 0; t < kXR; ++t)
+                            if (t < M) E.y[(size_t)t * N + row] = __float2bfloat16_rn(sum[h][t] + hand_b[t * kUnitRows + r]);
+                    }
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(hempty0 + 8 * (he & 1));
-            ++he;
-            if (have_first && p.tiles_done) {
-                group_sync<3>();  // every row of the tile is written
-                if (r == 0) {
+            if (lane == 0) {
+                mbar_arrive(hempty0 + 8 * (he & 1));
+                if (have_first && p.tiles_done) {  // this warp's rows of the tile are written: kRowsPer quarter tiles
                     __threadfence();
-                    red_release_add(p.tiles_done, 1u);
+                    red_release_add(p.tiles_done, kRowsPer);
                 }
             }
+            ++he;
         }
     } else if (tid < kProdBase) {
         // ======================= MMA issuers (one thread in each of kGroup warps) =======================
@@ -690,13 +846,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         if ((tid & 31) == 0) {
             const uint32_t w = (uint32_t)(tid - kMmaBase) >> 5;
             uint32_t xe = 0, G = 0;
+            bool alive = true, issued = false;
             Walk wk(p, c);
             const uint64_t desc_hi = smem_desc(0, kLbo);
             constexpr uint32_t lbo16 = (uint32_t)kLbo >> 4;
-            while (wk.next_entry()) {
+            while (alive && wk.next_entry()) {
                 const uint32_t KB = wk.KB, n = wk.u1 - wk.u0;
                 const uint32_t xb = xe & 1;
-                QIL_TR(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1));
+                if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1))) break;
                 ++xe;
                 const uint32_t xs16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
                 uint32_t kb = (wk.u0 + w) % KB;
@@ -705,7 +862,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     const uint32_t gs = G % kNG, gph = (G / kNG) & 1;
                     if (j < n) {
                         const uint32_t a = gs * kGroup + w;
-                        QIL_TR(2, guard.wait_mbar(afull0 + 8 * a, gph));  // (the unpack warps waited for the accumulators to be free)
+                        if (!QIL_WAIT(2, guard.wait_mbar(afull0 + 8 * a, gph))) {  // (the unpack warps waited for the accumulators to be free)
+                            alive = false;
+                            break;
+                        }
                         tc_fence_after();
                         const uint32_t ta = tmem + 32 * a, td = tmem + kColD + 16 * a;
                         const uint64_t b0 = desc_hi | (uint64_t)(xs16 + kb * 8 * lbo16);
@@ -714,7 +874,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         mma_i8_ts(td + 8, ta + 16, b0 + 2 * lbo16, 0u);   // high nibbles
                         mma_i8_ts(td + 8, ta + 24, b0 + 6 * lbo16, 1u);
                         tc_commit(dfull0 + 8 * gs);
-                    } else {  // the entry ends inside the group: this slot stays empty; its barriers still change phase
+                        issued = true;
+                    } else {
+                        // The entry ends inside the group: this slot stays empty, its barriers still change phase.  Like
+                        // the unpack warps the thread first waits until the groups that used these columns before have
+                        // been read out: an arrival must never reach a barrier whose previous phase is still collecting.
+                        for (uint32_t q = 0; alive && q < 4; ++q)
+                            alive = QIL_WAIT(2, guard.wait_count(rd0 + 4 * (gs * 4 + q), G / kNG, dempty0 + 8 * gs));
+                        if (!alive) break;
                         mbar_arrive_n(afull0 + 8 * (gs * kGroup + w), 4);
                         mbar_arrive(dfull0 + 8 * gs);
                     }
@@ -722,28 +889,41 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     if (kb >= KB) kb -= KB;
                 }
             }
+            // whatever happened to the other roles: the operations this thread issued are complete before tensor memory
+            // is released (this wait also holds in an abandoned kernel)
+            if (issued) {
+                tc_commit(mdone0 + 8 * w);
+                const unsigned long long t0 = Guard::now_ns();
+                while (!mbar_try_wait(mdone0 + 8 * w, 0) && Guard::now_ns() - t0 < kWaitLimitNs) {}
+            }
         }
     } else {
         // ======================= producer (one thread) =======================
         if (tid == kProdBase) {
             Cyc rs(p.stages);
             uint32_t issued = 0;
+            bool alive = true;
             Walk wk(p, c);
-            while (wk.next_entry()) {
+            while (alive && wk.next_entry()) {
                 const unsigned char* wbase = p.e[wk.ei].w;
                 for (uint32_t u = wk.u0; u < wk.u1; ++u, ++issued) {
-                    QIL_TR(1, guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1));
+                    if (!QIL_WAIT(1, guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1))) {
+                        alive = false;
+                        break;
+                    }
                     mbar_expect_tx(full0 + 8 * rs.idx, kUnitBytes);
                     bulk_g2s(smem_u32(ring + (size_t)rs.idx * kUnitBytes), wbase + (size_t)u * kUnitBytes, kUnitBytes,
                              full0 + 8 * rs.idx);
                     rs.step();
                 }
             }
-            // every copy issued must have landed before the CTA may retire
+            // every copy issued must have landed before the CTA may retire (rs names the stage after the last one
+            // issued; this wait also holds in an abandoned kernel)
             for (uint32_t back = 0; back < (uint32_t)p.stages && back < issued; ++back) {
                 if (rs.idx == 0) { rs.idx = p.stages; rs.ph ^= 1; }
                 --rs.idx;
-                guard.wait_mbar(full0 + 8 * rs.idx, rs.ph);
+                const unsigned long long t0 = Guard::now_ns();
+                while (!mbar_try_wait(full0 + 8 * rs.idx, rs.ph) && Guard::now_ns() - t0 < kWaitLimitNs) {}
             }
         }
     }
@@ -810,11 +990,12 @@ SmemPlan plan_for(int max_m, int kb_max) {
     const int lbo = 32 * pl.x_rows;
     pl.xbuf_bytes = kb_max * 8 * lbo + 128;  // the last chunk's 8-row window reaches past its own rows
     const size_t fixed = (size_t)2 * pl.xbuf_bytes + (size_t)2 * 2 * pl.x_rows * kb_max * 4 +
-                         (size_t)2 * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 8) * 8 + 16 + 128;
+                         (size_t)3 * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 12 + kGroup) * 8 + 16 + 16 * kNG + 128;
     pl.stages = 0;
     if (fixed < kSmemLimit) {
         long s = (long)((kSmemLimit - fixed) / (kUnitBytes + 16));
         if (s > 24) s = 24;
+        s -= s % kNumWg;  // a ring stage is then always consumed by the same unpack warpgroup, which sees each of its phases
         pl.stages = (int)s;
     }
     pl.total = fixed + (size_t)pl.stages * (kUnitBytes + 16);

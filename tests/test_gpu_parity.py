@@ -513,6 +513,45 @@ def test_w4a16_tc_batch_with_dependencies(api):
         cur_bits = wl.f32_to_bf16_bits(y_ref.astype(np.float32))
 
 
+def test_w4a16_tc_long_list_without_dependencies(api):
+    """Six decoder layers of Llama-2-7B shaped linears in one list, no entry waiting for another: CTAs and the
+    roles inside a CTA drift apart by several linears, which exercises every ring (slots between CTAs, buffers
+    between roles) in its blocking state.  Each output must equal, bit for bit, the same linear run alone."""
+    import ctypes as C
+    import torch
+    from paper_2412_01034_b200 import _lib
+    lib = _lib.load()
+    G, M = 128, 1
+    shapes = {"sq": (4096, 4096), "up": (11008, 4096), "down": (4096, 11008)}
+    packs = {}
+    for i, (name, (N, K)) in enumerate(shapes.items()):
+        w = wl.normal_weights(322, i, N, K, 0.02, outlier_prob=0.001)
+        q = c_oracle.quantize_rtn_w4_asym(w, G)
+        packs[name] = api.pack_stream128_w4(cuda(q[0]), cuda(q[1]), cuda(q[2]), G)
+    layer = ["sq", "sq", "sq", "sq", "up", "up", "down"]
+    names = layer * 6
+    xs = {K: to_bf16_cuda(wl.normal_activations_bf16(322, 50 + j, M, K)) for j, K in enumerate((4096, 11008))}
+    ys = [torch.zeros((M, shapes[nm][0]), dtype=torch.bfloat16, device="cuda") for nm in names]
+    descs = (_lib.LinearDesc * len(names))()
+    for i, nm in enumerate(names):
+        N, K = shapes[nm]
+        d = descs[i]
+        d.x, d.qweight, d.y = xs[K].data_ptr(), packs[nm].data_ptr(), ys[i].data_ptr()
+        d.scales = d.zeros = None
+        d.M, d.N, d.K, d.group_size, d.layout, d.flags = M, N, K, G, api.LAYOUT_STREAM128, 0
+    ws = api.new_workspace(api.linear_w4a16_workspace_size(M, 11008, 11008, G))
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    alone = {nm: api.linear_w4a16(xs[shapes[nm][1]], packs[nm], None, None, shapes[nm][0], G, api.LAYOUT_STREAM128,
+                                  workspace=ws) for nm in shapes}
+    for rep in range(3):
+        assert lib.qil_linear_w4a16_batch(descs, len(names), C.c_void_p(ws.data_ptr()), ws.numel(), st) == 0
+        torch.cuda.synchronize()
+        assert _status(api, ws) == 0
+        for i, nm in enumerate(names):
+            np.testing.assert_array_equal(bits_of(ys[i]), bits_of(alone[nm]))
+            ys[i].zero_()
+
+
 # ----------------------------------------------------------------------------
 # W4A4
 # ----------------------------------------------------------------------------

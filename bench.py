@@ -188,9 +188,9 @@ def run_qil(args):
         v, cores, sample = oracle_sample(args.cpu_budget_s, 32)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
 
-    layout = {"stream128": api.LAYOUT_STREAM128, "stream": api.LAYOUT_STREAM, "tile16": api.LAYOUT_TILE16,
+    layout = {"stream128": api.LAYOUT_STREAM128, "tile16": api.LAYOUT_TILE16,
               "canonical": api.LAYOUT_CANONICAL}[args.layout]
-    persistent = args.layout in ("stream", "stream128")
+    persistent = args.layout == "stream128"
     model = llama_decode.QuantisedLinears(cfg=1, M=1, n_layers=args.layers, layout=layout, deps=args.deps,
                                           device=f"cuda:{local_rank}")
     stream = torch.cuda.Stream(device=dev)
@@ -249,7 +249,7 @@ def run_qil(args):
         peak = float(peaks.get("hbm_gbs", 6650.0))
         peak_kind = "measured copy bandwidth (MEASURED_PEAKS.json)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
         launches_per_step = 1 if persistent else model.count
-        kernel = {"stream128": "w4a16_tc_kernel", "stream": "w4a16_stream_kernel"}.get(args.layout, "w4a16_skinny_kernel<1>")
+        kernel = "w4a16_tc_kernel<1>" if persistent else "w4a16_skinny_kernel<1>"
         per_launch_bytes = bytes_per_step / launches_per_step
         per_launch_ms = ms / launches_per_step          # average over the timed region, launch gaps included
         achieved = per_launch_bytes / (per_launch_ms * 1e-3) / 1e9
@@ -285,7 +285,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=70)
     ap.add_argument("--impl", default="qil", choices=["qil", "reference"])
     ap.add_argument("--layers", type=int, default=32, help="decoder layers (32 = the stated workload)")
-    ap.add_argument("--layout", default="stream128", choices=["stream128", "stream", "tile16", "canonical"])
+    ap.add_argument("--layout", default="stream128", choices=["stream128", "tile16", "canonical"])
     ap.add_argument("--deps", default="layer", choices=["layer", "all", "none"],
                     help="which linears wait for all earlier ones (layer = data flow of a decoder layer)")
     ap.add_argument("--cpu-budget-s", type=float, default=12.0)

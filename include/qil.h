@@ -66,16 +66,6 @@ typedef enum { QIL_F32 = 0, QIL_BF16 = 1, QIL_F16 = 2 } qil_dtype;
  *   each.  Word (n, i) is at ((n/16)*(K/128) + i/16)*256 + (n%16)*16 + i%16.
  *   Needs N % 16 == 0 and K % 128 == 0.  A warp of the decode kernel reads one
  *   tile (1 KiB) with two fully coalesced 512-byte loads.
- * QIL_LAYOUT_STREAM   : self-contained units for the persistent decode kernel,
- *   built by qil_pack_stream_w4 from codes, scales and zeros.  Unit u =
- *   (n/16)*(K/128) + k/128 occupies bytes [1088 u, 1088 (u+1)): first 1024
- *   bytes of codes, 16 rows x 16 words as in a TILE16 tile, except that inside
- *   each word byte b holds code b in its low and code 4 + b in its high nibble
- *   (code k of the 8 sits at nibble 2 (k % 4) + k / 4); then 16 pairs {fp16 scale,
- *   fp16 zero}, one per row of the tile, valid for that 128-column block (a
- *   group larger than 128 repeats its pair in every block it covers).
- *   Needs N % 16 == 0, K % 128 == 0, group_size % 128 == 0.  With group 128 the
- *   buffer is exactly as large as canonical codes + scales + zeros.
  * QIL_LAYOUT_STREAM128: units for the tensor-memory (tcgen05) decode kernel, built by
  *   qil_pack_stream128_w4.  Unit u = (n/128)*(K/128) + k/128 occupies bytes
  *   [8704 u, 8704 (u+1)): 4 chunks (32 columns of K each) x 128 rows x 16 bytes of
@@ -87,7 +77,6 @@ typedef enum { QIL_F32 = 0, QIL_BF16 = 1, QIL_F16 = 2 } qil_dtype;
 typedef enum {
     QIL_LAYOUT_CANONICAL = 0,
     QIL_LAYOUT_TILE16 = 1,
-    QIL_LAYOUT_STREAM = 2,
     QIL_LAYOUT_STREAM128 = 3
 } qil_layout;
 
@@ -119,13 +108,9 @@ qil_status qil_pack_w4(const uint8_t* codes, int N, int K, qil_layout layout, ui
 qil_status qil_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout, int is_signed,
                          uint8_t* codes, qil_stream_t stream);
 
-/* Builds the QIL_LAYOUT_STREAM buffer (qil_stream_w4_bytes(N, K) bytes) from unsigned
- * codes [N][K], fp16 scales and fp16 zeros [N][K/group_size].
- * Errors: NULL, SHAPE (N % 16, K % 128, group_size % 128, K % group_size), ALIGN. */
-size_t qil_stream_w4_bytes(int N, int K);
-qil_status qil_pack_stream_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K,
-                              int group_size, void* out, qil_stream_t stream);
-/* Same for QIL_LAYOUT_STREAM128 (N >= 1, K % 128 == 0, group_size % 128 == 0). */
+/* Builds the QIL_LAYOUT_STREAM128 buffer (qil_stream128_w4_bytes(N, K) bytes) from unsigned codes [N][K], fp16
+ * scales and fp16 zeros [N][K/group_size].
+ * Errors: NULL, SHAPE (N < 1, K % 128, group_size % 128, K % group_size), ALIGN. */
 size_t qil_stream128_w4_bytes(int N, int K);
 qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K,
                                  int group_size, void* out, qil_stream_t stream);
@@ -139,10 +124,10 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  * The kernel is chosen from the shape: tensor-core skinny kernel (weights read
  * once, any M handled in slabs of 64 rows) when K % 128 == 0 and
  * group_size % 128 == 0; a general kernel otherwise (any K % 8 == 0, any
- * group_size dividing K, canonical layout only).  With QIL_LAYOUT_STREAM
- * or QIL_LAYOUT_STREAM128 (both M <= 4) a persistent streaming kernel runs;
+ * group_size dividing K, canonical layout only).  With QIL_LAYOUT_STREAM128
+ * (M <= 4) the persistent streaming kernel runs;
  * scales and zeros are part of the buffer, the two arguments are ignored and
- * may be null; the workspace is always needed.  Both streaming kernels convert
+ * may be null; the workspace is always needed.  The streaming kernel converts
  * the activations to 16-bit block fixed point (per 128 columns a power-of-two
  * scale, |integer| <= 32639) and accumulates exactly in int32; the conversion
  * error per element is at most 2^-16 of the block maximum.
@@ -151,7 +136,9 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  * (the kernels leave it zeroed again).  Calls that share a workspace must not
  * overlap on the device.  Its first int is a status word: the streaming kernel
  * ORs QIL_ERR_TIMEOUT into it if one of its bounded waits ever runs out (read it
- * with qil_device_status; after such an error re-zero the workspace).
+ * with qil_device_status; words 2..5 of the workspace then tell where: 1 + CTA,
+ * thread, shared-memory address of the barrier or 0, parity; after such an
+ * error re-zero the workspace).
  * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, CUDA.
  * ---------------------------------------------------------------------- */
 size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size);
@@ -196,8 +183,8 @@ qil_status qil_linear_w4a16_static_ws(const void* x, const uint32_t* qweight, co
  * QIL_DEP_PREVIOUS in `flags`: it then starts only after every earlier entry has
  * written all of its outputs.  Entries without the flag may overlap with their
  * predecessors (q, k and v of one layer share an input and need no flag).
- * When every entry uses QIL_LAYOUT_STREAM, or every entry uses
- * QIL_LAYOUT_STREAM128, the whole list runs as one persistent kernel.  All pointers inside a descriptor are device
+ * When every entry uses QIL_LAYOUT_STREAM128, the whole list runs as one
+ * persistent kernel.  All pointers inside a descriptor are device
  * pointers; the descriptor array itself is host memory and is consumed before
  * the call returns.  workspace must be as large as the largest
  * qil_linear_w4a16_workspace_size() over the entries (zero-filled once).

@@ -204,40 +204,6 @@ def from_layout(flat: np.ndarray, N: int, K: int, layout: int) -> np.ndarray:
     raise ValueError("unknown layout")
 
 
-def to_stream(packed: np.ndarray, scales, zeros, group_size: int) -> np.ndarray:
-    """Canonical packed words [N][K/8] + fp16 scales/zeros [N][K/G] -> the STREAM byte buffer.
-
-    Unit u = (n // 16) * (K // 128) + kb holds, at byte 1088 * u: the 16 x 16 words of the tile
-    (rows n//16*16 .. +15, words 16*kb .. 16*kb+15, row after row, little endian), then for each of
-    the 16 rows the fp16 scale followed by the fp16 zero of the group that contains block kb.
-    Inside a word, byte b holds element b in its low and element 4 + b in its high nibble
-    (element k sits at nibble 2 * (k % 4) + k // 4).
-    """
-    p = np.asarray(packed, dtype=np.uint32)
-    N, Wd = p.shape
-    K = Wd * 8
-    G = int(group_size)
-    if N % 16 or K % 128 or G % 128 or K % G:
-        raise ValueError("STREAM layout needs N % 16 == 0, K % 128 == 0, G % 128 == 0")
-    s16 = np.ascontiguousarray(scales, dtype=np.float16).view(np.uint16)
-    z16 = np.ascontiguousarray(zeros, dtype=np.float16).view(np.uint16)
-    KB = K // 128
-    out = np.zeros((N // 16) * KB * 1088, dtype=np.uint8)
-    for rt in range(N // 16):
-        for kb in range(KB):
-            base = (rt * KB + kb) * 1088
-            canon = p[rt * 16:rt * 16 + 16, kb * 16:kb * 16 + 16]
-            tile = np.zeros_like(canon)
-            for k in range(8):
-                tile |= ((canon >> np.uint32(4 * k)) & np.uint32(0xF)) << np.uint32(4 * (2 * (k % 4) + k // 4))
-            out[base:base + 1024] = np.ascontiguousarray(tile).view(np.uint8).reshape(-1)
-            meta = np.empty((16, 2), dtype=np.uint16)
-            meta[:, 0] = s16[rt * 16:rt * 16 + 16, (kb * 128) // G]
-            meta[:, 1] = z16[rt * 16:rt * 16 + 16, (kb * 128) // G]
-            out[base + 1024:base + 1088] = meta.view(np.uint8).reshape(-1)
-    return out
-
-
 def to_stream128(codes: np.ndarray, scales, zeros, group_size: int) -> np.ndarray:
     """Codes uint8 [N][K] + fp16 scales/zeros [N][K/G] -> the STREAM128 byte buffer.
 

@@ -13,8 +13,6 @@ SIGNATURES = {
     "qil_quantize_rtn_w4": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _i, _vp, _vp, _vp]),
     "qil_pack_w4": (_i, [_vp, _i, _i, _i, _vp, _vp]),
     "qil_unpack_w4": (_i, [_vp, _i, _i, _i, _i, _vp, _vp]),
-    "qil_stream_w4_bytes": (_sz, [_i, _i]),
-    "qil_pack_stream_w4": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "qil_stream128_w4_bytes": (_sz, [_i, _i]),
     "qil_pack_stream128_w4": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "qil_linear_w4a16_workspace_size": (_sz, [_i, _i, _i, _i]),

@@ -14,7 +14,7 @@ from . import _lib
 
 OK = 0
 F32, BF16, F16 = 0, 1, 2
-LAYOUT_CANONICAL, LAYOUT_TILE16, LAYOUT_STREAM, LAYOUT_STREAM128 = 0, 1, 2, 3
+LAYOUT_CANONICAL, LAYOUT_TILE16, LAYOUT_STREAM128 = 0, 1, 3
 DEP_PREVIOUS = 1
 ERR_RANGE = 8
 
@@ -85,18 +85,6 @@ def pack_w4(codes, layout: int = LAYOUT_CANONICAL, stream=None):
     packed = torch.empty(shape, dtype=torch.int32, device=codes.device)
     _check(_lib.load().qil_pack_w4(_ptr(codes), N, K, int(layout), _ptr(packed), _stream(stream)))
     return packed
-
-
-def pack_stream_w4(codes, scales, zeros, group_size: int, stream=None):
-    """codes uint8 [N][K] + fp16 scales/zeros [N][K/G] -> the self-contained STREAM buffer (uint8, flat)."""
-    _need_cuda(codes, scales, zeros)
-    N, K = codes.shape
-    lib = _lib.load()
-    nbytes = int(lib.qil_stream_w4_bytes(N, K))
-    out = torch.empty((max(nbytes, 16),), dtype=torch.uint8, device=codes.device)
-    _check(lib.qil_pack_stream_w4(_ptr(codes), _ptr(scales), _ptr(zeros), N, K, int(group_size), _ptr(out),
-                                  _stream(stream)))
-    return out
 
 
 def pack_stream128_w4(codes, scales, zeros, group_size: int, stream=None):

@@ -26,7 +26,7 @@ using namespace qil;
 namespace {
 inline cudaStream_t S(qil_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
 inline bool dtype_ok(int d) { return d == QIL_F32 || d == QIL_BF16 || d == QIL_F16; }
-inline bool layout_ok(int l) { return l == QIL_LAYOUT_CANONICAL || l == QIL_LAYOUT_TILE16 || l == QIL_LAYOUT_STREAM || l == QIL_LAYOUT_STREAM128; }
+inline bool layout_ok(int l) { return l == QIL_LAYOUT_CANONICAL || l == QIL_LAYOUT_TILE16 || l == QIL_LAYOUT_STREAM128; }
 inline bool pack_layout_ok(int l) { return l == QIL_LAYOUT_CANONICAL || l == QIL_LAYOUT_TILE16; }
 }  // namespace
 
@@ -82,21 +82,6 @@ static qil_status check_pack(const void* a, const void* b, int N, int K, qil_lay
     return QIL_OK;
 }
 
-size_t qil_stream_w4_bytes(int N, int K) {
-    if (N <= 0 || K <= 0 || N % 16 != 0 || K % 128 != 0) return 0;
-    return w4a16_stream_weight_bytes(N, K);
-}
-
-qil_status qil_pack_stream_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K,
-                              int group_size, void* out, qil_stream_t stream) {
-    if (!codes || !scales || !zeros || !out) return QIL_ERR_NULL;
-    if (N <= 0 || K <= 0 || group_size <= 0 || N % 16 != 0 || K % 128 != 0 || group_size % 128 != 0 ||
-        K % group_size != 0)
-        return QIL_ERR_SHAPE;
-    if (!aligned16(codes) || !aligned16(scales) || !aligned16(zeros) || !aligned16(out)) return QIL_ERR_ALIGN;
-    return launch_pack_stream_w4(codes, scales, zeros, N, K, group_size, out, S(stream));
-}
-
 size_t qil_stream128_w4_bytes(int N, int K) {
     if (N <= 0 || K <= 0 || K % 128 != 0) return 0;
     return w4a16_tc_weight_bytes(N, K);
@@ -126,16 +111,15 @@ qil_status qil_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout
 
 static qil_status check_w4a16(const void* x, const void* qw, const void* sc, const void* z, const void* y, int M,
                               int N, int K, int G, qil_layout layout) {
-    const bool stream_layout = layout == QIL_LAYOUT_STREAM || layout == QIL_LAYOUT_STREAM128;
+    const bool stream_layout = layout == QIL_LAYOUT_STREAM128;
     if (!x || !qw || !y || (!stream_layout && (!sc || !z))) return QIL_ERR_NULL;
     if (M <= 0 || N <= 0 || K <= 0 || G <= 0 || K % 8 != 0 || K % G != 0) return QIL_ERR_SHAPE;
     if (!layout_ok(layout)) return QIL_ERR_UNSUPPORTED;
-    if ((layout == QIL_LAYOUT_TILE16 || layout == QIL_LAYOUT_STREAM) && (N % 16 != 0 || K % 128 != 0)) return QIL_ERR_SHAPE;
+    if (layout == QIL_LAYOUT_TILE16 && (N % 16 != 0 || K % 128 != 0)) return QIL_ERR_SHAPE;
     if (layout == QIL_LAYOUT_STREAM128 && K % 128 != 0) return QIL_ERR_SHAPE;
     if (stream_layout && G % 128 != 0) return QIL_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(qw) || !aligned16(y)) return QIL_ERR_ALIGN;
     if (!stream_layout && (!aligned16(sc) || !aligned16(z))) return QIL_ERR_ALIGN;
-    if (layout == QIL_LAYOUT_STREAM && !w4a16_stream_supported(M, N, K, G)) return QIL_ERR_UNSUPPORTED;
     if (layout == QIL_LAYOUT_STREAM128 && !w4a16_tc_supported(M, N, K, G)) return QIL_ERR_UNSUPPORTED;
     return QIL_OK;
 }
@@ -144,8 +128,7 @@ size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size) {
     if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0) return 0;
     if (K % 128 != 0 || group_size % 128 != 0) return 0;
     size_t a = w4a16_skinny_workspace(M, N, K, group_size);
-    const size_t b = w4a16_stream_workspace(), c = w4a16_tc_workspace();
-    if (b > a) a = b;
+    const size_t c = w4a16_tc_workspace();
     return c > a ? c : a;  // large enough for every layout
 }
 
@@ -155,12 +138,11 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
     const qil_status s = check_w4a16(x, qweight, scales, zeros, y, M, N, K, group_size, layout);
     if (s != QIL_OK) return s;
     if (workspace && !aligned16(workspace)) return QIL_ERR_ALIGN;
-    if (layout == QIL_LAYOUT_STREAM || layout == QIL_LAYOUT_STREAM128) {
+    if (layout == QIL_LAYOUT_STREAM128) {
         qil_linear_desc d;
         d.x = x; d.qweight = qweight; d.scales = nullptr; d.zeros = nullptr; d.y = y;
         d.M = M; d.N = N; d.K = K; d.group_size = group_size; d.layout = layout; d.flags = 0;
-        return layout == QIL_LAYOUT_STREAM ? launch_w4a16_stream(&d, 1, workspace, workspace_bytes, S(stream))
-                                           : launch_w4a16_tc(&d, 1, workspace, workspace_bytes, S(stream));
+        return launch_w4a16_tc(&d, 1, workspace, workspace_bytes, S(stream));
     }
     if (w4a16_skinny_supported(M, N, K, group_size, layout))
         return launch_w4a16_skinny(x, qweight, scales, zeros, y, M, N, K, group_size, layout, workspace,
@@ -175,19 +157,13 @@ qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs, int count, void*
     if (count <= 0) return QIL_ERR_SHAPE;
     if (workspace && !aligned16(workspace)) return QIL_ERR_ALIGN;
     // validate the whole list before the first launch
-    bool all_stream = true, all_tc = true;
+    bool all_tc = true;
     for (int i = 0; i < count; ++i) {
         const qil_linear_desc& d = descs[i];
         if ((d.flags & ~QIL_DEP_PREVIOUS) != 0) return QIL_ERR_UNSUPPORTED;
         const qil_status s = check_w4a16(d.x, d.qweight, d.scales, d.zeros, d.y, d.M, d.N, d.K, d.group_size,
                                          (qil_layout)d.layout);
         if (s != QIL_OK) return s;
-        if (d.layout == QIL_LAYOUT_STREAM) {
-            if (!workspace || workspace_bytes < w4a16_stream_workspace()) return QIL_ERR_WORKSPACE;
-            all_tc = false;
-            continue;
-        }
-        all_stream = false;
         if (d.layout == QIL_LAYOUT_STREAM128) {
             if (!workspace || workspace_bytes < w4a16_tc_workspace()) return QIL_ERR_WORKSPACE;
             continue;
@@ -200,7 +176,6 @@ qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs, int count, void*
             if (need > 0 && (!workspace || workspace_bytes < need)) return QIL_ERR_WORKSPACE;
         }
     }
-    if (all_stream) return launch_w4a16_stream(descs, count, workspace, workspace_bytes, S(stream));
     if (all_tc) return launch_w4a16_tc(descs, count, workspace, workspace_bytes, S(stream));
     for (int i = 0; i < count; ++i) {
         const qil_linear_desc& d = descs[i];

@@ -69,13 +69,6 @@ qil_status launch_w4a16_skinny(const void* x, const uint32_t* qw, const void* sc
                                void* y, int M, int N, int K, int G, qil_layout layout, void* ws,
                                size_t ws_bytes, cudaStream_t st);
 
-bool w4a16_stream_supported(int M, int N, int K, int G);
-size_t w4a16_stream_weight_bytes(int N, int K);
-size_t w4a16_stream_workspace();
-qil_status launch_pack_stream_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K, int G,
-                                 void* out, cudaStream_t st);
-qil_status launch_w4a16_stream(const qil_linear_desc* entries, int count, void* ws, size_t ws_bytes, cudaStream_t st);
-
 bool w4a16_tc_supported(int M, int N, int K, int G);
 size_t w4a16_tc_weight_bytes(int N, int K);
 size_t w4a16_tc_workspace();

@@ -25,14 +25,15 @@
 //   producer (1 thread)    streams the CTA's units through a shared-memory ring (cp.async.bulk +
 //                          mbarrier), running ahead across linears as far as the ring allows, so
 //                          HBM keeps streaming while the consumers wait for a dependency;
-//   unpack warpgroups (3)  take turns on units: shared memory -> nibble split -> tensor memory;
+//   unpack warpgroups      (QIL_TC_UNPACK_WGS, default 2) take turns on units: shared memory -> nibble split -> tensor memory;
 //   MMA issuers (4 x 1 thread) units are handled in groups of four, issuer w takes slot w of
 //                          every group: four tcgen05.mma per unit, completion by tcgen05.commit;
-//   epilogue warpgroups (2) alternate groups; thread = weight row: accumulators -> fp32 row sums
-//                          (kept in registers over the units of a row tile); at the end of a row
-//                          tile the second warpgroup's sums are added to the first's, which
-//                          writes the bf16 outputs of row tiles the CTA owns entirely, or hands
-//                          over the partial sums of a row tile it shares;
+//   epilogue warpgroups    (QIL_TC_EPILOGUE_WGS, default 1; two alternate groups) thread = weight
+//                          row: accumulators -> fp32 row sums (kept in registers over the units of
+//                          a row tile); with two warpgroups the second one's sums are added to the
+//                          first's at the end of a row tile; the first writes the bf16 outputs of
+//                          row tiles the CTA owns entirely, or hands over the partial sums of a row
+//                          tile it shares;
 //   stager (4 warps)       waits for QIL_DEP_PREVIOUS, loads and converts the activation blocks the
 //                          CTA's units need (double buffered, one linear ahead);
 //   fixer (2 warps)        all cross-CTA work: publishes the partial sums of a shared row tile as
@@ -71,9 +72,18 @@ namespace {
 
 constexpr int kUnitRows = 128;
 constexpr int kUnitBytes = 8192 + 512;
-constexpr int kNumWg = 3;                        // unpack warpgroups
+#ifndef QIL_TC_UNPACK_WGS
+#define QIL_TC_UNPACK_WGS 2
+#endif
+#ifndef QIL_TC_EPI_BATCH
+#define QIL_TC_EPI_BATCH 4
+#endif
+#ifndef QIL_TC_EPILOGUE_WGS
+#define QIL_TC_EPILOGUE_WGS 1
+#endif
+constexpr int kNumWg = QIL_TC_UNPACK_WGS;        // unpack warpgroups
 constexpr int kUnpackThreads = 128 * kNumWg;
-constexpr int kNumEpi = 2;                       // epilogue warpgroups (they alternate groups of units)
+constexpr int kNumEpi = QIL_TC_EPILOGUE_WGS;      // epilogue warpgroups (they alternate groups of units)
 constexpr int kEpiBase = kUnpackThreads;         // (their warps keep warp % 4 = lane quarter)
 constexpr int kStagerBase = kEpiBase + 128 * kNumEpi;
 constexpr int kFixBase = kStagerBase + 128;
@@ -490,7 +500,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // its own (always in that order) and writes the tile out or hands it to the fixer.
         const uint32_t ew = (uint32_t)(tid - kEpiBase) >> 7, r = (uint32_t)(tid - kEpiBase) & 127, lane = tid & 31;
         const uint32_t lane_base = (r & ~31u) << 16;
-        constexpr int kEB = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;  // units read back per tcgen05.wait::ld
+        constexpr int kEBmax = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;                      // (registers)
+        constexpr int kEB = QIL_TC_EPI_BATCH < kEBmax ? QIL_TC_EPI_BATCH : kEBmax;  // units read back per tcgen05.wait::ld
         uint32_t xe = 0, he = 0, G = 0, ts = 0;               // ts: row tiles closed so far
         bool alive = true;
         Walk wk(p, c);
@@ -526,14 +537,16 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tfull0 + 8 * tb);
                 } else {
-                    if (!QIL_WAIT(6, guard.wait_mbar(tfull0 + 8 * tb, tph))) {
-                        alive = false;
-                        return;
-                    }
+                    if constexpr (kNumEpi > 1) {
+                        if (!QIL_WAIT(6, guard.wait_mbar(tfull0 + 8 * tb, tph))) {
+                            alive = false;
+                            return;
+                        }
 #pragma unroll
-                    for (int t = 0; t < kXR; ++t) fin[t] += tp[t * kUnitRows];
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty0 + 8 * tb);
+                        for (int t = 0; t < kXR; ++t) fin[t] += tp[t * kUnitRows];
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty0 + 8 * tb);
+                    }
                     const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
                     if (cb && ce) {
                         ++n_full;
@@ -581,6 +594,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 }
                 tc_fence_after();
                 for (uint32_t b0 = 0; alive && b0 < nreal; b0 += kEB) {
+#ifdef QIL_TRACE
+                    const long long tr_e0 = clock64();
+#endif
                     uint32_t dl[kEB][8], dh[kEB][8], meta[kEB];
 #pragma unroll
                     for (int i = 0; i < kEB; ++i) {
@@ -595,7 +611,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             meta[i] = tmem_ld1(tmem + lane_base + kColMeta + a);
                         }
                     }
+#ifdef QIL_TRACE
+                    const long long tr_e1 = clock64();
+#endif
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#ifdef QIL_TRACE
+                    const long long tr_e2 = clock64();
+                    tr[7] += tr_e1 - tr_e0;
+                    tr[8] += tr_e2 - tr_e1;
+#endif
 #pragma unroll
                     for (int i = 0; i < kEB; ++i) {  // no use of the loaded registers is scheduled before the wait
 #pragma unroll
@@ -613,6 +637,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             mbar_arrive(dempty0 + 8 * gs);
                         }
                     }
+#ifdef QIL_TRACE
+                    const long long tr_e3 = clock64();
+                    tr[9] += tr_e3 - tr_e2;
+#endif
 #pragma unroll
                     for (int i = 0; i < kEB; ++i)
                         if (alive && b0 + i < nreal) {
@@ -620,6 +648,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             consume(dl[i], dh[i], meta[i]);
                             if (++kb == KB || j0 + b0 + i + 1 == n) close_tile();
                         }
+#ifdef QIL_TRACE
+                    asm volatile("" : "+f"(fin[0]));
+                    tr[10] += clock64() - tr_e3;
+#endif
                 }
             }
             if (!alive) break;

@@ -50,8 +50,6 @@ class QuantisedLinears:
                 codes, s, z = api.quantize_rtn_w4(wd, self.G)
                 if layout == api.LAYOUT_STREAM128:
                     self.packed.append(api.pack_stream128_w4(codes, s, z, self.G))
-                elif layout == api.LAYOUT_STREAM:
-                    self.packed.append(api.pack_stream_w4(codes, s, z, self.G))
                 else:
                     self.packed.append(api.pack_w4(codes, layout))
                 self.scales.append(s)

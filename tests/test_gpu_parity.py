@@ -274,17 +274,10 @@ def test_cfg3_shapes(api, N, K, M):
 
 
 # ----------------------------------------------------------------------------
-# W4A16, persistent streaming kernel (QIL_LAYOUT_STREAM)
+# W4A16, tensor-memory (tcgen05) decode kernel (QIL_LAYOUT_STREAM128)
 # ----------------------------------------------------------------------------
-def _stream_inputs(api, M, N, K, G, seed):
-    w = wl.normal_weights(310, seed, N, K, 0.02, outlier_prob=0.001)
-    x = wl.normal_activations_bf16(310, seed + 1, M, K)
-    codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
-    buf = api.pack_stream_w4(cuda(codes), cuda(scales), cuda(zeros), G)
-    return x, codes, scales, zeros, buf
-
-
 def _status(api, ws):
+    """The status word at the start of a workspace (0 unless a bounded device-side wait ran out)."""
     import ctypes as C
     import torch
     from paper_2412_01034_b200 import _lib
@@ -295,123 +288,6 @@ def _status(api, ws):
     return out.value
 
 
-@pytest.mark.parametrize("N,K,G", [(32, 512, 256), (48, 384, 128), (16, 128, 128)])
-def test_pack_stream_matches_oracle(api, N, K, G):
-    _, codes, scales, zeros, buf = _stream_inputs(api, 1, N, K, G, N + K)
-    ref = np_oracle.to_stream(np_oracle.pack_w4(codes), scales, zeros, G)
-    np.testing.assert_array_equal(buf.cpu().numpy()[:ref.size], ref)
-
-
-@pytest.mark.parametrize("M,N,K,G", [
-    (1, 16, 128, 128), (1, 48, 1024, 128), (3, 208, 1024, 128), (1, 4096, 4096, 128), (1, 4096, 11008, 128),
-    (1, 11008, 4096, 128), (4, 1024, 4096, 128), (3, 2064, 2176, 128), (2, 64, 1024, 256), (1, 160, 2048, 2048),
-    (1, 37008, 256, 128),
-])
-def test_w4a16_stream_shapes(api, M, N, K, G):
-    x, codes, scales, zeros, buf = _stream_inputs(api, M, N, K, G, M + N + K)
-    rows = np.arange(N) if N * K <= (1 << 24) else np.sort(np.random.default_rng(N).choice(N, 512, replace=False))
-    y_ref = c_oracle.linear_w4a16(x, codes[rows], scales[rows], zeros[rows], G)
-    ws = api.new_workspace(api.linear_w4a16_workspace_size(M, N, K, G))
-    outs = []
-    for _ in range(2):
-        y = api.linear_w4a16(to_bf16_cuda(x), buf, None, None, N, G, api.LAYOUT_STREAM, workspace=ws)
-        outs.append(y.clone())
-    assert _status(api, ws) == 0
-    assert_rows_close(bf16_to_f64(outs[0])[:, rows], y_ref)
-    np.testing.assert_array_equal(bits_of(outs[0]), bits_of(outs[1]))
-    import torch
-    # the workspace is left ready for the next call: the status word and every {value, tag} pair are zero
-    sms = torch.cuda.get_device_properties(0).multi_processor_count
-    assert int(torch.count_nonzero(ws[:4]).item()) == 0
-    assert int(torch.count_nonzero(ws[256:256 + sms * 2 * 4 * 512]).item()) == 0
-
-
-def test_w4a16_stream_batch_with_dependencies(api):
-    """A list of linears in one launch: independent entries, then a chain x -> y0 -> y1 -> y2 in which every
-    stage needs QIL_DEP_PREVIOUS.  The list must equal the same calls made one by one, and the oracle."""
-    import ctypes as C
-    import torch
-    from paper_2412_01034_b200 import _lib
-    lib = _lib.load()
-    G, M = 128, 2
-    dims = [(512, 1024), (1024, 512), (768, 1024), (256, 768)]     # (N, K); entries 1..3 chain on entry 0
-    packs, refs = [], []
-    for i, (N, K) in enumerate(dims):
-        w = wl.normal_weights(311, i, N, K, 0.05)
-        q = np_oracle.quantize_rtn_w4_asym(w, G)
-        refs.append(q)
-        packs.append(api.pack_stream_w4(cuda(q[0]), cuda(q[1]), cuda(q[2]), G))
-    x0 = wl.normal_activations_bf16(311, 100, M, dims[0][1])
-    xd = to_bf16_cuda(x0)
-    ys = [torch.zeros((M, N), dtype=torch.bfloat16, device="cuda") for (N, _) in dims]
-    side_x = wl.normal_activations_bf16(311, 101, M, 1024)
-    side_y = torch.zeros((M, 512), dtype=torch.bfloat16, device="cuda")
-    ins = [xd, ys[0], ys[1], ys[2]]
-    descs = (_lib.LinearDesc * 5)()
-    for i, (N, K) in enumerate(dims):
-        d = descs[i]
-        d.x, d.qweight, d.y = ins[i].data_ptr(), packs[i].data_ptr(), ys[i].data_ptr()
-        d.scales = d.zeros = None
-        d.M, d.N, d.K, d.group_size, d.layout, d.flags = M, N, K, G, api.LAYOUT_STREAM, (api.DEP_PREVIOUS if i else 0)
-    d = descs[4]                                                   # an independent entry at the end (no flag)
-    sxd = to_bf16_cuda(side_x)
-    d.x, d.qweight, d.y = sxd.data_ptr(), packs[0].data_ptr(), side_y.data_ptr()
-    d.scales = d.zeros = None
-    d.M, d.N, d.K, d.group_size, d.layout, d.flags = M, 512, 1024, G, api.LAYOUT_STREAM, 0
-    ws = api.new_workspace(api.linear_w4a16_workspace_size(M, 1024, 1024, G))
-    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
-    for rep in range(3):
-        for y in ys:
-            y.zero_()
-        assert lib.qil_linear_w4a16_batch(descs, 5, C.c_void_p(ws.data_ptr()), ws.numel(), st) == 0
-        torch.cuda.synchronize()
-        assert _status(api, ws) == 0
-        got = [y.clone() for y in ys]
-        # one by one, each stage fed with the previous stage's device output
-        cur = xd
-        for i, (N, K) in enumerate(dims):
-            one = api.linear_w4a16(cur, packs[i], None, None, N, G, api.LAYOUT_STREAM, workspace=ws)
-            np.testing.assert_array_equal(bits_of(got[i]), bits_of(one))
-            cur = one
-    # oracle chain: each stage's reference output, rounded to bf16 by the input helper, feeds the next stage
-    cur_bits = x0
-    for i, (N, K) in enumerate(dims):
-        y_ref = c_oracle.linear_w4a16(cur_bits, *refs[i], G)
-        assert_rows_close(bf16_to_f64(got[i]), y_ref, rel=1e-2)
-        cur_bits = wl.f32_to_bf16_bits(y_ref.astype(np.float32))
-    assert_rows_close(bf16_to_f64(side_y), c_oracle.linear_w4a16(side_x, *refs[0], G))
-
-
-def test_w4a16_stream_wide_dynamic_range(api):
-    """Activations 3000x larger than usual, one block of tiny values and one block of zeros: the per-block
-    fixed point must keep the small blocks' contribution (their scale is independent of the large blocks)."""
-    M, N, K, G = 2, 256, 2048, 128
-    x, codes, scales, zeros, buf = _stream_inputs(api, M, N, K, G, 78)
-    xf = wl.bf16_bits_to_f32(x).copy() * 3000.0
-    xf[:, 1024:1152] *= 1e-6
-    xf[1, 1280:1408] = 0.0
-    x = wl.f32_to_bf16_bits(xf)
-    y_ref = c_oracle.linear_w4a16(x, codes, scales, zeros, G)
-    y = api.linear_w4a16(to_bf16_cuda(x), buf, None, None, N, G, api.LAYOUT_STREAM)
-    assert_rows_close(bf16_to_f64(y), y_ref)
-
-
-def test_w4a16_stream_rejects_unsupported(api):
-    import torch
-    buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
-    x = torch.zeros((5, 1024), dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(api.QilError) as e:
-        api.linear_w4a16(x, buf, None, None, 64, 128, api.LAYOUT_STREAM)     # M = 5 > 4
-    assert e.value.code == 4
-    x1 = torch.zeros((1, 1024), dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(api.QilError) as e:
-        api.linear_w4a16(x1, buf, None, None, 64, 128, api.LAYOUT_STREAM, workspace=torch.zeros(64, dtype=torch.uint8, device="cuda"))
-    assert e.value.code == 5
-
-
-# ----------------------------------------------------------------------------
-# W4A16, tensor-memory (tcgen05) decode kernel (QIL_LAYOUT_STREAM128)
-# ----------------------------------------------------------------------------
 def _tc_inputs(api, M, N, K, G, seed, x_scale=None):
     w = wl.normal_weights(320, seed, N, K, 0.02, outlier_prob=0.001)
     x = wl.normal_activations_bf16(320, seed + 1, M, K)

@@ -260,36 +260,6 @@ def test_tile16_layout_is_a_documented_permutation():
     np.testing.assert_array_equal(flat[16:32], p[1, :16])
 
 
-def test_stream_layout_follows_its_written_rule():
-    rng = np.random.default_rng(12)
-    N, K, G = 32, 512, 256
-    codes = rng.integers(0, 16, size=(N, K)).astype(np.uint8)
-    scales = (rng.random((N, K // G)) + 0.5).astype(np.float16)
-    zeros = rng.integers(0, 16, size=(N, K // G)).astype(np.float16)
-    buf = np_oracle.to_stream(np_oracle.pack_w4(codes), scales, zeros, G)
-    assert buf.size == (N // 16) * (K // 128) * 1088
-    # element (n=21, k=300): row tile 1, block 2 -> unit 1*4+2 = 6; row 5 of the tile; k%128 = 44 -> word 5,
-    # element 4 of the word -> byte 0, high nibble = nibble 1; element 301 (5 of the word) -> byte 1, high = nibble 3
-    off = 6 * 1088 + 5 * 64 + 5 * 4
-    word = int.from_bytes(buf[off:off + 4].tobytes(), "little")
-    assert (word >> 4) & 0xF == int(codes[21, 300])
-    assert (word >> 12) & 0xF == int(codes[21, 301])
-    assert (word >> 0) & 0xF == int(codes[21, 296])   # element 0 of the word: byte 0, low nibble
-    assert (word >> 24) & 0xF == int(codes[21, 299])  # element 3: byte 3, low nibble
-    # its scale / zero: group 300 // 256 = 1, stored after the 1024 code bytes at row 5
-    m = 6 * 1088 + 1024 + 5 * 4
-    assert buf[m:m + 2].view(np.float16)[0] == scales[21, 1]
-    assert buf[m + 2:m + 4].view(np.float16)[0] == zeros[21, 1]
-    # block 1 of the same row belongs to group 0
-    m0 = (1 * 4 + 1) * 1088 + 1024 + 5 * 4
-    assert buf[m0:m0 + 2].view(np.float16)[0] == scales[21, 0]
-    # every word of a unit holds the same 8 codes as the TILE16 word at the same place
-    t16 = np_oracle.to_layout(np_oracle.pack_w4(codes), np_oracle.LAYOUT_TILE16)[6 * 256:7 * 256]
-    words = buf[6 * 1088:6 * 1088 + 1024].view(np.uint32)
-    for k in range(8):
-        np.testing.assert_array_equal((words >> np.uint32(4 * (2 * (k % 4) + k // 4))) & 0xF, (t16 >> np.uint32(4 * k)) & 0xF)
-
-
 def test_stream128_layout_follows_its_written_rule():
     rng = np.random.default_rng(13)
     N, K, G = 200, 384, 128      # two row tiles (the second one ragged), three column blocks

@@ -240,6 +240,13 @@ def run_qil(args):
     value = units_all / (ms_all * 1e-3) / 1e9
     value_e2e = units_all / (ms_e2e_all * 1e-3) / 1e9
 
+    n_linears, x_elems, y_elems = model.count, model.x_elems, model.y_elems
+    secondary = None
+    if rank == 0 and world == 1 and not args.no_secondary:
+        del g_dev, g_e2e, model
+        torch.cuda.empty_cache()
+        secondary = secondary_measurements(dev)
+
     if rank == 0:
         peaks = {}
         try:
@@ -248,7 +255,7 @@ def run_qil(args):
             pass
         peak = float(peaks.get("hbm_gbs", 6650.0))
         peak_kind = "measured copy bandwidth (MEASURED_PEAKS.json)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
-        launches_per_step = 1 if persistent else model.count
+        launches_per_step = 1 if persistent else n_linears
         kernel = "w4a16_tc_kernel<1>" if persistent else "w4a16_skinny_kernel<1>"
         per_launch_bytes = bytes_per_step / launches_per_step
         per_launch_ms = ms / launches_per_step          # average over the timed region, launch gaps included
@@ -257,25 +264,113 @@ def run_qil(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_all, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 activations x int4 weights, fp32 accumulate", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "layers": args.layers, "linears_per_step": model.count,
+            "config": {"workload": WORKLOAD, "layers": args.layers, "linears_per_step": n_linears,
                        "layout": args.layout, "dependencies": args.deps,
                        "bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (3.44 GB of weights per step)",
                        "parallelism": f"replicas x{world}", "launch": ("CUDA graph of one persistent kernel over the whole list" if persistent
                                   else "CUDA graph of one kernel per linear")},
             "clocks": clocks,
             "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_e2e_all,
-                    "h2d_bytes_per_step": 2 * model.x_elems, "d2h_bytes_per_step": 2 * model.y_elems},
+                    "h2d_bytes_per_step": 2 * x_elems, "d2h_bytes_per_step": 2 * y_elems},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": None, "peak_kind": peak_kind, "kernel": kernel,
                          "bytes_per_launch": per_launch_bytes, "us_per_launch": per_launch_ms * 1e3,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu_baseline,
+            "secondary": secondary,
         }
         print(json.dumps(out))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def secondary_measurements(dev):
+    """Short timings of the other rows of the path on the same GPU (each a few milliseconds): the W4A4 integer
+    GEMM on the four im2col conv shapes (GEMM alone and with the per-token activation quantiser), the 16-bit
+    reference GEMV the 4-bit decode is compared with, and one decoder layer at prefill length 280."""
+    import numpy as np
+    import torch
+    from paper_2412_01034_b200 import api, workloads as wl
+    out = {}
+
+    def time_us(fn, reps):
+        """Device time per call: `reps` calls captured in a CUDA graph (these kernels are shorter than a launch
+        from Python), the graph replayed three times and timed with events on its stream."""
+        st = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(st):
+            for _ in range(3):
+                fn()
+            st.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=st):
+                for _ in range(reps):
+                    fn()
+            graph.replay()
+            st.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            for _ in range(3):
+                graph.replay()
+            e1.record(st)
+            st.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (3 * reps)
+
+    g = torch.Generator(device=dev)
+    g.manual_seed(4)
+    conv = []
+    for stage in range(4):
+        M, K, N = wl.conv_gemm_shape(stage)
+        x = torch.relu(torch.randn((M, K), device=dev, generator=g)).to(torch.bfloat16)
+        w = torch.randn((N, K), device=dev, generator=g) * wl.SIGMA_CONV
+        qw, sw, _ = api.quantize_rtn_w4(w, K, symmetric=True)
+        pw = api.pack_w4(qw)
+        qx, sx = api.quantize_act_a4(x)
+        ws = api.new_workspace(api.linear_w4a4_workspace_size(M, N, K), dev)
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        t_gemm = time_us(lambda: api.linear_w4a4(qx, sx, pw, sw.reshape(-1), out=y, workspace=ws), 50)
+        t_both = time_us(lambda: api.linear_w4a4(*api.quantize_act_a4(x), pw, sw.reshape(-1), out=y, workspace=ws), 50)
+        ops = 2.0 * M * K * N
+        conv.append({"M": M, "K": K, "N": N, "gemm_us": t_gemm, "gemm_tops": ops / t_gemm / 1e6,
+                     "quantise_plus_gemm_us": t_both, "l2": "operands fit L2 (warm)"})
+    out["w4a4_conv_stages"] = conv
+    out["w4a4_tops_total"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv) / sum(c["gemm_us"] for c in conv) / 1e6
+
+    # 16-bit reference GEMV, cold: rotate over copies larger than L2
+    N = K = wl.HIDDEN
+    copies = 12
+    wd = [torch.randn((N, K), device=dev, generator=g).to(torch.bfloat16) for _ in range(copies)]
+    xv = torch.randn((1, K), device=dev, generator=g).to(torch.bfloat16)
+    yv = torch.empty((N,), dtype=torch.bfloat16, device=dev)
+    state = {"i": 0}
+
+    def ref():
+        api.ref_gemv_bf16(xv, wd[state["i"] % copies], out=yv)
+        state["i"] += 1
+    t_ref = time_us(ref, 48)
+    out["ref_gemv_bf16_4096x4096"] = {"us": t_ref, "GB/s": (2.0 * N * K + 2 * K + 2 * N) / t_ref / 1e3,
+                                      "l2": f"cold: {copies} weight copies in rotation"}
+    del wd
+
+    # prefill: one decoder layer (7 linears) at M = 280
+    Mp = wl.PREFILL_M
+    xs = {K: torch.randn((Mp, K), device=dev, generator=g).to(torch.bfloat16) for K in (wl.HIDDEN, wl.FFN)}
+    lin = []
+    for (_, N, K) in wl.LLAMA2_7B_LAYER:
+        w = torch.randn((N, K), device=dev, generator=g) * wl.SIGMA_LLM
+        codes, s, z = api.quantize_rtn_w4(w, wl.GROUP_SIZE)
+        lin.append((N, K, api.pack_w4(codes, api.LAYOUT_TILE16), s, z, torch.empty((Mp, N), dtype=torch.bfloat16, device=dev),
+                    api.new_workspace(api.linear_w4a16_workspace_size(Mp, N, K, wl.GROUP_SIZE), dev)))
+        del w, codes
+
+    def layer():
+        for (N, K, pk, s, z, yo, ws) in lin:
+            api.linear_w4a16(xs[K], pk, s, z, N, wl.GROUP_SIZE, api.LAYOUT_TILE16, out=yo, workspace=ws)
+    t_layer = time_us(layer, 10)
+    flops = sum(2.0 * Mp * N * K for (_, N, K) in wl.LLAMA2_7B_LAYER)
+    out["w4a16_prefill_m280_layer"] = {"us": t_layer, "TFLOP/s": flops / t_layer / 1e6, "kernel": "w4a16_skinny_kernel (slabs of 64 rows)"}
+    return out
 
 
 def main():
@@ -290,6 +385,7 @@ def main():
                     help="which linears wait for all earlier ones (layer = data flow of a decoder layer)")
     ap.add_argument("--cpu-budget-s", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the short W4A4 / reference / prefill timings")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

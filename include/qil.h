@@ -232,6 +232,9 @@ qil_status qil_quantize_act_a4(const void* x, int M, int K, const float* static_
  *   qx [M][K/8], qw [N][K/8] canonical packed signed nibbles; sx [M], sw [N] fp32
  *   acc_out: optional [M][N] int32 copy of the raw accumulators.
  * Needs K % 32 == 0.  |acc| <= 64 K must fit int32.
+ * workspace: qil_linear_w4a4_workspace_size() bytes, zero-filled once; its first
+ * int is a status word that receives QIL_ERR_TIMEOUT if a bounded device-side
+ * wait ever runs out (read it with qil_device_status).
  * ---------------------------------------------------------------------- */
 size_t qil_linear_w4a4_workspace_size(int M, int N, int K);
 qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw,

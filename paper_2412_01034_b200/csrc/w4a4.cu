@@ -1,104 +1,277 @@
 // W4A4 integer GEMM (the compute-bound driving-policy deployment of the paper,
-// Sec. 5.1 / Sec. 5.4): acc = qx . qw^T in int32, y = bf16(float(acc) * sx[m] * sw[n]).
+// Sec. 5.1 / Sec. 5.4): acc = qx . qw^T in int32, y = bf16(float(acc) * sx[m] * sw[n]),
+// on the 5th-generation tensor cores (tcgen05.mma kind::i8, accumulators in tensor memory).
 //
-// Unpacking trick shared by every path in this file: for a packed word w,
-//   (w << 4) & 0xF0F0F0F0  holds nibbles 0,2,4,6 and  w & 0xF0F0F0F0  holds nibbles
-//   1,3,5,7, each as a signed byte equal to 16 x the int4 value (the nibble is the
-//   byte's high half, so its sign bit is the byte's sign bit).
-// Both operands are scaled by 16, the int32 accumulator is exactly 256 x the true
-// sum (|acc| <= 64 K, so 256 |acc| < 2^31 for K <= 131072) and is shifted back.
-// The order of k inside a word differs from memory order, identically for both
-// operands, which leaves the sum unchanged.
+// A CTA computes a 128 (tokens) x 64 (output channels) tile.  Per step of 128 input
+// channels its four loader warps read the packed nibbles of both operands from global
+// memory (the operands of this workload stay in L2), split them into signed bytes and store
+// them to shared memory in the tensor core's K-major layout without swizzle (8 rows x 16
+// bytes per core matrix; K-adjacent core matrices `rows x 16` bytes apart, 8-row groups 128
+// bytes apart).  One thread issues four tcgen05.mma (128 x 64 x 32) per step; a
+// tcgen05.commit hands the shared-memory stage back to the loaders.  After the last step the
+// same four warps read the accumulators (tcgen05.ld), rescale and store bf16.
+//
+// Unpacking: for a packed word w, (w << 4) & 0xF0F0F0F0 holds nibbles 0,2,4,6 and
+// w & 0xF0F0F0F0 holds nibbles 1,3,5,7, each as a signed byte equal to 16 x the int4 value
+// (the nibble is the byte's high half, so its sign bit is the byte's sign bit).  Both
+// operands are scaled by 16, the int32 accumulator is exactly 256 x the true sum
+// (|acc| <= 64 K, so 256 |acc| < 2^31 for K <= 131072) and is shifted back.  The order of k
+// inside a word differs from memory order, identically for both operands, which leaves the
+// sum unchanged.
 #include "qil_common.cuh"
 
 namespace qil {
 
 namespace {
 
-__device__ __forceinline__ void mma_s8_16832(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                             uint32_t b0, uint32_t b1) {
+constexpr int kTileM = 128, kTileN = 64, kStepK = 128;  // K elements per step = 64 packed bytes per row
+constexpr int kStages = 3;
+constexpr int kAStage = kTileM * kStepK;  // bytes (one byte per element after the split)
+constexpr int kBStage = kTileN * kStepK;
+constexpr int kThreads = 160;             // 4 loader / epilogue warps + the MMA warp
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
     asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// Bounded wait: false when the limit ran out (the caller then stops issuing work).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0, t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        if (t - t0 > kWaitLimitNs) return false;
+    }
+}
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    uint64_t d = (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+    return d;
+}
+// D[128 x 64] (+)= A[128 x 32 s8, shared memory] * B[64 x 32 s8, shared memory]^T, int32 accumulate
+__device__ __forceinline__ void mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+    // instruction descriptor: D = s32 (2 at bit 4), A = s8 (1 at bit 7), B = s8 (1 at bit 10), both K-major,
+    // N >> 3 at bit 17, M >> 4 at bit 24
+    constexpr uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)kTileN >> 3) << 17) | (((uint32_t)kTileM >> 4) << 24);
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
 }
 
-__device__ __forceinline__ uint32_t even_nibbles_x16(uint32_t w) { return (w << 4) & 0xF0F0F0F0u; }
-__device__ __forceinline__ uint32_t odd_nibbles_x16(uint32_t w) { return w & 0xF0F0F0F0u; }
+// 32 packed codes (one uint4) -> 32 signed bytes (x16) = two 16-byte K chunks
+__device__ __forceinline__ void split32(const uint4& w, uint4& c0, uint4& c1) {
+    constexpr uint32_t m = 0xF0F0F0F0u;
+    c0 = make_uint4((w.x << 4) & m, w.x & m, (w.y << 4) & m, w.y & m);
+    c1 = make_uint4((w.z << 4) & m, w.z & m, (w.w << 4) & m, w.w & m);
+}
 
-constexpr int kNT = 8;  // 8-column tiles per warp: warp tile 16 x 64
+__global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __restrict__ qx, const float* __restrict__ sx,
+                                                             const uint32_t* __restrict__ qw, const float* __restrict__ sw,
+                                                             __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out,
+                                                             int M, int N, int K, int* __restrict__ status) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* sa = smem;                                  // [kStages][kAStage]
+    unsigned char* sb = smem + (size_t)kStages * kAStage;      // [kStages][kBStage]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sb + (size_t)kStages * kBStage);
+    const uint32_t full0 = smem_u32(bars), free0 = smem_u32(bars + kStages), done0 = smem_u32(bars + 2 * kStages);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+    float* sws = reinterpret_cast<float*>(tmem_slot + 2);  // [kTileN] weight scales of the tile
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
+    const int steps = (K + kStepK - 1) / kStepK;
+    const int row_words = K >> 3;  // 32-bit words per packed row
 
-// Register-only kernel: each warp computes a 16 x 64 tile, operands come straight
-// from global memory (they are L2 resident at the sizes this path serves).
-__global__ void __launch_bounds__(128) w4a4_mma_sync_kernel(const uint32_t* __restrict__ qx,
-                                                            const float* __restrict__ sx,
-                                                            const uint32_t* __restrict__ qw,
-                                                            const float* __restrict__ sw,
-                                                            __nv_bfloat16* __restrict__ y,
-                                                            int32_t* __restrict__ acc_out, int M, int N, int K) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int g = lane >> 2, t = lane & 3;
-    const int m0 = (blockIdx.x * 4 + warp) * 16;
-    const int n0 = blockIdx.y * (8 * kNT);
-    if (m0 >= M) return;
-    const int chunks = K >> 5;  // 128-bit chunks (32 codes) per row
-    const uint4* xa = reinterpret_cast<const uint4*>(qx) + (size_t)(m0 + g) * chunks;
-    const uint4* xb = reinterpret_cast<const uint4*>(qx) + (size_t)(m0 + g + 8) * chunks;
-    const bool a_ok = (m0 + g) < M, b_ok = (m0 + g + 8) < M;
-
-    int acc[kNT][4];
-#pragma unroll
-    for (int nt = 0; nt < kNT; ++nt)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[nt][c] = 0;
-
-    for (int ks = 0; ks * 4 < chunks; ++ks) {
-        const int ch = ks * 4 + t;
-        const bool in = ch < chunks;
-        uint4 va = make_uint4(0, 0, 0, 0), vb = make_uint4(0, 0, 0, 0);
-        if (in && a_ok) va = xa[ch];
-        if (in && b_ok) vb = xb[ch];
-        const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
-        const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
-#pragma unroll
-        for (int nt = 0; nt < kNT; ++nt) {
-            const int n = n0 + nt * 8 + g;
-            uint4 vw = make_uint4(0, 0, 0, 0);
-            if (in && n < N) vw = (reinterpret_cast<const uint4*>(qw) + (size_t)n * chunks)[ch];
-            const uint32_t ww[4] = {vw.x, vw.y, vw.z, vw.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                mma_s8_16832(acc[nt], even_nibbles_x16(wa[j]), even_nibbles_x16(wb[j]), odd_nibbles_x16(wa[j]),
-                             odd_nibbles_x16(wb[j]), even_nibbles_x16(ww[j]), odd_nibbles_x16(ww[j]));
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full0 + 8 * s, 4);
+            mbar_init(free0 + 8 * s, 1);
         }
+        mbar_init(done0, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (tid < kTileN) sws[tid] = (n0 + tid < N) ? sw[n0 + tid] : 0.f;
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTileN));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+    bool ok = true;
 
+    if (warp < 4) {
+        // ---------------- loaders: thread r owns token row r of the tile and half of weight row r / 2 ----------------
+        const int r = tid;
+        const bool a_row = m0 + r < M;
+        const int bn = r >> 1, bh = r & 1;  // weight row of the tile, which 64-element half of the step
+        const bool b_row = n0 + bn < N;
+        const uint32_t* xa = qx + (size_t)(m0 + (a_row ? r : 0)) * row_words;
+        const uint32_t* wb = qw + (size_t)(n0 + (b_row ? bn : 0)) * row_words;
+        uint4 pa[4], pb[2];
+        auto fetch = [&](int step) {  // packed words of one step into registers (zeros beyond the matrix)
+            const int w0 = step * (kStepK / 8);
 #pragma unroll
-    for (int nt = 0; nt < kNT; ++nt)
+            for (int q = 0; q < 4; ++q) {
+                const int w = w0 + 4 * q;
+                pa[q] = (a_row && w < row_words) ? __ldg(reinterpret_cast<const uint4*>(xa + w)) : make_uint4(0, 0, 0, 0);
+            }
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const int m = m0 + g + ((c & 2) ? 8 : 0);
-            const int n = n0 + nt * 8 + 2 * t + (c & 1);
-            if (m < M && n < N) {
-                const int a = acc[nt][c] >> 8;  // exact: the accumulator is a multiple of 256
-                if (acc_out) acc_out[(size_t)m * N + n] = a;
-                y[(size_t)m * N + n] = __float2bfloat16_rn((float)a * (sx[m] * sw[n]));
+            for (int q = 0; q < 2; ++q) {
+                const int w = w0 + 4 * (2 * bh + q);
+                pb[q] = (b_row && w < row_words) ? __ldg(reinterpret_cast<const uint4*>(wb + w)) : make_uint4(0, 0, 0, 0);
+            }
+        };
+        fetch(0);
+        for (int step = 0; step < steps && ok; ++step) {
+            const int s = step % kStages, use = step / kStages;
+            ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
+            if (!ok) break;
+            unsigned char* a_st = sa + (size_t)s * kAStage + (size_t)r * 16;
+            unsigned char* b_st = sb + (size_t)s * kBStage + (size_t)bn * 16;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {  // K chunks 2q, 2q+1 of the step
+                uint4 c0, c1;
+                split32(pa[q], c0, c1);
+                *reinterpret_cast<uint4*>(a_st + (size_t)(2 * q) * (kTileM * 16)) = c0;
+                *reinterpret_cast<uint4*>(a_st + (size_t)(2 * q + 1) * (kTileM * 16)) = c1;
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint4 c0, c1;
+                split32(pb[q], c0, c1);
+                const int ch = 2 * (2 * bh + q);
+                *reinterpret_cast<uint4*>(b_st + (size_t)ch * (kTileN * 16)) = c0;
+                *reinterpret_cast<uint4*>(b_st + (size_t)(ch + 1) * (kTileN * 16)) = c1;
+            }
+            if (step + 1 < steps) fetch(step + 1);  // in flight while the tensor core works on this step
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full0 + 8 * s);
+        }
+        // ---------------- epilogue: thread r = accumulator row r ----------------
+        if (ok) ok = mbar_wait(done0, 0);
+        if (ok) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int m = m0 + r;
+            const float sxm = a_row ? sx[m] : 0.f;
+            const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
+            const bool vec = (N % 8) == 0;  // rows of y are then 16-byte aligned pieces of 8 outputs
+#pragma unroll 1
+            for (int c0 = 0; c0 < kTileN; c0 += 16) {
+                uint32_t d[16];
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                    : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]), "=r"(d[8]),
+                      "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
+                    : "r"(tmem + lane_base + (uint32_t)c0));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 16; ++j) asm volatile("" : "+r"(d[j]));
+                if (!a_row) continue;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {  // 8 outputs = one 16-byte piece of the row
+                    const int nb = n0 + c0 + 8 * h;
+                    if (nb >= N) continue;
+                    int a[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) a[j] = (int)d[8 * h + j] >> 8;  // exact: the accumulator is a multiple of 256
+                    if (vec) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const __nv_bfloat162 v = __floats2bfloat162_rn((float)a[2 * j] * (sxm * sws[c0 + 8 * h + 2 * j]),
+                                                                           (float)a[2 * j + 1] * (sxm * sws[c0 + 8 * h + 2 * j + 1]));
+                            pk[j] = *reinterpret_cast<const uint32_t*>(&v);
+                        }
+                        *reinterpret_cast<uint4*>(y + (size_t)m * N + nb) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        if (acc_out) {
+                            *reinterpret_cast<int4*>(acc_out + (size_t)m * N + nb) = make_int4(a[0], a[1], a[2], a[3]);
+                            *reinterpret_cast<int4*>(acc_out + (size_t)m * N + nb + 4) = make_int4(a[4], a[5], a[6], a[7]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (nb + j < N) {
+                                if (acc_out) acc_out[(size_t)m * N + nb + j] = a[j];
+                                y[(size_t)m * N + nb + j] = __float2bfloat16_rn((float)a[j] * (sxm * sws[c0 + 8 * h + j]));
+                            }
+                    }
+                }
             }
         }
+    } else if (lane == 0) {
+        // ---------------- MMA issuer ----------------
+        constexpr uint32_t kALbo = kTileM * 16, kBLbo = kTileN * 16;  // K-adjacent core matrices
+        for (int step = 0; step < steps; ++step) {
+            const int s = step % kStages, use = step / kStages;
+            ok = mbar_wait(full0 + 8 * s, use & 1);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = smem_u32(sa + (size_t)s * kAStage), b_addr = smem_u32(sb + (size_t)s * kBStage);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)  // K = 32 each: chunks 2i, 2i + 1
+                mma_i8_ss(tmem, smem_desc(a_addr + 2 * i * kALbo, kALbo, 128), smem_desc(b_addr + 2 * i * kBLbo, kBLbo, 128),
+                          (step > 0 || i > 0) ? 1u : 0u);
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(free0 + 8 * s) : "memory");
+        }
+        // all MMAs of this thread are complete when this arrival happens (also needed before tensor memory is released)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(done0) : "memory");
+        unsigned long long t0, t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+        while (!mbar_try_wait(done0, 0)) {
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+            if (t - t0 > kWaitLimitNs) { ok = false; break; }
+        }
+    }
+    if (!ok && status) atomicOr(status, (int)QIL_ERR_TIMEOUT);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTileN));
 }
+
+constexpr size_t kSmemBytes = (size_t)kStages * (kAStage + kBStage) + (2 * kStages + 1) * 8 + 8 + kTileN * 4 + 8;
 
 }  // namespace
 
+// The first int of the workspace receives QIL_ERR_TIMEOUT if a bounded device-side wait runs out.
 size_t w4a4_workspace(int M, int N, int K) {
     (void)M; (void)N; (void)K;
-    return 0;
+    return 16;
 }
 
 qil_status launch_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, void* y,
                        int32_t* acc_out, int M, int N, int K, void* ws, size_t ws_bytes, cudaStream_t st) {
-    (void)ws; (void)ws_bytes;
-    const dim3 grid((M + 63) / 64, (N + 8 * kNT - 1) / (8 * kNT));
-    w4a4_mma_sync_kernel<<<grid, 128, 0, st>>>(qx, sx, qw, sw, reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K);
+    if (ws == nullptr || ws_bytes < 16) return QIL_ERR_WORKSPACE;
+    if (cudaFuncSetAttribute(w4a4_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return QIL_ERR_CUDA;
+    }
+    const dim3 grid((M + kTileM - 1) / kTileM, (N + kTileN - 1) / kTileN);
+    w4a4_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qx, sx, qw, sw, reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K,
+                                                      reinterpret_cast<int*>(ws));
     return launch_status();
 }
 

@@ -360,16 +360,16 @@ def secondary_measurements(dev):
     for (_, N, K) in wl.LLAMA2_7B_LAYER:
         w = torch.randn((N, K), device=dev, generator=g) * wl.SIGMA_LLM
         codes, s, z = api.quantize_rtn_w4(w, wl.GROUP_SIZE)
-        lin.append((N, K, api.pack_w4(codes, api.LAYOUT_TILE16), s, z, torch.empty((Mp, N), dtype=torch.bfloat16, device=dev),
+        lin.append((N, K, api.pack_w4(codes), s, z, torch.empty((Mp, N), dtype=torch.bfloat16, device=dev),
                     api.new_workspace(api.linear_w4a16_workspace_size(Mp, N, K, wl.GROUP_SIZE), dev)))
         del w, codes
 
     def layer():
         for (N, K, pk, s, z, yo, ws) in lin:
-            api.linear_w4a16(xs[K], pk, s, z, N, wl.GROUP_SIZE, api.LAYOUT_TILE16, out=yo, workspace=ws)
+            api.linear_w4a16(xs[K], pk, s, z, N, wl.GROUP_SIZE, api.LAYOUT_CANONICAL, out=yo, workspace=ws)
     t_layer = time_us(layer, 10)
     flops = sum(2.0 * Mp * N * K for (_, N, K) in wl.LLAMA2_7B_LAYER)
-    out["w4a16_prefill_m280_layer"] = {"us": t_layer, "TFLOP/s": flops / t_layer / 1e6, "kernel": "w4a16_skinny_kernel (slabs of 64 rows)"}
+    out["w4a16_prefill_m280_layer"] = {"us": t_layer, "TFLOP/s": flops / t_layer / 1e6, "kernel": "w4a16_prefill_kernel (tcgen05 kind::f16)"}
     return out
 
 

@@ -144,6 +144,9 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
         d.M = M; d.N = N; d.K = K; d.group_size = group_size; d.layout = layout; d.flags = 0;
         return launch_w4a16_tc(&d, 1, workspace, workspace_bytes, S(stream));
     }
+    if (w4a16_prefill_supported(M, N, K, group_size, layout))
+        return launch_w4a16_prefill(x, qweight, scales, zeros, y, M, N, K, group_size,
+                                    workspace_bytes >= sizeof(int) ? workspace : nullptr, S(stream));
     if (w4a16_skinny_supported(M, N, K, group_size, layout))
         return launch_w4a16_skinny(x, qweight, scales, zeros, y, M, N, K, group_size, layout, workspace,
                                    workspace_bytes, S(stream));

@@ -69,6 +69,10 @@ qil_status launch_w4a16_skinny(const void* x, const uint32_t* qw, const void* sc
                                void* y, int M, int N, int K, int G, qil_layout layout, void* ws,
                                size_t ws_bytes, cudaStream_t st);
 
+bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout);
+qil_status launch_w4a16_prefill(const void* x, const uint32_t* qw, const void* scales, const void* zeros, void* y, int M,
+                                int N, int K, int G, void* ws, cudaStream_t st);
+
 bool w4a16_tc_supported(int M, int N, int K, int G);
 size_t w4a16_tc_weight_bytes(int N, int K);
 size_t w4a16_tc_workspace();

@@ -11,7 +11,7 @@ import pytest
 
 from oracle import c_oracle, np_oracle
 from paper_2412_01034_b200 import workloads as wl
-from tests.util import assert_rows_close, bf16_to_f64, bits_of, cuda, to_bf16_cuda
+from tests.util import CONTRACT_REL, DERIVED_REL, assert_rows_close, bf16_to_f64, bits_of, cuda, to_bf16_cuda
 
 pytestmark = pytest.mark.gpu
 
@@ -161,6 +161,13 @@ def test_pack_unpack_layouts(api, N, K):
 # ----------------------------------------------------------------------------
 # W4A16
 # ----------------------------------------------------------------------------
+def _prefill_path(M, K, G, layout):
+    """Shapes that qil_linear_w4a16 serves with the tensor-core prefill GEMM: it rounds every dequantised weight and
+    every group scale to bf16 (each within 2^-9, independent signs), so its error is a random sum that the tests
+    hold to the contract's 1e-2 of the row maximum instead of the tighter figure derived for fp32 dequantisation."""
+    return layout == 0 and M > 64 and K % 64 == 0 and G % 64 == 0
+
+
 def _w4a16_case(api, M, N, K, G, layout, seed, outliers=True):
     w = wl.normal_weights(300, seed, N, K, 0.02, outlier_prob=0.001 if outliers else 0.0)
     x = wl.normal_activations_bf16(300, seed + 1, M, K)
@@ -169,7 +176,7 @@ def _w4a16_case(api, M, N, K, G, layout, seed, outliers=True):
     packed = api.pack_w4(cuda(codes), layout)
     y = api.linear_w4a16(to_bf16_cuda(x), packed, cuda(scales), cuda(zeros), N, G, layout)
     assert tuple(y.shape) == (M, N)
-    assert_rows_close(bf16_to_f64(y), y_ref)
+    assert_rows_close(bf16_to_f64(y), y_ref, rel=CONTRACT_REL if _prefill_path(M, K, G, layout) else DERIVED_REL)
     return y
 
 
@@ -198,6 +205,35 @@ def test_w4a16_skinny_m_sweep(api, M, layout):
 def test_w4a16_skinny_shapes(api, N, K, G, layout):
     for M in (1, 5):
         _w4a16_case(api, M, N, K, G, layout, seed=N + K + G)
+
+
+@pytest.mark.parametrize("M,N,K,G", [
+    (280, 512, 1024, 128), (130, 200, 256, 64), (65, 1000, 2176, 128), (129, 136, 128, 128), (300, 77, 192, 192),
+])
+def test_w4a16_prefill_shapes(api, M, N, K, G):
+    """The tcgen05 prefill GEMM (M > 64, canonical layout): ragged M and N, one to many K steps, groups of one or
+    several steps; run twice: the result must not depend on what the previous launch left behind."""
+    y1 = _w4a16_case(api, M, N, K, G, 0, seed=M + N + K)
+    y2 = _w4a16_case(api, M, N, K, G, 0, seed=M + N + K)
+    np.testing.assert_array_equal(bits_of(y1), bits_of(y2))
+
+
+@pytest.mark.parametrize("N,K", [(wl.HIDDEN, wl.HIDDEN), (wl.FFN, wl.HIDDEN), (wl.HIDDEN, wl.FFN)])
+def test_cfg2_prefill_shapes(api, N, K):
+    """Config 2: the Llama-2-7B linear shapes at prefill length 280; the oracle runs on 256 sampled output
+    features (the kernel computes all N)."""
+    M, G = wl.PREFILL_M, wl.GROUP_SIZE
+    w = wl.normal_weights(2, N + K, N, K, 0.02, outlier_prob=0.001)
+    x = wl.normal_activations_bf16(2, N + K + 1, M, K)
+    got = api.quantize_rtn_w4(cuda(w), G)
+    rows = np.sort(np.random.default_rng(N + K).choice(N, 256, replace=False))
+    codes, scales, zeros = got[0].cpu().numpy()[rows], got[1].cpu().numpy()[rows], got[2].cpu().numpy()[rows]
+    ref = np_oracle.quantize_rtn_w4_asym(w[rows], G)
+    np.testing.assert_array_equal(codes, ref[0])
+    y = api.linear_w4a16(to_bf16_cuda(x), api.pack_w4(got[0]), got[1], got[2], N, G)
+    y_ref = c_oracle.linear_w4a16(x, *ref, G)
+    # the row maximum over the sampled features lower-bounds the true row maximum: the check is stricter
+    assert_rows_close(bf16_to_f64(y)[:, rows], y_ref, rel=CONTRACT_REL)
 
 
 @pytest.mark.parametrize("N,K,G", [(24, 256, 32), (9, 40, 8), (17, 192, 64), (8, 320, 320)])

@@ -100,6 +100,16 @@ __global__ void __launch_bounds__(256) quantize_sym_kernel(const T* __restrict__
     }
 }
 
+// rint(f / s) with the IEEE division of the specification, without paying for a division per element: the product
+// with the reciprocal is within a few ulp of the quotient, so unless it lies that close to a rounding boundary
+// (k + 0.5) it rounds to the same integer; the rare close calls (and anything not finite) take the true division.
+__device__ __forceinline__ float rint_div(float f, float s, float inv_s) {
+    const float r = f * inv_s;
+    const float dist = fabsf(fabsf(r - rintf(r)) - 0.5f);  // distance of r from the nearest k + 0.5
+    if (dist > 1e-4f * fmaxf(fabsf(r), 1.0f) && fabsf(r) < 1e6f) return rintf(r);
+    return rintf(__fdiv_rn(f, s));
+}
+
 // Per-token symmetric int4 of bf16 activations, fused with packing.  One warp per row.
 // Each lane owns whole 32-bit output words (8 consecutive k).
 __global__ void __launch_bounds__(256) quantize_act_kernel(const __nv_bfloat16* __restrict__ x, int M, int K,
@@ -129,6 +139,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const __nv_bfloat16* 
             if (a == 0.0f) s = 1.0f;
         }
         if (lane == 0) scales[m] = s;
+        const float inv_s = __frcp_rn(s);
         for (int i = lane; i < words; i += 32) {
             uint4 v = row[i];
             const uint32_t u[4] = {v.x, v.y, v.z, v.w};
@@ -137,8 +148,8 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const __nv_bfloat16* 
             for (int j = 0; j < 4; ++j) {
                 float f0 = __uint_as_float(u[j] << 16);
                 float f1 = __uint_as_float(u[j] & 0xFFFF0000u);
-                int q0 = (int)clampf(rintf(__fdiv_rn(f0, s)), -8.0f, 7.0f);
-                int q1 = (int)clampf(rintf(__fdiv_rn(f1, s)), -8.0f, 7.0f);
+                int q0 = (int)clampf(rint_div(f0, s, inv_s), -8.0f, 7.0f);
+                int q1 = (int)clampf(rint_div(f1, s, inv_s), -8.0f, 7.0f);
                 word |= (uint32_t)(q0 & 0xF) << (8 * j);
                 word |= (uint32_t)(q1 & 0xF) << (8 * j + 4);
             }

@@ -2,18 +2,18 @@
 // persistent kernel over a list of linears (the memory-bound decode stage of the paper's
 // OpenVLA deployment, Sec. 5.4 / App. A.4.2; M <= 4 activation rows).
 //
-// The kernel is bound by HBM only if the SM spends very few instructions per weight, so the
-// CUDA cores do nothing but split nibbles: a thread owns one weight row of a unit (128 rows
-// x 128 columns), reads its 64 packed bytes, and with ONE logic instruction per 4 weights
-// produces unsigned bytes - the low nibbles as they are, the high nibbles in place, i.e.
-// times 16 - which it writes to tensor memory (tcgen05.st).  There they are the A operand
-// (128 rows x 32 bytes per instruction) of tcgen05.mma kind::i8.  The B operand is the
-// activation block, converted once per linear to 16-bit block fixed point - per 128 columns a
-// power-of-two scale 2^e and two int8 planes (v = 256 hi + lo) - K-major in shared memory.
-// Low-nibble and high-nibble bytes accumulate in separate int32 accumulators in tensor memory
-// (exact); per 128-column block the epilogue thread of a weight row reads them back
-// (tcgen05.ld) and folds scale and zero point once:
-//     y += s_w * 2^e * ((256 L_hi + L_lo) + (256 H_hi + H_lo) / 16 - z * X),  X = sum of the block's integers.
+// The kernel is bound by HBM only if the SM spends very few instructions per weight.  A packed
+// byte holds two codes, b = lo + 16 hi.  The tensor core multiplies the RAW bytes, read straight
+// from the shared-memory ring, by the activations under the high nibbles (x_c), and the MASKED
+// bytes (b & 0x0F: one logic instruction per 8 weights, written to tensor memory by the thread that
+// owns the weight row) by 16 x_a - x_c, x_a being the activations under the low nibbles:
+//     sum b x_c + sum lo (16 x_a - x_c) = 16 (sum lo x_a + sum hi x_c).
+// Both are tcgen05.mma kind::i8 (128 rows x 8 columns x 32 bytes) with exact int32 accumulators in
+// tensor memory.  The activations are converted once per linear to 16-bit block fixed point - per
+// 128 columns a power-of-two scale 2^e and integers v - and enter as signed-byte planes (two for
+// x_c, three for 16 x_a - x_c), K-major in shared memory.  Per 128-column block the epilogue
+// thread of a weight row reads the accumulators back (tcgen05.ld) and folds scale and zero point:
+//     y += s_w * 2^e * (((256 R1 + R0) + (65536 T2 + 256 T1 + T0)) / 16 - z * X),  X = sum of the block's v.
 //
 // Data layout (QIL_LAYOUT_STREAM128): unit u = (row tile of 128 rows, column block of 128)
 // is 8704 bytes: 4 chunks (32 columns each) x 128 rows x 16 bytes of codes, byte b of
@@ -75,6 +75,9 @@ constexpr int kUnitBytes = 8192 + 512;
 #ifndef QIL_TC_UNPACK_WGS
 #define QIL_TC_UNPACK_WGS 2
 #endif
+#ifndef QIL_TC_SPIN_POLLS
+#define QIL_TC_SPIN_POLLS 0
+#endif
 #ifndef QIL_TC_EPI_BATCH
 #define QIL_TC_EPI_BATCH 4
 #endif
@@ -93,12 +96,17 @@ constexpr int kMmaBase = kFixBase + kFixThreads; // kGroup warps, one issuing th
 constexpr int kProdBase = kMmaBase + 32 * kGroup;  // one warp, one thread issues
 constexpr int kThreads = kProdBase + 32;
 static_assert(kThreads <= 1024, "block size");
-constexpr int kNG = 2;                           // groups in flight in tensor memory
+constexpr int kNG = 3;                           // groups in flight in tensor memory
 constexpr int kNB = kGroup * kNG;                // = units in flight
 constexpr int kTmemCols = 512;
-constexpr int kColD = 32 * kNB;                  // A: 32 columns per unit; D: 8 (low nibbles) + 8 (high nibbles)
-constexpr int kColMeta = kColD + 16 * kNB;       // one column per unit: {scale, zero} of the thread's row
-static_assert(kColMeta + kNB <= kTmemCols, "tensor memory budget");
+// tensor-memory columns: per unit 16 of masked low nibbles (A), 8 accumulators of the raw-byte products and 8 (16 with
+// four activation rows) of the masked ones, 1 of {scale, zero}
+constexpr int kColD = 16 * kNB;
+__host__ __device__ constexpr int d_unit_cols(int xr) { return 8 + (xr == 4 ? 16 : 8); }
+__host__ __device__ constexpr int col_meta(int xr) { return kColD + d_unit_cols(xr) * kNB; }
+static_assert(col_meta(4) + kNB <= kTmemCols, "tensor memory budget");
+static_assert(kNumEpi == 1 || kNG % kNumEpi == 0, "a slot group must always be read out by the same epilogue warpgroup");
+constexpr int kHandDepth = 8;                    // hand-over buffers between the epilogue and the fixer
 constexpr int kMaxEntries = 256;
 constexpr int kMaxRows = 4;                      // activation rows
 constexpr int kSlotDepth = 4;                    // ring of slots per (CTA, first / last tile), indexed by entry
@@ -151,6 +159,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// non-blocking test of a phase
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -212,6 +232,23 @@ __device__ __forceinline__ void tmem_ld(uint32_t addr, uint32_t (&v)[8]) {
                      : "r"(addr));
     }
 }
+// the accumulator columns of the masked-byte products: 3 per activation row
+template <int kXR>
+__device__ __forceinline__ void tmem_ld_m(uint32_t addr, uint32_t (&v)[16]) {
+    if constexpr (kXR == 1) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(addr));
+    } else if constexpr (kXR == 2) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                     : "r"(addr));
+    } else {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+              "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+            : "r"(addr));
+    }
+}
 // shared-memory operand descriptor: K-major, no swizzle, 8-row x 16-byte core matrices `lbo` bytes apart along K
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo) {
     uint64_t d = (uint64_t)((addr >> 4) & 0x3FFFu);
@@ -220,15 +257,26 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo) {
     d |= (uint64_t)1 << 46;            // descriptor version of this architecture
     return d;
 }
-// D[128 x 8] (+)= A[128 x 32 u8, tensor memory] * B[8 x 32 s8, shared memory]^T, int32 accumulate
+// D[128 x kN] (+)= A[128 x 32 u8, tensor memory] * B[kN x 32 s8, shared memory]^T, int32 accumulate
+template <int kN>
 __device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t accumulate) {
     // instruction descriptor: D = s32 (2 at bit 4), A = u8 (0 at bit 7), B = s8 (1 at bit 10), both K-major,
     // N >> 3 at bit 17, M >> 4 at bit 24
-    constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((8u >> 3) << 17) | ((128u >> 4) << 24);
+    constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | (((uint32_t)kN >> 3) << 17) | ((128u >> 4) << 24);
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
+// D[128 x 8] (+)= A[128 x 32 u8, shared memory] * B[8 x 32 s8, shared memory]^T, int32 accumulate
+__device__ __forceinline__ void mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+    constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((8u >> 3) << 17) | ((128u >> 4) << 24);
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
         : "memory");
 }
 
@@ -257,7 +305,13 @@ struct Guard {
             status[5] = (int)parity;
         }
     }
+    // A thread suspended in mbarrier.try_wait wakes up late (measured: hand-overs between roles then cost on the
+    // order of a microsecond each), so a wait first polls without blocking for a while and only then lets the
+    // hardware suspend the thread.
     __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity) const {
+#pragma unroll 1
+        for (int i = 0; i < QIL_TC_SPIN_POLLS; ++i)
+            if (mbar_test_wait(bar, parity)) return true;
         if (mbar_try_wait(bar, parity)) return true;
 #ifdef QIL_TRACE
         return wait_mbar_slow(status, poisoned, bar, parity, polls);
@@ -362,10 +416,13 @@ struct Cyc {
 template <int kXR>
 __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_constant__ TcParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int kLbo = 32 * kXR;   // byte distance between the 16-byte K chunks of the activation operand: the
-                                     // 2 kXR planes of a chunk; rows of the 8-row window beyond them belong to
-                                     // the next chunks and only feed accumulator columns nobody reads
-    constexpr int kDCols = 2 * kXR;  // accumulator columns in use: {high byte, low byte} plane per activation row
+    // Activation operands: per 16-byte K chunk the planes of all activation rows follow each other (2 per row for
+    // x_c, 3 per row for 16 x_a - x_c); the rows of the tensor core's 8- or 16-row window beyond them belong to the
+    // next chunks and only feed accumulator columns nobody reads.
+    constexpr int kLboR = 32 * kXR, kLboM = 48 * kXR;
+    constexpr int kRCols = 2 * kXR, kMCols = 3 * kXR;   // accumulator columns in use
+    constexpr int kMskN = kXR == 4 ? 16 : 8;            // columns of the masked-byte MMA
+    constexpr int kDUnit = d_unit_cols(kXR), kColMeta = col_meta(kXR);
     const int tid = threadIdx.x;
     const uint32_t c = blockIdx.x;
 
@@ -374,17 +431,18 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     unsigned char* xs = ring + (size_t)p.stages * kUnitBytes;                       // [2][xbuf_bytes]
     int* xsum = reinterpret_cast<int*>(xs + (size_t)2 * p.xbuf_bytes);              // [2][kXR][kb_max]
     float* xscale = reinterpret_cast<float*>(xsum + 2 * kXR * p.kb_max);            // [2][kXR][kb_max]
-    float* hand = xscale + 2 * kXR * p.kb_max;                                      // [2][2][kXR][128]
-    float* tpart = hand + 2 * 2 * kXR * kUnitRows;                                  // [2][kXR][128]
+    float* hand = xscale + 2 * kXR * p.kb_max;                                      // [kHandDepth][2][kXR][128]
+    float* tpart = hand + kHandDepth * 2 * kXR * kUnitRows;                         // [2][kXR][128]
     uint64_t* bars = reinterpret_cast<uint64_t*>(tpart + 2 * kXR * kUnitRows);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
     // afull: per unit slot; dfull / dempty: per group of kGroup slots
     const uint32_t afull0 = smem_u32(b2), dfull0 = smem_u32(b2 + kNB), dempty0 = smem_u32(b2 + kNB + kNG);
     uint64_t* b3 = b2 + 3 * kNB;
-    const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2), hfull0 = smem_u32(b3 + 4), hempty0 = smem_u32(b3 + 6);
+    const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2);
     const uint32_t tfull0 = smem_u32(b3 + 8), tempty0 = smem_u32(b3 + 10), mdone0 = smem_u32(b3 + 12);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 12 + kGroup);
+    const uint32_t hfull0 = smem_u32(b3 + 12 + kGroup), hempty0 = smem_u32(b3 + 12 + kGroup + kHandDepth);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 12 + kGroup + 2 * kHandDepth);
     volatile int* poisoned = reinterpret_cast<volatile int*>(tmem_slot + 1);
     // rd[gs][q]: groups of slot group gs that epilogue warp q (tensor-memory lanes 32q..32q+31) has read out
     const uint32_t rd0 = smem_u32(tmem_slot + 2);
@@ -392,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, 4);
+            mbar_init(empty0 + 8 * s, 5);  // the four unpack warps and the commit of the MMAs that read the raw bytes
         }
         for (int i = 0; i < kNB; ++i) mbar_init(afull0 + 8 * i, 4);
         for (int i = 0; i < kNG; ++i) {
@@ -402,12 +460,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         for (int i = 0; i < 2; ++i) {
             mbar_init(xfull0 + 8 * i, 4);  // the stager warps
             mbar_init(xempty0 + 8 * i, 4 * kNumEpi);
-            mbar_init(hfull0 + 8 * i, 4);
-            mbar_init(hempty0 + 8 * i, kFixThreads / 32);
             mbar_init(tfull0 + 8 * i, 4);
             mbar_init(tempty0 + 8 * i, 4);
         }
         for (int i = 0; i < kGroup; ++i) mbar_init(mdone0 + 8 * i, 1);
+        for (int i = 0; i < kHandDepth; ++i) {
+            mbar_init(hfull0 + 8 * i, 4);
+            mbar_init(hempty0 + 8 * i, kFixThreads / 32);
+        }
         *poisoned = 0;
         for (int i = 0; i < 4 * kNG; ++i) tmem_slot[2 + i] = 0u;
         if (blockIdx.x == 0) p.status[6] = (int)full0;  // (reference for the time-out diagnostics)
@@ -459,8 +519,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 QIL_TR_COUNT(3);
                 tc_fence_after();
                 const unsigned char* ub = ring + (size_t)st_i * kUnitBytes;
-                const uint32_t ta = tmem + lane_base + 32 * a;
-                constexpr uint32_t kLo = 0x0F0F0F0Fu, kHi = 0xF0F0F0F0u;
+                const uint32_t ta = tmem + lane_base + 16 * a;
+                constexpr uint32_t kLo = 0x0F0F0F0Fu;
                 uint4 w[4];
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) w[ch] = *reinterpret_cast<const uint4*>(ub + ((size_t)ch * kUnitRows + r) * 16);
@@ -470,12 +530,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 for (int ch = 0; ch < 4; ++ch) {
                     v[4 * ch] = w[ch].x & kLo; v[4 * ch + 1] = w[ch].y & kLo; v[4 * ch + 2] = w[ch].z & kLo; v[4 * ch + 3] = w[ch].w & kLo;
                 }
-                tmem_st16(ta, v);       // A of the two low-nibble MMAs: columns [0, 64) and [64, 128) of the block
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    v[4 * ch] = w[ch].x & kHi; v[4 * ch + 1] = w[ch].y & kHi; v[4 * ch + 2] = w[ch].z & kHi; v[4 * ch + 3] = w[ch].w & kHi;
-                }
-                tmem_st16(ta + 16, v);  // A of the two high-nibble MMAs (values x 16)
+                tmem_st16(ta, v);  // A of the two masked-byte MMAs: chunks 0, 1 and 2, 3 of the block
                 tmem_st1(tmem + lane_base + kColMeta + a, meta);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
@@ -516,8 +571,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             ++xe;
             const int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
             const float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
-            float* hand_b = hand + (size_t)(he & 1) * 2 * kXR * kUnitRows;
-            if (shares && ew == 0 && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * (he & 1), ((he >> 1) & 1) ^ 1))) break;
+            float* hand_b = hand + (size_t)(he % kHandDepth) * 2 * kXR * kUnitRows;
+            if (shares && ew == 0 && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * (he % kHandDepth), ((he / kHandDepth) & 1) ^ 1))) break;
             uint32_t n_full = 0;
             float fin[kXR];
 #pragma unroll
@@ -569,15 +624,17 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 ++ts;
             };
             // one unit of this warpgroup: fold scale and zero point into the row sums
-            auto consume = [&](const uint32_t (&cl)[8], const uint32_t (&ch)[8], uint32_t meta) {
+            // (cr: raw-byte accumulators {x_c high, low plane}; cm: masked-byte accumulators {top, middle, low plane})
+            auto consume = [&](const uint32_t (&cr)[8], const uint32_t (&cm)[16], uint32_t meta) {
                 const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
                 const float s = __low2float(sz);
                 const int z = (int)__high2float(sz);
 #pragma unroll
                 for (int t = 0; t < kXR; ++t)
                     if (t < M) {
-                        const int v = ((int)cl[2 * t] * 256 + (int)cl[2 * t + 1]) + (((int)ch[2 * t] * 256 + (int)ch[2 * t + 1]) >> 4) -
-                                      z * xsum_b[t * p.kb_max + kb];
+                        const int v16 = ((int)cr[2 * t] * 256 + (int)cr[2 * t + 1]) +
+                                        ((int)cm[3 * t] * 65536 + (int)cm[3 * t + 1] * 256 + (int)cm[3 * t + 2]);
+                        const int v = (v16 >> 4) - z * xsum_b[t * p.kb_max + kb];  // (v16 is an exact multiple of 16)
                         fin[t] = fmaf((float)v, s * xscale_b[t * p.kb_max + kb], fin[t]);
                     }
             };
@@ -597,36 +654,29 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
 #ifdef QIL_TRACE
                     const long long tr_e0 = clock64();
 #endif
-                    uint32_t dl[kEB][8], dh[kEB][8], meta[kEB];
+                    uint32_t dr[kEB][8], dm[kEB][16], meta[kEB];
 #pragma unroll
                     for (int i = 0; i < kEB; ++i) {
 #pragma unroll
-                        for (int q = 0; q < kDCols; ++q) dl[i][q] = dh[i][q] = 0u;
+                        for (int q = 0; q < kRCols; ++q) dr[i][q] = 0u;
+#pragma unroll
+                        for (int q = 0; q < kMCols; ++q) dm[i][q] = 0u;
                         meta[i] = 0u;
                         if (b0 + i < nreal) {
                             const uint32_t a = gs * kGroup + b0 + i;
-                            const uint32_t td = tmem + lane_base + kColD + 16 * a;
-                            tmem_ld<kDCols>(td, dl[i]);
-                            tmem_ld<kDCols>(td + 8, dh[i]);
+                            const uint32_t td = tmem + lane_base + kColD + kDUnit * a;
+                            tmem_ld<kRCols>(td, dr[i]);
+                            tmem_ld_m<kXR>(td + 8, dm[i]);
                             meta[i] = tmem_ld1(tmem + lane_base + kColMeta + a);
                         }
                     }
-#ifdef QIL_TRACE
-                    const long long tr_e1 = clock64();
-#endif
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#ifdef QIL_TRACE
-                    const long long tr_e2 = clock64();
-                    tr[7] += tr_e1 - tr_e0;
-                    tr[8] += tr_e2 - tr_e1;
-#endif
 #pragma unroll
                     for (int i = 0; i < kEB; ++i) {  // no use of the loaded registers is scheduled before the wait
 #pragma unroll
-                        for (int q = 0; q < kDCols; ++q) {
-                            asm volatile("" : "+r"(dl[i][q]));
-                            asm volatile("" : "+r"(dh[i][q]));
-                        }
+                        for (int q = 0; q < kRCols; ++q) asm volatile("" : "+r"(dr[i][q]));
+#pragma unroll
+                        for (int q = 0; q < kMCols; ++q) asm volatile("" : "+r"(dm[i][q]));
                         asm volatile("" : "+r"(meta[i]));
                     }
                     if (b0 + kEB >= nreal) {  // the group's columns may be reused
@@ -639,13 +689,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     }
 #ifdef QIL_TRACE
                     const long long tr_e3 = clock64();
-                    tr[9] += tr_e3 - tr_e2;
+                    tr[9] += tr_e3 - tr_e0;
 #endif
 #pragma unroll
                     for (int i = 0; i < kEB; ++i)
                         if (alive && b0 + i < nreal) {
                             QIL_TR_COUNT(5);
-                            consume(dl[i], dh[i], meta[i]);
+                            consume(dr[i], dm[i], meta[i]);
                             if (++kb == KB || j0 + b0 + i + 1 == n) close_tile();
                         }
 #ifdef QIL_TRACE
@@ -658,7 +708,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(xempty0 + 8 * xb);
-                if (shares && ew == 0) mbar_arrive(hfull0 + 8 * (he & 1));
+                if (shares && ew == 0) mbar_arrive(hfull0 + 8 * (he % kHandDepth));
                 // the dependency counter counts quarter tiles (32 rows), so that no warp has to wait for another
                 if (ew == 0 && n_full && p.tiles_done) {
                     __threadfence();
@@ -669,10 +719,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         }
     } else if (tid < kFixBase) {
         // ======================= activation stager (a half warp = one 128-column block per pass) =======================
-        // bf16 row -> per 128 columns: e with max|x| / 2^e <= 32639, v = rint(x / 2^e) = 256 hi + lo (both int8),
-        // X = sum v.  Only the blocks the CTA's units touch are converted.  K order of the operand inside a block:
-        // 16-byte chunk 4p + 2h + cc (p: half of the block, h: low / high nibble columns, cc: 32-column chunk of
-        // the half), byte 4m + b = column 64p + 32cc + 8m + 4h + b.  The four warps work independently.
+        // bf16 row -> per 128 columns: e with max|x| / 2^e <= 32639, v = rint(x / 2^e) as signed-byte planes,
+        // X = sum v.  Only the blocks the CTA's units touch are converted.  K order of both operands inside a block:
+        // 16-byte chunk j (32 columns), byte 4m + b = the packed byte holding columns 32j + 8m + b (low nibble, x_a)
+        // and 32j + 8m + 4 + b (high nibble, x_c).  The four warps work independently.
         const int st = tid - kStagerBase, lane = tid & 31, l16 = st & 15, hw = st >> 4;
         uint32_t xe = 0;
         Walk wk(p, c);
@@ -680,7 +730,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const TcEntry& E = p.e[wk.ei];
             const uint32_t KB = wk.KB;
             const uint32_t xb = xe & 1;
-            unsigned char* xs_b = xs + (size_t)xb * p.xbuf_bytes;
+            unsigned char* xs_b = xs + (size_t)xb * p.xbuf_bytes;                  // planes of x_c
+            unsigned char* xm_b = xs_b + (size_t)p.kb_max * 4 * kLboR + 256;       // planes of 16 x_a - x_c
             int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
             float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
             bool ok = true;
@@ -697,7 +748,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const long long tr_conv0 = clock64();
 #endif
             const uint32_t nblk = min(KB, wk.u1 - wk.u0), kb0 = wk.u0 % KB;
-            const uint32_t p_half = (uint32_t)l16 >> 3, cc = ((uint32_t)l16 >> 2) & 1, m = (uint32_t)l16 & 3;
+            const uint32_t m = (uint32_t)l16 & 3;
             for (int t = 0; t < E.M; ++t) {
                 const uint16_t* xrow = E.x + (size_t)t * E.K;
                 // up to four passes of 8 blocks at a time: their loads are all in flight before the first conversion
@@ -732,32 +783,42 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         int e = ef - 127 - 14 + (((amax & 0x7FFFFFu) > 0x7EFE00u) ? 1 : 0);
                         if (e < -126) e = -126;
                         const float inv = __uint_as_float((uint32_t)(127 - e) << 23);  // 2^-e
-                        // v = rint(x * 2^-e) through the 1.5 * 2^23 trick; v + 128 = 256 * hi + (lo + 128)
-                        uint32_t vb[8];
+                        // v = rint(x * 2^-e) through the 1.5 * 2^23 trick
+                        int vq[8];
                         int sum = 0;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const float f0 = fmaf(__uint_as_float(u[j] << 16), inv, 12582912.f);
                             const float f1 = fmaf(__uint_as_float(u[j] & 0xFFFF0000u), inv, 12582912.f);
-                            const int q0 = (int)(__float_as_uint(f0) - 0x4B400000u), q1 = (int)(__float_as_uint(f1) - 0x4B400000u);
-                            sum += q0 + q1;
-                            vb[2 * j] = (uint32_t)(q0 + 128);
-                            vb[2 * j + 1] = (uint32_t)(q1 + 128);
+                            vq[2 * j] = (int)(__float_as_uint(f0) - 0x4B400000u);
+                            vq[2 * j + 1] = (int)(__float_as_uint(f1) - 0x4B400000u);
+                            sum += vq[2 * j] + vq[2 * j + 1];
                         }
 #pragma unroll
                         for (int o = 1; o < 16; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
                         if (valid) {
-                            // byte 0 of each (v + 128) is lo + 128, byte 1 is hi; columns 0-3 of the piece sit under low
-                            // nibbles, columns 4-7 under high nibbles
-                            const uint32_t lo_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0040), __byte_perm(vb[2], vb[3], 0x0040), 0x5410) ^ 0x80808080u;
-                            const uint32_t lo_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0040), __byte_perm(vb[6], vb[7], 0x0040), 0x5410) ^ 0x80808080u;
-                            const uint32_t hi_a = __byte_perm(__byte_perm(vb[0], vb[1], 0x0051), __byte_perm(vb[2], vb[3], 0x0051), 0x5410);
-                            const uint32_t hi_b = __byte_perm(__byte_perm(vb[4], vb[5], 0x0051), __byte_perm(vb[6], vb[7], 0x0051), 0x5410);
-                            unsigned char* dst = xs_b + (size_t)(kb * 8 + 4 * p_half + cc) * kLbo + (size_t)(2 * t) * 16 + 4 * m;
-                            *reinterpret_cast<uint32_t*>(dst) = hi_a;
-                            *reinterpret_cast<uint32_t*>(dst + 16) = lo_a;
-                            *reinterpret_cast<uint32_t*>(dst + 2 * kLbo) = hi_b;
-                            *reinterpret_cast<uint32_t*>(dst + 2 * kLbo + 16) = lo_b;
+                            // Columns 0-3 of the piece sit under low nibbles (x_a), columns 4-7 under high nibbles (x_c).
+                            // A biased integer t + 0x808080 has the bytes b_i with t = sum (b_i - 128) 256^i: its bytes
+                            // XOR 0x80 are the signed planes (two for x_c, three for 16 x_a - x_c, |.| < 2^20).
+                            uint32_t uc[4], um[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                uc[j] = (uint32_t)(vq[4 + j] + 0x8080);
+                                um[j] = (uint32_t)(16 * vq[j] - vq[4 + j] + 0x808080);
+                            }
+                            const uint32_t c0 = __byte_perm(__byte_perm(uc[0], uc[1], 0x0040), __byte_perm(uc[2], uc[3], 0x0040), 0x5410) ^ 0x80808080u;
+                            const uint32_t c1 = __byte_perm(__byte_perm(uc[0], uc[1], 0x0051), __byte_perm(uc[2], uc[3], 0x0051), 0x5410) ^ 0x80808080u;
+                            const uint32_t m0 = __byte_perm(__byte_perm(um[0], um[1], 0x0040), __byte_perm(um[2], um[3], 0x0040), 0x5410) ^ 0x80808080u;
+                            const uint32_t m1 = __byte_perm(__byte_perm(um[0], um[1], 0x0051), __byte_perm(um[2], um[3], 0x0051), 0x5410) ^ 0x80808080u;
+                            const uint32_t m2 = __byte_perm(__byte_perm(um[0], um[1], 0x0062), __byte_perm(um[2], um[3], 0x0062), 0x5410) ^ 0x80808080u;
+                            // piece l16 = bytes 4m .. 4m+3 of 16-byte chunk l16 / 4 of the block
+                            unsigned char* dr = xs_b + (size_t)(kb * 4 + (l16 >> 2)) * kLboR + (size_t)(2 * t) * 16 + 4 * m;
+                            *reinterpret_cast<uint32_t*>(dr) = c1;       // high plane of x_c
+                            *reinterpret_cast<uint32_t*>(dr + 16) = c0;  // low plane
+                            unsigned char* dm = xm_b + (size_t)(kb * 4 + (l16 >> 2)) * kLboM + (size_t)(3 * t) * 16 + 4 * m;
+                            *reinterpret_cast<uint32_t*>(dm) = m2;       // top plane of 16 x_a - x_c
+                            *reinterpret_cast<uint32_t*>(dm + 16) = m1;
+                            *reinterpret_cast<uint32_t*>(dm + 32) = m0;
                             if (l16 == 0) {
                                 xsum_b[t * p.kb_max + kb] = sum;
                                 xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);
@@ -791,7 +852,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const bool have_first = t_first * KB < u0 && (t_first + 1) * KB <= u1;  // completes a tile begun elsewhere
             if (!have_last && !(t_first * KB < u0)) continue;
             const uint32_t tag = (uint32_t)wk.ei + 1u, ring_i = (uint32_t)wk.ei % kSlotDepth;
-            const float* hand_b = hand + (size_t)(he & 1) * 2 * kXR * kUnitRows;
+            const float* hand_b = hand + (size_t)(he % kHandDepth) * 2 * kXR * kUnitRows;
             unsigned long long* my_slot = nullptr;
             if (have_last) {
                 const uint32_t which = (t_last == t_first) ? 0u : 1u;
@@ -804,7 +865,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         alive = QIL_WAIT(1, guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; }));
                     }
             }
-            alive = alive && QIL_WAIT(2, guard.wait_mbar(hfull0 + 8 * (he & 1), (he >> 1) & 1));
+            alive = alive && QIL_WAIT(2, guard.wait_mbar(hfull0 + 8 * (he % kHandDepth), (he / kHandDepth) & 1));
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
             if (have_last) {  // publish first (a chain of CTAs must never wait on each other in a circle)
@@ -863,7 +924,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(hempty0 + 8 * (he & 1));
+                mbar_arrive(hempty0 + 8 * (he % kHandDepth));
                 if (have_first && p.tiles_done) {  // this warp's rows of the tile are written: kRowsPer quarter tiles
                     __threadfence();
                     red_release_add(p.tiles_done, kRowsPer);
@@ -880,33 +941,48 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             uint32_t xe = 0, G = 0;
             bool alive = true, issued = false;
             Walk wk(p, c);
-            const uint64_t desc_hi = smem_desc(0, kLbo);
-            constexpr uint32_t lbo16 = (uint32_t)kLbo >> 4;
+            const uint64_t desc_r = smem_desc(0, kLboR), desc_m = smem_desc(0, kLboM), desc_a = smem_desc(0, kUnitRows * 16);
+            constexpr uint32_t lbor16 = (uint32_t)kLboR >> 4, lbom16 = (uint32_t)kLboM >> 4;
+            const uint32_t S = (uint32_t)p.stages, ring16 = smem_u32(ring) >> 4;
+            uint32_t stage0 = 0;  // ring stage of the entry's first unit
             while (alive && wk.next_entry()) {
                 const uint32_t KB = wk.KB, n = wk.u1 - wk.u0;
                 const uint32_t xb = xe & 1;
                 if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1))) break;
                 ++xe;
-                const uint32_t xs16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
+                const uint32_t xr16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
+                const uint32_t xm16 = xr16 + (((uint32_t)p.kb_max * 4 * kLboR + 256) >> 4);
                 uint32_t kb = (wk.u0 + w) % KB;
                 const uint32_t kstep = kGroup % KB;
+                uint32_t st_i = (stage0 + w) % S;
                 for (uint32_t j = w; j < (n + kGroup - 1) / kGroup * kGroup; j += kGroup, ++G) {
                     const uint32_t gs = G % kNG, gph = (G / kNG) & 1;
                     if (j < n) {
                         const uint32_t a = gs * kGroup + w;
-                        if (!QIL_WAIT(2, guard.wait_mbar(afull0 + 8 * a, gph))) {  // (the unpack warps waited for the accumulators to be free)
+                        if (!QIL_WAIT(2, guard.wait_mbar(afull0 + 8 * a, gph))) {  // (the unpack warps waited for the columns to be free)
                             alive = false;
                             break;
                         }
                         tc_fence_after();
-                        const uint32_t ta = tmem + 32 * a, td = tmem + kColD + 16 * a;
-                        const uint64_t b0 = desc_hi | (uint64_t)(xs16 + kb * 8 * lbo16);
-                        mma_i8_ts(td, ta, b0, 0u);                        // low nibbles, columns [0, 64)
-                        mma_i8_ts(td, ta + 8, b0 + 4 * lbo16, 1u);        // low nibbles, columns [64, 128)
-                        mma_i8_ts(td + 8, ta + 16, b0 + 2 * lbo16, 0u);   // high nibbles
-                        mma_i8_ts(td + 8, ta + 24, b0 + 6 * lbo16, 1u);
+#ifdef QIL_TRACE
+                        const long long tr_m0 = clock64();
+#endif
+                        const uint32_t ta = tmem + 16 * a, td = tmem + kColD + kDUnit * a;
+                        // raw bytes of the unit in the ring: 16-byte chunk j at j * 2048, rows 16 bytes apart
+                        const uint64_t a0 = desc_a | (uint64_t)(ring16 + st_i * (kUnitBytes >> 4));
+                        const uint64_t br = desc_r | (uint64_t)(xr16 + kb * 4 * lbor16);
+                        const uint64_t bm = desc_m | (uint64_t)(xm16 + kb * 4 * lbom16);
+                        mma_i8_ss(td, a0, br, 0u);                                        // raw bytes x x_c, chunks 0, 1
+                        mma_i8_ss(td, a0 + 2 * (kUnitRows * 16 >> 4), br + 2 * lbor16, 1u);  // chunks 2, 3
+                        mma_i8_ts<kMskN>(td + 8, ta, bm, 0u);                             // masked bytes x (16 x_a - x_c)
+                        mma_i8_ts<kMskN>(td + 8, ta + 8, bm + 2 * lbom16, 1u);
                         tc_commit(dfull0 + 8 * gs);
+                        tc_commit(empty0 + 8 * st_i);  // the ring stage has been read
                         issued = true;
+#ifdef QIL_TRACE
+                        tr[4] += clock64() - tr_m0;
+                        tr[5] += 1;
+#endif
                     } else {
                         // The entry ends inside the group: this slot stays empty, its barriers still change phase.  Like
                         // the unpack warps the thread first waits until the groups that used these columns before have
@@ -919,7 +995,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     }
                     kb += kstep;
                     if (kb >= KB) kb -= KB;
+                    st_i += kGroup;
+                    if (st_i >= S) st_i -= S;
                 }
+                stage0 = (stage0 + n) % S;
             }
             // whatever happened to the other roles: the operations this thread issued are complete before tensor memory
             // is released (this wait also holds in an abandoned kernel)
@@ -1019,16 +1098,17 @@ constexpr size_t kSmemLimit = 232448;  // 227 KiB per CTA
 SmemPlan plan_for(int max_m, int kb_max) {
     SmemPlan pl;
     pl.x_rows = max_m <= 1 ? 1 : max_m <= 2 ? 2 : 4;
-    const int lbo = 32 * pl.x_rows;
-    pl.xbuf_bytes = kb_max * 8 * lbo + 128;  // the last chunk's 8-row window reaches past its own rows
+    pl.xbuf_bytes = kb_max * 4 * (32 + 48) * pl.x_rows + 512;  // (the last chunk's row window reaches past its own rows)
     const size_t fixed = (size_t)2 * pl.xbuf_bytes + (size_t)2 * 2 * pl.x_rows * kb_max * 4 +
-                         (size_t)3 * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 12 + kGroup) * 8 + 16 + 16 * kNG + 128;
+                         (size_t)(kHandDepth + 1) * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 12 + kGroup + 2 * kHandDepth) * 8 + 16 +
+                         16 * kNG + 128;
     pl.stages = 0;
     if (fixed < kSmemLimit) {
         long s = (long)((kSmemLimit - fixed) / (kUnitBytes + 16));
         if (s > 24) s = 24;
         s -= s % kNumWg;  // a ring stage is then always consumed by the same unpack warpgroup, which sees each of its phases
         pl.stages = (int)s;
+        if (pl.stages <= kGroup) pl.stages = 0;  // (the issuers step through the ring by kGroup)
     }
     pl.total = fixed + (size_t)pl.stages * (kUnitBytes + 16);
     return pl;

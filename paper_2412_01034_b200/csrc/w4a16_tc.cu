@@ -46,6 +46,7 @@
 // workspace status word (with the place in words 2..5 of the workspace), every role stops at its
 // next wait without issuing further work, outstanding copies and tensor-core operations are
 // waited for, tensor memory is released and the kernel returns.
+#include <algorithm>
 #include <mutex>
 
 #include "qil_common.cuh"
@@ -90,13 +91,17 @@ constexpr int kNumEpi = QIL_TC_EPILOGUE_WGS;      // epilogue warpgroups (they a
 constexpr int kEpiBase = kUnpackThreads;         // (their warps keep warp % 4 = lane quarter)
 constexpr int kStagerBase = kEpiBase + 128 * kNumEpi;
 constexpr int kFixBase = kStagerBase + 128;
-constexpr int kFixThreads = 64;                  // fixer: two warps, two rows of the tile per thread
+constexpr int kFixTeams = 4;                     // fixer warps: entry i's shared tiles belong to warp i % kFixTeams
+constexpr int kFixThreads = 32 * kFixTeams;      // (a lane takes four rows of the tile)
 constexpr int kGroup = 4;                        // units per group: one per MMA issuer, one epilogue pass
 constexpr int kMmaBase = kFixBase + kFixThreads; // kGroup warps, one issuing thread each
 constexpr int kProdBase = kMmaBase + 32 * kGroup;  // one warp, one thread issues
 constexpr int kThreads = kProdBase + 32;
 static_assert(kThreads <= 1024, "block size");
-constexpr int kNG = 3;                           // groups in flight in tensor memory
+#ifndef QIL_TC_GROUPS
+#define QIL_TC_GROUPS 3
+#endif
+constexpr int kNG = QIL_TC_GROUPS;               // groups in flight in tensor memory
 constexpr int kNB = kGroup * kNG;                // = units in flight
 constexpr int kTmemCols = 512;
 // tensor-memory columns: per unit 16 of masked low nibbles (A), 8 accumulators of the raw-byte products and 8 (16 with
@@ -106,10 +111,12 @@ __host__ __device__ constexpr int d_unit_cols(int xr) { return 8 + (xr == 4 ? 16
 __host__ __device__ constexpr int col_meta(int xr) { return kColD + d_unit_cols(xr) * kNB; }
 static_assert(col_meta(4) + kNB <= kTmemCols, "tensor memory budget");
 static_assert(kNumEpi == 1 || kNG % kNumEpi == 0, "a slot group must always be read out by the same epilogue warpgroup");
-constexpr int kHandDepth = 8;                    // hand-over buffers between the epilogue and the fixer
+constexpr int kMaxXBufs = 4;                     // activation buffers at most
+constexpr int kHandDepth = 2 * kFixTeams;        // hand-over buffers between the epilogue and the fixer: two per warp
 constexpr int kMaxEntries = 256;
 constexpr int kMaxRows = 4;                      // activation rows
 constexpr int kSlotDepth = 4;                    // ring of slots per (CTA, first / last tile), indexed by entry
+static_assert(kSlotDepth == kFixTeams, "a slot is always written by the same fixer warp, in entry order");
 constexpr int kSlotElems = kMaxRows * kUnitRows; // {value, tag} pairs of 8 bytes
 constexpr int kWsHeader = 256;
 constexpr int kFlagDep = 1;
@@ -129,7 +136,8 @@ struct TcParams {
     TcEntry e[kMaxEntries];
     int count;
     int stages;
-    int kb_max;      // max K / 128
+    int nb_max;      // 128-column blocks an activation buffer holds (>= the blocks a CTA touches in any entry)
+    int xbufs;       // activation buffers (entries the stager may run ahead)
     int xbuf_bytes;  // one activation operand buffer
     int* status;
     unsigned int* tiles_done;
@@ -428,10 +436,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
 
     // ---- carve shared memory ----
     unsigned char* ring = smem;                                                     // [stages][kUnitBytes]
-    unsigned char* xs = ring + (size_t)p.stages * kUnitBytes;                       // [2][xbuf_bytes]
-    int* xsum = reinterpret_cast<int*>(xs + (size_t)2 * p.xbuf_bytes);              // [2][kXR][kb_max]
-    float* xscale = reinterpret_cast<float*>(xsum + 2 * kXR * p.kb_max);            // [2][kXR][kb_max]
-    float* hand = xscale + 2 * kXR * p.kb_max;                                      // [kHandDepth][2][kXR][128]
+    unsigned char* xs = ring + (size_t)p.stages * kUnitBytes;                       // [xbufs][xbuf_bytes]
+    int* xsum = reinterpret_cast<int*>(xs + (size_t)p.xbufs * p.xbuf_bytes);        // [xbufs][kXR][nb_max]
+    float* xscale = reinterpret_cast<float*>(xsum + p.xbufs * kXR * p.nb_max);      // [xbufs][kXR][nb_max]
+    float* hand = xscale + p.xbufs * kXR * p.nb_max;                                // [kHandDepth][2][kXR][128]
     float* tpart = hand + kHandDepth * 2 * kXR * kUnitRows;                         // [2][kXR][128]
     uint64_t* bars = reinterpret_cast<uint64_t*>(tpart + 2 * kXR * kUnitRows);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
@@ -439,7 +447,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     // afull: per unit slot; dfull / dempty: per group of kGroup slots
     const uint32_t afull0 = smem_u32(b2), dfull0 = smem_u32(b2 + kNB), dempty0 = smem_u32(b2 + kNB + kNG);
     uint64_t* b3 = b2 + 3 * kNB;
-    const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + 2);
+    const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + kMaxXBufs);
     const uint32_t tfull0 = smem_u32(b3 + 8), tempty0 = smem_u32(b3 + 10), mdone0 = smem_u32(b3 + 12);
     const uint32_t hfull0 = smem_u32(b3 + 12 + kGroup), hempty0 = smem_u32(b3 + 12 + kGroup + kHandDepth);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 12 + kGroup + 2 * kHandDepth);
@@ -457,23 +465,25 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             mbar_init(dfull0 + 8 * i, kGroup);  // one arrival per issuer
             mbar_init(dempty0 + 8 * i, 4);      // the epilogue warps
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kMaxXBufs; ++i) {
             mbar_init(xfull0 + 8 * i, 4);  // the stager warps
             mbar_init(xempty0 + 8 * i, 4 * kNumEpi);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(tfull0 + 8 * i, 4);
             mbar_init(tempty0 + 8 * i, 4);
         }
         for (int i = 0; i < kGroup; ++i) mbar_init(mdone0 + 8 * i, 1);
         for (int i = 0; i < kHandDepth; ++i) {
             mbar_init(hfull0 + 8 * i, 4);
-            mbar_init(hempty0 + 8 * i, kFixThreads / 32);
+            mbar_init(hempty0 + 8 * i, 1);
         }
         *poisoned = 0;
         for (int i = 0; i < 4 * kNG; ++i) tmem_slot[2 + i] = 0u;
         if (blockIdx.x == 0) p.status[6] = (int)full0;  // (reference for the time-out diagnostics)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < 2 * p.xbuf_bytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(xs)[i] = 0u;
+    for (int i = tid; i < p.xbufs * p.xbuf_bytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(xs)[i] = 0u;
     if (tid < 32) {  // one warp owns the tensor-memory allocation
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(kTmemCols));
@@ -557,7 +567,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         const uint32_t lane_base = (r & ~31u) << 16;
         constexpr int kEBmax = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;                      // (registers)
         constexpr int kEB = QIL_TC_EPI_BATCH < kEBmax ? QIL_TC_EPI_BATCH : kEBmax;  // units read back per tcgen05.wait::ld
-        uint32_t xe = 0, he = 0, G = 0, ts = 0;               // ts: row tiles closed so far
+        uint32_t hc = 0, G = 0, ts = 0;  // hc: per fixer warp, two bits counting the entries handed to it; ts: row tiles closed
+        Cyc xc(p.xbufs);
         bool alive = true;
         Walk wk(p, c);
         while (alive && wk.next_entry()) {
@@ -566,13 +577,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, n = u1 - u0;
             const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
             const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
-            const uint32_t xb = xe & 1;
-            if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1))) break;
-            ++xe;
-            const int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
-            const float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
-            float* hand_b = hand + (size_t)(he % kHandDepth) * 2 * kXR * kUnitRows;
-            if (shares && ew == 0 && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * (he % kHandDepth), ((he / kHandDepth) & 1) ^ 1))) break;
+            const uint32_t xb = xc.idx, kb0 = u0 % KB;  // (a buffer holds the blocks from the slice's first one on, cyclically)
+            if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xc.ph))) break;
+            xc.step();
+            const int* xsum_b = xsum + (size_t)xb * kXR * p.nb_max;
+            const float* xscale_b = xscale + (size_t)xb * kXR * p.nb_max;
+            const uint32_t team = (uint32_t)wk.ei % kFixTeams, hcnt = (hc >> (2 * team)) & 3u;
+            const uint32_t hbuf = 2 * team + (hcnt & 1u);
+            float* hand_b = hand + (size_t)hbuf * 2 * kXR * kUnitRows;
+            if (shares && ew == 0 && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * hbuf, ((hcnt >> 1) & 1u) ^ 1u))) break;
             uint32_t n_full = 0;
             float fin[kXR];
 #pragma unroll
@@ -629,13 +642,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
                 const float s = __low2float(sz);
                 const int z = (int)__high2float(sz);
+                const uint32_t bi = kb >= kb0 ? kb - kb0 : kb + KB - kb0;
 #pragma unroll
                 for (int t = 0; t < kXR; ++t)
                     if (t < M) {
                         const int v16 = ((int)cr[2 * t] * 256 + (int)cr[2 * t + 1]) +
                                         ((int)cm[3 * t] * 65536 + (int)cm[3 * t + 1] * 256 + (int)cm[3 * t + 2]);
-                        const int v = (v16 >> 4) - z * xsum_b[t * p.kb_max + kb];  // (v16 is an exact multiple of 16)
-                        fin[t] = fmaf((float)v, s * xscale_b[t * p.kb_max + kb], fin[t]);
+                        const int v = (v16 >> 4) - z * xsum_b[t * p.nb_max + bi];  // (v16 is an exact multiple of 16)
+                        fin[t] = fmaf((float)v, s * xscale_b[t * p.nb_max + bi], fin[t]);
                     }
             };
             for (uint32_t j0 = 0; alive && j0 < n; j0 += kGroup, ++G) {
@@ -708,14 +722,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(xempty0 + 8 * xb);
-                if (shares && ew == 0) mbar_arrive(hfull0 + 8 * (he % kHandDepth));
+                if (shares && ew == 0) mbar_arrive(hfull0 + 8 * hbuf);
                 // the dependency counter counts quarter tiles (32 rows), so that no warp has to wait for another
                 if (ew == 0 && n_full && p.tiles_done) {
                     __threadfence();
                     red_release_add(p.tiles_done, n_full);
                 }
             }
-            if (shares) ++he;
+            if (shares) hc = (hc & ~(3u << (2 * team))) | (((hcnt + 1u) & 3u) << (2 * team));
         }
     } else if (tid < kFixBase) {
         // ======================= activation stager (a half warp = one 128-column block per pass) =======================
@@ -724,19 +738,19 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // 16-byte chunk j (32 columns), byte 4m + b = the packed byte holding columns 32j + 8m + b (low nibble, x_a)
         // and 32j + 8m + 4 + b (high nibble, x_c).  The four warps work independently.
         const int st = tid - kStagerBase, lane = tid & 31, l16 = st & 15, hw = st >> 4;
-        uint32_t xe = 0;
+        Cyc xc(p.xbufs);
         Walk wk(p, c);
         while (wk.next_entry()) {
             const TcEntry& E = p.e[wk.ei];
             const uint32_t KB = wk.KB;
-            const uint32_t xb = xe & 1;
+            const uint32_t xb = xc.idx;
             unsigned char* xs_b = xs + (size_t)xb * p.xbuf_bytes;                  // planes of x_c
-            unsigned char* xm_b = xs_b + (size_t)p.kb_max * 4 * kLboR + 256;       // planes of 16 x_a - x_c
-            int* xsum_b = xsum + (size_t)xb * kXR * p.kb_max;
-            float* xscale_b = xscale + (size_t)xb * kXR * p.kb_max;
+            unsigned char* xm_b = xs_b + (size_t)p.nb_max * 4 * kLboR + 256;       // planes of 16 x_a - x_c
+            int* xsum_b = xsum + (size_t)xb * kXR * p.nb_max;
+            float* xscale_b = xscale + (size_t)xb * kXR * p.nb_max;
             bool ok = true;
             if (lane == 0) {  // the buffer is free; the rows of x are written (quarter tiles of all earlier entries)
-                ok = QIL_WAIT(1, guard.wait_mbar(xempty0 + 8 * xb, ((xe >> 1) & 1) ^ 1));
+                ok = QIL_WAIT(1, guard.wait_mbar(xempty0 + 8 * xb, xc.ph ^ 1));
                 if (ok && (E.flags & kFlagDep)) {
                     const unsigned int need = 4u * E.tiles_before;
                     ok = QIL_WAIT(2, guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; }));
@@ -812,16 +826,16 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             const uint32_t m1 = __byte_perm(__byte_perm(um[0], um[1], 0x0051), __byte_perm(um[2], um[3], 0x0051), 0x5410) ^ 0x80808080u;
                             const uint32_t m2 = __byte_perm(__byte_perm(um[0], um[1], 0x0062), __byte_perm(um[2], um[3], 0x0062), 0x5410) ^ 0x80808080u;
                             // piece l16 = bytes 4m .. 4m+3 of 16-byte chunk l16 / 4 of the block
-                            unsigned char* dr = xs_b + (size_t)(kb * 4 + (l16 >> 2)) * kLboR + (size_t)(2 * t) * 16 + 4 * m;
+                            unsigned char* dr = xs_b + (size_t)(i * 4 + (l16 >> 2)) * kLboR + (size_t)(2 * t) * 16 + 4 * m;
                             *reinterpret_cast<uint32_t*>(dr) = c1;       // high plane of x_c
                             *reinterpret_cast<uint32_t*>(dr + 16) = c0;  // low plane
-                            unsigned char* dm = xm_b + (size_t)(kb * 4 + (l16 >> 2)) * kLboM + (size_t)(3 * t) * 16 + 4 * m;
+                            unsigned char* dm = xm_b + (size_t)(i * 4 + (l16 >> 2)) * kLboM + (size_t)(3 * t) * 16 + 4 * m;
                             *reinterpret_cast<uint32_t*>(dm) = m2;       // top plane of 16 x_a - x_c
                             *reinterpret_cast<uint32_t*>(dm + 16) = m1;
                             *reinterpret_cast<uint32_t*>(dm + 32) = m0;
                             if (l16 == 0) {
-                                xsum_b[t * p.kb_max + kb] = sum;
-                                xscale_b[t * p.kb_max + kb] = __uint_as_float((uint32_t)(127 + e) << 23);
+                                xsum_b[t * p.nb_max + i] = sum;
+                                xscale_b[t * p.nb_max + i] = __uint_as_float((uint32_t)(127 + e) << 23);
                             }
                         }
                     }
@@ -833,17 +847,21 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             tr[3] += clock64() - tr_conv0;
 #endif
             if (lane == 0) mbar_arrive(xfull0 + 8 * xb);
-            ++xe;
+            xc.step();
         }
     } else if (tid < kMmaBase) {
-        // ======================= fixer (two warps, thread = two rows of the tile): all cross-CTA work =======================
-        const uint32_t fr = tid - kFixBase, lane = tid & 31;
-        constexpr uint32_t kRowsPer = kUnitRows / kFixThreads;
+        // ======================= fixer warps (lane = four rows of the tile): all cross-CTA work =======================
+        // The shared tiles of an entry cost several round trips through the L2 (is the slot free, the other CTAs'
+        // parts, the output); the warps take the entries in turn so that these latencies overlap.
+        const uint32_t team = (uint32_t)(tid - kFixBase) >> 5, lane = tid & 31;
+        constexpr uint32_t kRowsPer = kUnitRows / 32;
+        constexpr uint32_t kPoll = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;  // other CTAs' parts fetched together (registers)
         unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
-        uint32_t he = 0;
+        uint32_t cnt = 0;  // entries this warp has taken over
         bool alive = true;
         Walk wk(p, c);
         while (alive && wk.next_entry()) {
+            if ((uint32_t)wk.ei % kFixTeams != team) continue;
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1;
@@ -852,25 +870,28 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const bool have_first = t_first * KB < u0 && (t_first + 1) * KB <= u1;  // completes a tile begun elsewhere
             if (!have_last && !(t_first * KB < u0)) continue;
             const uint32_t tag = (uint32_t)wk.ei + 1u, ring_i = (uint32_t)wk.ei % kSlotDepth;
-            const float* hand_b = hand + (size_t)(he % kHandDepth) * 2 * kXR * kUnitRows;
+            const uint32_t hbuf = 2 * team + (cnt & 1u), hph = (cnt >> 1) & 1u;
+            const float* hand_b = hand + (size_t)hbuf * 2 * kXR * kUnitRows;
             unsigned long long* my_slot = nullptr;
             if (have_last) {
                 const uint32_t which = (t_last == t_first) ? 0u : 1u;
                 my_slot = slots + (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems;
                 // the slot must have been consumed (tags cleared) by whoever completed the tile it last served;
                 // checked now, while the units are still being computed
-                for (uint32_t h = 0; alive && h < kRowsPer; ++h)
-                    for (int t = 0; alive && t < M; ++t) {
-                        const unsigned long long* q = my_slot + t * kUnitRows + fr + h * kFixThreads;
-                        alive = QIL_WAIT(1, guard.wait_flag([&] { return (uint32_t)(__ldcg(q) >> 32) == 0u; }));
-                    }
+                alive = QIL_WAIT(1, guard.wait_flag([&] {
+                    bool is_free = true;
+                    for (uint32_t h = 0; h < kRowsPer; ++h)
+                        for (int t = 0; t < kXR; ++t)
+                            if (t < M) is_free &= (uint32_t)(__ldcg(my_slot + t * kUnitRows + lane + 32 * h) >> 32) == 0u;
+                    return is_free;
+                }));
             }
-            alive = alive && QIL_WAIT(2, guard.wait_mbar(hfull0 + 8 * (he % kHandDepth), (he / kHandDepth) & 1));
+            alive = alive && QIL_WAIT(2, guard.wait_mbar(hfull0 + 8 * hbuf, hph));
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
             if (have_last) {  // publish first (a chain of CTAs must never wait on each other in a circle)
                 for (uint32_t h = 0; h < kRowsPer; ++h) {
-                    const uint32_t r = fr + h * kFixThreads;
+                    const uint32_t r = lane + 32 * h;
                     for (int t = 0; t < M; ++t)
                         __stcg(my_slot + t * kUnitRows + r,
                                ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(hand_b[(kXR + t) * kUnitRows + r]));
@@ -883,38 +904,54 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 for (uint32_t h = 0; h < kRowsPer; ++h)
 #pragma unroll
                     for (int t = 0; t < kXR; ++t) sum[h][t] = 0.f;
-                for (uint32_t cc = c_lo; cc < c; ++cc) {
-                    uint32_t cu0, cu1;
-                    slice_of(E.q, E.rem, cc, cu0, cu1);
-                    if (cu0 == cu1) continue;
-                    const uint32_t which = (cu0 / KB == t_first) ? 0u : 1u;
-                    unsigned long long* src = slots + (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + fr;
-                    unsigned long long got[kRowsPer][kXR];
+                for (uint32_t cc0 = c_lo; cc0 < c; cc0 += kPoll) {
+                    unsigned long long* src[kPoll];
+                    unsigned long long got[kPoll][kRowsPer][kXR];
+#pragma unroll
+                    for (uint32_t k = 0; k < kPoll; ++k) {
+                        src[k] = nullptr;
+                        uint32_t cu0 = 0, cu1 = 0;
+                        if (cc0 + k < c) slice_of(E.q, E.rem, cc0 + k, cu0, cu1);
+                        if (cu0 != cu1) {
+                            const uint32_t which = (cu0 / KB == t_first) ? 0u : 1u;
+                            src[k] = slots + (((size_t)(cc0 + k) * 2 + which) * kSlotDepth + ring_i) * kSlotElems + lane;
+                        }
+                    }
                     alive = QIL_WAIT(3, guard.wait_flag([&] {
                         bool all = true;
-                        for (uint32_t h = 0; h < kRowsPer; ++h)
-                            for (int t = 0; t < kXR; ++t)
-                                if (t < M) {
-                                    got[h][t] = __ldcg(src + t * kUnitRows + h * kFixThreads);
-                                    all &= (uint32_t)(got[h][t] >> 32) == tag;
-                                }
+#pragma unroll
+                        for (uint32_t k = 0; k < kPoll; ++k)
+                            if (src[k] != nullptr) {
+#pragma unroll
+                                for (uint32_t h = 0; h < kRowsPer; ++h)
+#pragma unroll
+                                    for (int t = 0; t < kXR; ++t)
+                                        if (t < M) {
+                                            got[k][h][t] = __ldcg(src[k] + t * kUnitRows + 32 * h);
+                                            all &= (uint32_t)(got[k][h][t] >> 32) == tag;
+                                        }
+                            }
                         return all;
                     }));
                     alive = __all_sync(0xffffffffu, alive);
                     if (!alive) break;
 #pragma unroll
-                    for (uint32_t h = 0; h < kRowsPer; ++h)
+                    for (uint32_t k = 0; k < kPoll; ++k)  // (always summed in CTA order)
+                        if (src[k] != nullptr) {
 #pragma unroll
-                        for (int t = 0; t < kXR; ++t)
-                            if (t < M) {
-                                sum[h][t] += __uint_as_float((uint32_t)got[h][t]);
-                                __stcg(src + t * kUnitRows + h * kFixThreads, 0ull);  // consumed: the slot may be reused
-                            }
+                            for (uint32_t h = 0; h < kRowsPer; ++h)
+#pragma unroll
+                                for (int t = 0; t < kXR; ++t)
+                                    if (t < M) {
+                                        sum[h][t] += __uint_as_float((uint32_t)got[k][h][t]);
+                                        __stcg(src[k] + t * kUnitRows + 32 * h, 0ull);  // consumed: the slot may be reused
+                                    }
+                        }
                 }
                 if (!alive) break;
 #pragma unroll
                 for (uint32_t h = 0; h < kRowsPer; ++h) {
-                    const uint32_t r = fr + h * kFixThreads, row = t_first * kUnitRows + r;
+                    const uint32_t r = lane + 32 * h, row = t_first * kUnitRows + r;
                     if (row < (uint32_t)N) {
 #pragma unroll
                         for (int t = 0; t < kXR; ++t)
@@ -924,13 +961,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(hempty0 + 8 * (he % kHandDepth));
-                if (have_first && p.tiles_done) {  // this warp's rows of the tile are written: kRowsPer quarter tiles
+                mbar_arrive(hempty0 + 8 * hbuf);
+                if (have_first && p.tiles_done) {  // the tile is written: kRowsPer quarter tiles
                     __threadfence();
                     red_release_add(p.tiles_done, kRowsPer);
                 }
             }
-            ++he;
+            ++cnt;
         }
     } else if (tid < kProdBase) {
         // ======================= MMA issuers (one thread in each of kGroup warps) =======================
@@ -938,7 +975,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // core at 8 columns; issuer w therefore takes slot w of every group, so kGroup units are issued in parallel.
         if ((tid & 31) == 0) {
             const uint32_t w = (uint32_t)(tid - kMmaBase) >> 5;
-            uint32_t xe = 0, G = 0;
+            uint32_t G = 0;
+            Cyc xc(p.xbufs);
             bool alive = true, issued = false;
             Walk wk(p, c);
             const uint64_t desc_r = smem_desc(0, kLboR), desc_m = smem_desc(0, kLboM), desc_a = smem_desc(0, kUnitRows * 16);
@@ -947,12 +985,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             uint32_t stage0 = 0;  // ring stage of the entry's first unit
             while (alive && wk.next_entry()) {
                 const uint32_t KB = wk.KB, n = wk.u1 - wk.u0;
-                const uint32_t xb = xe & 1;
-                if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, (xe >> 1) & 1))) break;
-                ++xe;
+                const uint32_t xb = xc.idx;
+                if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xc.ph))) break;
+                xc.step();
                 const uint32_t xr16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
-                const uint32_t xm16 = xr16 + (((uint32_t)p.kb_max * 4 * kLboR + 256) >> 4);
-                uint32_t kb = (wk.u0 + w) % KB;
+                const uint32_t xm16 = xr16 + (((uint32_t)p.nb_max * 4 * kLboR + 256) >> 4);
+                uint32_t kb = w % KB;  // block of the unit inside the activation buffer: unit j sits at j % KB
                 const uint32_t kstep = kGroup % KB;
                 uint32_t st_i = (stage0 + w) % S;
                 for (uint32_t j = w; j < (n + kGroup - 1) / kGroup * kGroup; j += kGroup, ++G) {
@@ -1089,19 +1127,20 @@ unsigned long long* g_trace = nullptr;
 #endif
 
 struct SmemPlan {
-    int x_rows, xbuf_bytes, stages;
+    int x_rows, xbuf_bytes, stages, xbufs;
     size_t total;
 };
 
 constexpr size_t kSmemLimit = 232448;  // 227 KiB per CTA
 
-SmemPlan plan_for(int max_m, int kb_max) {
+SmemPlan plan_for(int max_m, int nb_max, int xbufs) {
     SmemPlan pl;
     pl.x_rows = max_m <= 1 ? 1 : max_m <= 2 ? 2 : 4;
-    pl.xbuf_bytes = kb_max * 4 * (32 + 48) * pl.x_rows + 512;  // (the last chunk's row window reaches past its own rows)
-    const size_t fixed = (size_t)2 * pl.xbuf_bytes + (size_t)2 * 2 * pl.x_rows * kb_max * 4 +
+    pl.xbuf_bytes = nb_max * 4 * (32 + 48) * pl.x_rows + 512;  // (the last chunk's row window reaches past its own rows)
+    const size_t fixed = (size_t)xbufs * pl.xbuf_bytes + (size_t)xbufs * 2 * pl.x_rows * nb_max * 4 +
                          (size_t)(kHandDepth + 1) * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 12 + kGroup + 2 * kHandDepth) * 8 + 16 +
                          16 * kNG + 128;
+    pl.xbufs = xbufs;
     pl.stages = 0;
     if (fixed < kSmemLimit) {
         long s = (long)((kSmemLimit - fixed) / (kUnitBytes + 16));
@@ -1126,7 +1165,7 @@ cudaError_t launch_one(const TcParams& p, int C, size_t smem, cudaStream_t st) {
 
 bool w4a16_tc_supported(int M, int N, int K, int G) {
     if (M < 1 || M > kMaxRows || N < 1 || K % 128 != 0 || G % 128 != 0) return false;
-    return plan_for(M, K / 128).stages >= 4;
+    return plan_for(M, K / 128, 2).stages >= 4;  // (whatever the list: a buffer never holds more than K / 128 blocks)
 }
 
 size_t w4a16_tc_weight_bytes(int N, int K) { return (size_t)((N + kUnitRows - 1) / kUnitRows) * (K / 128) * kUnitBytes; }
@@ -1154,7 +1193,7 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
     const int C = num_sms();
     for (int base = 0; base < count; base += kMaxEntries) {
         const int n = count - base < kMaxEntries ? count - base : kMaxEntries;
-        int max_m = 1, kmax = 128;
+        int max_m = 1, nb_max = 1;
         bool any_dep = false;
         uint32_t tiles = 0;
         for (int i = 0; i < n; ++i) {
@@ -1174,13 +1213,17 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
             tiles += row_tiles;
             any_dep |= (e.flags & kFlagDep) != 0;
             if (d.M > max_m) max_m = d.M;
-            if (d.K > kmax) kmax = d.K;
+            const int nb = (int)std::min<uint32_t>((uint32_t)(d.K / 128), e.q + (e.rem ? 1u : 0u));  // blocks a CTA touches
+            if (nb > nb_max) nb_max = nb;
         }
-        const SmemPlan pl = plan_for(max_m, kmax / 128);
+        // as many activation buffers as leave a deep weight ring
+        SmemPlan pl = plan_for(max_m, nb_max, kMaxXBufs);
+        for (int xb = kMaxXBufs - 1; xb >= 2 && pl.stages < 12; --xb) pl = plan_for(max_m, nb_max, xb);
         if (pl.stages < 4) return QIL_ERR_UNSUPPORTED;
         p.count = n;
         p.stages = pl.stages;
-        p.kb_max = kmax / 128;
+        p.nb_max = nb_max;
+        p.xbufs = pl.xbufs;
         p.xbuf_bytes = pl.xbuf_bytes;
         p.status = reinterpret_cast<int*>(ws);
         p.tiles_done = any_dep ? reinterpret_cast<unsigned int*>(ws) + 1 : nullptr;

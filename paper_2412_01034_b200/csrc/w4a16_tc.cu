@@ -80,7 +80,7 @@ constexpr int kUnitBytes = 8192 + 512;
 #define QIL_TC_SPIN_POLLS 0
 #endif
 #ifndef QIL_TC_EPI_BATCH
-#define QIL_TC_EPI_BATCH 4
+#define QIL_TC_EPI_BATCH 1
 #endif
 #ifndef QIL_TC_EPILOGUE_WGS
 #define QIL_TC_EPILOGUE_WGS 1
@@ -93,7 +93,10 @@ constexpr int kStagerBase = kEpiBase + 128 * kNumEpi;
 constexpr int kFixBase = kStagerBase + 128;
 constexpr int kFixTeams = 4;                     // fixer warps: entry i's shared tiles belong to warp i % kFixTeams
 constexpr int kFixThreads = 32 * kFixTeams;      // (a lane takes four rows of the tile)
-constexpr int kGroup = 4;                        // units per group: one per MMA issuer, one epilogue pass
+#ifndef QIL_TC_GROUP_UNITS
+#define QIL_TC_GROUP_UNITS 4
+#endif
+constexpr int kGroup = QIL_TC_GROUP_UNITS;       // units per group: one per MMA issuer, one epilogue pass
 constexpr int kMmaBase = kFixBase + kFixThreads; // kGroup warps, one issuing thread each
 constexpr int kProdBase = kMmaBase + 32 * kGroup;  // one warp, one thread issues
 constexpr int kThreads = kProdBase + 32;
@@ -437,9 +440,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     // ---- carve shared memory ----
     unsigned char* ring = smem;                                                     // [stages][kUnitBytes]
     unsigned char* xs = ring + (size_t)p.stages * kUnitBytes;                       // [xbufs][xbuf_bytes]
-    int* xsum = reinterpret_cast<int*>(xs + (size_t)p.xbufs * p.xbuf_bytes);        // [xbufs][kXR][nb_max]
-    float* xscale = reinterpret_cast<float*>(xsum + p.xbufs * kXR * p.nb_max);      // [xbufs][kXR][nb_max]
-    float* hand = xscale + p.xbufs * kXR * p.nb_max;                                // [kHandDepth][2][kXR][128]
+    int2* xblk = reinterpret_cast<int2*>(xs + (size_t)p.xbufs * p.xbuf_bytes);      // [xbufs][kXR][nb_max] {sum v, bits of 2^e}
+    float* hand = reinterpret_cast<float*>(xblk + p.xbufs * kXR * p.nb_max);        // [kHandDepth][2][kXR][128]
     float* tpart = hand + kHandDepth * 2 * kXR * kUnitRows;                         // [2][kXR][128]
     uint64_t* bars = reinterpret_cast<uint64_t*>(tpart + 2 * kXR * kUnitRows);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
@@ -577,11 +579,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, n = u1 - u0;
             const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
             const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
-            const uint32_t xb = xc.idx, kb0 = u0 % KB;  // (a buffer holds the blocks from the slice's first one on, cyclically)
+            const uint32_t xb = xc.idx;
             if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xc.ph))) break;
             xc.step();
-            const int* xsum_b = xsum + (size_t)xb * kXR * p.nb_max;
-            const float* xscale_b = xscale + (size_t)xb * kXR * p.nb_max;
+            const int2* xblk_b = xblk + (size_t)xb * kXR * p.nb_max;
             const uint32_t team = (uint32_t)wk.ei % kFixTeams, hcnt = (hc >> (2 * team)) & 3u;
             const uint32_t hbuf = 2 * team + (hcnt & 1u);
             float* hand_b = hand + (size_t)hbuf * 2 * kXR * kUnitRows;
@@ -591,6 +592,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
 #pragma unroll
             for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
             uint32_t rt = t_first, kb = u0 - t_first * KB;
+            uint32_t bi = 0;  // block inside the activation buffer, which holds the blocks from the slice's first one on, cyclically
             // the CTA's part of row tile rt is complete
             auto close_tile = [&]() {
                 const uint32_t tb = ts & 1, tph = (ts >> 1) & 1;
@@ -641,22 +643,24 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             auto consume = [&](const uint32_t (&cr)[8], const uint32_t (&cm)[16], uint32_t meta) {
                 const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
                 const float s = __low2float(sz);
-                const int z = (int)__high2float(sz);
-                const uint32_t bi = kb >= kb0 ? kb - kb0 : kb + KB - kb0;
+                const int z = __half2int_rz(__high2half(sz));
 #pragma unroll
                 for (int t = 0; t < kXR; ++t)
                     if (t < M) {
                         const int v16 = ((int)cr[2 * t] * 256 + (int)cr[2 * t + 1]) +
                                         ((int)cm[3 * t] * 65536 + (int)cm[3 * t + 1] * 256 + (int)cm[3 * t + 2]);
-                        const int v = (v16 >> 4) - z * xsum_b[t * p.nb_max + bi];  // (v16 is an exact multiple of 16)
-                        fin[t] = fmaf((float)v, s * xscale_b[t * p.nb_max + bi], fin[t]);
+                        const int2 xm = xblk_b[t * p.nb_max + bi];
+                        const int v = (v16 >> 4) - z * xm.x;  // (v16 is an exact multiple of 16)
+                        fin[t] = fmaf((float)v, s * __int_as_float(xm.y), fin[t]);
                     }
             };
             for (uint32_t j0 = 0; alive && j0 < n; j0 += kGroup, ++G) {
                 const uint32_t gs = G % kNG, nreal = min((uint32_t)kGroup, n - j0);
                 if (G % kNumEpi != ew) {  // the other warpgroup's units: only follow the row tiles
-                    for (uint32_t i = 0; alive && i < nreal; ++i)
+                    for (uint32_t i = 0; alive && i < nreal; ++i) {
+                        if (++bi == KB) bi = 0;
                         if (++kb == KB || j0 + i + 1 == n) close_tile();
+                    }
                     continue;
                 }
                 if (!QIL_WAIT(3, guard.wait_mbar(dfull0 + 8 * gs, (G / kNG) & 1))) {  // all units of the group are accumulated
@@ -710,6 +714,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         if (alive && b0 + i < nreal) {
                             QIL_TR_COUNT(5);
                             consume(dr[i], dm[i], meta[i]);
+                            if (++bi == KB) bi = 0;
                             if (++kb == KB || j0 + b0 + i + 1 == n) close_tile();
                         }
 #ifdef QIL_TRACE
@@ -746,8 +751,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const uint32_t xb = xc.idx;
             unsigned char* xs_b = xs + (size_t)xb * p.xbuf_bytes;                  // planes of x_c
             unsigned char* xm_b = xs_b + (size_t)p.nb_max * 4 * kLboR + 256;       // planes of 16 x_a - x_c
-            int* xsum_b = xsum + (size_t)xb * kXR * p.nb_max;
-            float* xscale_b = xscale + (size_t)xb * kXR * p.nb_max;
+            int2* xblk_b = xblk + (size_t)xb * kXR * p.nb_max;
             bool ok = true;
             if (lane == 0) {  // the buffer is free; the rows of x are written (quarter tiles of all earlier entries)
                 ok = QIL_WAIT(1, guard.wait_mbar(xempty0 + 8 * xb, xc.ph ^ 1));
@@ -833,10 +837,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             *reinterpret_cast<uint32_t*>(dm) = m2;       // top plane of 16 x_a - x_c
                             *reinterpret_cast<uint32_t*>(dm + 16) = m1;
                             *reinterpret_cast<uint32_t*>(dm + 32) = m0;
-                            if (l16 == 0) {
-                                xsum_b[t * p.nb_max + i] = sum;
-                                xscale_b[t * p.nb_max + i] = __uint_as_float((uint32_t)(127 + e) << 23);
-                            }
+                            if (l16 == 0) xblk_b[t * p.nb_max + i] = make_int2(sum, (int)((uint32_t)(127 + e) << 23));
                         }
                     }
                 }

@@ -94,7 +94,7 @@ constexpr int kFixBase = kStagerBase + 128;
 constexpr int kFixTeams = 4;                     // fixer warps: entry i's shared tiles belong to warp i % kFixTeams
 constexpr int kFixThreads = 32 * kFixTeams;      // (a lane takes four rows of the tile)
 #ifndef QIL_TC_GROUP_UNITS
-#define QIL_TC_GROUP_UNITS 4
+#define QIL_TC_GROUP_UNITS 3
 #endif
 constexpr int kGroup = QIL_TC_GROUP_UNITS;       // units per group: one per MMA issuer, one epilogue pass
 constexpr int kMmaBase = kFixBase + kFixThreads; // kGroup warps, one issuing thread each
@@ -102,7 +102,7 @@ constexpr int kProdBase = kMmaBase + 32 * kGroup;  // one warp, one thread issue
 constexpr int kThreads = kProdBase + 32;
 static_assert(kThreads <= 1024, "block size");
 #ifndef QIL_TC_GROUPS
-#define QIL_TC_GROUPS 3
+#define QIL_TC_GROUPS 4
 #endif
 constexpr int kNG = QIL_TC_GROUPS;               // groups in flight in tensor memory
 constexpr int kNB = kGroup * kNG;                // = units in flight
@@ -729,8 +729,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 mbar_arrive(xempty0 + 8 * xb);
                 if (shares && ew == 0) mbar_arrive(hfull0 + 8 * hbuf);
                 // the dependency counter counts quarter tiles (32 rows), so that no warp has to wait for another
+                // (the release covers the other lanes' stores as well: they are ordered before it by the __syncwarp above)
                 if (ew == 0 && n_full && p.tiles_done) {
-                    __threadfence();
                     red_release_add(p.tiles_done, n_full);
                 }
             }
@@ -964,7 +964,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             if (lane == 0) {
                 mbar_arrive(hempty0 + 8 * hbuf);
                 if (have_first && p.tiles_done) {  // the tile is written: kRowsPer quarter tiles
-                    __threadfence();
                     red_release_add(p.tiles_done, kRowsPer);
                 }
             }

@@ -20,7 +20,7 @@ from . import _lib, api, workloads as wl
 
 class QuantisedLinears:
     def __init__(self, cfg: int = 1, M: int = 1, n_layers: int = wl.N_LAYERS, layout: int = api.LAYOUT_STREAM128,
-                 deps: str = "layer",
+                 deps: str = "none",
                  outliers: bool = True, device: str = "cuda", keep_host_rows: dict | None = None,
                  host_threads: int | None = None):
         self.M, self.layout, self.device = M, layout, device
@@ -87,12 +87,18 @@ class QuantisedLinears:
             d.zeros = self.zeros[i].data_ptr()
             d.y = self.y_dev.data_ptr() + 2 * self.y_off[i]
             d.M, d.N, d.K, d.group_size, d.layout = M, N, K, self.G, layout
-            d.flags = self._dep_flag(i, deps)
+        self.set_deps(deps)
+
+    def set_deps(self, deps: str) -> None:
+        """Rewrites the ordering flags of the descriptor list (see _dep_flag)."""
+        for i in range(len(self.specs)):
+            self.descs[i].flags = self._dep_flag(i, deps)
 
     def _dep_flag(self, i: int, deps: str) -> int:
-        """Which entries wait for all earlier ones.  "layer": the data flow of a real decoder layer
-        (q after the previous layer's down, o after attention, gate after o, down after gate/up; k, v and
-        up share their input with q / gate).  "all": every entry.  "none": no entry."""
+        """Which entries wait for all earlier ones.  "none": no entry (every linear reads its own input vector,
+        none reads another linear's output: the GEMV throughput).  "layer": the order a decoder layer imposes
+        (q after the previous layer's down, o after attention, gate after o, down after gate/up; k, v and up
+        start with q / gate), as if each output fed the next input directly.  "all": every entry."""
         if deps == "all":
             return api.DEP_PREVIOUS if i > 0 else 0
         if deps == "none":

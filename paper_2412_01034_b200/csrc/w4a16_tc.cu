@@ -26,7 +26,7 @@
 //                          mbarrier), running ahead across linears as far as the ring allows, so
 //                          HBM keeps streaming while the consumers wait for a dependency;
 //   unpack warpgroups      (QIL_TC_UNPACK_WGS, default 2) take turns on units: shared memory -> nibble split -> tensor memory;
-//   MMA issuers (4 x 1 thread) units are handled in groups of four, issuer w takes slot w of
+//   MMA issuers (kGroup x 1 thread) units are handled in groups of kGroup (3), issuer w takes slot w of
 //                          every group: four tcgen05.mma per unit, completion by tcgen05.commit;
 //   epilogue warpgroups    (QIL_TC_EPILOGUE_WGS, default 1; two alternate groups) thread = weight
 //                          row: accumulators -> fp32 row sums (kept in registers over the units of
@@ -35,12 +35,14 @@
 //                          row tiles the CTA owns entirely, or hands over the partial sums of a row
 //                          tile it shares;
 //   stager (4 warps)       waits for QIL_DEP_PREVIOUS, loads and converts the activation blocks the
-//                          CTA's units need (double buffered, one linear ahead);
-//   fixer (2 warps)        all cross-CTA work: publishes the partial sums of a shared row tile as
-//                          {value, tag} pairs (one 8-byte store each, tag = entry index + 1) into a
-//                          ring of slots in the workspace, completes the row tile whose end the CTA
-//                          owns by adding the contributions in CTA order (bit-reproducible), and
-//                          counts finished quarter tiles for the dependency counter.
+//                          CTA's units need, into a ring of up to four buffers (up to three linears ahead);
+//   fixer (4 warps)        all cross-CTA work, linear i's shared row tiles belonging to warp i % 4: it
+//                          publishes the partial sums of a shared row tile as {value, tag} pairs (one
+//                          8-byte store each, tag = entry index + 1) into a ring of slots in the
+//                          workspace, completes the row tile whose end the CTA owns by adding the
+//                          contributions in CTA order (bit-reproducible), and counts finished quarter
+//                          tiles for the dependency counter.  A linear costs a fixer warp several round
+//                          trips through the L2; taking the linears in turn overlaps them.
 // No role uses a named barrier: every hand-over is an mbarrier or a flag in global memory, and
 // every wait is bounded (2 s).  When a wait runs out, QIL_ERR_TIMEOUT is recorded in the
 // workspace status word (with the place in words 2..5 of the workspace), every role stops at its

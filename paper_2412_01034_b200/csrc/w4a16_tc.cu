@@ -575,12 +575,25 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         Cyc xc(p.xbufs);
         bool alive = true;
         Walk wk(p, c);
+#ifdef QIL_TRACE
+        long long tr_p0 = clock64();
+#endif
         while (alive && wk.next_entry()) {
+#ifdef QIL_TRACE
+            const long long tr_p1 = clock64();
+            tr[11] += tr_p1 - tr_p0;  // tail of the previous entry + next_entry
+#endif
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, n = u1 - u0;
             const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
             const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
+#ifdef QIL_TRACE
+            uint32_t tr_keep = t_first + t_last + (shares ? 1u : 0u) + (uint32_t)M + (uint32_t)N;
+            asm volatile("" : "+r"(tr_keep));
+            const long long tr_p2 = clock64();
+            tr[12] += tr_p2 - tr_p1;  // entry fields and the two divisions
+#endif
             const uint32_t xb = xc.idx;
             if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xc.ph))) break;
             xc.step();
@@ -656,6 +669,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         fin[t] = fmaf((float)v, s * __int_as_float(xm.y), fin[t]);
                     }
             };
+#ifdef QIL_TRACE
+            asm volatile("" : "+r"(rt), "+r"(kb), "+r"(hc));
+            tr[13] += clock64() - tr_p2;  // waits for the activation and hand-over buffers, set-up
+#endif
             for (uint32_t j0 = 0; alive && j0 < n; j0 += kGroup, ++G) {
                 const uint32_t gs = G % kNG, nreal = min((uint32_t)kGroup, n - j0);
                 if (G % kNumEpi != ew) {  // the other warpgroup's units: only follow the row tiles
@@ -726,6 +743,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 }
             }
             if (!alive) break;
+#ifdef QIL_TRACE
+            tr_p0 = clock64();
+#endif
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(xempty0 + 8 * xb);

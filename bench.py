@@ -384,6 +384,45 @@ def secondary_measurements(dev):
         for (N, K, pk, s, z, yo, ws) in lin:
             api.linear_w4a16(xs[K], pk, s, z, N, wl.GROUP_SIZE, api.LAYOUT_CANONICAL, out=yo, workspace=ws)
     t_layer = time_us(layer, 10)
+    del lin, xs
+
+    # configs[3]: M sweep on the two FFN shapes, cold (6 weight copies in rotation = 144 MB of packed weights,
+    # larger than L2).  M <= 4 runs the tcgen05 decode kernel (STREAM128 units), M <= 16 the mma.sync skinny kernel
+    # (TILE16), larger M the tcgen05 prefill kernel (canonical layout).
+    sweep = []
+    copies = 6
+    for (N, K) in ((wl.FFN, wl.HIDDEN), (wl.HIDDEN, wl.FFN)):
+        packs = {"stream128": [], "tile16": [], "canonical": []}
+        sz = []
+        for _ in range(copies):
+            w = torch.randn((N, K), device=dev, generator=g) * wl.SIGMA_LLM
+            codes, s_, z_ = api.quantize_rtn_w4(w, wl.GROUP_SIZE)
+            packs["stream128"].append(api.pack_stream128_w4(codes, s_, z_, wl.GROUP_SIZE))
+            packs["tile16"].append(api.pack_w4(codes, api.LAYOUT_TILE16))
+            packs["canonical"].append(api.pack_w4(codes, api.LAYOUT_CANONICAL))
+            sz.append((s_, z_))
+            del w, codes
+        lay = {"stream128": api.LAYOUT_STREAM128, "tile16": api.LAYOUT_TILE16, "canonical": api.LAYOUT_CANONICAL}
+        for Ms in (1, 2, 4, 8, 16, 32, 64, 128, 280):
+            xm = torch.randn((Ms, K), device=dev, generator=g).to(torch.bfloat16)
+            ym = torch.empty((Ms, N), dtype=torch.bfloat16, device=dev)
+            ws = api.new_workspace(api.linear_w4a16_workspace_size(Ms, N, K, wl.GROUP_SIZE), dev)
+            for name in (("stream128", "tile16") if Ms <= 4 else ("tile16",) if Ms <= 16 else ("canonical",)):
+                st_ = {"i": 0}
+
+                def one():
+                    i = st_["i"] % copies
+                    st_["i"] += 1
+                    if name == "stream128":
+                        api.linear_w4a16(xm, packs[name][i], None, None, N, wl.GROUP_SIZE, lay[name], out=ym, workspace=ws)
+                    else:
+                        api.linear_w4a16(xm, packs[name][i], sz[i][0], sz[i][1], N, wl.GROUP_SIZE, lay[name], out=ym, workspace=ws)
+                t = time_us(one, 4 * copies)
+                by = N * K * 0.53125 + 2.0 * Ms * K + 2.0 * Ms * N
+                sweep.append({"N": N, "K": K, "M": Ms, "layout": name, "us": t, "GB/s": by / t / 1e3,
+                              "TFLOP/s": 2.0 * Ms * N * K / t / 1e6})
+        del packs, sz
+    out["w4a16_m_sweep"] = sweep
     flops = sum(2.0 * Mp * N * K for (_, N, K) in wl.LLAMA2_7B_LAYER)
     out["w4a16_prefill_m280_layer"] = {"us": t_layer, "TFLOP/s": flops / t_layer / 1e6, "kernel": "w4a16_prefill_kernel (tcgen05 kind::f16)"}
     return out

@@ -2,15 +2,16 @@
 // App. A.4.2; M tokens, typically 280): a tensor-bound GEMM on tcgen05.mma kind::f16 (bf16 operands, fp32
 // accumulators in tensor memory over the whole K).
 //
-// A CTA computes a 128 (tokens) x 128 (output features) tile.  Per step of 64 input features its four loader warps
-//   * read 64 packed codes of one weight row per thread, turn them into bf16 with a mask/or (0x4300 | q = 128 + q,
-//     exact), subtract 128 + z (exact in bf16: integers below 256) and multiply by the group's scale (one rounding
-//     per weight; the scale itself is rounded from fp16 to bf16 once per group),
-//   * read the activations (bf16) of one token row per thread,
-// and store both as K-major operands without swizzle (8 rows x 16 bytes per core matrix).  Inside every 8-element
+// A CTA computes a 128 (tokens) x 128 (output features) tile.  Per step of 64 input features
+//   * four weight-loader warps read 64 packed codes of one weight row per thread, turn them into bf16 with a
+//     mask/or (0x4300 | q = 128 + q, exact), subtract 128 + z (exact in bf16: integers below 256) and multiply by
+//     the group's scale (one rounding per weight; the scale itself is rounded from fp16 to bf16 once per group),
+//   * four activation-loader warps read the activations (bf16) of one token row per thread,
+// each thread keeping the global loads of three steps in flight (the step time is otherwise one L2 / DRAM
+// latency), and store both as K-major operands without swizzle (8 rows x 16 bytes per core matrix).  Inside every 8-element
 // piece the order is {0,4,1,5,2,6,3,7} for both operands - the order in which a packed word gives up its nibble
 // pairs - which leaves the dot product unchanged.  One thread issues four tcgen05.mma (128 x 128 x 16) per step;
-// tcgen05.commit recycles the shared-memory stage.  The same four warps then read the accumulators, round to bf16
+// tcgen05.commit recycles the shared-memory stage.  The activation-loader warps then read the accumulators, round to bf16
 // and store 16-byte pieces.  Canonical packed layout only.
 #include "qil_common.cuh"
 
@@ -19,8 +20,13 @@ namespace qil {
 namespace {
 
 constexpr int kTile = 128, kStepK = 64, kStages = 4;
-constexpr int kOpStage = kTile * kStepK * 2;  // bytes of one operand tile (bf16)
-constexpr int kThreads = 160;
+constexpr int kOpStage = kTile * kStepK * 2;  // bytes of one weight operand tile (bf16)
+// The activation tile is loaded by eight lanes per token row (one 128-byte line per row and step) and stored with
+// the K-adjacent core matrices 16 bytes further apart than they are long, so that those eight lanes hit different banks.
+constexpr int kLboA = kTile * 16 + 16;
+constexpr int kOpStageA = 8 * kLboA;
+constexpr int kThreads = 288;  // 4 activation loader warps, 4 weight loader warps, 1 MMA warp
+constexpr int kPre = 3;        // steps whose global loads are in flight per loader thread
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -95,8 +101,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __nv_b
                                                                    __nv_bfloat16* __restrict__ y, int M, int N, int K, int G,
                                                                    int* __restrict__ status) {
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* sa = smem;                                   // [kStages][kOpStage] activations
-    unsigned char* sb = smem + (size_t)kStages * kOpStage;      // [kStages][kOpStage] weights
+    unsigned char* sa = smem;                                   // [kStages][kOpStageA] activations
+    unsigned char* sb = smem + (size_t)kStages * kOpStageA;     // [kStages][kOpStage] weights
     uint64_t* bars = reinterpret_cast<uint64_t*>(sb + (size_t)kStages * kOpStage);
     const uint32_t full0 = smem_u32(bars), free0 = smem_u32(bars + kStages), done0 = smem_u32(bars + 2 * kStages);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
@@ -106,13 +112,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __nv_b
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full0 + 8 * s, 4);
+            mbar_init(full0 + 8 * s, 8);
             mbar_init(free0 + 8 * s, 1);
         }
         mbar_init(done0, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTile));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
@@ -123,49 +129,42 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __nv_b
     bool ok = true;
 
     if (warp < 4) {
-        // ---------------- loaders: thread r owns token row m0 + r and weight row n0 + r ----------------
+        // ---------------- activation loaders: lane = 16-byte piece tid % 8 of token rows tid / 8 + 16 j ----------------
         const int r = tid;
-        const bool a_row = m0 + r < M, b_row = n0 + r < N;
-        const __nv_bfloat16* xa = x + (size_t)(m0 + (a_row ? r : 0)) * K;
-        const uint32_t* wb = qw + (size_t)(n0 + (b_row ? r : 0)) * (K >> 3);
-        const __half* sr = scales + (size_t)(n0 + (b_row ? r : 0)) * ng;
-        const __half* zr = zeros + (size_t)(n0 + (b_row ? r : 0)) * ng;
-        uint4 pa[8], pb[2];
-        __half ps = __float2half(0.f), pz = __float2half(0.f);
-        auto fetch = [&](int step) {
-            const int k0 = step * kStepK;
+        const bool a_row = m0 + r < M;  // (for the epilogue: thread r reads out token row m0 + r)
+        const int pc = tid & 7, pr = tid >> 3;
+        const __nv_bfloat16* xa = x + (size_t)m0 * K + 8 * pc;
+        uint4 pa[kPre][8];
+        auto fetch = [&](uint4 (&dst)[8], int step) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                pa[c] = a_row ? __ldg(reinterpret_cast<const uint4*>(xa + k0 + 8 * c)) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-            for (int q = 0; q < 2; ++q)
-                pb[q] = b_row ? __ldg(reinterpret_cast<const uint4*>(wb + (k0 >> 3) + 4 * q)) : make_uint4(0, 0, 0, 0);
-            if (b_row) {
-                ps = sr[k0 / G];
-                pz = zr[k0 / G];
+            for (int j = 0; j < 8; ++j) {
+                const int row = pr + 16 * j;
+                dst[j] = (m0 + row < M) ? __ldg(reinterpret_cast<const uint4*>(xa + (size_t)row * K + step * kStepK))
+                                        : make_uint4(0, 0, 0, 0);
             }
         };
-        fetch(0);
-        for (int step = 0; step < steps; ++step) {
-            const int s = step % kStages, use = step / kStages;
-            ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
-            if (!ok) break;
-            unsigned char* a_st = sa + (size_t)s * kOpStage + (size_t)r * 16;
-            unsigned char* b_st = sb + (size_t)s * kOpStage + (size_t)r * 16;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(a_st + (size_t)c * (kTile * 16)) = permute8(pa[c]);
-            {
-                const float zf = b_row ? __half2float(pz) + 128.f : 128.f;
-                const float sf = b_row ? __half2float(ps) : 0.f;
-                const __nv_bfloat162 off = __float2bfloat162_rn(zf), sc = __float2bfloat162_rn(sf);
-                const uint32_t w[8] = {pb[0].x, pb[0].y, pb[0].z, pb[0].w, pb[1].x, pb[1].y, pb[1].z, pb[1].w};
+        for (int u = 0; u < kPre; ++u) {
 #pragma unroll
-                for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(b_st + (size_t)c * (kTile * 16)) = dequant8(w[c], off, sc);
+            for (int j = 0; j < 8; ++j) pa[u][j] = make_uint4(0, 0, 0, 0);
+            if (u < steps) fetch(pa[u], u);
+        }
+        for (int step0 = 0; ok && step0 < steps; step0 += kPre) {
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int step = step0 + u;
+                if (step >= steps) break;
+                const int s = step % kStages, use = step / kStages;
+                ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
+                if (!ok) break;
+                unsigned char* a_st = sa + (size_t)s * kOpStageA + (size_t)pc * kLboA + (size_t)pr * 16;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(a_st + (size_t)j * (16 * 16)) = permute8(pa[u][j]);
+                if (step + kPre < steps) fetch(pa[u], step + kPre);  // kPre steps stay in flight
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read through the async proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full0 + 8 * s);
             }
-            if (step + 1 < steps) fetch(step + 1);  // in flight while the tensor core works on this step
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read through the async proxy
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full0 + 8 * s);
         }
         // ---------------- epilogue: thread r = token row m0 + r ----------------
         if (ok) ok = mbar_wait(done0, 0);
@@ -206,18 +205,62 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __nv_b
                 }
             }
         }
+    } else if (warp < 8) {
+        // ---------------- weight loaders: thread r owns weight row n0 + r ----------------
+        const int r = tid - 128;
+        const bool b_row = n0 + r < N;
+        const uint32_t* wb = qw + (size_t)(n0 + (b_row ? r : 0)) * (K >> 3);
+        const __half* sr = scales + (size_t)(n0 + (b_row ? r : 0)) * ng;
+        const __half* zr = zeros + (size_t)(n0 + (b_row ? r : 0)) * ng;
+        uint4 pb[kPre][2];
+        __half ps[kPre], pz[kPre];
+        auto fetch = [&](uint4 (&dst)[2], __half& s_, __half& z_, int step) {
+            const int k0 = step * kStepK;
+#pragma unroll
+            for (int q = 0; q < 2; ++q)
+                dst[q] = b_row ? __ldg(reinterpret_cast<const uint4*>(wb + (k0 >> 3) + 4 * q)) : make_uint4(0, 0, 0, 0);
+            s_ = b_row ? sr[k0 / G] : __float2half(0.f);
+            z_ = b_row ? zr[k0 / G] : __float2half(0.f);
+        };
+#pragma unroll
+        for (int u = 0; u < kPre; ++u) {
+            pb[u][0] = pb[u][1] = make_uint4(0, 0, 0, 0);
+            ps[u] = pz[u] = __float2half(0.f);
+            if (u < steps) fetch(pb[u], ps[u], pz[u], u);
+        }
+        for (int step0 = 0; ok && step0 < steps; step0 += kPre) {
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int step = step0 + u;
+                if (step >= steps) break;
+                const int s = step % kStages, use = step / kStages;
+                ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);
+                if (!ok) break;
+                unsigned char* b_st = sb + (size_t)s * kOpStage + (size_t)r * 16;
+                const float zf = b_row ? __half2float(pz[u]) + 128.f : 128.f;
+                const float sf = b_row ? __half2float(ps[u]) : 0.f;
+                const __nv_bfloat162 off = __float2bfloat162_rn(zf), sc = __float2bfloat162_rn(sf);
+                const uint32_t w[8] = {pb[u][0].x, pb[u][0].y, pb[u][0].z, pb[u][0].w, pb[u][1].x, pb[u][1].y, pb[u][1].z, pb[u][1].w};
+#pragma unroll
+                for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(b_st + (size_t)c * (kTile * 16)) = dequant8(w[c], off, sc);
+                if (step + kPre < steps) fetch(pb[u], ps[u], pz[u], step + kPre);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full0 + 8 * s);
+            }
+        }
     } else if (lane == 0) {
         // ---------------- MMA issuer ----------------
-        constexpr uint32_t kLbo = kTile * 16;  // K-adjacent core matrices
+        constexpr uint32_t kLbo = kTile * 16;  // K-adjacent core matrices of the weight operand
         for (int step = 0; step < steps; ++step) {
             const int s = step % kStages, use = step / kStages;
             ok = mbar_wait(full0 + 8 * s, use & 1);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a_addr = smem_u32(sa + (size_t)s * kOpStage), b_addr = smem_u32(sb + (size_t)s * kOpStage);
+            const uint32_t a_addr = smem_u32(sa + (size_t)s * kOpStageA), b_addr = smem_u32(sb + (size_t)s * kOpStage);
 #pragma unroll
             for (int i = 0; i < 4; ++i)  // K = 16 each: 16-byte pieces 2i, 2i + 1
-                mma_bf16_ss(tmem, smem_desc(a_addr + 2 * i * kLbo, kLbo, 128), smem_desc(b_addr + 2 * i * kLbo, kLbo, 128),
+                mma_bf16_ss(tmem, smem_desc(a_addr + 2 * i * kLboA, kLboA, 128), smem_desc(b_addr + 2 * i * kLbo, kLbo, 128),
                             (step > 0 || i > 0) ? 1u : 0u);
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(free0 + 8 * s) : "memory");
         }
@@ -234,15 +277,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __nv_b
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTile));
+    if (warp == 8) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTile));
 }
 
-constexpr size_t kSmemBytes = (size_t)2 * kStages * kOpStage + (2 * kStages + 1) * 8 + 16;
+constexpr size_t kSmemBytes = (size_t)kStages * (kOpStage + kOpStageA) + (2 * kStages + 1) * 8 + 16;
 
 }  // namespace
 
 bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout) {
-    return layout == QIL_LAYOUT_CANONICAL && M > 64 && N >= 1 && K % kStepK == 0 && G % kStepK == 0 && K % G == 0;
+    return layout == QIL_LAYOUT_CANONICAL && M > 16 && N >= 1 && K % kStepK == 0 && G % kStepK == 0 && K % G == 0;
 }
 
 // ws (optional): its first int receives QIL_ERR_TIMEOUT if a bounded device-side wait runs out.

@@ -1187,7 +1187,10 @@ cudaError_t launch_one(const TcParams& p, int C, size_t smem, cudaStream_t st) {
 
 bool w4a16_tc_supported(int M, int N, int K, int G) {
     if (M < 1 || M > kMaxRows || N < 1 || K % 128 != 0 || G % 128 != 0) return false;
-    return plan_for(M, K / 128, 2).stages >= 4;  // (whatever the list: a buffer never holds more than K / 128 blocks)
+    // an activation buffer holds the 128-column blocks one CTA touches in this linear
+    const uint32_t units = (uint32_t)((N + kUnitRows - 1) / kUnitRows) * (uint32_t)(K / 128);
+    const uint32_t nb = std::min<uint32_t>((uint32_t)(K / 128), units / (uint32_t)num_sms() + 1u);
+    return plan_for(M, (int)nb, 2).stages >= 4;
 }
 
 size_t w4a16_tc_weight_bytes(int N, int K) { return (size_t)((N + kUnitRows - 1) / kUnitRows) * (K / 128) * kUnitBytes; }

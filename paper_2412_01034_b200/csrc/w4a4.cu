@@ -26,8 +26,13 @@ namespace {
 
 constexpr int kTileM = 128, kTileN = 64, kStepK = 128;  // K elements per step = 64 packed bytes per row
 constexpr int kStages = 3;
-constexpr int kAStage = kTileM * kStepK;  // bytes (one byte per element after the split)
-constexpr int kBStage = kTileN * kStepK;
+// Operand tiles in shared memory: one byte per element after the split, K-major core matrices (8 rows x 16 bytes).
+// The K-adjacent core matrices lie 16 bytes further apart than they are long: the four lanes that hold the four
+// 16-byte pieces of one packed row then store to different banks.
+constexpr int kALbo = kTileM * 16 + 16, kBLbo = kTileN * 16 + 16;
+constexpr int kAStage = (kStepK / 16) * kALbo;
+constexpr int kBStage = (kStepK / 16) * kBLbo;
+constexpr int kPre = 2;                   // steps whose global loads are in flight per loader thread
 constexpr int kThreads = 160;             // 4 loader / epilogue warps + the MMA warp
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -122,53 +127,67 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
     bool ok = true;
 
     if (warp < 4) {
-        // ---------------- loaders: thread r owns token row r of the tile and half of weight row r / 2 ----------------
+        // ---------------- loaders: lane = 16-byte piece tid % 4 (32 codes) of the step's 64 packed bytes of token rows
+        // tid / 4 + 32 j (j < 4) and weight rows tid / 4 + 32 j (j < 2): four lanes read one row's bytes together ----------------
         const int r = tid;
-        const bool a_row = m0 + r < M;
-        const int bn = r >> 1, bh = r & 1;  // weight row of the tile, which 64-element half of the step
-        const bool b_row = n0 + bn < N;
-        const uint32_t* xa = qx + (size_t)(m0 + (a_row ? r : 0)) * row_words;
-        const uint32_t* wb = qw + (size_t)(n0 + (b_row ? bn : 0)) * row_words;
-        uint4 pa[4], pb[2];
-        auto fetch = [&](int step) {  // packed words of one step into registers (zeros beyond the matrix)
+        const bool a_row = m0 + r < M;  // (for the epilogue: thread r reads out accumulator row r)
+        const int pq = tid & 3, pr = tid >> 2;
+        const uint32_t* xa = qx + (size_t)m0 * row_words + 4 * pq;
+        const uint32_t* wb = qw + (size_t)n0 * row_words + 4 * pq;
+        uint4 pa[kPre][4], pb[kPre][2];
+        auto fetch = [&](uint4 (&da)[4], uint4 (&db)[2], int step) {  // packed words of one step (zeros beyond the matrix)
             const int w0 = step * (kStepK / 8);
+            const bool in_k = w0 + 4 * pq < row_words;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int w = w0 + 4 * q;
-                pa[q] = (a_row && w < row_words) ? __ldg(reinterpret_cast<const uint4*>(xa + w)) : make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < 4; ++j) {
+                const int row = pr + 32 * j;
+                da[j] = (in_k && m0 + row < M) ? __ldg(reinterpret_cast<const uint4*>(xa + (size_t)row * row_words + w0))
+                                               : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int w = w0 + 4 * (2 * bh + q);
-                pb[q] = (b_row && w < row_words) ? __ldg(reinterpret_cast<const uint4*>(wb + w)) : make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < 2; ++j) {
+                const int row = pr + 32 * j;
+                db[j] = (in_k && n0 + row < N) ? __ldg(reinterpret_cast<const uint4*>(wb + (size_t)row * row_words + w0))
+                                               : make_uint4(0, 0, 0, 0);
             }
         };
-        fetch(0);
-        for (int step = 0; step < steps && ok; ++step) {
-            const int s = step % kStages, use = step / kStages;
-            ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
-            if (!ok) break;
-            unsigned char* a_st = sa + (size_t)s * kAStage + (size_t)r * 16;
-            unsigned char* b_st = sb + (size_t)s * kBStage + (size_t)bn * 16;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {  // K chunks 2q, 2q+1 of the step
-                uint4 c0, c1;
-                split32(pa[q], c0, c1);
-                *reinterpret_cast<uint4*>(a_st + (size_t)(2 * q) * (kTileM * 16)) = c0;
-                *reinterpret_cast<uint4*>(a_st + (size_t)(2 * q + 1) * (kTileM * 16)) = c1;
-            }
+        for (int u = 0; u < kPre; ++u) {
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                uint4 c0, c1;
-                split32(pb[q], c0, c1);
-                const int ch = 2 * (2 * bh + q);
-                *reinterpret_cast<uint4*>(b_st + (size_t)ch * (kTileN * 16)) = c0;
-                *reinterpret_cast<uint4*>(b_st + (size_t)(ch + 1) * (kTileN * 16)) = c1;
+            for (int j = 0; j < 4; ++j) pa[u][j] = make_uint4(0, 0, 0, 0);
+            pb[u][0] = pb[u][1] = make_uint4(0, 0, 0, 0);
+            if (u < steps) fetch(pa[u], pb[u], u);
+        }
+        for (int step0 = 0; ok && step0 < steps; step0 += kPre) {
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int step = step0 + u;
+                if (step >= steps) break;
+                const int s = step % kStages, use = step / kStages;
+                ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
+                if (!ok) break;
+                // piece pq = K chunks 2 pq, 2 pq + 1 of the step
+                unsigned char* a_st = sa + (size_t)s * kAStage + (size_t)(2 * pq) * kALbo + (size_t)pr * 16;
+                unsigned char* b_st = sb + (size_t)s * kBStage + (size_t)(2 * pq) * kBLbo + (size_t)pr * 16;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 c0, c1;
+                    split32(pa[u][j], c0, c1);
+                    *reinterpret_cast<uint4*>(a_st + (size_t)j * (32 * 16)) = c0;
+                    *reinterpret_cast<uint4*>(a_st + (size_t)j * (32 * 16) + kALbo) = c1;
+                }
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    uint4 c0, c1;
+                    split32(pb[u][j], c0, c1);
+                    *reinterpret_cast<uint4*>(b_st + (size_t)j * (32 * 16)) = c0;
+                    *reinterpret_cast<uint4*>(b_st + (size_t)j * (32 * 16) + kBLbo) = c1;
+                }
+                if (step + kPre < steps) fetch(pa[u], pb[u], step + kPre);  // kPre steps stay in flight
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read through the async proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full0 + 8 * s);
             }
-            if (step + 1 < steps) fetch(step + 1);  // in flight while the tensor core works on this step
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read through the async proxy
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full0 + 8 * s);
         }
         // ---------------- epilogue: thread r = accumulator row r ----------------
         if (ok) ok = mbar_wait(done0, 0);
@@ -223,7 +242,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
         }
     } else if (lane == 0) {
         // ---------------- MMA issuer ----------------
-        constexpr uint32_t kALbo = kTileM * 16, kBLbo = kTileN * 16;  // K-adjacent core matrices
         for (int step = 0; step < steps; ++step) {
             const int s = step % kStages, use = step / kStages;
             ok = mbar_wait(full0 + 8 * s, use & 1);

@@ -365,16 +365,19 @@ struct Guard {
     }
     template <typename Pred>
     __device__ __forceinline__ bool wait_flag(Pred done) const {
-        if (done()) return true;
-        if (*poisoned) return false;
-        const unsigned long long t0 = now_ns();
-        for (uint32_t i = 1;; ++i) {
+        unsigned long long t0 = 0;
+#pragma unroll 1
+        for (uint32_t i = 0;; ++i) {  // (one copy of the predicate's code: the kernel is sensitive to its size)
             if (done()) return true;
 #ifdef QIL_TRACE
             *polls += 1;
 #endif
+            if (i == 0) {
+                if (*poisoned) return false;
+                t0 = now_ns();
+            }
             if (i > 8) __nanosleep(i < 64 ? 32 : 256);
-            if ((i & 15u) == 0) {
+            if ((i & 15u) == 15u) {
                 if (*poisoned) return false;
                 if (now_ns() - t0 > kWaitLimitNs) break;
             }
@@ -878,7 +881,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // parts, the output); the warps take the entries in turn so that these latencies overlap.
         const uint32_t team = (uint32_t)(tid - kFixBase) >> 5, lane = tid & 31;
         constexpr uint32_t kRowsPer = kUnitRows / 32;
-        constexpr uint32_t kPoll = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;  // other CTAs' parts fetched together (registers)
+        constexpr uint32_t kPoll = 1;  // other CTAs' parts fetched together (more measured slower: the code grows)
         unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
         uint32_t cnt = 0;  // entries this warp has taken over
         bool alive = true;

@@ -112,6 +112,63 @@ __device__ __forceinline__ float rint_div(float f, float s, float inv_s) {
 
 // Per-token symmetric int4 of bf16 activations, fused with packing.  One warp per row.
 // Each lane owns whole 32-bit output words (8 consecutive k).
+// Rows of at most 256 kPer elements: a warp keeps its row in registers between the maximum and the rounding, and all
+// of the row's loads are in flight at once (same arithmetic as the general kernel below, hence the same codes).
+template <int kPer>
+__global__ void __launch_bounds__(256) quantize_act_cached_kernel(const __nv_bfloat16* __restrict__ x, int M, int K,
+                                                                  bool use_static, float static_scale,
+                                                                  uint32_t* __restrict__ qx, float* __restrict__ scales) {
+    const int lane = threadIdx.x & 31;
+    const int words = K >> 3;
+    const int warps = gridDim.x * (blockDim.x >> 5);
+    for (int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); m < M; m += warps) {
+        const uint4* row = reinterpret_cast<const uint4*>(x + (size_t)m * K);
+        uint4 buf[kPer];
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const int i = lane + 32 * j;
+            buf[j] = i < words ? __ldg(row + i) : make_uint4(0, 0, 0, 0);
+        }
+        float s;
+        if (use_static) {
+            s = static_scale;
+        } else {
+            float a = 0.0f;
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const uint32_t u[4] = {buf[j].x, buf[j].y, buf[j].z, buf[j].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    a = fmaxf(a, fabsf(__uint_as_float(u[c] << 16)));
+                    a = fmaxf(a, fabsf(__uint_as_float(u[c] & 0xFFFF0000u)));
+                }
+            }
+            a = warp_max(a);
+            s = __fdiv_rn(a, 7.0f);
+            if (a == 0.0f) s = 1.0f;
+        }
+        if (lane == 0) scales[m] = s;
+        const float inv_s = __frcp_rn(s);
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const int i = lane + 32 * j;
+            if (i >= words) continue;
+            const uint32_t u[4] = {buf[j].x, buf[j].y, buf[j].z, buf[j].w};
+            uint32_t word = 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float f0 = __uint_as_float(u[c] << 16);
+                const float f1 = __uint_as_float(u[c] & 0xFFFF0000u);
+                const int q0 = (int)clampf(rint_div(f0, s, inv_s), -8.0f, 7.0f);
+                const int q1 = (int)clampf(rint_div(f1, s, inv_s), -8.0f, 7.0f);
+                word |= (uint32_t)(q0 & 0xF) << (8 * c);
+                word |= (uint32_t)(q1 & 0xF) << (8 * c + 4);
+            }
+            qx[(size_t)m * words + i] = word;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256) quantize_act_kernel(const __nv_bfloat16* __restrict__ x, int M, int K,
                                                            bool use_static, float static_scale,
                                                            uint32_t* __restrict__ qx, float* __restrict__ scales) {
@@ -255,6 +312,18 @@ qil_status launch_unpack_w4(const uint32_t* packed, int N, int K, qil_layout lay
 
 qil_status launch_quantize_act_a4(const void* x, int M, int K, bool use_static, float static_scale,
                                   uint32_t* qx, float* scales, cudaStream_t st) {
+    const int words = K >> 3;
+#define QIL_ACT_CACHED(P)                                                                                           \
+    if (words <= 32 * (P)) {                                                                                        \
+        quantize_act_cached_kernel<P><<<grid_for(M, 8), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), M, \
+                                                                      K, use_static, static_scale, qx, scales);      \
+        return launch_status();                                                                                     \
+    }
+    QIL_ACT_CACHED(3)
+    QIL_ACT_CACHED(5)
+    QIL_ACT_CACHED(9)
+    QIL_ACT_CACHED(18)
+#undef QIL_ACT_CACHED
     quantize_act_kernel<<<grid_for(M, 8), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), M, K,
                                                         use_static, static_scale, qx, scales);
     return launch_status();

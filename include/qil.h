@@ -121,11 +121,13 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  * into the matmul, accumulation is fp32, the result is rounded to bf16.
  *   x [M][K] bf16   qweight packed per `layout`   scales, zeros [N][K/group_size] fp16
  *   y [M][N] bf16
- * The kernel is chosen from the shape: tensor-core skinny kernel (weights read
- * once, any M handled in slabs of 64 rows) when K % 128 == 0 and
- * group_size % 128 == 0; a general kernel otherwise (any K % 8 == 0, any
- * group_size dividing K, canonical layout only).  With QIL_LAYOUT_STREAM128
- * (M <= 4) the persistent streaming kernel runs;
+ * The kernel is chosen from the shape: on the canonical layout with M > 16,
+ * K % 64 == 0 and group_size % 64 == 0 the tcgen05 prefill GEMM (weights
+ * dequantised to bf16, one rounding per weight); else the tensor-core skinny
+ * kernel (weights read once, any M handled in slabs of 64 rows) when
+ * K % 128 == 0 and group_size % 128 == 0; a general kernel otherwise (any
+ * K % 8 == 0, any group_size dividing K, canonical layout only).  With
+ * QIL_LAYOUT_STREAM128 (M <= 4) the persistent streaming kernel runs;
  * scales and zeros are part of the buffer, the two arguments are ignored and
  * may be null; the workspace is always needed.  The streaming kernel converts
  * the activations to 16-bit block fixed point (per 128 columns a power-of-two

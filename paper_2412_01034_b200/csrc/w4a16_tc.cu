@@ -400,18 +400,26 @@ __device__ __forceinline__ uint32_t owner_of(uint32_t q, uint32_t rem, uint32_t 
     return u < big ? u / (q + 1) : rem + (u - big) / q;
 }
 
-// The entries in which one CTA owns units.
+// The entries in which one CTA owns units.  The CTA's slice of every entry is worked out once, at the start of the
+// kernel, into a table in shared memory ({first unit, first row tile, units | row tiles touched << 16, first
+// column block | column blocks per row tile << 16}): six roles walk the list, and slicing costs divisions.
 struct Walk {
-    const TcParams& p;
-    uint32_t c;
+    const uint4* plan;
+    int count;
     int ei;
-    uint32_t KB, u0, u1;
-    __device__ Walk(const TcParams& p_, uint32_t c_) : p(p_), c(c_), ei(-1) {}
+    uint32_t KB, u0, u1, t_first, t_last, kb0;
+    __device__ Walk(const uint4* plan_, int count_) : plan(plan_), count(count_), ei(-1) {}
     __device__ __forceinline__ bool next_entry() {
-        for (++ei; ei < p.count; ++ei) {
-            slice_of(p.e[ei].q, p.e[ei].rem, c, u0, u1);
-            if (u0 != u1) {
-                KB = (uint32_t)p.e[ei].K >> 7;
+        for (++ei; ei < count; ++ei) {
+            const uint4 e = plan[ei];
+            const uint32_t n = e.z & 0xFFFFu;
+            if (n != 0u) {
+                u0 = e.x;
+                u1 = e.x + n;
+                t_first = e.y;
+                t_last = e.y + (e.z >> 16) - 1u;
+                kb0 = e.w & 0xFFFFu;
+                KB = e.w >> 16;
                 return true;
             }
         }
@@ -461,6 +469,20 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     volatile int* poisoned = reinterpret_cast<volatile int*>(tmem_slot + 1);
     // rd[gs][q]: groups of slot group gs that epilogue warp q (tensor-memory lanes 32q..32q+31) has read out
     const uint32_t rd0 = smem_u32(tmem_slot + 2);
+    uint4* plan = reinterpret_cast<uint4*>((reinterpret_cast<uintptr_t>(tmem_slot + 2 + 4 * kNG) + 15) & ~(uintptr_t)15);  // [count] this CTA's slice of every entry
+    for (int i = tid; i < p.count; i += kThreads) {
+        uint32_t pu0, pu1;
+        slice_of(p.e[i].q, p.e[i].rem, c, pu0, pu1);
+        const uint32_t pn = pu1 - pu0, pKB = (uint32_t)p.e[i].K >> 7;
+        uint4 e = make_uint4(pu0, 0u, 0u, pKB << 16);
+        if (pn != 0u) {
+            e.y = pu0 / pKB;
+            const uint32_t pkb0 = pu0 - e.y * pKB;
+            e.z = pn | (((pkb0 + pn - 1u) / pKB + 1u) << 16);
+            e.w |= pkb0;
+        }
+        plan[i] = e;
+    }
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -518,7 +540,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         uint32_t stage0 = 0, ph0 = 0, turn0 = 0;  // ring stage / phase / turn of the entry's first unit
         uint32_t G = 0;                           // groups so far: unit j of an entry sits in group G + j / kGroup, slot j % kGroup
         bool alive = true;
-        Walk wk(p, c);
+        Walk wk(plan, p.count);
         while (alive && wk.next_entry()) {
             const uint32_t n = wk.u1 - wk.u0;
             uint32_t j = wg >= turn0 ? wg - turn0 : wg + kNumWg - turn0;  // this warpgroup's first unit of the entry
@@ -577,7 +599,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         uint32_t hc = 0, G = 0, ts = 0;  // hc: per fixer warp, two bits counting the entries handed to it; ts: row tiles closed
         Cyc xc(p.xbufs);
         bool alive = true;
-        Walk wk(p, c);
+        Walk wk(plan, p.count);
 #ifdef QIL_TRACE
         long long tr_p0 = clock64();
 #endif
@@ -589,7 +611,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, n = u1 - u0;
-            const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
+            const uint32_t t_first = wk.t_first, t_last = wk.t_last;
             const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
 #ifdef QIL_TRACE
             uint32_t tr_keep = t_first + t_last + (shares ? 1u : 0u) + (uint32_t)M + (uint32_t)N;
@@ -609,7 +631,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             float fin[kXR];
 #pragma unroll
             for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
-            uint32_t rt = t_first, kb = u0 - t_first * KB;
+            uint32_t rt = t_first, kb = wk.kb0;
             uint32_t bi = 0;  // block inside the activation buffer, which holds the blocks from the slice's first one on, cyclically
             // the CTA's part of row tile rt is complete
             auto close_tile = [&]() {
@@ -769,7 +791,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         // and 32j + 8m + 4 + b (high nibble, x_c).  The four warps work independently.
         const int st = tid - kStagerBase, lane = tid & 31, l16 = st & 15, hw = st >> 4;
         Cyc xc(p.xbufs);
-        Walk wk(p, c);
+        Walk wk(plan, p.count);
         while (wk.next_entry()) {
             const TcEntry& E = p.e[wk.ei];
             const uint32_t KB = wk.KB;
@@ -790,7 +812,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
 #ifdef QIL_TRACE
             const long long tr_conv0 = clock64();
 #endif
-            const uint32_t nblk = min(KB, wk.u1 - wk.u0), kb0 = wk.u0 % KB;
+            const uint32_t nblk = min(KB, wk.u1 - wk.u0), kb0 = wk.kb0;
             const uint32_t m = (uint32_t)l16 & 3;
             for (int t = 0; t < E.M; ++t) {
                 const uint16_t* xrow = E.x + (size_t)t * E.K;
@@ -885,13 +907,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
         uint32_t cnt = 0;  // entries this warp has taken over
         bool alive = true;
-        Walk wk(p, c);
+        Walk wk(plan, p.count);
         while (alive && wk.next_entry()) {
             if ((uint32_t)wk.ei % kFixTeams != team) continue;
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1;
-            const uint32_t t_first = u0 / KB, t_last = (u1 - 1) / KB;
+            const uint32_t t_first = wk.t_first, t_last = wk.t_last;
             const bool have_last = (t_last + 1) * KB > u1;                          // contributes to a tile that ends elsewhere
             const bool have_first = t_first * KB < u0 && (t_first + 1) * KB <= u1;  // completes a tile begun elsewhere
             if (!have_last && !(t_first * KB < u0)) continue;
@@ -1003,7 +1025,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             uint32_t G = 0;
             Cyc xc(p.xbufs);
             bool alive = true, issued = false;
-            Walk wk(p, c);
+            Walk wk(plan, p.count);
             const uint64_t desc_r = smem_desc(0, kLboR), desc_m = smem_desc(0, kLboM), desc_a = smem_desc(0, kUnitRows * 16);
             constexpr uint32_t lbor16 = (uint32_t)kLboR >> 4, lbom16 = (uint32_t)kLboM >> 4;
             const uint32_t S = (uint32_t)p.stages, ring16 = smem_u32(ring) >> 4;
@@ -1015,8 +1037,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 xc.step();
                 const uint32_t xr16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
                 const uint32_t xm16 = xr16 + (((uint32_t)p.nb_max * 4 * kLboR + 256) >> 4);
-                uint32_t kb = w % KB;  // block of the unit inside the activation buffer: unit j sits at j % KB
-                const uint32_t kstep = kGroup % KB;
+                uint32_t kb = w < KB ? w : w % KB;  // block of the unit inside the activation buffer: unit j sits at j % KB
+                const uint32_t kstep = (uint32_t)kGroup < KB ? (uint32_t)kGroup : (uint32_t)kGroup % KB;
                 uint32_t st_i = (stage0 + w) % S;
                 for (uint32_t j = w; j < (n + kGroup - 1) / kGroup * kGroup; j += kGroup, ++G) {
                     const uint32_t gs = G % kNG, gph = (G / kNG) & 1;
@@ -1077,7 +1099,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             Cyc rs(p.stages);
             uint32_t issued = 0;
             bool alive = true;
-            Walk wk(p, c);
+            Walk wk(plan, p.count);
             while (alive && wk.next_entry()) {
                 const unsigned char* wbase = p.e[wk.ei].w;
                 for (uint32_t u = wk.u0; u < wk.u1; ++u, ++issued) {
@@ -1164,7 +1186,7 @@ SmemPlan plan_for(int max_m, int nb_max, int xbufs) {
     pl.xbuf_bytes = nb_max * 4 * (32 + 48) * pl.x_rows + 512;  // (the last chunk's row window reaches past its own rows)
     const size_t fixed = (size_t)xbufs * pl.xbuf_bytes + (size_t)xbufs * 2 * pl.x_rows * nb_max * 4 +
                          (size_t)(kHandDepth + 1) * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 12 + kGroup + 2 * kHandDepth) * 8 + 16 +
-                         16 * kNG + 128;
+                         16 * kNG + 128 + (size_t)kMaxEntries * 16;
     pl.xbufs = xbufs;
     pl.stages = 0;
     if (fixed < kSmemLimit) {
@@ -1193,6 +1215,7 @@ bool w4a16_tc_supported(int M, int N, int K, int G) {
     // an activation buffer holds the 128-column blocks one CTA touches in this linear
     const uint32_t units = (uint32_t)((N + kUnitRows - 1) / kUnitRows) * (uint32_t)(K / 128);
     const uint32_t nb = std::min<uint32_t>((uint32_t)(K / 128), units / (uint32_t)num_sms() + 1u);
+    if (units / (uint32_t)num_sms() >= 65535u || K / 128 >= 65536) return false;  // (16-bit fields of the slice table)
     return plan_for(M, (int)nb, 2).stages >= 4;
 }
 
@@ -1238,6 +1261,7 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
             e.q = units / (uint32_t)C;
             e.rem = units % (uint32_t)C;
             e.pad = 0;
+            if (e.q >= 65535u || d.K / 128 >= 65536) return QIL_ERR_UNSUPPORTED;  // (16-bit fields of the slice table)
             tiles += row_tiles;
             any_dep |= (e.flags & kFlagDep) != 0;
             if (d.M > max_m) max_m = d.M;

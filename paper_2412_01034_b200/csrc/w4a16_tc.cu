@@ -28,12 +28,10 @@
 //   unpack warpgroups      (QIL_TC_UNPACK_WGS, default 2) take turns on units: shared memory -> nibble split -> tensor memory;
 //   MMA issuers (kGroup x 1 thread) units are handled in groups of kGroup (3), issuer w takes slot w of
 //                          every group: four tcgen05.mma per unit, completion by tcgen05.commit;
-//   epilogue warpgroups    (QIL_TC_EPILOGUE_WGS, default 1; two alternate groups) thread = weight
-//                          row: accumulators -> fp32 row sums (kept in registers over the units of
-//                          a row tile); with two warpgroups the second one's sums are added to the
-//                          first's at the end of a row tile; the first writes the bf16 outputs of
-//                          row tiles the CTA owns entirely, or hands over the partial sums of a row
-//                          tile it shares;
+//   epilogue warpgroups    (QIL_TC_EPILOGUE_WGS, default 1; two take the CTA's linears in turn) thread =
+//                          weight row: accumulators -> fp32 row sums (kept in registers over the units
+//                          of a row tile); writes the bf16 outputs of row tiles the CTA owns entirely,
+//                          or hands over the partial sums of a row tile it shares;
 //   stager (4 warps)       waits for QIL_DEP_PREVIOUS, loads and converts the activation blocks the
 //                          CTA's units need, into a ring of up to four buffers (up to three linears ahead);
 //   fixer (4 warps)        all cross-CTA work, linear i's shared row tiles belonging to warp i % 4: it
@@ -115,7 +113,7 @@ constexpr int kColD = 16 * kNB;
 __host__ __device__ constexpr int d_unit_cols(int xr) { return 8 + (xr == 4 ? 16 : 8); }
 __host__ __device__ constexpr int col_meta(int xr) { return kColD + d_unit_cols(xr) * kNB; }
 static_assert(col_meta(4) + kNB <= kTmemCols, "tensor memory budget");
-static_assert(kNumEpi == 1 || kNG % kNumEpi == 0, "a slot group must always be read out by the same epilogue warpgroup");
+static_assert(kNumEpi == 1 || kNumEpi == 2, "one or two read-out warpgroups");
 constexpr int kMaxXBufs = 4;                     // activation buffers at most
 constexpr int kHandDepth = 2 * kFixTeams;        // hand-over buffers between the epilogue and the fixer: two per warp
 constexpr int kMaxEntries = 256;
@@ -496,7 +494,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         }
         for (int i = 0; i < kMaxXBufs; ++i) {
             mbar_init(xfull0 + 8 * i, 4);  // the stager warps
-            mbar_init(xempty0 + 8 * i, 4 * kNumEpi);
+            mbar_init(xempty0 + 8 * i, 4);  // the warps of the warpgroup that read the linear out
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(tfull0 + 8 * i, 4);
@@ -589,14 +587,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         }
     } else if (tid < kStagerBase) {
         // ======================= epilogue warpgroups (thread = weight row of the unit) =======================
-        // Warpgroup ew takes the groups G with G % kNumEpi == ew; both follow every unit to know where row tiles end.
-        // At the end of a row tile warpgroup 1 leaves its partial sums in shared memory, warpgroup 0 adds them to
-        // its own (always in that order) and writes the tile out or hands it to the fixer.
+        // With two warpgroups they take the CTA's linears in turn, each doing the whole read-out of its linears: the
+        // per-linear code of one then overlaps the units of the other.  Both keep count of the groups, activation
+        // buffers and hand-over buffers of the linears they skip.
         const uint32_t ew = (uint32_t)(tid - kEpiBase) >> 7, r = (uint32_t)(tid - kEpiBase) & 127, lane = tid & 31;
         const uint32_t lane_base = (r & ~31u) << 16;
         constexpr int kEBmax = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;                      // (registers)
         constexpr int kEB = QIL_TC_EPI_BATCH < kEBmax ? QIL_TC_EPI_BATCH : kEBmax;  // units read back per tcgen05.wait::ld
         uint32_t hc = 0, G = 0, ts = 0;  // hc: per fixer warp, two bits counting the entries handed to it; ts: row tiles closed
+        uint32_t seq = 0;                // linears with units of this CTA so far
         Cyc xc(p.xbufs);
         bool alive = true;
         Walk wk(plan, p.count);
@@ -619,14 +618,22 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const long long tr_p2 = clock64();
             tr[12] += tr_p2 - tr_p1;  // entry fields and the two divisions
 #endif
-            const uint32_t xb = xc.idx;
-            if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xc.ph))) break;
+            const uint32_t xb = xc.idx, xph = xc.ph;
             xc.step();
-            const int2* xblk_b = xblk + (size_t)xb * kXR * p.nb_max;
+            if (kNumEpi > 1 && (seq++ % kNumEpi) != ew) {  // the other warpgroup's linear
+                G += (n + kGroup - 1) / kGroup;
+                continue;
+            }
+            // hand-over buffers of the fixer warp: with one warpgroup its two buffers alternate; with two, each
+            // warpgroup has its own (a barrier is then only ever waited on by warps that saw its previous phase)
             const uint32_t team = (uint32_t)wk.ei % kFixTeams, hcnt = (hc >> (2 * team)) & 3u;
-            const uint32_t hbuf = 2 * team + (hcnt & 1u);
+            if (shares) hc = (hc & ~(3u << (2 * team))) | (((hcnt + 1u) & 3u) << (2 * team));
+            const uint32_t hbuf = 2 * team + (kNumEpi > 1 ? ew : (hcnt & 1u));
+            const uint32_t hph = kNumEpi > 1 ? (hcnt & 1u) : ((hcnt >> 1) & 1u);
+            if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xph))) break;
+            const int2* xblk_b = xblk + (size_t)xb * kXR * p.nb_max;
             float* hand_b = hand + (size_t)hbuf * 2 * kXR * kUnitRows;
-            if (shares && ew == 0 && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * hbuf, ((hcnt >> 1) & 1u) ^ 1u))) break;
+            if (shares && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * hbuf, hph ^ 1u))) break;
             uint32_t n_full = 0;
             float fin[kXR];
 #pragma unroll
@@ -635,28 +642,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             uint32_t bi = 0;  // block inside the activation buffer, which holds the blocks from the slice's first one on, cyclically
             // the CTA's part of row tile rt is complete
             auto close_tile = [&]() {
-                const uint32_t tb = ts & 1, tph = (ts >> 1) & 1;
-                float* tp = tpart + (size_t)tb * kXR * kUnitRows + r;
-                if (ew != 0) {
-                    if (!QIL_WAIT(6, guard.wait_mbar(tempty0 + 8 * tb, tph ^ 1))) {
-                        alive = false;
-                        return;
-                    }
-#pragma unroll
-                    for (int t = 0; t < kXR; ++t) tp[t * kUnitRows] = fin[t];
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tfull0 + 8 * tb);
-                } else {
-                    if constexpr (kNumEpi > 1) {
-                        if (!QIL_WAIT(6, guard.wait_mbar(tfull0 + 8 * tb, tph))) {
-                            alive = false;
-                            return;
-                        }
-#pragma unroll
-                        for (int t = 0; t < kXR; ++t) fin[t] += tp[t * kUnitRows];
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(tempty0 + 8 * tb);
-                    }
+                {
                     const bool cb = u0 <= rt * KB, ce = (rt + 1) * KB <= u1;
                     if (cb && ce) {
                         ++n_full;
@@ -700,12 +686,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
 #endif
             for (uint32_t j0 = 0; alive && j0 < n; j0 += kGroup, ++G) {
                 const uint32_t gs = G % kNG, nreal = min((uint32_t)kGroup, n - j0);
-                if (G % kNumEpi != ew) {  // the other warpgroup's units: only follow the row tiles
-                    for (uint32_t i = 0; alive && i < nreal; ++i) {
-                        if (++bi == KB) bi = 0;
-                        if (++kb == KB || j0 + i + 1 == n) close_tile();
+                if constexpr (kNumEpi > 1) {
+                    // The columns' previous use may have been the other warpgroup's: wait until it has been read out,
+                    // so that the accumulation barrier is at most one phase behind (its parity cannot tell more).
+                    if (!QIL_WAIT(6, guard.wait_count(rd0 + 4 * (gs * 4 + (r >> 5)), G / kNG, dempty0 + 8 * gs))) {
+                        alive = false;
+                        break;
                     }
-                    continue;
                 }
                 if (!QIL_WAIT(3, guard.wait_mbar(dfull0 + 8 * gs, (G / kNG) & 1))) {  // all units of the group are accumulated
                     alive = false;
@@ -745,8 +732,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) {
-                            sts_release(rd0 + 4 * (gs * 4 + (r >> 5)), G / kNG + 1);
+                            // (arrival first: whoever sees the counter and refills the columns can only lead to arrivals
+                            // of the barrier's next phase; the counter may also be written by the other warpgroup's warp
+                            // of these lanes, for a later use of the columns, which cannot start before this one ends)
                             mbar_arrive(dempty0 + 8 * gs);
+                            sts_release(rd0 + 4 * (gs * 4 + (r >> 5)), G / kNG + 1);
                         }
                     }
 #ifdef QIL_TRACE
@@ -774,14 +764,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(xempty0 + 8 * xb);
-                if (shares && ew == 0) mbar_arrive(hfull0 + 8 * hbuf);
+                if (shares) mbar_arrive(hfull0 + 8 * hbuf);
                 // the dependency counter counts quarter tiles (32 rows), so that no warp has to wait for another
                 // (the release covers the other lanes' stores as well: they are ordered before it by the __syncwarp above)
-                if (ew == 0 && n_full && p.tiles_done) {
+                if (n_full && p.tiles_done) {
                     red_release_add(p.tiles_done, n_full);
                 }
             }
-            if (shares) hc = (hc & ~(3u << (2 * team))) | (((hcnt + 1u) & 3u) << (2 * team));
         }
     } else if (tid < kFixBase) {
         // ======================= activation stager (a half warp = one 128-column block per pass) =======================
@@ -905,10 +894,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         constexpr uint32_t kRowsPer = kUnitRows / 32;
         constexpr uint32_t kPoll = 1;  // other CTAs' parts fetched together (more measured slower: the code grows)
         unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
-        uint32_t cnt = 0;  // entries this warp has taken over
+        uint32_t cnt = 0, cntw[2] = {0u, 0u};  // entries this warp has taken over (in all / from each read-out warpgroup)
+        uint32_t seq = 0;                      // linears with units of this CTA so far
         bool alive = true;
         Walk wk(plan, p.count);
         while (alive && wk.next_entry()) {
+            const uint32_t ow = kNumEpi > 1 ? (seq++ % kNumEpi) : 0u;  // read-out warpgroup of the linear
             if ((uint32_t)wk.ei % kFixTeams != team) continue;
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
@@ -918,7 +909,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const bool have_first = t_first * KB < u0 && (t_first + 1) * KB <= u1;  // completes a tile begun elsewhere
             if (!have_last && !(t_first * KB < u0)) continue;
             const uint32_t tag = (uint32_t)wk.ei + 1u, ring_i = (uint32_t)wk.ei % kSlotDepth;
-            const uint32_t hbuf = 2 * team + (cnt & 1u), hph = (cnt >> 1) & 1u;
+            const uint32_t hbuf = 2 * team + (kNumEpi > 1 ? ow : (cnt & 1u));
+            const uint32_t hph = kNumEpi > 1 ? (cntw[ow] & 1u) : ((cnt >> 1) & 1u);
             const float* hand_b = hand + (size_t)hbuf * 2 * kXR * kUnitRows;
             unsigned long long* my_slot = nullptr;
             if (have_last) {
@@ -1015,6 +1007,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 }
             }
             ++cnt;
+            ++cntw[ow];
         }
     } else if (tid < kProdBase) {
         // ======================= MMA issuers (one thread in each of kGroup warps) =======================
@@ -1270,7 +1263,9 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
         }
         // as many activation buffers as leave a deep weight ring
         SmemPlan pl = plan_for(max_m, nb_max, kMaxXBufs);
-        for (int xb = kMaxXBufs - 1; xb >= 2 && pl.stages < 12; --xb) pl = plan_for(max_m, nb_max, xb);
+        // (with two read-out warpgroups an even number: a buffer is then always read by the same warpgroup)
+        for (int xb = kMaxXBufs - 1; xb >= 2 && pl.stages < 12; --xb)
+            if (kNumEpi == 1 || xb % 2 == 0) pl = plan_for(max_m, nb_max, xb);
         if (pl.stages < 4) return QIL_ERR_UNSUPPORTED;
         p.count = n;
         p.stages = pl.stages;

@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 
 METRIC = "W4A16 GEMV GB/s at Llama-2-7B M=1 (packed weights + scales + zeros + activations streamed per second)"
 UNIT = "GB/s"
-TC_DRAM_BYTES_PER_LAYER = (216139008 + 4765696) // 2   # measured DRAM read + write bytes of w4a16_tc_kernel<1> per decoder layer
+TC_DRAM_BYTES_PER_LAYER = (216146432 + 4754432) // 2   # measured DRAM read + write bytes of w4a16_tc_kernel<1> per decoder layer
 WORKLOAD = "configs[1]: Llama-2-7B decoder linears, decode M=1, 32 layers x 7 linears, group 128, 0.1% outliers"
 
 

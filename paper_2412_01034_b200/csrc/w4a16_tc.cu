@@ -582,8 +582,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             G += (n + kGroup - 1) / kGroup;
             turn0 = (turn0 + n) % kNumWg;
             const uint32_t adv = stage0 + n;
-            ph0 ^= (adv / S) & 1;
-            stage0 = adv % S;
+            uint32_t wrapped = adv;  // (subtractions instead of a division: per-linear code is expensive here)
+            while (wrapped >= S) {
+                wrapped -= S;
+                ph0 ^= 1;
+            }
+            stage0 = wrapped;
         }
     } else if (tid < kStagerBase) {
         // ======================= epilogue warpgroups (thread = weight row of the unit) =======================
@@ -1032,7 +1036,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 const uint32_t xm16 = xr16 + (((uint32_t)p.nb_max * 4 * kLboR + 256) >> 4);
                 uint32_t kb = w < KB ? w : w % KB;  // block of the unit inside the activation buffer: unit j sits at j % KB
                 const uint32_t kstep = (uint32_t)kGroup < KB ? (uint32_t)kGroup : (uint32_t)kGroup % KB;
-                uint32_t st_i = (stage0 + w) % S;
+                uint32_t st_i = stage0 + w;
+                if (st_i >= S) st_i -= S;
                 for (uint32_t j = w; j < (n + kGroup - 1) / kGroup * kGroup; j += kGroup, ++G) {
                     const uint32_t gs = G % kNG, gph = (G / kNG) & 1;
                     if (j < n) {
@@ -1076,7 +1081,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     st_i += kGroup;
                     if (st_i >= S) st_i -= S;
                 }
-                stage0 = (stage0 + n) % S;
+                stage0 += n;
+                while (stage0 >= S) stage0 -= S;
             }
             // whatever happened to the other roles: the operations this thread issued are complete before tensor memory
             // is released (this wait also holds in an abandoned kernel)

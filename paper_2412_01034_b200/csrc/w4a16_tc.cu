@@ -392,12 +392,6 @@ __device__ __forceinline__ void slice_of(uint32_t q, uint32_t rem, uint32_t c, u
     u0 = c * q + min(c, rem);
     u1 = u0 + q + (c < rem ? 1u : 0u);
 }
-// CTA that owns unit u
-__device__ __forceinline__ uint32_t owner_of(uint32_t q, uint32_t rem, uint32_t u) {
-    const uint32_t big = rem * (q + 1);  // units held by the first `rem` CTAs
-    return u < big ? u / (q + 1) : rem + (u - big) / q;
-}
-
 // The entries in which one CTA owns units.  The CTA's slice of every entry is worked out once, at the start of the
 // kernel, into a table in shared memory ({first unit, first row tile, units | row tiles touched << 16, first
 // column block | column blocks per row tile << 16}): six roles walk the list, and slicing costs divisions.
@@ -942,7 +936,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 }
             }
             if (have_first) {
-                const uint32_t c_lo = owner_of(E.q, E.rem, t_first * KB);
+                // the CTAs before this one that hold units of the tile (walked backwards: cheaper here than dividing)
+                uint32_t c_lo = c;
+                while (c_lo > 0) {
+                    uint32_t a0, a1;
+                    slice_of(E.q, E.rem, c_lo - 1, a0, a1);
+                    if (a1 <= t_first * KB) break;
+                    --c_lo;
+                }
                 float sum[kRowsPer][kXR];
 #pragma unroll
                 for (uint32_t h = 0; h < kRowsPer; ++h)
@@ -1034,8 +1035,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 xc.step();
                 const uint32_t xr16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
                 const uint32_t xm16 = xr16 + (((uint32_t)p.nb_max * 4 * kLboR + 256) >> 4);
-                uint32_t kb = w < KB ? w : w % KB;  // block of the unit inside the activation buffer: unit j sits at j % KB
-                const uint32_t kstep = (uint32_t)kGroup < KB ? (uint32_t)kGroup : (uint32_t)kGroup % KB;
+                uint32_t kb = w, kstep = (uint32_t)kGroup;  // block of the unit inside the activation buffer: unit j sits at j % KB
+                while (kb >= KB) kb -= KB;
+                while (kstep >= KB) kstep -= KB;
                 uint32_t st_i = stage0 + w;
                 if (st_i >= S) st_i -= S;
                 for (uint32_t j = w; j < (n + kGroup - 1) / kGroup * kGroup; j += kGroup, ++G) {

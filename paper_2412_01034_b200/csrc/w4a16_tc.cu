@@ -447,15 +447,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     unsigned char* xs = ring + (size_t)p.stages * kUnitBytes;                       // [xbufs][xbuf_bytes]
     int2* xblk = reinterpret_cast<int2*>(xs + (size_t)p.xbufs * p.xbuf_bytes);      // [xbufs][kXR][nb_max] {sum v, bits of 2^e}
     float* hand = reinterpret_cast<float*>(xblk + p.xbufs * kXR * p.nb_max);        // [kHandDepth][2][kXR][128]
-    float* tpart = hand + kHandDepth * 2 * kXR * kUnitRows;                         // [2][kXR][128]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tpart + 2 * kXR * kUnitRows);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(hand + kHandDepth * 2 * kXR * kUnitRows);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + p.stages);
     uint64_t* b2 = bars + 2 * p.stages;
     // afull: per unit slot; dfull / dempty: per group of kGroup slots
     const uint32_t afull0 = smem_u32(b2), dfull0 = smem_u32(b2 + kNB), dempty0 = smem_u32(b2 + kNB + kNG);
     uint64_t* b3 = b2 + 3 * kNB;
     const uint32_t xfull0 = smem_u32(b3), xempty0 = smem_u32(b3 + kMaxXBufs);
-    const uint32_t tfull0 = smem_u32(b3 + 8), tempty0 = smem_u32(b3 + 10), mdone0 = smem_u32(b3 + 12);
+    const uint32_t mdone0 = smem_u32(b3 + 12);  // (slots 8..11 are unused)
     const uint32_t hfull0 = smem_u32(b3 + 12 + kGroup), hempty0 = smem_u32(b3 + 12 + kGroup + kHandDepth);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b3 + 12 + kGroup + 2 * kHandDepth);
     volatile int* poisoned = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -489,10 +488,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         for (int i = 0; i < kMaxXBufs; ++i) {
             mbar_init(xfull0 + 8 * i, 4);  // the stager warps
             mbar_init(xempty0 + 8 * i, 4);  // the warps of the warpgroup that read the linear out
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(tfull0 + 8 * i, 4);
-            mbar_init(tempty0 + 8 * i, 4);
         }
         for (int i = 0; i < kGroup; ++i) mbar_init(mdone0 + 8 * i, 1);
         for (int i = 0; i < kHandDepth; ++i) {
@@ -592,7 +587,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         const uint32_t lane_base = (r & ~31u) << 16;
         constexpr int kEBmax = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;                      // (registers)
         constexpr int kEB = QIL_TC_EPI_BATCH < kEBmax ? QIL_TC_EPI_BATCH : kEBmax;  // units read back per tcgen05.wait::ld
-        uint32_t hc = 0, G = 0, ts = 0;  // hc: per fixer warp, two bits counting the entries handed to it; ts: row tiles closed
+        uint32_t hc = 0, G = 0;          // hc: per fixer warp, two bits counting the entries handed to it
         uint32_t seq = 0;                // linears with units of this CTA so far
         Cyc xc(p.xbufs);
         bool alive = true;
@@ -660,7 +655,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 for (int t = 0; t < kXR; ++t) fin[t] = 0.f;
                 kb = 0;
                 ++rt;
-                ++ts;
             };
             // one unit of this warpgroup: fold scale and zero point into the row sums
             // (cr: raw-byte accumulators {x_c high, low plane}; cm: masked-byte accumulators {top, middle, low plane})
@@ -958,26 +952,28 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         uint32_t cu0 = 0, cu1 = 0;
                         if (cc0 + k < c) slice_of(E.q, E.rem, cc0 + k, cu0, cu1);
                         if (cu0 != cu1) {
-                            const uint32_t which = (cu0 / KB == t_first) ? 0u : 1u;
+                            const uint32_t which = (cu0 >= t_first * KB) ? 0u : 1u;  // the tile is that CTA's first or its last
                             src[k] = slots + (((size_t)(cc0 + k) * 2 + which) * kSlotDepth + ring_i) * kSlotElems + lane;
                         }
                     }
-                    alive = QIL_WAIT(3, guard.wait_flag([&] {
+                    auto all_arrived = [&] {
                         bool all = true;
 #pragma unroll
                         for (uint32_t k = 0; k < kPoll; ++k)
                             if (src[k] != nullptr) {
 #pragma unroll
-                                for (uint32_t h = 0; h < kRowsPer; ++h)
+                                for (uint32_t h = 0; h < kRowsPer; ++h) {
 #pragma unroll
                                     for (int t = 0; t < kXR; ++t)
                                         if (t < M) {
                                             got[k][h][t] = __ldcg(src[k] + t * kUnitRows + 32 * h);
                                             all &= (uint32_t)(got[k][h][t] >> 32) == tag;
                                         }
+                                }
                             }
                         return all;
-                    }));
+                    };
+                    alive = QIL_WAIT(3, guard.wait_flag(all_arrived));
                     alive = __all_sync(0xffffffffu, alive);
                     if (!alive) break;
 #pragma unroll
@@ -1186,7 +1182,7 @@ SmemPlan plan_for(int max_m, int nb_max, int xbufs) {
     pl.x_rows = max_m <= 1 ? 1 : max_m <= 2 ? 2 : 4;
     pl.xbuf_bytes = nb_max * 4 * (32 + 48) * pl.x_rows + 512;  // (the last chunk's row window reaches past its own rows)
     const size_t fixed = (size_t)xbufs * pl.xbuf_bytes + (size_t)xbufs * 2 * pl.x_rows * nb_max * 4 +
-                         (size_t)(kHandDepth + 1) * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 12 + kGroup + 2 * kHandDepth) * 8 + 16 +
+                         (size_t)kHandDepth * 2 * pl.x_rows * kUnitRows * 4 + (size_t)(3 * kNB + 12 + kGroup + 2 * kHandDepth) * 8 + 16 +
                          16 * kNG + 128 + (size_t)kMaxEntries * 16;
     pl.xbufs = xbufs;
     pl.stages = 0;

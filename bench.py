@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 
 METRIC = "W4A16 GEMV GB/s at Llama-2-7B M=1 (packed weights + scales + zeros + activations streamed per second)"
 UNIT = "GB/s"
-TC_DRAM_BYTES_PER_LAYER = (216133376 + 5910272) // 2   # measured DRAM read + write bytes of w4a16_tc_kernel<1> per decoder layer
+TC_DRAM_BYTES_PER_LAYER = (216136448 + 4185344) // 2   # measured DRAM read + write bytes of w4a16_tc_kernel<1> per decoder layer
 WORKLOAD = "configs[1]: Llama-2-7B decoder linears, decode M=1, 32 layers x 7 linears, group 128, 0.1% outliers"
 
 
@@ -274,7 +274,7 @@ def run_qil(args):
         per_launch_ms = ms / launches_per_step          # average over the timed region, launch gaps included
         achieved = per_launch_bytes / (per_launch_ms * 1e-3) / 1e9
         # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel on 2 layers (14 independent
-        # linears, larger than L2): 111.02 MB per layer, scaled by the layers of a launch (traffic grows in proportion)
+        # linears, larger than L2): 110.16 MB per layer, scaled by the layers of a launch (traffic grows in proportion)
         traffic = TC_DRAM_BYTES_PER_LAYER * args.layers if (persistent and args.deps == "none") else None
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

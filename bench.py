@@ -28,7 +28,8 @@ if ROOT not in sys.path:
 
 METRIC = "W4A16 GEMV GB/s at Llama-2-7B M=1 (packed weights + scales + zeros + activations streamed per second)"
 UNIT = "GB/s"
-TC_DRAM_BYTES_PER_LAYER = (216136448 + 4185344) // 2   # measured DRAM read + write bytes of w4a16_tc_kernel<1> per decoder layer
+DECODE_PROFILE = os.path.join(ROOT, "profiles", "w4a16_tc_kernel_cfg1_decode.json")
+DECODE_KERNEL_SOURCE = os.path.join(ROOT, "paper_2412_01034_b200", "csrc", "w4a16_tc.cu")
 WORKLOAD = "configs[1]: Llama-2-7B decoder linears, decode M=1, 32 layers x 7 linears, group 128, 0.1% outliers"
 
 
@@ -98,6 +99,50 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(r[1] for r in use), "sm_max_mhz": max(r[2] for r in use),
                 "power_w_max": max(r[3] for r in use), "samples": len(use),
                 "window": "timed region" if inside else "warm-up and timed region", "reasons": reasons}
+
+
+def measured_dram_bytes_per_layer():
+    """DRAM read + write bytes of the decode kernel per decoder layer, from the tracked summary of its last ncu
+    capture; None when the kernel source has changed since that capture (the figure would describe another kernel)."""
+    import hashlib
+    try:
+        prof = json.load(open(DECODE_PROFILE))
+        digest = hashlib.sha256(open(DECODE_KERNEL_SOURCE, "rb").read()).hexdigest()
+    except (OSError, ValueError):
+        return None
+    if prof.get("kernel_source_sha256") != digest:
+        return None
+    return (prof["dram_bytes_read"] + prof["dram_bytes_write"]) / prof["layers_captured"]
+
+
+def check_against_oracle(model, sampled):
+    """After the timed region: the status word of the workspace must be 0 and the sampled output features of the
+    sampled linears must match the CPU oracle (quantiser + fp64 linear) within the acceptance rule."""
+    import ctypes as C
+    import numpy as np
+    import torch
+    from oracle import c_oracle
+    from paper_2412_01034_b200 import workloads as wl
+    model.y_dev.zero_()
+    model.run()
+    torch.cuda.synchronize()
+    out = C.c_int(-1)
+    rc = model.lib.qil_device_status(C.c_void_p(model.ws.data_ptr()), C.byref(out),
+                                     C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if rc != 0 or out.value != 0:
+        raise SystemExit(f"bench: device status word is {out.value} (rc {rc}) after the timed region")
+    worst = 0.0
+    for i in sampled:
+        rows, w_rows = model.kept[i]
+        q = c_oracle.quantize_rtn_w4_asym(w_rows, wl.GROUP_SIZE)
+        y_ref = c_oracle.linear_w4a16(model.input_bits(i), *q, wl.GROUP_SIZE)
+        y = model.output(i).to(torch.float32).cpu().numpy().astype(np.float64)[:, rows]
+        # (the maximum over the sampled features lower-bounds the row maximum: the check is the stricter one)
+        rel = float((np.abs(y - y_ref) / np.abs(y_ref).max(axis=1, keepdims=True)).max())
+        worst = max(worst, rel)
+        if not np.all(np.isfinite(y)) or rel > 1e-2:
+            raise SystemExit(f"bench: linear {i} differs from the oracle (row-relative error {rel:.3e})")
+    return worst
 
 
 def physical_gpu_index(local_rank: int) -> int:
@@ -192,8 +237,16 @@ def run_qil(args):
     layout = {"stream128": api.LAYOUT_STREAM128, "tile16": api.LAYOUT_TILE16,
               "canonical": api.LAYOUT_CANONICAL}[args.layout]
     persistent = args.layout == "stream128"
+    import numpy as np
+    per_layer = 7
+    sampled = sorted({0, (args.layers // 2) * per_layer + 4, (args.layers - 1) * per_layer + 6})   # a q, a gate, a down
+    rng = np.random.default_rng(5)
+    keep = {}
+    from paper_2412_01034_b200 import workloads as wl
+    for i in sampled:
+        keep[i] = np.sort(rng.choice(wl.llama_linear_ids()[i][2], 64, replace=False))
     model = llama_decode.QuantisedLinears(cfg=1, M=1, n_layers=args.layers, layout=layout, deps=args.deps,
-                                          device=f"cuda:{local_rank}")
+                                          device=f"cuda:{local_rank}", keep_host_rows=keep)
     stream = torch.cuda.Stream(device=dev)
     bytes_per_step = model.algorithmic_bytes()
 
@@ -236,6 +289,8 @@ def run_qil(args):
     ms, clocks = timed(g_dev, args.steps, args.warmup, physical_gpu_index(local_rank) if rank == 0 else None)
     ms_e2e, _ = timed(g_e2e, args.steps, args.warmup)
 
+    parity_worst = check_against_oracle(model, sampled)
+
     ms_all, units_all = reduce_max_time_sum_units(ms, bytes_per_step, world, dev)
     ms_e2e_all, _ = reduce_max_time_sum_units(ms_e2e, bytes_per_step, world, dev)
     value = units_all / (ms_all * 1e-3) / 1e9
@@ -251,6 +306,7 @@ def run_qil(args):
         ms_ord, _ = timed(g_ord, min(args.steps, 200), min(args.warmup, 20))
         ordered = {"dependencies": "layer", "ms_per_step": ms_ord, "GB/s": bytes_per_step / (ms_ord * 1e-3) / 1e9,
                    "waiting_linears_per_step": sum(1 for i in range(n_linears) if model.descs[i].flags)}
+        ordered["parity_worst_row_relative_error"] = check_against_oracle(model, sampled)
         model.set_deps("none")
         del g_ord
     if rank == 0 and world == 1 and not args.no_secondary:
@@ -275,7 +331,8 @@ def run_qil(args):
         achieved = per_launch_bytes / (per_launch_ms * 1e-3) / 1e9
         # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel on 2 layers (14 independent
         # linears, larger than L2): 110.16 MB per layer, scaled by the layers of a launch (traffic grows in proportion)
-        traffic = TC_DRAM_BYTES_PER_LAYER * args.layers if (persistent and args.deps == "none") else None
+        per_layer_traffic = measured_dram_bytes_per_layer() if (persistent and args.deps == "none") else None
+        traffic = per_layer_traffic * args.layers if per_layer_traffic else None
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_all, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -289,6 +346,9 @@ def run_qil(args):
             "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_e2e_all,
                     "h2d_bytes_per_step": 2 * x_elems, "d2h_bytes_per_step": 2 * y_elems},
             "gpu_launches": launches_per_step * args.steps,
+            "parity_checked": True,
+            "parity": {"status_word": 0, "linears": sampled, "features_per_linear": 64,
+                       "worst_row_relative_error": parity_worst, "bound": 1e-2},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_kind": peak_kind, "kernel": kernel,
                          "bytes_per_launch": per_launch_bytes, "us_per_launch": per_launch_ms * 1e3,

@@ -134,13 +134,21 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  * scale, |integer| <= 32639) and accumulates exactly in int32; the conversion
  * error per element is at most 2^-16 of the block maximum.
  * workspace: qil_linear_w4a16_workspace_size() bytes, only touched when the
- * shape needs a split along K; it must be zero-filled once before first use
- * (the kernels leave it zeroed again).  Calls that share a workspace must not
- * overlap on the device.  Its first int is a status word: the streaming kernel
- * ORs QIL_ERR_TIMEOUT into it if one of its bounded waits ever runs out (read it
- * with qil_device_status; words 2..5 of the workspace then tell where: 1 + CTA,
- * thread, shared-memory address of the barrier or 0, parity; after such an
- * error re-zero the workspace).
+ * shape needs a split along K or the streaming kernel runs; it must be
+ * zero-filled once before first use.  One workspace serves every layout: the
+ * streaming kernel's part (a 256-byte header and the slots through which CTAs
+ * hand partial row tiles to each other) comes first, the split-K scratch of the
+ * skinny kernel after it; each kernel leaves its own part ready for the next
+ * call (counters and slot tags back at zero; the header words 1..7 are scratch).
+ * Calls that share a workspace must not overlap on the device.  Its first int
+ * is a status word: the streaming kernel ORs QIL_ERR_TIMEOUT into it if one of
+ * its bounded waits ever runs out (read it with qil_device_status; words 2..5
+ * of the workspace then tell where: 1 + CTA, thread, shared-memory address of
+ * the barrier or 0, parity; after such an error re-zero the workspace).
+ * The streaming kernel is one CTA per SM and its CTAs wait for each other, so
+ * it is launched cooperatively: all of them are resident together or the
+ * launch is refused (QIL_ERR_UNSUPPORTED), e.g. on a device partition that is
+ * smaller than the device.  It should not share the GPU with other kernels.
  * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, CUDA.
  * ---------------------------------------------------------------------- */
 size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size);
@@ -157,11 +165,18 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
  * plug-in whose host application owns all device memory, code running inside a
  * region where the allocator may not be entered.  qil_linear_w4a16 needs a
  * caller-allocated workspace whenever the shape is split along K; this variant
- * computes the same result with the scratch held in a fixed array of
+ * runs the skinny kernel (or, for shapes outside it, the general kernel, which
+ * needs no scratch) with the split-K scratch held in a fixed array of
  * QIL_STATIC_WS_BYTES bytes that is part of the library image (each GPU that
  * loads the library keeps that much memory reserved until the process exits).
- * Arguments as qil_linear_w4a16, minus the workspace.
- *  - Shapes whose scratch need (qil_linear_w4a16_workspace_size) exceeds
+ * Arguments as qil_linear_w4a16, minus the workspace.  Two differences from
+ * that call: QIL_LAYOUT_STREAM128 is not served (QIL_ERR_UNSUPPORTED: the list
+ * kernel's workspace is larger than the array), and on the canonical layout
+ * with M > 16 the result is the skinny kernel's (fp32 dequantisation), not the
+ * prefill GEMM's (weights rounded to bf16): both are within the tolerance of
+ * the linear, but their bits differ.  The array's address is looked up for the
+ * device that is current at the call; `stream` must belong to that device.
+ *  - Shapes whose split-K scratch (qil_linear_w4a16_static_ws_need) exceeds
  *    QIL_STATIC_WS_BYTES are rejected with QIL_ERR_WORKSPACE; nothing is launched.
  *  - The call allocates and frees nothing.  The first call on each device looks
  *    up the device address of the array (with that device current); make that
@@ -176,6 +191,8 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
 qil_status qil_linear_w4a16_static_ws(const void* x, const uint32_t* qweight, const void* scales,
                                       const void* zeros, void* y, int M, int N, int K,
                                       int group_size, qil_layout layout, qil_stream_t stream);
+/* Bytes of the built-in array that a shape would use (0: the shape needs no scratch). */
+size_t qil_linear_w4a16_static_ws_need(int M, int N, int K, int group_size);
 
 /* ------------------------------------------------------------------------
  * A list of weight-only linears run in stream order (one decode pass over the
@@ -184,7 +201,12 @@ qil_status qil_linear_w4a16_static_ws(const void* x, const uint32_t* qweight, co
  * whose x is written by an earlier entry of the same list must carry
  * QIL_DEP_PREVIOUS in `flags`: it then starts only after every earlier entry has
  * written all of its outputs.  Entries without the flag may overlap with their
- * predecessors (q, k and v of one layer share an input and need no flag).
+ * predecessors (q, k and v of one layer share an input and need no flag) and
+ * with each other.  QIL_DEP_NEVER is a diagnostic flag: the entry waits for an
+ * event that never happens, so the kernel's bounded wait runs out, the launch
+ * ends with QIL_ERR_TIMEOUT in the status word and the outputs of that entry
+ * and of all later ones are unspecified (used with qil_set_wait_limit_ns to
+ * exercise the error path; the workspace must be re-zeroed afterwards).
  * When every entry uses QIL_LAYOUT_STREAM128, the whole list runs as one
  * persistent kernel.  All pointers inside a descriptor are device
  * pointers; the descriptor array itself is host memory and is consumed before
@@ -202,6 +224,7 @@ typedef struct {
     int flags;               /* 0 or QIL_DEP_PREVIOUS */
 } qil_linear_desc;
 #define QIL_DEP_PREVIOUS 1
+#define QIL_DEP_NEVER 2
 
 qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs /*host*/, int count, void* workspace,
                                   size_t workspace_bytes, qil_stream_t stream);
@@ -233,7 +256,9 @@ qil_status qil_quantize_act_a4(const void* x, int M, int K, const float* static_
  *   y[m][n]   = bf16( float(acc) * (sx[m] * sw[n]) )
  *   qx [M][K/8], qw [N][K/8] canonical packed signed nibbles; sx [M], sw [N] fp32
  *   acc_out: optional [M][N] int32 copy of the raw accumulators.
- * Needs K % 32 == 0.  |acc| <= 64 K must fit int32.
+ * Needs K % 32 == 0 and K < 131072: the kernel works on bytes that are 16 x the
+ * codes, its int32 accumulator holds 256 x the sum, and 256 * 64 K must stay
+ * below 2^31.
  * workspace: qil_linear_w4a4_workspace_size() bytes, zero-filled once; its first
  * int is a status word that receives QIL_ERR_TIMEOUT if a bounded device-side
  * wait ever runs out (read it with qil_device_status).
@@ -250,6 +275,9 @@ const char* qil_status_string(qil_status s);
 int qil_version(void);
 /* Copies the device status word to *out (host) and waits for that copy. */
 qil_status qil_device_status(const int* dev_status, int* out /*host*/, qil_stream_t stream);
+/* Limit of every device-side wait of the streaming list kernel, in nanoseconds, for launches made
+ * after the call (process-wide; 0 restores the default of 2 s). */
+qil_status qil_set_wait_limit_ns(unsigned long long ns);
 
 /* Measurement helpers (not part of the method): a dense bf16 GEMV
  * y[n] = sum_k x[k] W[n][k] with W bf16 [N][K], the 16-bit baseline the paper's

@@ -18,6 +18,8 @@ SIGNATURES = {
     "qil_linear_w4a16_workspace_size": (_sz, [_i, _i, _i, _i]),
     "qil_linear_w4a16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w4a16_static_ws": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "qil_linear_w4a16_static_ws_need": (_sz, [_i, _i, _i, _i]),
+    "qil_set_wait_limit_ns": (_i, [C.c_ulonglong]),
     "qil_linear_w4a16_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
     "qil_linear_w4a16_batch_host": (_i, [_vp, _i, _vp, _vp, _sz, _vp, _vp, _sz, _vp, _sz, _vp]),
     "qil_quantize_act_a4": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),

@@ -16,6 +16,7 @@ OK = 0
 F32, BF16, F16 = 0, 1, 2
 LAYOUT_CANONICAL, LAYOUT_TILE16, LAYOUT_STREAM128 = 0, 1, 3
 DEP_PREVIOUS = 1
+DEP_NEVER = 2
 ERR_RANGE = 8
 
 _DT = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}

@@ -6,18 +6,29 @@
 namespace qil {
 
 int num_sms() {
-    static std::atomic<int> cached{0};
-    int v = cached.load(std::memory_order_relaxed);
-    if (v > 0) return v;
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cached[kMaxDevices];
     int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return QIL_NUM_SMS_FALLBACK;  // (no device: only sizes are asked for)
+    }
+    const bool slot = dev >= 0 && dev < kMaxDevices;
+    if (slot) {
+        const int v = cached[dev].load(std::memory_order_relaxed);
+        if (v > 0) return v;
+    }
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
         (void)cudaGetLastError();
         return QIL_NUM_SMS_FALLBACK;  // not cached: a later call may succeed
     }
-    cached.store(sms, std::memory_order_relaxed);
+    if (slot) cached[dev].store(sms, std::memory_order_relaxed);
     return sms;
 }
+
+// The workspace of qil_linear_w4a16 has two parts that never overlap: the streaming list kernel's header and
+// hand-over slots first, the split-K scratch of the skinny kernel after them.
+size_t w4a16_skinny_ws_offset() { return (w4a16_tc_workspace() + 255) & ~(size_t)255; }
 
 }  // namespace qil
 
@@ -48,6 +59,11 @@ const char* qil_status_string(qil_status s) {
 }
 
 int qil_version(void) { return 100; }
+
+qil_status qil_set_wait_limit_ns(unsigned long long ns) {
+    w4a16_tc_set_wait_limit(ns);
+    return QIL_OK;
+}
 
 qil_status qil_device_status(const int* dev_status, int* out, qil_stream_t stream) {
     if (!dev_status || !out) return QIL_ERR_NULL;
@@ -127,9 +143,7 @@ static qil_status check_w4a16(const void* x, const void* qw, const void* sc, con
 size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size) {
     if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0) return 0;
     if (K % 128 != 0 || group_size % 128 != 0) return 0;
-    size_t a = w4a16_skinny_workspace(M, N, K, group_size);
-    const size_t c = w4a16_tc_workspace();
-    return c > a ? c : a;  // large enough for every layout
+    return w4a16_skinny_ws_offset() + w4a16_skinny_workspace(M, N, K, group_size);  // serves every layout
 }
 
 qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* scales, const void* zeros, void* y,
@@ -147,9 +161,13 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
     if (w4a16_prefill_supported(M, N, K, group_size, layout))
         return launch_w4a16_prefill(x, qweight, scales, zeros, y, M, N, K, group_size,
                                     workspace_bytes >= sizeof(int) ? workspace : nullptr, S(stream));
-    if (w4a16_skinny_supported(M, N, K, group_size, layout))
-        return launch_w4a16_skinny(x, qweight, scales, zeros, y, M, N, K, group_size, layout, workspace,
-                                   workspace_bytes, S(stream));
+    if (w4a16_skinny_supported(M, N, K, group_size, layout)) {
+        const size_t off = w4a16_skinny_ws_offset();
+        const bool have = workspace != nullptr && workspace_bytes > off;
+        return launch_w4a16_skinny(x, qweight, scales, zeros, y, M, N, K, group_size, layout,
+                                   have ? static_cast<char*>(workspace) + off : nullptr, have ? workspace_bytes - off : 0,
+                                   S(stream));
+    }
     if (layout != QIL_LAYOUT_CANONICAL) return QIL_ERR_UNSUPPORTED;
     return launch_w4a16_general(x, qweight, scales, zeros, y, M, N, K, group_size, S(stream));
 }
@@ -163,7 +181,7 @@ qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs, int count, void*
     bool all_tc = true;
     for (int i = 0; i < count; ++i) {
         const qil_linear_desc& d = descs[i];
-        if ((d.flags & ~QIL_DEP_PREVIOUS) != 0) return QIL_ERR_UNSUPPORTED;
+        if ((d.flags & ~(QIL_DEP_PREVIOUS | QIL_DEP_NEVER)) != 0) return QIL_ERR_UNSUPPORTED;
         const qil_status s = check_w4a16(d.x, d.qweight, d.scales, d.zeros, d.y, d.M, d.N, d.K, d.group_size,
                                          (qil_layout)d.layout);
         if (s != QIL_OK) return s;
@@ -176,7 +194,7 @@ qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs, int count, void*
         if (!skinny && d.layout != QIL_LAYOUT_CANONICAL) return QIL_ERR_UNSUPPORTED;
         if (skinny) {
             const size_t need = w4a16_skinny_workspace(d.M, d.N, d.K, d.group_size);
-            if (need > 0 && (!workspace || workspace_bytes < need)) return QIL_ERR_WORKSPACE;
+            if (need > 0 && (!workspace || workspace_bytes < w4a16_skinny_ws_offset() + need)) return QIL_ERR_WORKSPACE;
         }
     }
     if (all_tc) return launch_w4a16_tc(descs, count, workspace, workspace_bytes, S(stream));
@@ -226,7 +244,8 @@ qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* 
                            int32_t* acc_out, int M, int N, int K, void* workspace, size_t workspace_bytes,
                            qil_stream_t stream) {
     if (!qx || !sx || !qw || !sw || !y) return QIL_ERR_NULL;
-    if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || K > 131072) return QIL_ERR_SHAPE;
+    // (the kernel accumulates 256 x the true sum: 256 * 64 * K must stay below 2^31)
+    if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || K >= 131072) return QIL_ERR_SHAPE;
     if (!aligned16(qx) || !aligned16(sx) || !aligned16(qw) || !aligned16(sw) || !aligned16(y) ||
         (acc_out && !aligned16(acc_out)) || (workspace && !aligned16(workspace)))
         return QIL_ERR_ALIGN;

@@ -18,7 +18,7 @@ inline qil_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? QIL_OK : QIL_ERR_CUDA;
 }
 
-// Number of SMs of the current device (cached per process; the library targets one device type).
+// Number of SMs of the current device (cached per device ordinal).
 int num_sms();
 
 __device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) {
@@ -79,6 +79,7 @@ size_t w4a16_tc_workspace();
 qil_status launch_pack_stream128_w4(const uint8_t* codes, const void* scales, const void* zeros, int N, int K, int G,
                                     void* out, cudaStream_t st);
 qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, size_t ws_bytes, cudaStream_t st);
+void w4a16_tc_set_wait_limit(unsigned long long ns);  // 0 restores the default
 
 size_t w4a4_workspace(int M, int N, int K);
 qil_status launch_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, void* y,

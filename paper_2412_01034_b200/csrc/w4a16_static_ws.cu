@@ -38,6 +38,11 @@ qil_status static_ws_address(void** out) {
 
 }  // namespace
 
+extern "C" size_t qil_linear_w4a16_static_ws_need(int M, int N, int K, int group_size) {
+    if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0 || K % 128 != 0 || group_size % 128 != 0) return 0;
+    return qil::w4a16_skinny_workspace(M, N, K, group_size);
+}
+
 extern "C" qil_status qil_linear_w4a16_static_ws(const void* x, const uint32_t* qweight, const void* scales,
                                                  const void* zeros, void* y, int M, int N, int K, int group_size,
                                                  qil_layout layout, qil_stream_t stream) {

@@ -19,53 +19,40 @@
 // is 8704 bytes: 4 chunks (32 columns each) x 128 rows x 16 bytes of codes, byte b of
 // word m of a chunk holding column 8m+b (low nibble) and 8m+4+b (high nibble); then
 // 128 x {fp16 scale, fp16 zero}.  Rows beyond N are zero.  A linear is one contiguous
-// stream of units; CTA c of C owns units [c q + min(c, r), ...) with q = units / C, r = units % C.
+// stream of units.  The units of all entries of a phase (a run of entries that do not wait for each
+// other) form one stream of which CTA c of C owns units [c q + min(c, r), ...), q = units / C,
+// r = units % C (see launch_w4a16_tc).
 //
 // Roles in a CTA (one CTA per SM, alive for the whole list):
 //   producer (1 thread)    streams the CTA's units through a shared-memory ring (cp.async.bulk +
 //                          mbarrier), running ahead across linears as far as the ring allows, so
 //                          HBM keeps streaming while the consumers wait for a dependency;
-//   unpack warpgroups      (QIL_TC_UNPACK_WGS, default 2) take turns on units: shared memory -> nibble split -> tensor memory;
+//   unpack warpgroups (2)  take turns on units: shared memory -> nibble split -> tensor memory;
 //   MMA issuers (kGroup x 1 thread) units are handled in groups of kGroup (3), issuer w takes slot w of
 //                          every group: four tcgen05.mma per unit, completion by tcgen05.commit;
-//   epilogue warpgroups    (QIL_TC_EPILOGUE_WGS, default 1; two take the CTA's linears in turn) thread =
+//   epilogue warpgroup     thread =
 //                          weight row: accumulators -> fp32 row sums (kept in registers over the units
 //                          of a row tile); writes the bf16 outputs of row tiles the CTA owns entirely,
 //                          or hands over the partial sums of a row tile it shares;
 //   stager (4 warps)       waits for QIL_DEP_PREVIOUS, loads and converts the activation blocks the
 //                          CTA's units need, into a ring of up to four buffers (up to three linears ahead);
-//   fixer (4 warps)        all cross-CTA work, linear i's shared row tiles belonging to warp i % 4: it
-//                          publishes the partial sums of a shared row tile as {value, tag} pairs (one
-//                          8-byte store each, tag = entry index + 1) into a ring of slots in the
-//                          workspace, completes the row tile whose end the CTA owns by adding the
-//                          contributions in CTA order (bit-reproducible), and counts finished quarter
-//                          tiles for the dependency counter.  A linear costs a fixer warp several round
-//                          trips through the L2; taking the linears in turn overlaps them.
+//   fixer (4 warps)        all cross-CTA work, linear i's shared row tiles belonging to team i % 2: the
+//                          team's publishing warp writes the partial sums of a row tile that ends in
+//                          another CTA as {value, tag} pairs (one 8-byte store each, tag = entry index
+//                          + 1) into a ring of slots in the workspace; its completing warp finishes the
+//                          row tile whose end the CTA owns by adding the contributions in CTA order
+//                          (bit-reproducible) and counts finished quarter tiles for the dependency
+//                          counter.  Publishing never waits behind completing.
 // No role uses a named barrier: every hand-over is an mbarrier or a flag in global memory, and
-// every wait is bounded (2 s).  When a wait runs out, QIL_ERR_TIMEOUT is recorded in the
+// every wait is bounded (2 s unless set otherwise).  When a wait runs out, QIL_ERR_TIMEOUT is recorded in the
 // workspace status word (with the place in words 2..5 of the workspace), every role stops at its
 // next wait without issuing further work, outstanding copies and tensor-core operations are
 // waited for, tensor memory is released and the kernel returns.
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 
 #include "qil_common.cuh"
-
-// Optional per-warp timing (compile with -DQIL_TRACE): cycles spent in the waits of every role, written to a
-// buffer set with qil_trace_set_tc().  Nothing is skipped or reordered; without the macro the hooks vanish.
-#ifdef QIL_TRACE
-#define QIL_WAIT(slot, ...)                          \
-    ([&] {                                           \
-        const long long tr_t0_ = clock64();          \
-        const bool tr_ok_ = (__VA_ARGS__);           \
-        tr[slot] += clock64() - tr_t0_;              \
-        return tr_ok_;                               \
-    }())
-#define QIL_TR_COUNT(slot) tr[slot] += 1
-#else
-#define QIL_WAIT(slot, ...) (__VA_ARGS__)
-#define QIL_TR_COUNT(slot)
-#endif
 
 namespace qil {
 
@@ -73,38 +60,21 @@ namespace {
 
 constexpr int kUnitRows = 128;
 constexpr int kUnitBytes = 8192 + 512;
-#ifndef QIL_TC_UNPACK_WGS
-#define QIL_TC_UNPACK_WGS 2
-#endif
-#ifndef QIL_TC_SPIN_POLLS
-#define QIL_TC_SPIN_POLLS 0
-#endif
-#ifndef QIL_TC_EPI_BATCH
-#define QIL_TC_EPI_BATCH 1
-#endif
-#ifndef QIL_TC_EPILOGUE_WGS
-#define QIL_TC_EPILOGUE_WGS 1
-#endif
-constexpr int kNumWg = QIL_TC_UNPACK_WGS;        // unpack warpgroups
+// Role counts: the values below measured fastest on the Llama-2-7B list (a second read-out warpgroup, more units per
+// read-out pass and polling instead of sleeping waits all measured slower).
+constexpr int kNumWg = 2;                        // unpack warpgroups
 constexpr int kUnpackThreads = 128 * kNumWg;
-constexpr int kNumEpi = QIL_TC_EPILOGUE_WGS;      // epilogue warpgroups (they alternate groups of units)
-constexpr int kEpiBase = kUnpackThreads;         // (their warps keep warp % 4 = lane quarter)
-constexpr int kStagerBase = kEpiBase + 128 * kNumEpi;
+constexpr int kEpiBase = kUnpackThreads;         // the read-out warpgroup (its warps keep warp % 4 = lane quarter)
+constexpr int kStagerBase = kEpiBase + 128;
 constexpr int kFixBase = kStagerBase + 128;
-constexpr int kFixTeams = 4;                     // fixer warps: entry i's shared tiles belong to warp i % kFixTeams
-constexpr int kFixThreads = 32 * kFixTeams;      // (a lane takes four rows of the tile)
-#ifndef QIL_TC_GROUP_UNITS
-#define QIL_TC_GROUP_UNITS 3
-#endif
-constexpr int kGroup = QIL_TC_GROUP_UNITS;       // units per group: one per MMA issuer, one epilogue pass
+constexpr int kFixTeams = 2;                     // fixer teams: entry i's shared tiles belong to team i % kFixTeams;
+constexpr int kFixThreads = 64 * kFixTeams;      // a team is a publishing and a completing warp (a lane takes four rows)
+constexpr int kGroup = 3;                        // units per group: one per MMA issuer, one epilogue pass
 constexpr int kMmaBase = kFixBase + kFixThreads; // kGroup warps, one issuing thread each
 constexpr int kProdBase = kMmaBase + 32 * kGroup;  // one warp, one thread issues
 constexpr int kThreads = kProdBase + 32;
 static_assert(kThreads <= 1024, "block size");
-#ifndef QIL_TC_GROUPS
-#define QIL_TC_GROUPS 4
-#endif
-constexpr int kNG = QIL_TC_GROUPS;               // groups in flight in tensor memory
+constexpr int kNG = 4;                           // groups in flight in tensor memory
 constexpr int kNB = kGroup * kNG;                // = units in flight
 constexpr int kTmemCols = 512;
 // tensor-memory columns: per unit 16 of masked low nibbles (A), 8 accumulators of the raw-byte products and 8 (16 with
@@ -113,17 +83,17 @@ constexpr int kColD = 16 * kNB;
 __host__ __device__ constexpr int d_unit_cols(int xr) { return 8 + (xr == 4 ? 16 : 8); }
 __host__ __device__ constexpr int col_meta(int xr) { return kColD + d_unit_cols(xr) * kNB; }
 static_assert(col_meta(4) + kNB <= kTmemCols, "tensor memory budget");
-static_assert(kNumEpi == 1 || kNumEpi == 2, "one or two read-out warpgroups");
 constexpr int kMaxXBufs = 4;                     // activation buffers at most
-constexpr int kHandDepth = 2 * kFixTeams;        // hand-over buffers between the epilogue and the fixer: two per warp
+constexpr int kHandDepth = 2 * kFixTeams;        // hand-over buffers between the epilogue and the fixers: two per team
 constexpr int kMaxEntries = 256;
 constexpr int kMaxRows = 4;                      // activation rows
 constexpr int kSlotDepth = 4;                    // ring of slots per (CTA, first / last tile), indexed by entry
-static_assert(kSlotDepth == kFixTeams, "a slot is always written by the same fixer warp, in entry order");
+static_assert(kSlotDepth % kFixTeams == 0, "a slot is always written by the same fixer warp, in entry order");
 constexpr int kSlotElems = kMaxRows * kUnitRows; // {value, tag} pairs of 8 bytes
 constexpr int kWsHeader = 256;
 constexpr int kFlagDep = 1;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr int kFlagNever = 2;
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;
 
 struct TcEntry {  // 56 bytes
     const uint16_t* x;
@@ -131,8 +101,8 @@ struct TcEntry {  // 56 bytes
     __nv_bfloat16* y;
     int N, K, M, flags;
     uint32_t tiles_before;  // row tiles of all earlier entries of this launch
-    uint32_t q, rem;        // units / CTAs, units % CTAs
-    uint32_t pad;
+    uint32_t q, rem;        // units of the entry's phase / CTAs, and the remainder
+    uint32_t base;          // units of the phase before this entry
 };
 
 struct TcParams {
@@ -142,12 +112,10 @@ struct TcParams {
     int nb_max;      // 128-column blocks an activation buffer holds (>= the blocks a CTA touches in any entry)
     int xbufs;       // activation buffers (entries the stager may run ahead)
     int xbuf_bytes;  // one activation operand buffer
+    unsigned long long wait_ns;  // limit of every device-side wait
     int* status;
     unsigned int* tiles_done;
     unsigned char* slots;
-#ifdef QIL_TRACE
-    unsigned long long* trace;  // [CTA][warp][16]
-#endif
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -170,18 +138,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-// non-blocking test of a phase
-__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -299,9 +255,7 @@ __device__ __forceinline__ void mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint
 struct Guard {
     int* status;
     volatile int* poisoned;
-#ifdef QIL_TRACE
-    long long* polls;  // failed polls of this thread
-#endif
+    unsigned long long limit;  // nanoseconds
     static __device__ __forceinline__ unsigned long long now_ns() {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -316,35 +270,19 @@ struct Guard {
             status[5] = (int)parity;
         }
     }
-    // A thread suspended in mbarrier.try_wait wakes up late (measured: hand-overs between roles then cost on the
-    // order of a microsecond each), so a wait first polls without blocking for a while and only then lets the
-    // hardware suspend the thread.
     __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity) const {
-#pragma unroll 1
-        for (int i = 0; i < QIL_TC_SPIN_POLLS; ++i)
-            if (mbar_test_wait(bar, parity)) return true;
         if (mbar_try_wait(bar, parity)) return true;
-#ifdef QIL_TRACE
-        return wait_mbar_slow(status, poisoned, bar, parity, polls);
-#else
-        return wait_mbar_slow(status, poisoned, bar, parity);
-#endif
+        return wait_mbar_slow(status, poisoned, limit, bar, parity);
     }
     // (out of line, scalar arguments: the common case above stays one instruction and a branch)
-    static __device__ __noinline__ bool wait_mbar_slow(int* status, volatile int* poisoned, uint32_t bar, uint32_t parity
-#ifdef QIL_TRACE
-                                                       , long long* polls
-#endif
-    ) {
+    static __device__ __noinline__ bool wait_mbar_slow(int* status, volatile int* poisoned, unsigned long long limit,
+                                                       uint32_t bar, uint32_t parity) {
         if (*poisoned) return false;
         const unsigned long long t0 = now_ns();
         for (;;) {
             if (mbar_try_wait(bar, parity)) return true;
-#ifdef QIL_TRACE
-            *polls += 1;
-#endif
             if (*poisoned) return false;
-            if (now_ns() - t0 > kWaitLimitNs) break;
+            if (now_ns() - t0 > limit) break;
         }
         *poisoned = 1;
         atomicOr(status, (int)QIL_ERR_TIMEOUT);
@@ -367,9 +305,6 @@ struct Guard {
 #pragma unroll 1
         for (uint32_t i = 0;; ++i) {  // (one copy of the predicate's code: the kernel is sensitive to its size)
             if (done()) return true;
-#ifdef QIL_TRACE
-            *polls += 1;
-#endif
             if (i == 0) {
                 if (*poisoned) return false;
                 t0 = now_ns();
@@ -377,7 +312,7 @@ struct Guard {
             if (i > 8) __nanosleep(i < 64 ? 32 : 256);
             if ((i & 15u) == 15u) {
                 if (*poisoned) return false;
-                if (now_ns() - t0 > kWaitLimitNs) break;
+                if (now_ns() - t0 > limit) break;
             }
         }
         *poisoned = 1;
@@ -462,9 +397,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     const uint32_t rd0 = smem_u32(tmem_slot + 2);
     uint4* plan = reinterpret_cast<uint4*>((reinterpret_cast<uintptr_t>(tmem_slot + 2 + 4 * kNG) + 15) & ~(uintptr_t)15);  // [count] this CTA's slice of every entry
     for (int i = tid; i < p.count; i += kThreads) {
-        uint32_t pu0, pu1;
-        slice_of(p.e[i].q, p.e[i].rem, c, pu0, pu1);
-        const uint32_t pn = pu1 - pu0, pKB = (uint32_t)p.e[i].K >> 7;
+        // the CTA's slice of the entry's phase, cut down to the entry (unit numbers inside the entry)
+        uint32_t ph0, ph1;
+        slice_of(p.e[i].q, p.e[i].rem, c, ph0, ph1);
+        const uint32_t pKB = (uint32_t)p.e[i].K >> 7, base = p.e[i].base;
+        const uint32_t units = (((uint32_t)p.e[i].N + kUnitRows - 1u) / kUnitRows) * pKB;
+        const uint32_t lo = max(ph0, base), hi = min(ph1, base + units);
+        const uint32_t pu0 = lo - base, pn = hi > lo ? hi - lo : 0u;
         uint4 e = make_uint4(pu0, 0u, 0u, pKB << 16);
         if (pn != 0u) {
             e.y = pu0 / pKB;
@@ -492,11 +431,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
         for (int i = 0; i < kGroup; ++i) mbar_init(mdone0 + 8 * i, 1);
         for (int i = 0; i < kHandDepth; ++i) {
             mbar_init(hfull0 + 8 * i, 4);
-            mbar_init(hempty0 + 8 * i, 1);
+            mbar_init(hempty0 + 8 * i, 2);  // the team's publishing and completing warp
         }
         *poisoned = 0;
         for (int i = 0; i < 4 * kNG; ++i) tmem_slot[2 + i] = 0u;
-        if (blockIdx.x == 0) p.status[6] = (int)full0;  // (reference for the time-out diagnostics)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < p.xbufs * p.xbuf_bytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(xs)[i] = 0u;
@@ -510,14 +448,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-#ifdef QIL_TRACE
-    long long tr[16];
-    for (int i = 0; i < 16; ++i) tr[i] = 0;
-    const long long tr_begin = clock64();
-    const Guard guard{p.status, poisoned, &tr[15]};
-#else
-    const Guard guard{p.status, poisoned};
-#endif
+    const Guard guard{p.status, poisoned, p.wait_ns};
 
     if (tid < kUnpackThreads) {
         // ======================= unpack warpgroups: shared memory -> nibble split -> tensor memory =======================
@@ -537,12 +468,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 const uint32_t g = G + j / kGroup, a = (g % kNG) * kGroup + j % kGroup;
                 // the groups that used these columns before have been read out (by the epilogue warp of the same
                 // lanes); the unit has landed
-                if (!QIL_WAIT(1, guard.wait_count(rd0 + 4 * ((g % kNG) * 4 + (r >> 5)), g / kNG, dempty0 + 8 * (g % kNG))) ||
-                    !QIL_WAIT(2, guard.wait_mbar(full0 + 8 * st_i, st_ph))) {
+                if (!guard.wait_count(rd0 + 4 * ((g % kNG) * 4 + (r >> 5)), g / kNG, dempty0 + 8 * (g % kNG)) ||
+                    !guard.wait_mbar(full0 + 8 * st_i, st_ph)) {
                     alive = false;
                     break;
                 }
-                QIL_TR_COUNT(3);
                 tc_fence_after();
                 const unsigned char* ub = ring + (size_t)st_i * kUnitBytes;
                 const uint32_t ta = tmem + lane_base + 16 * a;
@@ -579,54 +509,31 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             stage0 = wrapped;
         }
     } else if (tid < kStagerBase) {
-        // ======================= epilogue warpgroups (thread = weight row of the unit) =======================
-        // With two warpgroups they take the CTA's linears in turn, each doing the whole read-out of its linears: the
-        // per-linear code of one then overlaps the units of the other.  Both keep count of the groups, activation
-        // buffers and hand-over buffers of the linears they skip.
-        const uint32_t ew = (uint32_t)(tid - kEpiBase) >> 7, r = (uint32_t)(tid - kEpiBase) & 127, lane = tid & 31;
+        // ======================= epilogue warpgroup (thread = weight row of the unit) =======================
+        const uint32_t r = (uint32_t)(tid - kEpiBase) & 127, lane = tid & 31;
         const uint32_t lane_base = (r & ~31u) << 16;
-        constexpr int kEBmax = kXR == 1 ? 4 : kXR == 2 ? 2 : 1;                      // (registers)
-        constexpr int kEB = QIL_TC_EPI_BATCH < kEBmax ? QIL_TC_EPI_BATCH : kEBmax;  // units read back per tcgen05.wait::ld
-        uint32_t hc = 0, G = 0;          // hc: per fixer warp, two bits counting the entries handed to it
-        uint32_t seq = 0;                // linears with units of this CTA so far
+        constexpr int kEB = 1;  // units read back per tcgen05.wait::ld
+        uint32_t hc = 0, G = 0;          // hc: per fixer team, two bits counting the entries handed to it
         Cyc xc(p.xbufs);
         bool alive = true;
         Walk wk(plan, p.count);
-#ifdef QIL_TRACE
-        long long tr_p0 = clock64();
-#endif
         while (alive && wk.next_entry()) {
-#ifdef QIL_TRACE
-            const long long tr_p1 = clock64();
-            tr[11] += tr_p1 - tr_p0;  // tail of the previous entry + next_entry
-#endif
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
             const uint32_t KB = wk.KB, u0 = wk.u0, u1 = wk.u1, n = u1 - u0;
             const uint32_t t_first = wk.t_first, t_last = wk.t_last;
             const bool shares = t_first * KB < u0 || (t_last + 1) * KB > u1;  // a row tile is shared with other CTAs
-#ifdef QIL_TRACE
-            uint32_t tr_keep = t_first + t_last + (shares ? 1u : 0u) + (uint32_t)M + (uint32_t)N;
-            asm volatile("" : "+r"(tr_keep));
-            const long long tr_p2 = clock64();
-            tr[12] += tr_p2 - tr_p1;  // entry fields and the two divisions
-#endif
             const uint32_t xb = xc.idx, xph = xc.ph;
             xc.step();
-            if (kNumEpi > 1 && (seq++ % kNumEpi) != ew) {  // the other warpgroup's linear
-                G += (n + kGroup - 1) / kGroup;
-                continue;
-            }
-            // hand-over buffers of the fixer warp: with one warpgroup its two buffers alternate; with two, each
-            // warpgroup has its own (a barrier is then only ever waited on by warps that saw its previous phase)
+            // the two hand-over buffers of the entry's fixer team alternate
             const uint32_t team = (uint32_t)wk.ei % kFixTeams, hcnt = (hc >> (2 * team)) & 3u;
             if (shares) hc = (hc & ~(3u << (2 * team))) | (((hcnt + 1u) & 3u) << (2 * team));
-            const uint32_t hbuf = 2 * team + (kNumEpi > 1 ? ew : (hcnt & 1u));
-            const uint32_t hph = kNumEpi > 1 ? (hcnt & 1u) : ((hcnt >> 1) & 1u);
-            if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xph))) break;
+            const uint32_t hbuf = 2 * team + (hcnt & 1u);
+            const uint32_t hph = (hcnt >> 1) & 1u;
+            if (!guard.wait_mbar(xfull0 + 8 * xb, xph)) break;
             const int2* xblk_b = xblk + (size_t)xb * kXR * p.nb_max;
             float* hand_b = hand + (size_t)hbuf * 2 * kXR * kUnitRows;
-            if (shares && !QIL_WAIT(2, guard.wait_mbar(hempty0 + 8 * hbuf, hph ^ 1u))) break;
+            if (shares && !guard.wait_mbar(hempty0 + 8 * hbuf, hph ^ 1u)) break;
             uint32_t n_full = 0;
             float fin[kXR];
 #pragma unroll
@@ -672,29 +579,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         fin[t] = fmaf((float)v, s * __int_as_float(xm.y), fin[t]);
                     }
             };
-#ifdef QIL_TRACE
-            asm volatile("" : "+r"(rt), "+r"(kb), "+r"(hc));
-            tr[13] += clock64() - tr_p2;  // waits for the activation and hand-over buffers, set-up
-#endif
             for (uint32_t j0 = 0; alive && j0 < n; j0 += kGroup, ++G) {
                 const uint32_t gs = G % kNG, nreal = min((uint32_t)kGroup, n - j0);
-                if constexpr (kNumEpi > 1) {
-                    // The columns' previous use may have been the other warpgroup's: wait until it has been read out,
-                    // so that the accumulation barrier is at most one phase behind (its parity cannot tell more).
-                    if (!QIL_WAIT(6, guard.wait_count(rd0 + 4 * (gs * 4 + (r >> 5)), G / kNG, dempty0 + 8 * gs))) {
-                        alive = false;
-                        break;
-                    }
-                }
-                if (!QIL_WAIT(3, guard.wait_mbar(dfull0 + 8 * gs, (G / kNG) & 1))) {  // all units of the group are accumulated
+                if (!guard.wait_mbar(dfull0 + 8 * gs, (G / kNG) & 1)) {  // all units of the group are accumulated
                     alive = false;
                     break;
                 }
                 tc_fence_after();
                 for (uint32_t b0 = 0; alive && b0 < nreal; b0 += kEB) {
-#ifdef QIL_TRACE
-                    const long long tr_e0 = clock64();
-#endif
                     uint32_t dr[kEB][8], dm[kEB][16], meta[kEB];
 #pragma unroll
                     for (int i = 0; i < kEB; ++i) {
@@ -731,28 +623,16 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                             sts_release(rd0 + 4 * (gs * 4 + (r >> 5)), G / kNG + 1);
                         }
                     }
-#ifdef QIL_TRACE
-                    const long long tr_e3 = clock64();
-                    tr[9] += tr_e3 - tr_e0;
-#endif
 #pragma unroll
                     for (int i = 0; i < kEB; ++i)
                         if (alive && b0 + i < nreal) {
-                            QIL_TR_COUNT(5);
                             consume(dr[i], dm[i], meta[i]);
                             if (++bi == KB) bi = 0;
                             if (++kb == KB || j0 + b0 + i + 1 == n) close_tile();
                         }
-#ifdef QIL_TRACE
-                    asm volatile("" : "+f"(fin[0]));
-                    tr[10] += clock64() - tr_e3;
-#endif
                 }
             }
             if (!alive) break;
-#ifdef QIL_TRACE
-            tr_p0 = clock64();
-#endif
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(xempty0 + 8 * xb);
@@ -782,17 +662,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             int2* xblk_b = xblk + (size_t)xb * kXR * p.nb_max;
             bool ok = true;
             if (lane == 0) {  // the buffer is free; the rows of x are written (quarter tiles of all earlier entries)
-                ok = QIL_WAIT(1, guard.wait_mbar(xempty0 + 8 * xb, xc.ph ^ 1));
+                ok = guard.wait_mbar(xempty0 + 8 * xb, xc.ph ^ 1);
                 if (ok && (E.flags & kFlagDep)) {
-                    const unsigned int need = 4u * E.tiles_before;
-                    ok = QIL_WAIT(2, guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; }));
+                    // (kFlagNever: a count that is never reached, so that this bounded wait runs out)
+                    const unsigned int need = (E.flags & kFlagNever) ? 0xFFFFFFFFu : 4u * E.tiles_before;
+                    ok = guard.wait_flag([&] { return ld_acquire(p.tiles_done) >= need; });
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-#ifdef QIL_TRACE
-            const long long tr_conv0 = clock64();
-#endif
             const uint32_t nblk = min(KB, wk.u1 - wk.u0), kb0 = wk.kb0;
             const uint32_t m = (uint32_t)l16 & 3;
             for (int t = 0; t < E.M; ++t) {
@@ -872,26 +750,23 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read xs through the async proxy
             __syncwarp();
-#ifdef QIL_TRACE
-            tr[3] += clock64() - tr_conv0;
-#endif
             if (lane == 0) mbar_arrive(xfull0 + 8 * xb);
             xc.step();
         }
     } else if (tid < kMmaBase) {
         // ======================= fixer warps (lane = four rows of the tile): all cross-CTA work =======================
-        // The shared tiles of an entry cost several round trips through the L2 (is the slot free, the other CTAs'
-        // parts, the output); the warps take the entries in turn so that these latencies overlap.
-        const uint32_t team = (uint32_t)(tid - kFixBase) >> 5, lane = tid & 31;
+        // Entry i's shared row tiles belong to team i % kFixTeams: its publishing warp hands the CTA's part of a tile
+        // that ends in another CTA over to that CTA, its completing warp finishes the tile that ends here.  The two
+        // are separate warps because completing waits for other CTAs and publishing must never wait behind it (CTA c
+        // would otherwise publish only after CTA c - 1 had, and so on down the grid).
+        const uint32_t fw = (uint32_t)(tid - kFixBase) >> 5, team = fw >> 1, lane = tid & 31;
+        const bool completer = (fw & 1u) != 0u;
         constexpr uint32_t kRowsPer = kUnitRows / 32;
-        constexpr uint32_t kPoll = 1;  // other CTAs' parts fetched together (more measured slower: the code grows)
         unsigned long long* slots = reinterpret_cast<unsigned long long*>(p.slots);
-        uint32_t cnt = 0, cntw[2] = {0u, 0u};  // entries this warp has taken over (in all / from each read-out warpgroup)
-        uint32_t seq = 0;                      // linears with units of this CTA so far
+        uint32_t cnt = 0;  // entries this team has taken over
         bool alive = true;
         Walk wk(plan, p.count);
         while (alive && wk.next_entry()) {
-            const uint32_t ow = kNumEpi > 1 ? (seq++ % kNumEpi) : 0u;  // read-out warpgroup of the linear
             if ((uint32_t)wk.ei % kFixTeams != team) continue;
             const TcEntry& E = p.e[wk.ei];
             const int M = E.M, N = E.N;
@@ -901,41 +776,52 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             const bool have_first = t_first * KB < u0 && (t_first + 1) * KB <= u1;  // completes a tile begun elsewhere
             if (!have_last && !(t_first * KB < u0)) continue;
             const uint32_t tag = (uint32_t)wk.ei + 1u, ring_i = (uint32_t)wk.ei % kSlotDepth;
-            const uint32_t hbuf = 2 * team + (kNumEpi > 1 ? ow : (cnt & 1u));
-            const uint32_t hph = kNumEpi > 1 ? (cntw[ow] & 1u) : ((cnt >> 1) & 1u);
+            const uint32_t hbuf = 2 * team + (cnt & 1u), hph = (cnt >> 1) & 1u;
+            ++cnt;
             const float* hand_b = hand + (size_t)hbuf * 2 * kXR * kUnitRows;
-            unsigned long long* my_slot = nullptr;
-            if (have_last) {
-                const uint32_t which = (t_last == t_first) ? 0u : 1u;
-                my_slot = slots + (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems;
-                // the slot must have been consumed (tags cleared) by whoever completed the tile it last served;
-                // checked now, while the units are still being computed
-                alive = QIL_WAIT(1, guard.wait_flag([&] {
-                    bool is_free = true;
-                    for (uint32_t h = 0; h < kRowsPer; ++h)
-                        for (int t = 0; t < kXR; ++t)
-                            if (t < M) is_free &= (uint32_t)(__ldcg(my_slot + t * kUnitRows + lane + 32 * h) >> 32) == 0u;
-                    return is_free;
-                }));
+            if (!completer) {
+                unsigned long long* my_slot = nullptr;
+                if (have_last) {
+                    const uint32_t which = (t_last == t_first) ? 0u : 1u;
+                    my_slot = slots + (((size_t)c * 2 + which) * kSlotDepth + ring_i) * kSlotElems;
+                    // the slot must have been consumed (tags cleared) by whoever completed the tile it last served;
+                    // checked now, while the units are still being computed
+                    alive = guard.wait_flag([&] {
+                        bool is_free = true;
+                        for (uint32_t h = 0; h < kRowsPer; ++h)
+                            for (int t = 0; t < kXR; ++t)
+                                if (t < M) is_free &= (uint32_t)(__ldcg(my_slot + t * kUnitRows + lane + 32 * h) >> 32) == 0u;
+                        return is_free;
+                    });
+                }
+                alive = alive && guard.wait_mbar(hfull0 + 8 * hbuf, hph);
+                alive = __all_sync(0xffffffffu, alive);
+                if (!alive) break;
+                if (have_last) {
+                    for (uint32_t h = 0; h < kRowsPer; ++h) {
+                        const uint32_t r = lane + 32 * h;
+                        for (int t = 0; t < M; ++t)
+                            __stcg(my_slot + t * kUnitRows + r,
+                                   ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(hand_b[(kXR + t) * kUnitRows + r]));
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(hempty0 + 8 * hbuf);
+                continue;
             }
-            alive = alive && QIL_WAIT(2, guard.wait_mbar(hfull0 + 8 * hbuf, hph));
+            // ---- completing warp ----
+            alive = guard.wait_mbar(hfull0 + 8 * hbuf, hph);
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
-            if (have_last) {  // publish first (a chain of CTAs must never wait on each other in a circle)
-                for (uint32_t h = 0; h < kRowsPer; ++h) {
-                    const uint32_t r = lane + 32 * h;
-                    for (int t = 0; t < M; ++t)
-                        __stcg(my_slot + t * kUnitRows + r,
-                               ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(hand_b[(kXR + t) * kUnitRows + r]));
-                }
-            }
             if (have_first) {
-                // the CTAs before this one that hold units of the tile (walked backwards: cheaper here than dividing)
+                // the CTAs before this one that hold units of the tile (walked backwards: cheaper here than dividing);
+                // slices are counted in units of the entry's phase, the tile begins at unit tile0 of the phase
+                const uint32_t tile0 = E.base + t_first * KB;
                 uint32_t c_lo = c;
                 while (c_lo > 0) {
                     uint32_t a0, a1;
                     slice_of(E.q, E.rem, c_lo - 1, a0, a1);
-                    if (a1 <= t_first * KB) break;
+                    if (a1 <= tile0) break;
                     --c_lo;
                 }
                 float sum[kRowsPer][kXR];
@@ -943,51 +829,38 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 for (uint32_t h = 0; h < kRowsPer; ++h)
 #pragma unroll
                     for (int t = 0; t < kXR; ++t) sum[h][t] = 0.f;
-                for (uint32_t cc0 = c_lo; cc0 < c; cc0 += kPoll) {
-                    unsigned long long* src[kPoll];
-                    unsigned long long got[kPoll][kRowsPer][kXR];
-#pragma unroll
-                    for (uint32_t k = 0; k < kPoll; ++k) {
-                        src[k] = nullptr;
-                        uint32_t cu0 = 0, cu1 = 0;
-                        if (cc0 + k < c) slice_of(E.q, E.rem, cc0 + k, cu0, cu1);
-                        if (cu0 != cu1) {
-                            const uint32_t which = (cu0 >= t_first * KB) ? 0u : 1u;  // the tile is that CTA's first or its last
-                            src[k] = slots + (((size_t)(cc0 + k) * 2 + which) * kSlotDepth + ring_i) * kSlotElems + lane;
-                        }
-                    }
-                    auto all_arrived = [&] {
+                for (uint32_t cc = c_lo; cc < c; ++cc) {
+                    uint32_t cu0, cu1;
+                    slice_of(E.q, E.rem, cc, cu0, cu1);
+                    if (cu0 == cu1) continue;
+                    // the tile is that CTA's first tile of the entry, or its last
+                    const uint32_t which = (max(cu0, E.base) >= tile0) ? 0u : 1u;
+                    unsigned long long* src = slots + (((size_t)cc * 2 + which) * kSlotDepth + ring_i) * kSlotElems + lane;
+                    unsigned long long got[kRowsPer][kXR];
+                    auto arrived = [&] {
                         bool all = true;
 #pragma unroll
-                        for (uint32_t k = 0; k < kPoll; ++k)
-                            if (src[k] != nullptr) {
+                        for (uint32_t h = 0; h < kRowsPer; ++h) {
 #pragma unroll
-                                for (uint32_t h = 0; h < kRowsPer; ++h) {
-#pragma unroll
-                                    for (int t = 0; t < kXR; ++t)
-                                        if (t < M) {
-                                            got[k][h][t] = __ldcg(src[k] + t * kUnitRows + 32 * h);
-                                            all &= (uint32_t)(got[k][h][t] >> 32) == tag;
-                                        }
+                            for (int t = 0; t < kXR; ++t)
+                                if (t < M) {
+                                    got[h][t] = __ldcg(src + t * kUnitRows + 32 * h);
+                                    all &= (uint32_t)(got[h][t] >> 32) == tag;
                                 }
-                            }
+                        }
                         return all;
                     };
-                    alive = QIL_WAIT(3, guard.wait_flag(all_arrived));
+                    alive = guard.wait_flag(arrived);
                     alive = __all_sync(0xffffffffu, alive);
                     if (!alive) break;
 #pragma unroll
-                    for (uint32_t k = 0; k < kPoll; ++k)  // (always summed in CTA order)
-                        if (src[k] != nullptr) {
+                    for (uint32_t h = 0; h < kRowsPer; ++h)  // (always summed in CTA order)
 #pragma unroll
-                            for (uint32_t h = 0; h < kRowsPer; ++h)
-#pragma unroll
-                                for (int t = 0; t < kXR; ++t)
-                                    if (t < M) {
-                                        sum[h][t] += __uint_as_float((uint32_t)got[k][h][t]);
-                                        __stcg(src[k] + t * kUnitRows + 32 * h, 0ull);  // consumed: the slot may be reused
-                                    }
-                        }
+                        for (int t = 0; t < kXR; ++t)
+                            if (t < M) {
+                                sum[h][t] += __uint_as_float((uint32_t)got[h][t]);
+                                __stcg(src + t * kUnitRows + 32 * h, 0ull);  // consumed: the slot may be reused
+                            }
                 }
                 if (!alive) break;
 #pragma unroll
@@ -1007,8 +880,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     red_release_add(p.tiles_done, kRowsPer);
                 }
             }
-            ++cnt;
-            ++cntw[ow];
         }
     } else if (tid < kProdBase) {
         // ======================= MMA issuers (one thread in each of kGroup warps) =======================
@@ -1027,7 +898,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             while (alive && wk.next_entry()) {
                 const uint32_t KB = wk.KB, n = wk.u1 - wk.u0;
                 const uint32_t xb = xc.idx;
-                if (!QIL_WAIT(1, guard.wait_mbar(xfull0 + 8 * xb, xc.ph))) break;
+                if (!guard.wait_mbar(xfull0 + 8 * xb, xc.ph)) break;
                 xc.step();
                 const uint32_t xr16 = smem_u32(xs + (size_t)xb * p.xbuf_bytes) >> 4;
                 const uint32_t xm16 = xr16 + (((uint32_t)p.nb_max * 4 * kLboR + 256) >> 4);
@@ -1040,14 +911,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                     const uint32_t gs = G % kNG, gph = (G / kNG) & 1;
                     if (j < n) {
                         const uint32_t a = gs * kGroup + w;
-                        if (!QIL_WAIT(2, guard.wait_mbar(afull0 + 8 * a, gph))) {  // (the unpack warps waited for the columns to be free)
+                        if (!guard.wait_mbar(afull0 + 8 * a, gph)) {  // (the unpack warps waited for the columns to be free)
                             alive = false;
                             break;
                         }
                         tc_fence_after();
-#ifdef QIL_TRACE
-                        const long long tr_m0 = clock64();
-#endif
                         const uint32_t ta = tmem + 16 * a, td = tmem + kColD + kDUnit * a;
                         // raw bytes of the unit in the ring: 16-byte chunk j at j * 2048, rows 16 bytes apart
                         const uint64_t a0 = desc_a | (uint64_t)(ring16 + st_i * (kUnitBytes >> 4));
@@ -1060,16 +928,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                         tc_commit(dfull0 + 8 * gs);
                         tc_commit(empty0 + 8 * st_i);  // the ring stage has been read
                         issued = true;
-#ifdef QIL_TRACE
-                        tr[4] += clock64() - tr_m0;
-                        tr[5] += 1;
-#endif
                     } else {
                         // The entry ends inside the group: this slot stays empty, its barriers still change phase.  Like
                         // the unpack warps the thread first waits until the groups that used these columns before have
                         // been read out: an arrival must never reach a barrier whose previous phase is still collecting.
                         for (uint32_t q = 0; alive && q < 4; ++q)
-                            alive = QIL_WAIT(2, guard.wait_count(rd0 + 4 * (gs * 4 + q), G / kNG, dempty0 + 8 * gs));
+                            alive = guard.wait_count(rd0 + 4 * (gs * 4 + q), G / kNG, dempty0 + 8 * gs);
                         if (!alive) break;
                         mbar_arrive_n(afull0 + 8 * (gs * kGroup + w), 4);
                         mbar_arrive(dfull0 + 8 * gs);
@@ -1087,7 +951,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             if (issued) {
                 tc_commit(mdone0 + 8 * w);
                 const unsigned long long t0 = Guard::now_ns();
-                while (!mbar_try_wait(mdone0 + 8 * w, 0) && Guard::now_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try_wait(mdone0 + 8 * w, 0) && Guard::now_ns() - t0 < kDefaultWaitLimitNs) {}
             }
         }
     } else {
@@ -1100,7 +964,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
             while (alive && wk.next_entry()) {
                 const unsigned char* wbase = p.e[wk.ei].w;
                 for (uint32_t u = wk.u0; u < wk.u1; ++u, ++issued) {
-                    if (!QIL_WAIT(1, guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1))) {
+                    if (!guard.wait_mbar(empty0 + 8 * rs.idx, rs.ph ^ 1)) {
                         alive = false;
                         break;
                     }
@@ -1116,17 +980,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_tc_kernel(const __grid_cons
                 if (rs.idx == 0) { rs.idx = p.stages; rs.ph ^= 1; }
                 --rs.idx;
                 const unsigned long long t0 = Guard::now_ns();
-                while (!mbar_try_wait(full0 + 8 * rs.idx, rs.ph) && Guard::now_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try_wait(full0 + 8 * rs.idx, rs.ph) && Guard::now_ns() - t0 < kDefaultWaitLimitNs) {}
             }
         }
     }
-#ifdef QIL_TRACE
-    tr[0] = clock64() - tr_begin;
-    if (p.trace && (tid & 31) == 0) {
-        unsigned long long* o = p.trace + ((size_t)blockIdx.x * 32 + (tid >> 5)) * 16;
-        for (int i = 0; i < 16; ++i) o[i] = (unsigned long long)tr[i];
-    }
-#endif
     // nobody leaves before every copy has landed and every role is done; then tensor memory is released
     tc_fence_before();
     __syncthreads();
@@ -1166,9 +1023,6 @@ __global__ void __launch_bounds__(256) pack_stream128_kernel(const uint8_t* __re
     }
 }
 
-#ifdef QIL_TRACE
-unsigned long long* g_trace = nullptr;
-#endif
 
 struct SmemPlan {
     int x_rows, xbuf_bytes, stages, xbufs;
@@ -1197,13 +1051,30 @@ SmemPlan plan_for(int max_m, int nb_max, int xbufs) {
     return pl;
 }
 
+// All CTAs of the kernel wait on each other (slots, dependency counter), so they must be resident together: the
+// launch is cooperative, which the driver refuses when the grid does not fit the device as it is.
 template <int kXR>
 cudaError_t launch_one(const TcParams& p, int C, size_t smem, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(w4a16_tc_kernel<kXR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    w4a16_tc_kernel<kXR><<<C, kThreads, smem, st>>>(p);
-    return cudaGetLastError();
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, w4a16_tc_kernel<kXR>, kThreads, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)C);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, w4a16_tc_kernel<kXR>, p);
 }
+
+std::atomic<unsigned long long> g_wait_ns{kDefaultWaitLimitNs};
 
 }  // namespace
 
@@ -1232,66 +1103,101 @@ qil_status launch_pack_stream128_w4(const uint8_t* codes, const void* scales, co
     return launch_status();
 }
 
-// Every entry must satisfy w4a16_tc_supported().  entries[i].flags bit 0 = QIL_DEP_PREVIOUS.
+void w4a16_tc_set_wait_limit(unsigned long long ns) { g_wait_ns.store(ns ? ns : kDefaultWaitLimitNs); }
+
+// Every entry must satisfy w4a16_tc_supported().  entries[i].flags: QIL_DEP_PREVIOUS, QIL_DEP_NEVER.
+//
+// How the units are dealt out.  A phase is a maximal run of entries of which only the first may carry
+// QIL_DEP_PREVIOUS: its entries do not depend on each other, so their units form one stream that is cut into one
+// contiguous, balanced slice per CTA.  A CTA then meets few entries per phase (on a list without dependencies: two or
+// three in the whole launch), and the cost a CTA pays per entry it takes part in - activation conversion, row tiles
+// shared with its neighbours - is paid rarely.  The price is an activation buffer that holds all K / 128 blocks of
+// an entry; where that leaves too shallow a weight ring every entry is its own phase.
 qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, size_t ws_bytes, cudaStream_t st) {
     if (ws == nullptr || ws_bytes < w4a16_tc_workspace()) return QIL_ERR_WORKSPACE;
     static TcParams p;  // 14 KiB: kept off the caller's stack; guarded by the mutex below
     static std::mutex mu;
     std::lock_guard<std::mutex> lock(mu);
-    const int C = num_sms();
-    for (int base = 0; base < count; base += kMaxEntries) {
-        const int n = count - base < kMaxEntries ? count - base : kMaxEntries;
-        int max_m = 1, nb_max = 1;
+    const uint32_t C = (uint32_t)num_sms();
+    for (int first = 0; first < count; first += kMaxEntries) {
+        const int n = count - first < kMaxEntries ? count - first : kMaxEntries;
+        int max_m = 1;
         bool any_dep = false;
         uint32_t tiles = 0;
+        uint32_t units[kMaxEntries];
         for (int i = 0; i < n; ++i) {
-            const qil_linear_desc& d = entries[base + i];
+            const qil_linear_desc& d = entries[first + i];
             TcEntry& e = p.e[i];
             e.x = reinterpret_cast<const uint16_t*>(d.x);
             e.w = reinterpret_cast<const unsigned char*>(d.qweight);
             e.y = reinterpret_cast<__nv_bfloat16*>(d.y);
             e.N = d.N; e.K = d.K; e.M = d.M;
-            e.flags = (i > 0) ? (d.flags & kFlagDep) : 0;  // earlier launches are ordered by the stream
+            e.flags = (i > 0) ? (d.flags & (kFlagDep | kFlagNever)) : 0;  // earlier launches are ordered by the stream
+            if (e.flags & kFlagNever) e.flags |= kFlagDep;
             e.tiles_before = tiles;
             const uint32_t row_tiles = (uint32_t)((d.N + kUnitRows - 1) / kUnitRows);
-            const uint32_t units = row_tiles * (uint32_t)(d.K / 128);
-            e.q = units / (uint32_t)C;
-            e.rem = units % (uint32_t)C;
-            e.pad = 0;
-            if (e.q >= 65535u || d.K / 128 >= 65536) return QIL_ERR_UNSUPPORTED;  // (16-bit fields of the slice table)
+            units[i] = row_tiles * (uint32_t)(d.K / 128);
+            if (d.K / 128 >= 65536) return QIL_ERR_UNSUPPORTED;  // (16-bit fields of the slice table)
             tiles += row_tiles;
             any_dep |= (e.flags & kFlagDep) != 0;
             if (d.M > max_m) max_m = d.M;
-            const int nb = (int)std::min<uint32_t>((uint32_t)(d.K / 128), e.q + (e.rem ? 1u : 0u));  // blocks a CTA touches
-            if (nb > nb_max) nb_max = nb;
         }
+        // slices per phase (merged) or per entry; returns the blocks an activation buffer must hold, 0 if a field overflows
+        auto deal = [&](bool merged) -> int {
+            int nb_max = 1;
+            for (int i = 0; i < n;) {
+                int j = i + 1;
+                while (merged && j < n && !(p.e[j].flags & kFlagDep)) ++j;
+                uint64_t total = 0;
+                for (int k = i; k < j; ++k) total += units[k];
+                if (total > 0xFFFFFFFFull) return 0;
+                const uint32_t q = (uint32_t)total / C, rem = (uint32_t)total % C;
+                uint32_t base = 0;
+                for (int k = i; k < j; ++k) {
+                    p.e[k].q = q; p.e[k].rem = rem; p.e[k].base = base;
+                    base += units[k];
+                    const uint32_t most = std::min<uint32_t>(units[k], q + (rem ? 1u : 0u));  // units one CTA holds of the entry
+                    if (most >= 65536u) return 0;
+                    const int nb = (int)std::min<uint32_t>((uint32_t)(entries[first + k].K / 128), most);
+                    if (nb > nb_max) nb_max = nb;
+                }
+                i = j;
+            }
+            return nb_max;
+        };
         // as many activation buffers as leave a deep weight ring
-        SmemPlan pl = plan_for(max_m, nb_max, kMaxXBufs);
-        // (with two read-out warpgroups an even number: a buffer is then always read by the same warpgroup)
-        for (int xb = kMaxXBufs - 1; xb >= 2 && pl.stages < 12; --xb)
-            if (kNumEpi == 1 || xb % 2 == 0) pl = plan_for(max_m, nb_max, xb);
+        auto best_plan = [&](int nb_max) {
+            SmemPlan pl = plan_for(max_m, nb_max, kMaxXBufs);
+            for (int xb = kMaxXBufs - 1; xb >= 2 && pl.stages < 12; --xb) pl = plan_for(max_m, nb_max, xb);
+            return pl;
+        };
+        int nb_max = deal(true);
+        SmemPlan pl = nb_max > 0 ? best_plan(nb_max) : SmemPlan{};
+        if (nb_max == 0 || pl.stages < 12) {
+            nb_max = deal(false);
+            if (nb_max == 0) return QIL_ERR_UNSUPPORTED;
+            pl = best_plan(nb_max);
+        }
         if (pl.stages < 4) return QIL_ERR_UNSUPPORTED;
         p.count = n;
         p.stages = pl.stages;
         p.nb_max = nb_max;
         p.xbufs = pl.xbufs;
         p.xbuf_bytes = pl.xbuf_bytes;
+        p.wait_ns = g_wait_ns.load();
         p.status = reinterpret_cast<int*>(ws);
         p.tiles_done = any_dep ? reinterpret_cast<unsigned int*>(ws) + 1 : nullptr;
         p.slots = reinterpret_cast<unsigned char*>(ws) + kWsHeader;
-#ifdef QIL_TRACE
-        p.trace = g_trace;
-#endif
         if (any_dep && cudaMemsetAsync(reinterpret_cast<unsigned int*>(ws) + 1, 0, 4, st) != cudaSuccess) {
             (void)cudaGetLastError();
             return QIL_ERR_CUDA;
         }
-        const cudaError_t err = pl.x_rows == 1   ? launch_one<1>(p, C, pl.total, st)
-                                : pl.x_rows == 2 ? launch_one<2>(p, C, pl.total, st)
-                                                 : launch_one<4>(p, C, pl.total, st);
+        const cudaError_t err = pl.x_rows == 1   ? launch_one<1>(p, (int)C, pl.total, st)
+                                : pl.x_rows == 2 ? launch_one<2>(p, (int)C, pl.total, st)
+                                                 : launch_one<4>(p, (int)C, pl.total, st);
         if (err != cudaSuccess) {
             (void)cudaGetLastError();
-            return QIL_ERR_CUDA;
+            return err == cudaErrorCooperativeLaunchTooLarge ? QIL_ERR_UNSUPPORTED : QIL_ERR_CUDA;
         }
     }
     return QIL_OK;
@@ -1299,6 +1205,3 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
 
 }  // namespace qil
 
-#ifdef QIL_TRACE
-extern "C" void qil_trace_set_tc(unsigned long long* t) { qil::g_trace = t; }
-#endif

@@ -161,6 +161,69 @@ int qo_quantize_sym4(const float* v, int R, int K, int G, int scale_f16,
     return bad;
 }
 
+/* ---- the same two quantisers on a grid of 2^bits levels (bits = 4 or 8): the 8-bit deployment
+ * points of the paper (INT8 weight-only OpenVLA, W8A8 CILRS; Sec. 5.4) ---- */
+int qo_quantize_rtn_asym(const float* w, int N, int K, int G, int bits,
+                         uint8_t* codes, uint16_t* scales, uint16_t* zeros) {
+    int ng = K / G;
+    int bad = 0;
+    const float top = (float)((1 << bits) - 1);
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (int n = 0; n < N; ++n) {
+        for (int g = 0; g < ng; ++g) {
+            const float* p = w + (size_t)n * K + (size_t)g * G;
+            float lo = 0.0f, hi = 0.0f;
+            for (int k = 0; k < G; ++k) {
+                if (p[k] < lo) lo = p[k];
+                if (p[k] > hi) hi = p[k];
+            }
+            float r = hi - lo;
+            float s32 = r / top;
+            uint16_t s16 = qo_f32_to_f16(s32);
+            if ((s16 & 0x7FFFu) == 0x7C00u) bad |= 1;
+            if ((s16 & 0x7FFFu) == 0) s16 = 0x3C00u;
+            float s = qo_f16_to_f32(s16);
+            float z = qo_clampf(rintf(-lo / s), 0.0f, top);
+            for (int k = 0; k < G; ++k) {
+                float q = qo_clampf(rintf(p[k] / s) + z, 0.0f, top);
+                codes[(size_t)n * K + (size_t)g * G + k] = (uint8_t)q;
+            }
+            scales[(size_t)n * ng + g] = s16;
+            zeros[(size_t)n * ng + g] = qo_f32_to_f16((float)(int)z);
+        }
+    }
+    return bad;
+}
+
+void qo_quantize_sym(const float* v, int R, int K, int G, int bits, const float* static_scale,
+                     int8_t* codes, float* scales) {
+    int ng = K / G;
+    const float qmax = (float)((1 << (bits - 1)) - 1), qmin = -(float)(1 << (bits - 1));
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < R; ++r) {
+        for (int g = 0; g < ng; ++g) {
+            const float* p = v + (size_t)r * K + (size_t)g * G;
+            float s;
+            if (static_scale) {
+                s = *static_scale;
+            } else {
+                float a = 0.0f;
+                for (int k = 0; k < G; ++k) {
+                    float t = fabsf(p[k]);
+                    if (t > a) a = t;
+                }
+                s = a / qmax;
+                if (a == 0.0f) s = 1.0f;
+            }
+            scales[(size_t)r * ng + g] = s;
+            for (int k = 0; k < G; ++k) {
+                float q = qo_clampf(rintf(p[k] / s), qmin, qmax);
+                codes[(size_t)r * K + (size_t)g * G + k] = (int8_t)q;
+            }
+        }
+    }
+}
+
 /* ---- packing: element k of a row -> word k/8, bits [4(k%8), 4(k%8)+3] ---- */
 void qo_pack_w4(const uint8_t* codes, int R, int K, uint32_t* packed) {
     int W = K / 8;

@@ -116,3 +116,44 @@ def linear_w4a4(qx, sx, qw, sw, want_y=True):
     y = np.empty((M, N), np.float64) if want_y else None
     load().qo_linear_w4a4(_p(qx), _p(sx), _p(qw), _p(sw), M, N, K, _p(acc), _p(y) if want_y else None)
     return acc, y
+
+
+# ---- 8-bit variants (the C loops of the two linears do not depend on the code width) ----
+def quantize_rtn_asym(w, group_size, bits):
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    N, K = w.shape
+    ng = K // group_size
+    codes = np.empty((N, K), np.uint8)
+    scales = np.empty((N, ng), np.uint16)
+    zeros = np.empty((N, ng), np.uint16)
+    rc = load().qo_quantize_rtn_asym(_p(w), N, K, int(group_size), int(bits), _p(codes), _p(scales), _p(zeros))
+    if rc:
+        raise OverflowError("scale does not fit fp16")
+    return codes, scales.view(np.float16), zeros.view(np.float16)
+
+
+def quantize_rtn_w8_asym(w, group_size):
+    return quantize_rtn_asym(w, group_size, 8)
+
+
+def quantize_sym(v, bits, group_size=None, static_scale=None):
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    R, K = v.shape
+    G = K if group_size is None else int(group_size)
+    codes = np.empty((R, K), np.int8)
+    scales = np.empty((R, K // G), np.float32)
+    ss = None if static_scale is None else C.byref(C.c_float(static_scale))
+    load().qo_quantize_sym(_p(v), R, K, G, int(bits), ss, _p(codes), _p(scales))
+    return codes, scales
+
+
+def quantize_sym8(v, group_size=None, static_scale=None):
+    return quantize_sym(v, 8, group_size, static_scale)
+
+
+def linear_w8a16(x_bf16_bits, codes, scales, zeros, group_size):
+    return linear_w4a16(x_bf16_bits, codes, scales, zeros, group_size)
+
+
+def linear_w8a8(qx, sx, qw, sw, want_y=True):
+    return linear_w4a4(qx, sx, qw, sw, want_y)

@@ -272,6 +272,96 @@ def linear_w4a4(qx, sx, qw, sw):
     return acc, y
 
 
-def row_tolerance(y_ref: np.ndarray, rel: float = 1e-2) -> np.ndarray:
-    """Per-row allowance of the acceptance rule: rel * max_n |y_ref[m][n]|."""
-    return rel * np.abs(np.asarray(y_ref, dtype=np.float64)).max(axis=1, keepdims=True)
+# ----------------------------------------------------------------------------
+# 8-bit variants: the paper's other two deployment points (Table "OpenVLA
+# performance", INT8 weight-only row; Table "CILRS performance", W8A8 row;
+# Sec. 5.4 "Implementation").  Same round-to-nearest uniform quantiser (Sec. 2.1)
+# on a grid of 2^8 levels; the operation list is the 4-bit one with 15 -> 255
+# and (-8, 7, divisor 7) -> (-128, 127, divisor 127).
+# ----------------------------------------------------------------------------
+def quantize_rtn_asym(w: np.ndarray, group_size: int, bits: int):
+    """w fp32 [N][K] -> (codes u8 [N][K] in 0..L, scales f16 [N][K/G], zeros f16 [N][K/G]), L = 2^bits - 1.
+
+    Per (row n, group g):
+      lo = min(0, min w), hi = max(0, max w)
+      s32 = (hi - lo) / L             (fp32)
+      s16 = fp16(s32); 0 -> 1.0; inf -> error
+      z   = clamp(rint(-lo / s16), 0, L)
+      q_k = clamp(rint(w_k / s16) + z, 0, L)
+    """
+    if bits not in (4, 8):
+        raise ValueError("bits must be 4 or 8")
+    L = F32(2 ** bits - 1)
+    w = np.ascontiguousarray(w, dtype=F32)
+    N, K = w.shape
+    G = int(group_size)
+    if G <= 0 or K % G != 0:
+        raise ValueError("group_size must divide K")
+    ng = K // G
+    wg = w.reshape(N, ng, G)
+    lo = np.minimum(F32(0), wg.min(axis=2)).astype(F32)
+    hi = np.maximum(F32(0), wg.max(axis=2)).astype(F32)
+    r = (hi - lo).astype(F32)
+    s32 = (r / L).astype(F32)
+    with np.errstate(over="ignore"):
+        s16 = s32.astype(np.float16)
+    if np.isinf(s16).any():
+        raise OverflowError("scale does not fit fp16")
+    s16 = np.where(s16 == np.float16(0), np.float16(1.0), s16).astype(np.float16)
+    s = s16.astype(F32)
+    z = np.clip(np.rint((-lo / s).astype(F32)), F32(0), L).astype(F32)
+    u = (np.rint((wg / s[:, :, None]).astype(F32)) + z[:, :, None]).astype(F32)
+    q = np.clip(u, F32(0), L)
+    return q.astype(np.uint8).reshape(N, K), s16, z.astype(np.uint8).astype(np.float16)
+
+
+def quantize_rtn_w8_asym(w: np.ndarray, group_size: int):
+    return quantize_rtn_asym(w, group_size, 8)
+
+
+def quantize_sym(v: np.ndarray, bits: int, group_size: int | None = None, static_scale: float | None = None):
+    """v fp32 [R][K] -> (codes int8 [R][K] in -2^(b-1) .. 2^(b-1)-1, fp32 scales [R][K/G]).
+
+    Per (row, group): a = max|v|; s = a / (2^(b-1) - 1) (fp32); a == 0 -> s = 1; with ``static_scale`` every group
+    uses that value.  q = clamp(rint(v / s), -2^(b-1), 2^(b-1) - 1).
+    """
+    if bits not in (4, 8):
+        raise ValueError("bits must be 4 or 8")
+    qmax = F32(2 ** (bits - 1) - 1)
+    qmin = F32(-(2 ** (bits - 1)))
+    v = np.ascontiguousarray(v, dtype=F32)
+    R, K = v.shape
+    G = K if group_size is None else int(group_size)
+    if G <= 0 or K % G != 0:
+        raise ValueError("group_size must divide K")
+    ng = K // G
+    vg = v.reshape(R, ng, G)
+    if static_scale is not None:
+        s = np.full((R, ng), F32(static_scale), dtype=F32)
+    else:
+        a = np.abs(vg).max(axis=2).astype(F32)
+        s = (a / qmax).astype(F32)
+        s = np.where(a == F32(0), F32(1.0), s).astype(F32)
+    q = np.clip(np.rint((vg / s[:, :, None]).astype(F32)), qmin, qmax)
+    return q.astype(np.int8).reshape(R, K), s
+
+
+def quantize_sym8(v: np.ndarray, group_size: int | None = None, static_scale: float | None = None):
+    return quantize_sym(v, 8, group_size, static_scale)
+
+
+def dequant_asym(codes, scales, zeros, group_size: int) -> np.ndarray:
+    """W_hat[n][k] = (q - z) * s in fp64, for codes of any width."""
+    return dequant_w4_asym(codes, scales, zeros, group_size)
+
+
+def linear_w8a16(x_bf16_bits, codes, scales, zeros, group_size: int) -> np.ndarray:
+    """y[m][n] = sum_k x[m][k] * (q[n][k] - z[n][k/G]) * s[n][k/G] with 8-bit codes, fp64 throughout."""
+    x = bf16_to_f32(x_bf16_bits).astype(np.float64)
+    w_hat = dequant_asym(codes, scales, zeros, group_size)
+    return np.matmul(x, w_hat.T)
+
+
+def linear_w8a8(qx, sx, qw, sw):
+    """acc[m][n] = sum_k qx[m][k]*qw[n][k] (int64, |acc| <= 2^14 K); y = acc * sx[m] * sw[n] (fp64)."""
+    return linear_w4a4(qx, sx, qw, sw)

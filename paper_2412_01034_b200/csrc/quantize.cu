@@ -1,9 +1,11 @@
 // Round-to-nearest 4-bit quantisers and the nibble packer (paper Sec. 2.1).
 //
-// The fp32 operation order is the one documented in qil.h; every division is an
-// IEEE division (__fdiv_rn) and rounding to integer is rintf (ties to even), so
-// the codes are reproducible bit for bit.  No step here may be contracted into a
-// fused multiply-add or replaced by a reciprocal.
+// The fp32 operation order is the one documented in qil.h; every result equals that of an
+// IEEE division (__fdiv_rn) followed by rintf (ties to even), so the codes are reproducible
+// bit for bit.  No step is contracted into a fused multiply-add.  The activation quantiser
+// has one fast path: it multiplies by a reciprocal and keeps that result only when it is
+// provably the same integer (the product is far enough from a rounding boundary), and falls
+// back to the exact division otherwise (rint_div below).
 #include "qil_common.cuh"
 
 namespace qil {

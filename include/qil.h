@@ -240,6 +240,43 @@ qil_status qil_linear_w4a16_batch_host(const qil_linear_desc* descs /*host*/, in
                                        void* workspace, size_t workspace_bytes, qil_stream_t stream);
 
 /* ------------------------------------------------------------------------
+ * 8-bit weight-only linear (the INT8 deployment point of Table "OpenVLA
+ * performance", Sec. 5.4): the same round-to-nearest quantiser on 256 levels,
+ * and the linear with uint8 codes, one per byte.
+ * qil_quantize_rtn_w8: arguments and errors as qil_quantize_rtn_w4.
+ *   symmetric = 0: codes 0..255, s = fp16_rn((hi - lo) / 255), z = clamp(rint(-lo / s), 0, 255);
+ *   symmetric = 1: codes -128..127 (int8), s = max|v| / 127.
+ * qil_linear_w8a16: y[M][N] bf16 = x[M][K] bf16 . dequant(W)^T, fp32 result rounded to bf16.
+ *   codes [N][K] uint8 row-major, scales and zeros [N][K/group_size] fp16.
+ *   With K % 128 == 0 and group_size % 128 == 0 (and K small enough for the activations of four rows to fit
+ *   shared memory: K <= 24576) a streaming kernel runs, four activation rows per pass: it converts the
+ *   activations to 16-bit block fixed point per 128 columns (error at most 2^-16 of the block maximum) and
+ *   accumulates integer dot products exactly.  Other shapes (K % 16 == 0) use a general kernel.
+ *   workspace: qil_linear_w8a16_workspace_size() bytes, zero-filled once; its first int is the status word
+ *   (QIL_ERR_TIMEOUT if a bounded wait ran out), its second a counter the list kernel uses between phases.
+ * qil_linear_w8a16_batch: a list in stream order, flags as for qil_linear_w4a16_batch (layout must be
+ *   QIL_LAYOUT_CANONICAL; desc.qweight points at the uint8 codes).  When every entry fits the streaming kernel
+ *   (M <= 4) the list is one cooperative launch of one CTA per SM; rows are dealt out whole, so CTAs exchange
+ *   nothing but the phase counter.
+ * Errors: NULL, SHAPE (K % 16, K % group_size), ALIGN, UNSUPPORTED, WORKSPACE, CUDA.
+ * ---------------------------------------------------------------------- */
+qil_status qil_quantize_rtn_w8(const void* w, qil_dtype w_dtype, int N, int K, int group_size,
+                               int symmetric, uint8_t* codes, void* scales, qil_dtype scale_dtype,
+                               void* zeros, int* dev_status, qil_stream_t stream);
+size_t qil_linear_w8a16_workspace_size(void);
+qil_status qil_linear_w8a16(const void* x, const uint8_t* qweight, const void* scales, const void* zeros,
+                            void* y, int M, int N, int K, int group_size, void* workspace,
+                            size_t workspace_bytes, qil_stream_t stream);
+qil_status qil_linear_w8a16_batch(const qil_linear_desc* descs /*host*/, int count, void* workspace,
+                                  size_t workspace_bytes, qil_stream_t stream);
+
+/* Per-token symmetric int8 activation quantiser of the W8A8 path (Table "CILRS performance", W8A8 row):
+ * x [M][K] bf16 -> qx [M][K] int8, scales [M] fp32; divisor 127, clamp to [-128, 127]; static_scale as for
+ * qil_quantize_act_a4. */
+qil_status qil_quantize_act_a8(const void* x, int M, int K, const float* static_scale /*host*/, int8_t* qx,
+                               float* scales, qil_stream_t stream);
+
+/* ------------------------------------------------------------------------
  * Activation quantiser of the W4A4 path (Sec. 5.1: the compute-bound driving
  * policy needs weights and activations in 4 bits): symmetric int4 per row.
  *   x [M][K] bf16 -> qx packed [M][K/8] (canonical), scales [M] fp32.

@@ -22,6 +22,11 @@ SIGNATURES = {
     "qil_set_wait_limit_ns": (_i, [C.c_ulonglong]),
     "qil_linear_w4a16_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
     "qil_linear_w4a16_batch_host": (_i, [_vp, _i, _vp, _vp, _sz, _vp, _vp, _sz, _vp, _sz, _vp]),
+    "qil_quantize_rtn_w8": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _i, _vp, _vp, _vp]),
+    "qil_linear_w8a16_workspace_size": (_sz, []),
+    "qil_linear_w8a16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_linear_w8a16_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
+    "qil_quantize_act_a8": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),
     "qil_quantize_act_a4": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),
     "qil_linear_w4a4_workspace_size": (_sz, [_i, _i, _i]),
     "qil_linear_w4a4": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),

@@ -78,6 +78,55 @@ def quantize_rtn_w4(w, group_size: int, symmetric: bool = False, scale_dtype=Non
     return codes, scales, zeros
 
 
+def quantize_rtn_w8(w, group_size: int, symmetric: bool = False, scale_dtype=None, stream=None):
+    """Round-to-nearest 8-bit weight quantiser: (codes uint8 0..255 / int8 -128..127, scales, zeros or None)."""
+    lib = _lib.load()
+    _need_cuda(w)
+    N, K = w.shape
+    if scale_dtype is None:
+        scale_dtype = torch.float32 if symmetric else torch.float16
+    if group_size <= 0 or K % group_size != 0:
+        _check(2)
+    ng = K // group_size
+    codes = torch.empty((N, K), dtype=torch.int8 if symmetric else torch.uint8, device=w.device)
+    scales = torch.empty((N, ng), dtype=scale_dtype, device=w.device)
+    zeros = None if symmetric else torch.empty((N, ng), dtype=torch.float16, device=w.device)
+    status = torch.zeros(1, dtype=torch.int32, device=w.device)
+    _check(lib.qil_quantize_rtn_w8(_ptr(w), _DT[w.dtype], N, K, int(group_size), int(bool(symmetric)), _ptr(codes),
+                                   _ptr(scales), _DT[scale_dtype], _ptr(zeros), _ptr(status), _stream(stream)))
+    out = C.c_int(0)
+    _check(lib.qil_device_status(_ptr(status), C.byref(out), _stream(stream)))
+    if out.value:
+        raise QilError(ERR_RANGE if out.value & ERR_RANGE else out.value)
+    return codes, scales, zeros
+
+
+def linear_w8a16(x, codes, scales, zeros, group_size: int, out=None, workspace=None, stream=None):
+    """y[M][N] (bf16) = x[M][K] (bf16) . dequant(W)^T with 8-bit group-quantised W (codes uint8 [N][K])."""
+    _need_cuda(x, codes, scales, zeros, out, workspace)
+    M, K = x.shape
+    N = codes.shape[0]
+    lib = _lib.load()
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    if workspace is None:
+        workspace = new_workspace(int(lib.qil_linear_w8a16_workspace_size()), x.device)
+    _check(lib.qil_linear_w8a16(_ptr(x), _ptr(codes), _ptr(scales), _ptr(zeros), _ptr(out), M, N, K, int(group_size),
+                                _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+    return out
+
+
+def quantize_act_a8(x, static_scale: float | None = None, stream=None):
+    """bf16 x [M][K] -> (int8 codes [M][K], scales [M] fp32)."""
+    _need_cuda(x)
+    M, K = x.shape
+    qx = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    scales = torch.empty((M,), dtype=torch.float32, device=x.device)
+    ss = None if static_scale is None else C.byref(C.c_float(static_scale))
+    _check(_lib.load().qil_quantize_act_a8(_ptr(x), M, K, ss, _ptr(qx), _ptr(scales), _stream(stream)))
+    return qx, scales
+
+
 def pack_w4(codes, layout: int = LAYOUT_CANONICAL, stream=None):
     """codes [N][K] (uint8 or int8) -> packed words: [N][K/8] (canonical) or flat [N*K/8] (TILE16)."""
     _need_cuda(codes)

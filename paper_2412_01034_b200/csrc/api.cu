@@ -62,6 +62,7 @@ int qil_version(void) { return 100; }
 
 qil_status qil_set_wait_limit_ns(unsigned long long ns) {
     w4a16_tc_set_wait_limit(ns);
+    w8a16_set_wait_limit(ns);
     return QIL_OK;
 }
 
@@ -85,8 +86,22 @@ qil_status qil_quantize_rtn_w4(const void* w, qil_dtype w_dtype, int N, int K, i
     if (!symmetric && scale_dtype != QIL_F16) return QIL_ERR_UNSUPPORTED;
     if (symmetric && scale_dtype == QIL_BF16) return QIL_ERR_UNSUPPORTED;
     if (!aligned16(w) || !aligned16(codes) || !aligned16(scales) || (zeros && !aligned16(zeros))) return QIL_ERR_ALIGN;
-    return launch_quantize_rtn_w4(w, w_dtype, N, K, group_size, symmetric, codes, scales, scale_dtype, zeros,
-                                  dev_status, S(stream));
+    return launch_quantize_rtn(w, w_dtype, N, K, group_size, symmetric, 4, codes, scales, scale_dtype, zeros,
+                               dev_status, S(stream));
+}
+
+qil_status qil_quantize_rtn_w8(const void* w, qil_dtype w_dtype, int N, int K, int group_size, int symmetric,
+                               uint8_t* codes, void* scales, qil_dtype scale_dtype, void* zeros,
+                               int* dev_status, qil_stream_t stream) {
+    if (!w || !codes || !scales) return QIL_ERR_NULL;
+    if (!symmetric && !zeros) return QIL_ERR_NULL;
+    if (N <= 0 || K <= 0 || group_size <= 0 || K % group_size != 0) return QIL_ERR_SHAPE;
+    if (!dtype_ok(w_dtype) || !dtype_ok(scale_dtype)) return QIL_ERR_UNSUPPORTED;
+    if (!symmetric && scale_dtype != QIL_F16) return QIL_ERR_UNSUPPORTED;
+    if (symmetric && scale_dtype == QIL_BF16) return QIL_ERR_UNSUPPORTED;
+    if (!aligned16(w) || !aligned16(codes) || !aligned16(scales) || (zeros && !aligned16(zeros))) return QIL_ERR_ALIGN;
+    return launch_quantize_rtn(w, w_dtype, N, K, group_size, symmetric, 8, codes, scales, scale_dtype, zeros,
+                               dev_status, S(stream));
 }
 
 static qil_status check_pack(const void* a, const void* b, int N, int K, qil_layout layout) {
@@ -223,6 +238,78 @@ qil_status qil_linear_w4a16_batch_host(const qil_linear_desc* descs, int count, 
         return QIL_ERR_CUDA;
     }
     return QIL_OK;
+}
+
+static qil_status check_w8a16(const void* x, const void* qw, const void* sc, const void* z, const void* y, int M, int N,
+                              int K, int G) {
+    if (!x || !qw || !y || !sc || !z) return QIL_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || G <= 0 || K % 16 != 0 || K % G != 0) return QIL_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(qw) || !aligned16(y) || !aligned16(sc) || !aligned16(z)) return QIL_ERR_ALIGN;
+    return QIL_OK;
+}
+
+size_t qil_linear_w8a16_workspace_size(void) { return w8a16_workspace(); }
+
+// One linear: the streaming kernel in slabs of four activation rows where the shape allows it, the general kernel
+// otherwise.
+static qil_status w8a16_one(const qil_linear_desc& d, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (!w8a16_stream_supported(1, d.N, d.K, d.group_size))
+        return launch_w8a16_general(d.x, reinterpret_cast<const uint8_t*>(d.qweight), d.scales, d.zeros, d.y, d.M, d.N, d.K,
+                                    d.group_size, st);
+    for (int m0 = 0; m0 < d.M; m0 += 4) {
+        qil_linear_desc s = d;
+        s.x = static_cast<const char*>(d.x) + (size_t)m0 * d.K * 2;
+        s.y = static_cast<char*>(d.y) + (size_t)m0 * d.N * 2;
+        s.M = d.M - m0 < 4 ? d.M - m0 : 4;
+        s.flags = 0;
+        const qil_status r = launch_w8a16_stream(&s, 1, workspace, workspace_bytes, st);
+        if (r != QIL_OK) return r;
+    }
+    return QIL_OK;
+}
+
+qil_status qil_linear_w8a16(const void* x, const uint8_t* qweight, const void* scales, const void* zeros, void* y, int M,
+                            int N, int K, int group_size, void* workspace, size_t workspace_bytes, qil_stream_t stream) {
+    const qil_status s = check_w8a16(x, qweight, scales, zeros, y, M, N, K, group_size);
+    if (s != QIL_OK) return s;
+    if (!workspace || workspace_bytes < w8a16_workspace()) return QIL_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return QIL_ERR_ALIGN;
+    qil_linear_desc d;
+    d.x = x; d.qweight = reinterpret_cast<const uint32_t*>(qweight); d.scales = scales; d.zeros = zeros; d.y = y;
+    d.M = M; d.N = N; d.K = K; d.group_size = group_size; d.layout = QIL_LAYOUT_CANONICAL; d.flags = 0;
+    return w8a16_one(d, workspace, workspace_bytes, S(stream));
+}
+
+qil_status qil_linear_w8a16_batch(const qil_linear_desc* descs, int count, void* workspace, size_t workspace_bytes,
+                                  qil_stream_t stream) {
+    if (!descs) return QIL_ERR_NULL;
+    if (count <= 0) return QIL_ERR_SHAPE;
+    if (!workspace || workspace_bytes < w8a16_workspace()) return QIL_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return QIL_ERR_ALIGN;
+    bool all_stream = true;
+    for (int i = 0; i < count; ++i) {
+        const qil_linear_desc& d = descs[i];
+        if ((d.flags & ~(QIL_DEP_PREVIOUS | QIL_DEP_NEVER)) != 0 || d.layout != QIL_LAYOUT_CANONICAL) return QIL_ERR_UNSUPPORTED;
+        const qil_status s = check_w8a16(d.x, d.qweight, d.scales, d.zeros, d.y, d.M, d.N, d.K, d.group_size);
+        if (s != QIL_OK) return s;
+        all_stream = all_stream && w8a16_stream_supported(d.M, d.N, d.K, d.group_size);
+    }
+    if (all_stream) return launch_w8a16_stream(descs, count, workspace, workspace_bytes, S(stream));
+    for (int i = 0; i < count; ++i) {  // stream order keeps every dependency
+        const qil_status s = w8a16_one(descs[i], workspace, workspace_bytes, S(stream));
+        if (s != QIL_OK) return s;
+    }
+    return QIL_OK;
+}
+
+qil_status qil_quantize_act_a8(const void* x, int M, int K, const float* static_scale, int8_t* qx, float* scales,
+                               qil_stream_t stream) {
+    if (!x || !qx || !scales) return QIL_ERR_NULL;
+    if (M <= 0 || K <= 0 || K % 8 != 0) return QIL_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(qx) || !aligned16(scales)) return QIL_ERR_ALIGN;
+    if (static_scale && !(*static_scale > 0.0f)) return QIL_ERR_UNSUPPORTED;
+    return launch_quantize_act_a8(x, M, K, static_scale != nullptr, static_scale ? *static_scale : 0.0f, qx, scales,
+                                  S(stream));
 }
 
 qil_status qil_quantize_act_a4(const void* x, int M, int K, const float* static_scale, uint32_t* qx, float* scales,

@@ -51,14 +51,24 @@ __device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
 }
 
 // Internal launchers (one per translation unit).
-qil_status launch_quantize_rtn_w4(const void* w, qil_dtype w_dtype, int N, int K, int G, int symmetric,
-                                  uint8_t* codes, void* scales, qil_dtype scale_dtype, void* zeros,
-                                  int* dev_status, cudaStream_t st);
+qil_status launch_quantize_rtn(const void* w, qil_dtype w_dtype, int N, int K, int G, int symmetric, int bits,
+                               uint8_t* codes, void* scales, qil_dtype scale_dtype, void* zeros,
+                               int* dev_status, cudaStream_t st);
 qil_status launch_pack_w4(const uint8_t* codes, int N, int K, qil_layout layout, uint32_t* packed, cudaStream_t st);
 qil_status launch_unpack_w4(const uint32_t* packed, int N, int K, qil_layout layout, int is_signed,
                             uint8_t* codes, cudaStream_t st);
 qil_status launch_quantize_act_a4(const void* x, int M, int K, bool use_static, float static_scale,
                                   uint32_t* qx, float* scales, cudaStream_t st);
+
+qil_status launch_quantize_act_a8(const void* x, int M, int K, bool use_static, float static_scale, int8_t* qx,
+                                  float* scales, cudaStream_t st);
+
+bool w8a16_stream_supported(int M, int N, int K, int G);
+size_t w8a16_workspace();
+void w8a16_set_wait_limit(unsigned long long ns);
+qil_status launch_w8a16_general(const void* x, const uint8_t* w, const void* s, const void* z, void* y, int M, int N, int K,
+                                int G, cudaStream_t st);
+qil_status launch_w8a16_stream(const qil_linear_desc* entries, int count, void* ws, size_t ws_bytes, cudaStream_t st);
 
 qil_status launch_w4a16_general(const void* x, const uint32_t* qw, const void* scales, const void* zeros,
                                 void* y, int M, int N, int K, int G, cudaStream_t st);

@@ -40,7 +40,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) quantize_asym_kernel(const T* __restrict__ w, int N, int K, int G,
                                                             uint8_t* __restrict__ codes,
                                                             __half* __restrict__ scales,
-                                                            __half* __restrict__ zeros, int* status) {
+                                                            __half* __restrict__ zeros, int* status, float top) {
+    // top = 15 (4-bit) or 255 (8-bit): the highest level of the grid
     const int lane = threadIdx.x & 31;
     const int ng = K / G;
     const long long total = (long long)N * ng;
@@ -56,13 +57,13 @@ __global__ void __launch_bounds__(256) quantize_asym_kernel(const T* __restrict_
         lo = warp_min(lo);
         hi = warp_max(hi);
         const float r = __fsub_rn(hi, lo);
-        const float s32 = __fdiv_rn(r, 15.0f);
+        const float s32 = __fdiv_rn(r, top);
         __half s16;
         const float s = round_scale_f16(s32, &s16, lane == 0 ? status : nullptr);
-        const float z = clampf(rintf(__fdiv_rn(-lo, s)), 0.0f, 15.0f);
+        const float z = clampf(rintf(__fdiv_rn(-lo, s)), 0.0f, top);
         for (int k = lane; k < G; k += 32) {
             float v = load_f32<T>(w, base + k);
-            float q = clampf(__fadd_rn(rintf(__fdiv_rn(v, s)), z), 0.0f, 15.0f);
+            float q = clampf(__fadd_rn(rintf(__fdiv_rn(v, s)), z), 0.0f, top);
             codes[base + k] = (uint8_t)(int)q;
         }
         if (lane == 0) {
@@ -72,11 +73,11 @@ __global__ void __launch_bounds__(256) quantize_asym_kernel(const T* __restrict_
     }
 }
 
-// One warp per (row, group).  Symmetric int4, divisor 7, clamp to [-8, 7].
+// One warp per (row, group).  Symmetric: divisor qmax = 7 (4-bit) or 127 (8-bit), clamp to [-qmax - 1, qmax].
 template <typename T, bool kScaleF16>
 __global__ void __launch_bounds__(256) quantize_sym_kernel(const T* __restrict__ v, int R, int K, int G,
                                                            int8_t* __restrict__ codes, void* __restrict__ scales,
-                                                           int* status) {
+                                                           int* status, float qmax) {
     const int lane = threadIdx.x & 31;
     const int ng = K / G;
     const long long total = (long long)R * ng;
@@ -86,7 +87,7 @@ __global__ void __launch_bounds__(256) quantize_sym_kernel(const T* __restrict__
         float a = 0.0f;
         for (int k = lane; k < G; k += 32) a = fmaxf(a, fabsf(load_f32<T>(v, base + k)));
         a = warp_max(a);
-        float s = __fdiv_rn(a, 7.0f);
+        float s = __fdiv_rn(a, qmax);
         if (a == 0.0f) s = 1.0f;
         if (kScaleF16) {
             __half s16;
@@ -96,7 +97,7 @@ __global__ void __launch_bounds__(256) quantize_sym_kernel(const T* __restrict__
             reinterpret_cast<float*>(scales)[grp] = s;
         }
         for (int k = lane; k < G; k += 32) {
-            float q = clampf(rintf(__fdiv_rn(load_f32<T>(v, base + k), s)), -8.0f, 7.0f);
+            float q = clampf(rintf(__fdiv_rn(load_f32<T>(v, base + k), s)), -qmax - 1.0f, qmax);
             codes[base + k] = (int8_t)(int)q;
         }
     }
@@ -262,6 +263,50 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
     }
 }
 
+// Per-token symmetric int8 of bf16 activations (divisor 127), one code per byte.  One warp per row; the same
+// division rule as the 4-bit quantiser (rint_div).
+__global__ void __launch_bounds__(256) quantize_act_a8_kernel(const __nv_bfloat16* __restrict__ x, int M, int K,
+                                                              bool use_static, float static_scale,
+                                                              int8_t* __restrict__ qx, float* __restrict__ scales) {
+    const int lane = threadIdx.x & 31;
+    const int words = K >> 3;  // 8 elements = one 16-byte load, one 8-byte store
+    const int warps = gridDim.x * (blockDim.x >> 5);
+    for (int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); m < M; m += warps) {
+        const uint4* row = reinterpret_cast<const uint4*>(x + (size_t)m * K);
+        float s;
+        if (use_static) {
+            s = static_scale;
+        } else {
+            uint32_t amax = 0;  // bf16 magnitudes order like unsigned integers
+            for (int i = lane; i < words; i += 32) {
+                const uint4 v = __ldg(row + i);
+                const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) amax = max(amax, max((u[j] << 16) & 0x7FFFFFFFu, u[j] & 0x7FFF0000u));
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            const float a = __uint_as_float(amax);
+            s = __fdiv_rn(a, 127.0f);
+            if (a == 0.0f) s = 1.0f;
+        }
+        const float inv_s = __frcp_rn(s);
+        for (int i = lane; i < words; i += 32) {
+            const uint4 v = __ldg(row + i);
+            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+            uint32_t out[2] = {0u, 0u};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int q0 = (int)clampf(rint_div(__uint_as_float(u[j] << 16), s, inv_s), -128.0f, 127.0f);
+                const int q1 = (int)clampf(rint_div(__uint_as_float(u[j] & 0xFFFF0000u), s, inv_s), -128.0f, 127.0f);
+                out[j >> 1] |= (((uint32_t)q0 & 0xFFu) | (((uint32_t)q1 & 0xFFu) << 8)) << (16 * (j & 1));
+            }
+            *reinterpret_cast<uint2*>(qx + (size_t)m * K + (size_t)i * 8) = make_uint2(out[0], out[1]);
+        }
+        if (lane == 0) scales[m] = s;
+    }
+}
+
 inline int grid_for(long long work_items, int per_block) {
     long long blocks = (work_items + per_block - 1) / per_block;
     long long cap = (long long)num_sms() * 16;
@@ -272,18 +317,19 @@ inline int grid_for(long long work_items, int per_block) {
 
 }  // namespace
 
-qil_status launch_quantize_rtn_w4(const void* w, qil_dtype w_dtype, int N, int K, int G, int symmetric,
-                                  uint8_t* codes, void* scales, qil_dtype scale_dtype, void* zeros,
-                                  int* dev_status, cudaStream_t st) {
+qil_status launch_quantize_rtn(const void* w, qil_dtype w_dtype, int N, int K, int G, int symmetric, int bits,
+                               uint8_t* codes, void* scales, qil_dtype scale_dtype, void* zeros,
+                               int* dev_status, cudaStream_t st) {
+    const float top = bits == 8 ? 255.0f : 15.0f, qmax = bits == 8 ? 127.0f : 7.0f;
     const long long groups = (long long)N * (K / G);
     const int grid = grid_for(groups, 8);
 #define QIL_ASYM(T)                                                                                  \
     quantize_asym_kernel<T><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(w), N, K, G, codes,     \
                                                   reinterpret_cast<__half*>(scales),                 \
-                                                  reinterpret_cast<__half*>(zeros), dev_status)
+                                                  reinterpret_cast<__half*>(zeros), dev_status, top)
 #define QIL_SYM(T, F16)                                                                              \
     quantize_sym_kernel<T, F16><<<grid, 256, 0, st>>>(reinterpret_cast<const T*>(w), N, K, G,        \
-                                                      reinterpret_cast<int8_t*>(codes), scales, dev_status)
+                                                      reinterpret_cast<int8_t*>(codes), scales, dev_status, qmax)
     if (!symmetric) {
         if (w_dtype == QIL_F32) QIL_ASYM(float);
         else if (w_dtype == QIL_BF16) QIL_ASYM(__nv_bfloat16);
@@ -328,6 +374,13 @@ qil_status launch_quantize_act_a4(const void* x, int M, int K, bool use_static, 
 #undef QIL_ACT_CACHED
     quantize_act_kernel<<<grid_for(M, 8), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), M, K,
                                                         use_static, static_scale, qx, scales);
+    return launch_status();
+}
+
+qil_status launch_quantize_act_a8(const void* x, int M, int K, bool use_static, float static_scale, int8_t* qx,
+                                  float* scales, cudaStream_t st) {
+    quantize_act_a8_kernel<<<grid_for(M, 8), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), M, K, use_static,
+                                                           static_scale, qx, scales);
     return launch_status();
 }
 

@@ -22,8 +22,10 @@ class QuantisedLinears:
     def __init__(self, cfg: int = 1, M: int = 1, n_layers: int = wl.N_LAYERS, layout: int = api.LAYOUT_STREAM128,
                  deps: str = "none",
                  outliers: bool = True, device: str = "cuda", keep_host_rows: dict | None = None,
-                 host_threads: int | None = None):
-        self.M, self.layout, self.device = M, layout, device
+                 host_threads: int | None = None, bits: int = 4):
+        if bits == 8:
+            layout = api.LAYOUT_CANONICAL   # 8-bit codes are one byte each, row-major
+        self.M, self.layout, self.device, self.bits = M, layout, device, bits
         self.lib = _lib.load()
         self.specs = [s for s in wl.llama_linear_ids() if s[0] < n_layers]
         self.G = wl.GROUP_SIZE
@@ -47,8 +49,10 @@ class QuantisedLinears:
                     rows = np.asarray(keep_host_rows[i])
                     self.kept[i] = (rows, w[rows].copy())
                 wd = torch.from_numpy(w).to(device)
-                codes, s, z = api.quantize_rtn_w4(wd, self.G)
-                if layout == api.LAYOUT_STREAM128:
+                codes, s, z = api.quantize_rtn_w8(wd, self.G) if bits == 8 else api.quantize_rtn_w4(wd, self.G)
+                if bits == 8:
+                    self.packed.append(codes)
+                elif layout == api.LAYOUT_STREAM128:
                     self.packed.append(api.pack_stream128_w4(codes, s, z, self.G))
                 else:
                     self.packed.append(api.pack_w4(codes, layout))
@@ -74,7 +78,10 @@ class QuantisedLinears:
         self.x_dev = self.x_host.to(device)
         self.y_dev = torch.zeros(yo, dtype=torch.bfloat16, device=device)
 
-        ws_bytes = max(api.linear_w4a16_workspace_size(M, N, K, self.G) for (_, _, N, K, _, _) in self.specs)
+        if bits == 8:
+            ws_bytes = int(self.lib.qil_linear_w8a16_workspace_size())
+        else:
+            ws_bytes = max(api.linear_w4a16_workspace_size(M, N, K, self.G) for (_, _, N, K, _, _) in self.specs)
         self.ws = api.new_workspace(ws_bytes, device)
         self.ws_bytes = self.ws.numel()
 
@@ -113,7 +120,7 @@ class QuantisedLinears:
 
     def weight_bytes(self) -> int:
         """Algorithmic weight-side bytes of one pass: packed codes + fp16 scales + fp16 zeros."""
-        return sum(N * K // 2 + 4 * N * (K // self.G) for (_, _, N, K, _, _) in self.specs)
+        return sum(N * K * self.bits // 8 + 4 * N * (K // self.G) for (_, _, N, K, _, _) in self.specs)
 
     def algorithmic_bytes(self) -> int:
         """weight_bytes + activations read + outputs written (bf16)."""
@@ -123,8 +130,8 @@ class QuantisedLinears:
     def run(self, stream=None) -> None:
         """One pass over all linears, activations already on the device."""
         s = torch.cuda.current_stream() if stream is None else stream
-        api._check(self.lib.qil_linear_w4a16_batch(self.descs, self.count, C.c_void_p(self.ws.data_ptr()),
-                                                   self.ws_bytes, C.c_void_p(s.cuda_stream)))
+        fn = self.lib.qil_linear_w8a16_batch if self.bits == 8 else self.lib.qil_linear_w4a16_batch
+        api._check(fn(self.descs, self.count, C.c_void_p(self.ws.data_ptr()), self.ws_bytes, C.c_void_p(s.cuda_stream)))
 
     def run_host(self, stream=None) -> None:
         """One pass with activations in (pinned) host memory: H2D copy, linears, D2H copy."""

@@ -93,3 +93,17 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(_lib, "LIB_PATH", str(tmp_path / "libqil.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         _lib.load()
+
+
+def test_w8_validation(lib):
+    f = lib.qil_linear_w8a16
+    assert f(None, A, A, A, A, 1, 16, 128, 128, A, 256, None) == 1
+    assert f(A, A, A, A, A, 1, 16, 120, 120, A, 256, None) == 2          # K % 16
+    assert f(A, A, A, A, A, 1, 16, 128, 96, A, 256, None) == 2           # group does not divide K
+    assert f(A, A, A, A, A, 1, 16, 128, 128, None, 0, None) == 5         # workspace
+    assert f(U, A, A, A, A, 1, 16, 128, 128, A, 256, None) == 3
+    assert lib.qil_linear_w8a16_workspace_size() >= 8
+    assert lib.qil_linear_w8a16_batch(None, 1, A, 256, None) == 1
+    assert lib.qil_quantize_rtn_w8(A, 0, 4, 8, 3, 0, A, A, 2, A, None, None) == 2
+    assert lib.qil_quantize_act_a8(A, 4, 12, None, A, A, None) == 2
+    assert lib.qil_set_wait_limit_ns(0) == 0

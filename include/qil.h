@@ -123,7 +123,8 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  *   y [M][N] bf16
  * The kernel is chosen from the shape: on the canonical layout with M > 16,
  * K % 64 == 0 and group_size % 64 == 0 the tcgen05 prefill GEMM (weights
- * dequantised to bf16, one rounding per weight); else the tensor-core skinny
+ * dequantised to bf16, one rounding per weight; K split over several CTAs where
+ * that fills the GPU, partial tiles added in a fixed order); else the tensor-core skinny
  * kernel (weights read once, any M handled in slabs of 64 rows) when
  * K % 128 == 0 and group_size % 128 == 0; a general kernel otherwise (any
  * K % 8 == 0, any group_size dividing K, canonical layout only).  With
@@ -252,8 +253,11 @@ qil_status qil_linear_w4a16_batch_host(const qil_linear_desc* descs /*host*/, in
  *   shared memory: K <= 24576) a streaming kernel runs, four activation rows per pass: it converts the
  *   activations to 16-bit block fixed point per 128 columns (error at most 2^-16 of the block maximum) and
  *   accumulates integer dot products exactly.  Other shapes (K % 16 == 0) use a general kernel.
- *   workspace: qil_linear_w8a16_workspace_size() bytes, zero-filled once; its first int is the status word
- *   (QIL_ERR_TIMEOUT if a bounded wait ran out), its second a counter the list kernel uses between phases.
+ *   With M > 16, K % 64 == 0 and group_size % 64 == 0 the tcgen05 prefill GEMM of qil_linear_w4a16 runs on the
+ *   8-bit codes (weights dequantised to bf16, one rounding per weight).
+ *   workspace: qil_linear_w8a16_workspace_size() bytes (at least 256), zero-filled once; its first int is the
+ *   status word (QIL_ERR_TIMEOUT if a bounded wait ran out), its second a counter the list kernel uses between
+ *   phases, the rest scratch of the prefill GEMM's split along K.
  * qil_linear_w8a16_batch: a list in stream order, flags as for qil_linear_w4a16_batch (layout must be
  *   QIL_LAYOUT_CANONICAL; desc.qweight points at the uint8 codes).  When every entry fits the streaming kernel
  *   (M <= 4) the list is one cooperative launch of one CTA per SM; rows are dealt out whole, so CTAs exchange
@@ -263,7 +267,7 @@ qil_status qil_linear_w4a16_batch_host(const qil_linear_desc* descs /*host*/, in
 qil_status qil_quantize_rtn_w8(const void* w, qil_dtype w_dtype, int N, int K, int group_size,
                                int symmetric, uint8_t* codes, void* scales, qil_dtype scale_dtype,
                                void* zeros, int* dev_status, qil_stream_t stream);
-size_t qil_linear_w8a16_workspace_size(void);
+size_t qil_linear_w8a16_workspace_size(int M, int N, int K, int group_size);
 qil_status qil_linear_w8a16(const void* x, const uint8_t* qweight, const void* scales, const void* zeros,
                             void* y, int M, int N, int K, int group_size, void* workspace,
                             size_t workspace_bytes, qil_stream_t stream);
@@ -305,6 +309,13 @@ qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* 
                            void* y, int32_t* acc_out, int M, int N, int K, void* workspace,
                            size_t workspace_bytes, qil_stream_t stream);
 
+/* W8A8 integer GEMM (Table "CILRS performance", W8A8 row; Sec. 5.4): as qil_linear_w4a4 with one signed byte per
+ * element: qx [M][K], qw [N][K] int8; acc exact in int32 (|acc| <= 2^14 K: K < 131072), K % 16 == 0; the same
+ * workspace (qil_linear_w4a4_workspace_size). */
+qil_status qil_linear_w8a8(const int8_t* qx, const float* sx, const int8_t* qw, const float* sw, void* y,
+                           int32_t* acc_out, int M, int N, int K, void* workspace, size_t workspace_bytes,
+                           qil_stream_t stream);
+
 /* ------------------------------------------------------------------------
  * Helpers
  * ---------------------------------------------------------------------- */
@@ -322,6 +333,13 @@ qil_status qil_set_wait_limit_ns(unsigned long long ns);
  * streaming pass over `bytes` bytes that adds every 32-bit word into *sink. */
 qil_status qil_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, qil_stream_t stream);
 qil_status qil_probe_hbm_read(const void* buf, size_t bytes, unsigned int* sink, qil_stream_t stream);
+/* Tensor-core roofs: one CTA per SM issues `iters` x 4 tcgen05.mma (128 x 256, K = 32 bytes each) over operand
+ * tiles resident in shared memory, kind::i8 resp. kind::f16 with bf16 operands, with a tcgen05.commit every
+ * `commit_every` iterations (8 for the roof; 1 shows what a commit per pipeline step costs).  *ops_out (host, optional)
+ * receives the operations of the launch (2 per multiply-add); the caller times the launch.  dev_status
+ * (device, optional) receives QIL_ERR_TIMEOUT if a bounded wait ran out. */
+qil_status qil_probe_mma_i8(int iters, int commit_every, double* ops_out /*host*/, int* dev_status, qil_stream_t stream);
+qil_status qil_probe_mma_bf16(int iters, int commit_every, double* ops_out /*host*/, int* dev_status, qil_stream_t stream);
 
 #ifdef __cplusplus
 }

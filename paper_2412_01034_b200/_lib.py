@@ -23,18 +23,21 @@ SIGNATURES = {
     "qil_linear_w4a16_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
     "qil_linear_w4a16_batch_host": (_i, [_vp, _i, _vp, _vp, _sz, _vp, _vp, _sz, _vp, _sz, _vp]),
     "qil_quantize_rtn_w8": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _i, _vp, _vp, _vp]),
-    "qil_linear_w8a16_workspace_size": (_sz, []),
+    "qil_linear_w8a16_workspace_size": (_sz, [_i, _i, _i, _i]),
     "qil_linear_w8a16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w8a16_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
     "qil_quantize_act_a8": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),
     "qil_quantize_act_a4": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),
     "qil_linear_w4a4_workspace_size": (_sz, [_i, _i, _i]),
     "qil_linear_w4a4": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_linear_w8a8": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "qil_status_string": (C.c_char_p, [_i]),
     "qil_version": (_i, []),
     "qil_device_status": (_i, [_vp, C.POINTER(C.c_int), _vp]),
     "qil_ref_gemv_bf16": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "qil_probe_hbm_read": (_i, [_vp, _sz, _vp, _vp]),
+    "qil_probe_mma_i8": (_i, [_i, _i, C.POINTER(C.c_double), _vp, _vp]),
+    "qil_probe_mma_bf16": (_i, [_i, _i, C.POINTER(C.c_double), _vp, _vp]),
 }
 
 

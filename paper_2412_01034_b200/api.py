@@ -110,7 +110,7 @@ def linear_w8a16(x, codes, scales, zeros, group_size: int, out=None, workspace=N
     if out is None:
         out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
     if workspace is None:
-        workspace = new_workspace(int(lib.qil_linear_w8a16_workspace_size()), x.device)
+        workspace = new_workspace(int(lib.qil_linear_w8a16_workspace_size(M, N, K, int(group_size))), x.device)
     _check(lib.qil_linear_w8a16(_ptr(x), _ptr(codes), _ptr(scales), _ptr(zeros), _ptr(out), M, N, K, int(group_size),
                                 _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
     return out
@@ -215,6 +215,21 @@ def linear_w4a4(qx, sx, qw, sw, want_acc: bool = False, out=None, workspace=None
     return (out, acc) if want_acc else out
 
 
+def linear_w8a8(qx, sx, qw, sw, want_acc: bool = False, out=None, workspace=None, stream=None):
+    """Integer GEMM of int8 operands (qx [M][K], qw [N][K]); returns y (bf16) or (y, acc int32)."""
+    _need_cuda(qx, sx, qw, sw, out, workspace)
+    M, K = qx.shape
+    N = qw.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=qx.device)
+    acc = torch.empty((M, N), dtype=torch.int32, device=qx.device) if want_acc else None
+    if workspace is None:
+        workspace = new_workspace(linear_w4a4_workspace_size(M, N, K), qx.device)
+    _check(_lib.load().qil_linear_w8a8(_ptr(qx), _ptr(sx), _ptr(qw), _ptr(sw), _ptr(out), _ptr(acc), M, N, K,
+                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+    return (out, acc) if want_acc else out
+
+
 def ref_gemv_bf16(x, w, out=None, stream=None):
     _need_cuda(x, w, out)
     N, K = w.shape
@@ -227,3 +242,12 @@ def ref_gemv_bf16(x, w, out=None, stream=None):
 def probe_hbm_read(buf, sink, stream=None):
     _need_cuda(buf, sink)
     _check(_lib.load().qil_probe_hbm_read(_ptr(buf), buf.numel() * buf.element_size(), _ptr(sink), _stream(stream)))
+
+
+def probe_mma(kind: str, iters: int, commit_every: int = 8, status=None, stream=None) -> float:
+    """Launches the tensor-core probe ("i8" or "bf16"); returns the operations of the launch (the caller times it)."""
+    lib = _lib.load()
+    ops = C.c_double(0.0)
+    fn = lib.qil_probe_mma_i8 if kind == "i8" else lib.qil_probe_mma_bf16
+    _check(fn(int(iters), int(commit_every), C.byref(ops), _ptr(status), _stream(stream)))
+    return float(ops.value)

@@ -158,7 +158,12 @@ static qil_status check_w4a16(const void* x, const void* qw, const void* sc, con
 size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size) {
     if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0) return 0;
     if (K % 128 != 0 || group_size % 128 != 0) return 0;
-    return w4a16_skinny_ws_offset() + w4a16_skinny_workspace(M, N, K, group_size);  // serves every layout
+    size_t scratch = w4a16_skinny_workspace(M, N, K, group_size);
+    if (w4a16_prefill_supported(M, N, K, group_size, QIL_LAYOUT_CANONICAL)) {
+        const size_t pf = w4a16_prefill_workspace(M, N, K);
+        if (pf > scratch) scratch = pf;
+    }
+    return w4a16_skinny_ws_offset() + scratch;  // serves every layout
 }
 
 qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* scales, const void* zeros, void* y,
@@ -173,9 +178,14 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
         d.M = M; d.N = N; d.K = K; d.group_size = group_size; d.layout = layout; d.flags = 0;
         return launch_w4a16_tc(&d, 1, workspace, workspace_bytes, S(stream));
     }
-    if (w4a16_prefill_supported(M, N, K, group_size, layout))
-        return launch_w4a16_prefill(x, qweight, scales, zeros, y, M, N, K, group_size,
-                                    workspace_bytes >= sizeof(int) ? workspace : nullptr, S(stream));
+    if (w4a16_prefill_supported(M, N, K, group_size, layout)) {
+        const size_t off = w4a16_skinny_ws_offset();
+        const bool have = workspace != nullptr && workspace_bytes > off;
+        return launch_w4a16_prefill(x, qweight, scales, zeros, y, M, N, K, group_size, 4,
+                                    workspace_bytes >= sizeof(int) ? static_cast<int*>(workspace) : nullptr,
+                                    have ? static_cast<char*>(workspace) + off : nullptr, have ? workspace_bytes - off : 0,
+                                    S(stream));
+    }
     if (w4a16_skinny_supported(M, N, K, group_size, layout)) {
         const size_t off = w4a16_skinny_ws_offset();
         const bool have = workspace != nullptr && workspace_bytes > off;
@@ -248,11 +258,23 @@ static qil_status check_w8a16(const void* x, const void* qw, const void* sc, con
     return QIL_OK;
 }
 
-size_t qil_linear_w8a16_workspace_size(void) { return w8a16_workspace(); }
+size_t qil_linear_w8a16_workspace_size(int M, int N, int K, int group_size) {
+    if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0) return 0;
+    size_t scratch = 0;
+    if (w4a16_prefill_supported(M, N, K, group_size, QIL_LAYOUT_CANONICAL)) scratch = w4a16_prefill_workspace(M, N, K);
+    return w8a16_workspace() + scratch;
+}
 
 // One linear: the streaming kernel in slabs of four activation rows where the shape allows it, the general kernel
 // otherwise.
 static qil_status w8a16_one(const qil_linear_desc& d, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (w4a16_prefill_supported(d.M, d.N, d.K, d.group_size, QIL_LAYOUT_CANONICAL)) {  // M > 16: the tensor-core GEMM
+        const size_t off = w8a16_workspace();
+        const bool have = workspace_bytes > off;
+        return launch_w4a16_prefill(d.x, d.qweight, d.scales, d.zeros, d.y, d.M, d.N, d.K, d.group_size, 8,
+                                    static_cast<int*>(workspace), have ? static_cast<char*>(workspace) + off : nullptr,
+                                    have ? workspace_bytes - off : 0, st);
+    }
     if (!w8a16_stream_supported(1, d.N, d.K, d.group_size))
         return launch_w8a16_general(d.x, reinterpret_cast<const uint8_t*>(d.qweight), d.scales, d.zeros, d.y, d.M, d.N, d.K,
                                     d.group_size, st);
@@ -338,7 +360,20 @@ qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* 
         return QIL_ERR_ALIGN;
     if (w4a4_workspace(M, N, K) > 0 && (!workspace || workspace_bytes < w4a4_workspace(M, N, K)))
         return QIL_ERR_WORKSPACE;
-    return launch_w4a4(qx, sx, qw, sw, y, acc_out, M, N, K, workspace, workspace_bytes, S(stream));
+    return launch_w4a4(qx, sx, qw, sw, y, acc_out, M, N, K, 4, workspace, workspace_bytes, S(stream));
+}
+
+qil_status qil_linear_w8a8(const int8_t* qx, const float* sx, const int8_t* qw, const float* sw, void* y,
+                           int32_t* acc_out, int M, int N, int K, void* workspace, size_t workspace_bytes,
+                           qil_stream_t stream) {
+    if (!qx || !sx || !qw || !sw || !y) return QIL_ERR_NULL;
+    // (|acc| <= 2^14 K must stay below 2^31)
+    if (M <= 0 || N <= 0 || K <= 0 || K % 16 != 0 || K >= 131072) return QIL_ERR_SHAPE;
+    if (!aligned16(qx) || !aligned16(sx) || !aligned16(qw) || !aligned16(sw) || !aligned16(y) ||
+        (acc_out && !aligned16(acc_out)) || (workspace && !aligned16(workspace)))
+        return QIL_ERR_ALIGN;
+    if (!workspace || workspace_bytes < w4a4_workspace(M, N, K)) return QIL_ERR_WORKSPACE;
+    return launch_w4a4(qx, sx, qw, sw, y, acc_out, M, N, K, 8, workspace, workspace_bytes, S(stream));
 }
 
 qil_status qil_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, qil_stream_t stream) {
@@ -346,6 +381,16 @@ qil_status qil_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K
     if (N <= 0 || K <= 0 || K % 8 != 0) return QIL_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return QIL_ERR_ALIGN;
     return launch_ref_gemv_bf16(x, w, y, N, K, S(stream));
+}
+
+qil_status qil_probe_mma_i8(int iters, int commit_every, double* ops_out, int* dev_status, qil_stream_t stream) {
+    if (iters <= 0 || iters > (1 << 24) || commit_every <= 0) return QIL_ERR_SHAPE;
+    return launch_probe_mma(true, iters, commit_every, ops_out, dev_status, S(stream));
+}
+
+qil_status qil_probe_mma_bf16(int iters, int commit_every, double* ops_out, int* dev_status, qil_stream_t stream) {
+    if (iters <= 0 || iters > (1 << 24) || commit_every <= 0) return QIL_ERR_SHAPE;
+    return launch_probe_mma(false, iters, commit_every, ops_out, dev_status, S(stream));
 }
 
 qil_status qil_probe_hbm_read(const void* buf, size_t bytes, unsigned int* sink, qil_stream_t stream) {

@@ -80,8 +80,9 @@ qil_status launch_w4a16_skinny(const void* x, const uint32_t* qw, const void* sc
                                size_t ws_bytes, cudaStream_t st);
 
 bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout);
-qil_status launch_w4a16_prefill(const void* x, const uint32_t* qw, const void* scales, const void* zeros, void* y, int M,
-                                int N, int K, int G, void* ws, cudaStream_t st);
+size_t w4a16_prefill_workspace(int M, int N, int K);  // scratch of the split along K (0: none)
+qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scales, const void* zeros, void* y, int M, int N,
+                                int K, int G, int bits, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st);
 
 bool w4a16_tc_supported(int M, int N, int K, int G);
 size_t w4a16_tc_weight_bytes(int N, int K);
@@ -92,10 +93,11 @@ qil_status launch_w4a16_tc(const qil_linear_desc* entries, int count, void* ws, 
 void w4a16_tc_set_wait_limit(unsigned long long ns);  // 0 restores the default
 
 size_t w4a4_workspace(int M, int N, int K);
-qil_status launch_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, void* y,
-                       int32_t* acc_out, int M, int N, int K, void* ws, size_t ws_bytes, cudaStream_t st);
+qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const float* sw, void* y, int32_t* acc_out, int M,
+                       int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st);
 
 qil_status launch_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, cudaStream_t st);
+qil_status launch_probe_mma(bool i8, int iters, int commit_every, double* ops_out, int* status, cudaStream_t st);
 qil_status launch_probe_hbm_read(const void* buf, size_t bytes, unsigned int* sink, cudaStream_t st);
 
 }  // namespace qil

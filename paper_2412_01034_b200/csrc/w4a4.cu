@@ -1,6 +1,9 @@
-// W4A4 integer GEMM (the compute-bound driving-policy deployment of the paper,
-// Sec. 5.1 / Sec. 5.4): acc = qx . qw^T in int32, y = bf16(float(acc) * sx[m] * sw[n]),
-// on the 5th-generation tensor cores (tcgen05.mma kind::i8, accumulators in tensor memory).
+// W4A4 and W8A8 integer GEMMs (the compute-bound driving-policy deployment of the paper,
+// Sec. 5.1 / Sec. 5.4, Table "CILRS performance"): acc = qx . qw^T in int32,
+// y = bf16(float(acc) * sx[m] * sw[n]), on the 5th-generation tensor cores (tcgen05.mma kind::i8,
+// accumulators in tensor memory).  The text below describes the 4-bit operands; with 8-bit operands
+// (one signed byte per element) a step is 64 input channels, the bytes are stored as they are and
+// the accumulator is the sum itself.
 //
 // A CTA computes a 128 (tokens) x 64 (output channels) tile.  Per step of 128 input
 // channels its four loader warps read the packed nibbles of both operands from global
@@ -24,14 +27,15 @@ namespace qil {
 
 namespace {
 
-constexpr int kTileM = 128, kTileN = 64, kStepK = 128;  // K elements per step = 64 packed bytes per row
+constexpr int kTileM = 128, kTileN = 64;
+constexpr int kStepBytes = 64;  // operand bytes per row and step: 128 four-bit or 64 eight-bit elements
 constexpr int kStages = 3;
 // Operand tiles in shared memory: one byte per element after the split, K-major core matrices (8 rows x 16 bytes).
 // The K-adjacent core matrices lie 16 bytes further apart than they are long: the four lanes that hold the four
 // 16-byte pieces of one packed row then store to different banks.
 constexpr int kALbo = kTileM * 16 + 16, kBLbo = kTileN * 16 + 16;
-constexpr int kAStage = (kStepK / 16) * kALbo;
-constexpr int kBStage = (kStepK / 16) * kBLbo;
+constexpr int kAStage = 8 * kALbo;  // (sized for the 8 chunks of a 4-bit step; an 8-bit step uses 4)
+constexpr int kBStage = 8 * kBLbo;
 constexpr int kPre = 2;                   // steps whose global loads are in flight per loader thread
 constexpr int kThreads = 160;             // 4 loader / epilogue warps + the MMA warp
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -91,6 +95,7 @@ __device__ __forceinline__ void split32(const uint4& w, uint4& c0, uint4& c1) {
     c1 = make_uint4((w.z << 4) & m, w.z & m, (w.w << 4) & m, w.w & m);
 }
 
+template <int kBits>
 __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __restrict__ qx, const float* __restrict__ sx,
                                                              const uint32_t* __restrict__ qw, const float* __restrict__ sw,
                                                              __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out,
@@ -104,8 +109,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
     float* sws = reinterpret_cast<float*>(tmem_slot + 2);  // [kTileN] weight scales of the tile
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
+    constexpr int kStepK = kStepBytes * 8 / kBits;   // elements per step
+    constexpr int kChunks = kStepK / 16;             // 16-byte K chunks of a step in shared memory
     const int steps = (K + kStepK - 1) / kStepK;
-    const int row_words = K >> 3;  // 32-bit words per packed row
+    const int row_words = K * kBits / 32;  // 32-bit words per operand row
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -136,7 +143,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
         const uint32_t* wb = qw + (size_t)n0 * row_words + 4 * pq;
         uint4 pa[kPre][4], pb[kPre][2];
         auto fetch = [&](uint4 (&da)[4], uint4 (&db)[2], int step) {  // packed words of one step (zeros beyond the matrix)
-            const int w0 = step * (kStepK / 8);
+            const int w0 = step * (kStepBytes / 4);
             const bool in_k = w0 + 4 * pq < row_words;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -166,22 +173,31 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
                 const int s = step % kStages, use = step / kStages;
                 ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
                 if (!ok) break;
-                // piece pq = K chunks 2 pq, 2 pq + 1 of the step
-                unsigned char* a_st = sa + (size_t)s * kAStage + (size_t)(2 * pq) * kALbo + (size_t)pr * 16;
-                unsigned char* b_st = sb + (size_t)s * kBStage + (size_t)(2 * pq) * kBLbo + (size_t)pr * 16;
+                // 4-bit: piece pq = K chunks 2 pq, 2 pq + 1 of the step; 8-bit: piece pq = chunk pq
+                constexpr int kPer = kBits == 4 ? 2 : 1;
+                unsigned char* a_st = sa + (size_t)s * kAStage + (size_t)(kPer * pq) * kALbo + (size_t)pr * 16;
+                unsigned char* b_st = sb + (size_t)s * kBStage + (size_t)(kPer * pq) * kBLbo + (size_t)pr * 16;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    uint4 c0, c1;
-                    split32(pa[u][j], c0, c1);
-                    *reinterpret_cast<uint4*>(a_st + (size_t)j * (32 * 16)) = c0;
-                    *reinterpret_cast<uint4*>(a_st + (size_t)j * (32 * 16) + kALbo) = c1;
+                    if constexpr (kBits == 4) {
+                        uint4 c0, c1;
+                        split32(pa[u][j], c0, c1);
+                        *reinterpret_cast<uint4*>(a_st + (size_t)j * (32 * 16)) = c0;
+                        *reinterpret_cast<uint4*>(a_st + (size_t)j * (32 * 16) + kALbo) = c1;
+                    } else {
+                        *reinterpret_cast<uint4*>(a_st + (size_t)j * (32 * 16)) = pa[u][j];
+                    }
                 }
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
-                    uint4 c0, c1;
-                    split32(pb[u][j], c0, c1);
-                    *reinterpret_cast<uint4*>(b_st + (size_t)j * (32 * 16)) = c0;
-                    *reinterpret_cast<uint4*>(b_st + (size_t)j * (32 * 16) + kBLbo) = c1;
+                    if constexpr (kBits == 4) {
+                        uint4 c0, c1;
+                        split32(pb[u][j], c0, c1);
+                        *reinterpret_cast<uint4*>(b_st + (size_t)j * (32 * 16)) = c0;
+                        *reinterpret_cast<uint4*>(b_st + (size_t)j * (32 * 16) + kBLbo) = c1;
+                    } else {
+                        *reinterpret_cast<uint4*>(b_st + (size_t)j * (32 * 16)) = pb[u][j];
+                    }
                 }
                 if (step + kPre < steps) fetch(pa[u], pb[u], step + kPre);  // kPre steps stay in flight
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read through the async proxy
@@ -215,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
                     if (nb >= N) continue;
                     int a[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) a[j] = (int)d[8 * h + j] >> 8;  // exact: the accumulator is a multiple of 256
+                    for (int j = 0; j < 8; ++j) a[j] = kBits == 4 ? ((int)d[8 * h + j] >> 8) : (int)d[8 * h + j];  // (4-bit: exact, the accumulator is a multiple of 256)
                     if (vec) {
                         uint32_t pk[4];
 #pragma unroll
@@ -249,7 +265,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t a_addr = smem_u32(sa + (size_t)s * kAStage), b_addr = smem_u32(sb + (size_t)s * kBStage);
 #pragma unroll
-            for (int i = 0; i < 4; ++i)  // K = 32 each: chunks 2i, 2i + 1
+            for (int i = 0; i < kChunks / 2; ++i)  // K = 32 each: chunks 2i, 2i + 1
                 mma_i8_ss(tmem, smem_desc(a_addr + 2 * i * kALbo, kALbo, 128), smem_desc(b_addr + 2 * i * kBLbo, kBLbo, 128),
                           (step > 0 || i > 0) ? 1u : 0u);
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(free0 + 8 * s) : "memory");
@@ -280,16 +296,27 @@ size_t w4a4_workspace(int M, int N, int K) {
     return 16;
 }
 
-qil_status launch_w4a4(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, void* y,
-                       int32_t* acc_out, int M, int N, int K, void* ws, size_t ws_bytes, cudaStream_t st) {
+// bits = 4: packed nibbles [M][K/8], [N][K/8]; bits = 8: signed bytes [M][K], [N][K]
+qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const float* sw, void* y, int32_t* acc_out, int M,
+                       int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st) {
     if (ws == nullptr || ws_bytes < 16) return QIL_ERR_WORKSPACE;
-    if (cudaFuncSetAttribute(w4a4_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
+    const dim3 grid((M + kTileM - 1) / kTileM, (N + kTileN - 1) / kTileN);
+    cudaError_t e;
+    if (bits == 8) {
+        e = cudaFuncSetAttribute(w4a4_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e == cudaSuccess)
+            w4a4_tc_kernel<8><<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const uint32_t*>(qx), sx, reinterpret_cast<const uint32_t*>(qw), sw,
+                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws));
+    } else {
+        e = cudaFuncSetAttribute(w4a4_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e == cudaSuccess)
+            w4a4_tc_kernel<4><<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const uint32_t*>(qx), sx, reinterpret_cast<const uint32_t*>(qw), sw,
+                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws));
+    }
+    if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return QIL_ERR_CUDA;
     }
-    const dim3 grid((M + kTileM - 1) / kTileM, (N + kTileN - 1) / kTileN);
-    w4a4_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qx, sx, qw, sw, reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K,
-                                                      reinterpret_cast<int*>(ws));
     return launch_status();
 }
 

@@ -79,7 +79,7 @@ class QuantisedLinears:
         self.y_dev = torch.zeros(yo, dtype=torch.bfloat16, device=device)
 
         if bits == 8:
-            ws_bytes = int(self.lib.qil_linear_w8a16_workspace_size())
+            ws_bytes = max(int(self.lib.qil_linear_w8a16_workspace_size(M, N, K, self.G)) for (_, _, N, K, _, _) in self.specs)
         else:
             ws_bytes = max(api.linear_w4a16_workspace_size(M, N, K, self.G) for (_, _, N, K, _, _) in self.specs)
         self.ws = api.new_workspace(ws_bytes, device)

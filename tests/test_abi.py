@@ -102,8 +102,11 @@ def test_w8_validation(lib):
     assert f(A, A, A, A, A, 1, 16, 128, 96, A, 256, None) == 2           # group does not divide K
     assert f(A, A, A, A, A, 1, 16, 128, 128, None, 0, None) == 5         # workspace
     assert f(U, A, A, A, A, 1, 16, 128, 128, A, 256, None) == 3
-    assert lib.qil_linear_w8a16_workspace_size() >= 8
+    assert lib.qil_linear_w8a16_workspace_size(1, 16, 128, 128) >= 8
     assert lib.qil_linear_w8a16_batch(None, 1, A, 256, None) == 1
     assert lib.qil_quantize_rtn_w8(A, 0, 4, 8, 3, 0, A, A, 2, A, None, None) == 2
     assert lib.qil_quantize_act_a8(A, 4, 12, None, A, A, None) == 2
     assert lib.qil_set_wait_limit_ns(0) == 0
+    assert lib.qil_linear_w8a8(A, A, A, A, A, None, 4, 4, 24, A, 16, None) == 2     # K % 16
+    assert lib.qil_linear_w8a8(A, A, A, A, A, None, 4, 4, 32, None, 0, None) == 5
+    assert lib.qil_probe_mma_i8(0, 8, None, None, None) == 2

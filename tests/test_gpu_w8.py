@@ -9,7 +9,7 @@ import pytest
 
 from oracle import c_oracle, np_oracle
 from paper_2412_01034_b200 import workloads as wl
-from tests.util import assert_rows_close, bf16_to_f64, bits_of, cuda, to_bf16_cuda
+from tests.util import CONTRACT_REL, DERIVED_REL, assert_rows_close, bf16_to_f64, bits_of, cuda, to_bf16_cuda
 
 pytestmark = pytest.mark.gpu
 
@@ -87,14 +87,16 @@ def _w8_case(api, M, N, K, G, seed, x_scale=None):
     y_ref = c_oracle.linear_w8a16(x, q[0][rows], q[1][rows], q[2][rows], G)
     y = api.linear_w8a16(to_bf16_cuda(x), cuda(q[0]), cuda(q[1]), cuda(q[2]), G)
     assert tuple(y.shape) == (M, N)
-    assert_rows_close(bf16_to_f64(y)[:, rows], y_ref)
+    # M > 16 runs the tensor-core GEMM, which rounds every dequantised weight to bf16: judged by the contract's bound
+    gemm = M > 16 and K % 64 == 0 and G % 64 == 0
+    assert_rows_close(bf16_to_f64(y)[:, rows], y_ref, rel=CONTRACT_REL if gemm else DERIVED_REL)
     return y
 
 
 @pytest.mark.parametrize("M,N,K,G", [
     (1, 128, 128, 128), (1, 257, 1024, 128), (2, 200, 384, 128), (3, 1000, 2176, 128), (4, 512, 1024, 256),
     (1, 4096, 4096, 128), (1, 4096, 11008, 128), (1, 11008, 4096, 128), (4, 4096, 4096, 128), (1, 160, 2048, 2048),
-    (5, 300, 1024, 128), (16, 64, 512, 128), (33, 48, 256, 128),
+    (5, 300, 1024, 128), (16, 64, 512, 128), (33, 48, 256, 128), (280, 1000, 2176, 128), (130, 4096, 4096, 128),
 ])
 def test_w8a16_stream_shapes(api, M, N, K, G):
     y1 = _w8_case(api, M, N, K, G, M + N + K)
@@ -145,7 +147,7 @@ def test_w8a16_batch_with_and_without_dependencies(api):
     names = ["sq", "sq", "sq", "sq", "up", "up", "down"] * 2
     ys = [torch.zeros((M, shapes[nm][0]), dtype=torch.bfloat16, device="cuda") for nm in names]
     descs = (_lib.LinearDesc * len(names))()
-    ws = api.new_workspace(int(lib.qil_linear_w8a16_workspace_size()))
+    ws = api.new_workspace(int(lib.qil_linear_w8a16_workspace_size(4, 11008, 11008, 128)))
     st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     for deps in ("none", "layer"):
         for i, nm in enumerate(names):
@@ -207,7 +209,7 @@ def test_w8a16_wait_that_runs_out_is_reported(api):
         d.scales, d.zeros = dq[1].data_ptr(), dq[2].data_ptr()
         d.M, d.N, d.K, d.group_size, d.layout = M, N, K, G, api.LAYOUT_CANONICAL
     descs[0].flags, descs[1].flags = 0, api.DEP_PREVIOUS | api.DEP_NEVER
-    ws = api.new_workspace(int(lib.qil_linear_w8a16_workspace_size()))
+    ws = api.new_workspace(int(lib.qil_linear_w8a16_workspace_size(4, 11008, 11008, 128)))
     st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     try:
         assert lib.qil_set_wait_limit_ns(5_000_000) == 0
@@ -224,3 +226,47 @@ def test_w8a16_wait_that_runs_out_is_reported(api):
     torch.cuda.synchronize()
     assert int(ws[:4].view(torch.int32).item()) == 0
     assert_rows_close(bf16_to_f64(ys[1]), y_ref)
+
+
+# ----------------------------------------------------------------------------
+# W8A8 integer GEMM
+# ----------------------------------------------------------------------------
+def test_w8a8_extreme_codes(api):
+    """All-(-128) rows against all-(-128) and all-127 rows: 2^14 K and -128 * 127 K exactly."""
+    M, N, K = 19, 70, 4608
+    qx = np.full((M, K), -128, np.int8)
+    qw = np.full((N, K), -128, np.int8)
+    qw[1] = 127
+    one = np.ones(max(M, N), np.float32)
+    _, acc = api.linear_w8a8(cuda(qx), cuda(one[:M]), cuda(qw), cuda(one[:N]), want_acc=True)
+    a = acc.cpu().numpy()
+    assert np.all(a[:, 0] == 16384 * K) and np.all(a[:, 1] == -128 * 127 * K) and np.all(a[:, 2:] == 16384 * K)
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 16), (17, 9, 96), (130, 200, 160), (64, 64, 1152), (300, 70, 48)])
+def test_w8a8_ragged_shapes(api, M, N, K):
+    rng = np.random.default_rng(M * N + K)
+    qx = rng.integers(-128, 128, size=(M, K)).astype(np.int8)
+    qw = rng.integers(-128, 128, size=(N, K)).astype(np.int8)
+    sx = rng.random(M).astype(np.float32) + 0.1
+    sw = rng.random(N).astype(np.float32) + 0.1
+    acc_ref, y_ref = np_oracle.linear_w8a8(qx, sx, qw, sw)
+    y, acc = api.linear_w8a8(cuda(qx), cuda(sx), cuda(qw), cuda(sw), want_acc=True)
+    np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert_rows_close(bf16_to_f64(y), y_ref)
+
+
+@pytest.mark.parametrize("stage,batch", [(0, 32), (1, 32), (2, 32), (3, 32), (3, 2)])
+def test_w8a8_conv_stages(api, stage, batch):
+    """The im2col conv GEMMs of config 4 with 8-bit operands: quantisers, accumulators (bit-exact) and outputs."""
+    x, w = wl.conv_stage(stage, batch=batch)
+    qx_ref, sx_ref = np_oracle.quantize_sym8(wl.bf16_bits_to_f32(x))
+    qw_ref, sw_ref = np_oracle.quantize_sym8(w)
+    acc_ref, y_ref = c_oracle.linear_w8a8(qx_ref, sx_ref, qw_ref, sw_ref)
+    qx, sx = api.quantize_act_a8(to_bf16_cuda(x))
+    qw, sw, _ = api.quantize_rtn_w8(cuda(w), w.shape[1], symmetric=True)
+    np.testing.assert_array_equal(qx.cpu().numpy(), qx_ref)
+    np.testing.assert_array_equal(qw.cpu().numpy(), qw_ref)
+    y, acc = api.linear_w8a8(qx, sx, qw, sw.reshape(-1), want_acc=True)
+    np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert_rows_close(bf16_to_f64(y), y_ref)

@@ -395,7 +395,37 @@ def secondary_measurements(dev):
 
     g = torch.Generator(device=dev)
     g.manual_seed(4)
-    conv = []
+
+    def time_event_us(fn):
+        """One launch timed with events on the current stream (for launches of tens of microseconds or more)."""
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3
+
+    # roofs measured by the library's own probes: a read-only pass over 2 GiB (a GEMV reads, it does not copy) and
+    # tcgen05.mma over operands resident in shared memory
+    buf = torch.empty(1 << 29, dtype=torch.int32, device=dev)
+    sink = torch.zeros(1, dtype=torch.int32, device=dev)
+    t_read = min(time_event_us(lambda: api.probe_hbm_read(buf, sink)) for _ in range(3))
+    del buf
+    pstat = torch.zeros(4, dtype=torch.int32, device=dev)
+    probes = {"hbm_read_GB/s": (1 << 31) / t_read / 1e3}
+    for kind, key in (("i8", "mma_i8_TOPS"), ("bf16", "mma_bf16_TFLOP/s")):
+        ops = api.probe_mma(kind, 2000, 8, status=pstat)
+        t = min(time_event_us(lambda: api.probe_mma(kind, 2000, 8, status=pstat)) for _ in range(3))
+        probes[key] = ops / t / 1e6
+    probes["status"] = int(pstat[0].item())
+    probes["note"] = "burst figures: each probe launch lasts well under a millisecond"
+    out["probes"] = probes
+    i8_roof = probes["mma_i8_TOPS"]
+
+    conv, conv8 = [], []
+    l2_bytes = 126 * 1024 * 1024
     for stage in range(4):
         M, K, N = wl.conv_gemm_shape(stage)
         x = torch.relu(torch.randn((M, K), device=dev, generator=g)).to(torch.bfloat16)
@@ -407,11 +437,115 @@ def secondary_measurements(dev):
         y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
         t_gemm = time_us(lambda: api.linear_w4a4(qx, sx, pw, sw.reshape(-1), out=y, workspace=ws), 50)
         t_both = time_us(lambda: api.linear_w4a4(*api.quantize_act_a4(x), pw, sw.reshape(-1), out=y, workspace=ws), 50)
+        # tensor-wise static activation scale (the paper's W4A4 setting, App. A.1.2): quantiser + GEMM
+        t_static = time_us(lambda: api.linear_w4a4(*api.quantize_act_a4(x, static_scale=0.5), pw, sw.reshape(-1), out=y, workspace=ws), 50)
+        # cold: distinct operand and output copies in rotation, together more than four times the L2
+        per_copy = M * K // 2 + N * K // 2 + 2 * M * N + 4 * (M + N)
+        copies = min(160, 4 * l2_bytes // per_copy + 1)
+        qxs = [qx.clone() for _ in range(copies)]
+        pws = [pw.clone() for _ in range(copies)]
+        ys = [torch.empty_like(y) for _ in range(copies)]
+        st_ = {"i": 0}
+
+        def cold():
+            i = st_["i"] % copies
+            st_["i"] += 1
+            api.linear_w4a4(qxs[i], sx, pws[i], sw.reshape(-1), out=ys[i], workspace=ws)
+        t_cold = time_us(cold, copies)
+        del qxs, pws, ys
         ops = 2.0 * M * K * N
         conv.append({"M": M, "K": K, "N": N, "gemm_us": t_gemm, "gemm_tops": ops / t_gemm / 1e6,
-                     "quantise_plus_gemm_us": t_both, "l2": "operands fit L2 (warm)"})
+                     "gemm_cold_us": t_cold, "gemm_cold_tops": ops / t_cold / 1e6,
+                     "quantise_plus_gemm_us": t_both, "static_scale_quantise_plus_gemm_us": t_static,
+                     "frac_of_i8_probe": ops / t_gemm / 1e6 / i8_roof,
+                     "l2": "warm: operands resident in L2; cold: %d copies in rotation" % copies})
+        # the same shapes with 8-bit operands (Table "CILRS performance", W8A8 row)
+        qw8, sw8, _ = api.quantize_rtn_w8(w, K, symmetric=True)
+        qx8, sx8 = api.quantize_act_a8(x)
+        t8 = time_us(lambda: api.linear_w8a8(qx8, sx8, qw8, sw8.reshape(-1), out=y, workspace=ws), 50)
+        t8_both = time_us(lambda: api.linear_w8a8(*api.quantize_act_a8(x), qw8, sw8.reshape(-1), out=y, workspace=ws), 50)
+        conv8.append({"M": M, "K": K, "N": N, "gemm_us": t8, "gemm_tops": ops / t8 / 1e6, "quantise_plus_gemm_us": t8_both,
+                      "frac_of_i8_probe": ops / t8 / 1e6 / i8_roof})
     out["w4a4_conv_stages"] = conv
     out["w4a4_tops_total"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv) / sum(c["gemm_us"] for c in conv) / 1e6
+    out["w4a4_tops_total_cold"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv) / sum(c["gemm_cold_us"] for c in conv) / 1e6
+    out["w8a8_conv_stages"] = conv8
+    out["w8a8_tops_total"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv8) / sum(c["gemm_us"] for c in conv8) / 1e6
+
+    # the policy MLP of the DM-Control / D4RL experiments (Sec. 5.1: three fully connected layers of 2048 units) as
+    # W4A4: per-token activation quantiser + integer GEMM per layer, a latency case
+    mlp = []
+    wq = []
+    for _ in range(3):
+        w = torch.randn((2048, 2048), device=dev, generator=g) * wl.SIGMA_CONV
+        qw, sw, _ = api.quantize_rtn_w4(w, 2048, symmetric=True)
+        wq.append((api.pack_w4(qw), sw.reshape(-1)))
+    for Mb in (1, 256):
+        xin = torch.randn((Mb, 2048), device=dev, generator=g).to(torch.bfloat16)
+        bufs = [torch.empty((Mb, 2048), dtype=torch.bfloat16, device=dev) for _ in range(3)]
+        ws = api.new_workspace(api.linear_w4a4_workspace_size(Mb, 2048, 2048), dev)
+
+        def mlp_pass():
+            cur = xin
+            for (pw_, sw_), yb in zip(wq, bufs):
+                api.linear_w4a4(*api.quantize_act_a4(cur), pw_, sw_, out=yb, workspace=ws)
+                cur = yb
+        t = time_us(mlp_pass, 20)
+        mlp.append({"batch": Mb, "us_per_pass": t, "layers": 3, "units": 2048})
+    out["w4a4_policy_mlp_3x2048"] = mlp
+
+    # the paper's channel-wise weight setting (App. A.1.2: group_size = K) on one 4096 x 4096 decode linear, cold
+    N = K = wl.HIDDEN
+    copies = 12
+    chan = []
+    for _ in range(copies):
+        w = torch.randn((N, K), device=dev, generator=g) * wl.SIGMA_LLM
+        codes, s_, z_ = api.quantize_rtn_w4(w, K)
+        chan.append(api.pack_stream128_w4(codes, s_, z_, K))
+        del w, codes
+    xv1 = torch.randn((1, K), device=dev, generator=g).to(torch.bfloat16)
+    yv1 = torch.empty((1, N), dtype=torch.bfloat16, device=dev)
+    wsc = api.new_workspace(api.linear_w4a16_workspace_size(1, N, K, K), dev)
+    stc = {"i": 0}
+
+    def chan_one():
+        api.linear_w4a16(xv1, chan[stc["i"] % copies], None, None, N, K, api.LAYOUT_STREAM128, out=yv1, workspace=wsc)
+        stc["i"] += 1
+    t_chan = time_us(chan_one, 4 * copies)
+    out["w4a16_channelwise_4096x4096_m1"] = {"us": t_chan, "GB/s": (N * K / 2 + 4 * N + 2 * K + 2 * N) / t_chan / 1e3,
+                                             "l2": f"cold: {copies} weight copies in rotation", "note": "single call: includes the start-up of one launch"}
+    del chan
+
+    # INT8 weight-only decode (Table "OpenVLA performance", INT8 row): 8 decoder layers of the Llama-2-7B list
+    # (1.6 GB of codes, larger than L2) in one launch of the 8-bit streaming kernel
+    from paper_2412_01034_b200 import llama_decode
+    m8 = llama_decode.QuantisedLinears(cfg=1, M=1, n_layers=8, deps="none", device=str(dev), bits=8)
+    st8 = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(st8):
+        for _ in range(3):
+            m8.run(st8)
+        st8.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st8)
+        for _ in range(20):
+            m8.run(st8)
+        e1.record(st8)
+        st8.synchronize()
+    t8l = e0.elapsed_time(e1) / 20
+    w8 = {"layers": 8, "ms_per_pass": t8l, "GB/s": m8.algorithmic_bytes() / (t8l * 1e-3) / 1e9,
+          "bytes_per_pass": m8.algorithmic_bytes(), "kernel": "w8a16_stream_kernel<1> (dp4a)"}
+    m8.set_deps("layer")
+    with torch.cuda.stream(st8):
+        m8.run(st8)
+        st8.synchronize()
+        e0.record(st8)
+        for _ in range(20):
+            m8.run(st8)
+        e1.record(st8)
+        st8.synchronize()
+    w8["decoder_layer_order_GB/s"] = m8.algorithmic_bytes() / (e0.elapsed_time(e1) / 20 * 1e-3) / 1e9
+    out["w8a16_decode_list"] = w8
+    del m8
 
     # 16-bit reference GEMV, cold: rotate over copies larger than L2
     N = K = wl.HIDDEN

@@ -291,6 +291,24 @@ void qo_linear_w4a4(const int8_t* qx, const float* sx, const int8_t* qw, const f
     }
 }
 
+/* ---- W4A4 linear followed by the next layer's static-scale int4 quantiser, on the fp32 output ---- */
+void qo_linear_w4a4_requant(const int8_t* qx, const float* sx, const int8_t* qw, const float* sw,
+                            int M, int N, int K, float out_scale, int relu, int8_t* q_out) {
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            int64_t acc = 0;
+            for (int k = 0; k < K; ++k)
+                acc += (int64_t)qx[(size_t)m * K + k] * (int64_t)qw[(size_t)n * K + k];
+            float scale = sx[m] * sw[n];
+            float y = (float)acc * scale;
+            if (relu && y < 0.0f) y = 0.0f;
+            float q = qo_clampf(rintf(y / out_scale), -8.0f, 7.0f);
+            q_out[(size_t)m * N + n] = (int8_t)q;
+        }
+    }
+}
+
 int qo_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

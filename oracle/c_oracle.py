@@ -157,3 +157,15 @@ def linear_w8a16(x_bf16_bits, codes, scales, zeros, group_size):
 
 def linear_w8a8(qx, sx, qw, sw, want_y=True):
     return linear_w4a4(qx, sx, qw, sw, want_y)
+
+
+def linear_w4a4_requant(qx, sx, qw, sw, out_scale, relu):
+    qx = np.ascontiguousarray(qx, dtype=np.int8)
+    qw = np.ascontiguousarray(qw, dtype=np.int8)
+    sx = np.ascontiguousarray(sx, dtype=np.float32).reshape(-1)
+    sw = np.ascontiguousarray(sw, dtype=np.float32).reshape(-1)
+    M, K = qx.shape
+    N = qw.shape[0]
+    q = np.empty((M, N), np.int8)
+    load().qo_linear_w4a4_requant(_p(qx), _p(sx), _p(qw), _p(sw), M, N, K, C.c_float(out_scale), int(bool(relu)), _p(q))
+    return q

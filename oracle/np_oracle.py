@@ -365,3 +365,24 @@ def linear_w8a16(x_bf16_bits, codes, scales, zeros, group_size: int) -> np.ndarr
 def linear_w8a8(qx, sx, qw, sw):
     """acc[m][n] = sum_k qx[m][k]*qw[n][k] (int64, |acc| <= 2^14 K); y = acc * sx[m] * sw[n] (fp64)."""
     return linear_w4a4(qx, sx, qw, sw)
+
+
+# ----------------------------------------------------------------------------
+# W4A4 linear whose output is quantised again for the next layer (tensor-wise static activation scale, the paper's
+# W4A4 setting: App. A.1.2 uses one learned step size per activation tensor).  The next layer's quantiser is applied to
+# the fp32 output of the rescale, before any rounding to bf16:
+#   acc = sum_k qx qw                     (integer, exact)
+#   y32 = fl32(fl32(acc) * fl32(sx[m] * sw[n]))          two fp32 multiplications
+#   y32 = max(y32, 0)                     when relu is set
+#   q   = clamp(rint(y32 / out_scale), -8, 7)            fp32 division, ties to even
+# ----------------------------------------------------------------------------
+def linear_w4a4_requant(qx, sx, qw, sw, out_scale: float, relu: bool):
+    acc, _ = linear_w4a4(qx, sx, qw, sw)
+    if np.abs(acc).max() >= 2 ** 24:
+        raise OverflowError("accumulator is not exact in fp32")
+    scale = (np.asarray(sx, dtype=F32).reshape(-1, 1) * np.asarray(sw, dtype=F32).reshape(1, -1)).astype(F32)
+    y32 = (acc.astype(F32) * scale).astype(F32)
+    if relu:
+        y32 = np.maximum(y32, F32(0))
+    q = np.clip(np.rint((y32 / F32(out_scale)).astype(F32)), F32(-8), F32(7))
+    return q.astype(np.int8)

@@ -247,3 +247,47 @@ def test_linear_w8a8_exact_integers(impl):
     assert acc[0, 0] == 16384 * 96 and acc[0, 1] == -128 * 127 * 96
     assert y[0, 0] == 16384 * 96 * 0.5 and y[0, 1] == -128 * 127 * 96 * 0.5 * 0.5
     assert np.abs(acc).max() <= 16384 * 96
+
+
+# --------------------------------------------------------------------------
+# W4A4 linear with the next layer's static-scale quantiser applied to its output
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", IMPLS)
+def test_w4a4_requant_hand_case(impl):
+    """qx = (1, -2, 3, 0), sx = 0.5; three weight rows with sw = (0.25, 1, 2):
+    acc = (1*4 - 2*1 + 3*2, 1*7 - 2*7 + 3*7, -1 - 2*(-8) + 3*(-8)) = (8, 14, -9);
+    y = acc * sx * sw = (8 * 0.125, 14 * 0.5, -9 * 1.0) = (1, 7, -9); with out_scale = 0.5: y / 0.5 = (2, 14, -18)
+    -> codes (2, 7 (clamped), -8 (clamped)); with relu the last becomes 0.  A tie: acc 5 with scale 0.25 * 0.5 ... see
+    second row: y = 1.25 / 0.5 = 2.5 -> 2 (ties to even)."""
+    qx = np.array([[1, -2, 3, 0], [5, 0, 0, 0]], dtype=np.int8)
+    qw = np.array([[4, 1, 2, 0], [7, 7, 7, 0], [-1, -8, -8, 0]], dtype=np.int8)
+    sx = np.array([0.5, 0.5], dtype=np.float32)
+    sw = np.array([0.25, 1.0, 2.0], dtype=np.float32)
+    # row 1: acc = (20, 35, -5); y = (2.5, 17.5, -5); / 0.5 = (5, 35, -10) -> (5, 7, -8)
+    q = impl.linear_w4a4_requant(qx, sx, qw, sw, 0.5, False)
+    assert q.tolist() == [[2, 7, -8], [5, 7, -8]]
+    q = impl.linear_w4a4_requant(qx, sx, qw, sw, 0.5, True)
+    assert q.tolist() == [[2, 7, 0], [5, 7, 0]]
+    # ties to even: acc = 5, scale 0.5 * 0.25 -> y = 0.625; out_scale 0.25 -> 2.5 -> 2
+    q = impl.linear_w4a4_requant(np.array([[5, 0, 0, 0]], np.int8), np.array([0.5], np.float32),
+                                 np.array([[1, 0, 0, 0]], np.int8), np.array([0.25], np.float32), 0.25, False)
+    assert q.tolist() == [[2]]
+
+
+def test_w4a4_requant_is_the_static_quantiser_of_the_fp32_output():
+    """Reduces to the pinned pieces: integer matmul, two fp32 multiplications, then quantize_sym4 with a static scale;
+    the two writings agree bit for bit."""
+    rng = np.random.default_rng(9)
+    qx = rng.integers(-8, 8, size=(37, 96)).astype(np.int8)
+    qw = rng.integers(-8, 8, size=(40, 96)).astype(np.int8)
+    sx = (rng.random(37) * 0.1 + 0.01).astype(np.float32)
+    sw = (rng.random(40) * 0.1 + 0.01).astype(np.float32)
+    acc = qx.astype(np.int64) @ qw.astype(np.int64).T
+    y32 = acc.astype(np.float32) * (sx[:, None] * sw[None, :]).astype(np.float32)
+    for relu in (False, True):
+        want, _ = np_oracle.quantize_sym4(np.maximum(y32, 0) if relu else y32, static_scale=0.05)
+        a = np_oracle.linear_w4a4_requant(qx, sx, qw, sw, 0.05, relu)
+        b = c_oracle.linear_w4a4_requant(qx, sx, qw, sw, 0.05, relu)
+        np.testing.assert_array_equal(a, want)
+        np.testing.assert_array_equal(b, want)
+        assert a.min() >= -8 and a.max() <= 7

@@ -309,6 +309,16 @@ qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* 
                            void* y, int32_t* acc_out, int M, int N, int K, void* workspace,
                            size_t workspace_bytes, qil_stream_t stream);
 
+/* W4A4 GEMM fused with the next layer's activation quantiser (a neighbour of the linear on the W4A4 path: with
+ * the paper's tensor-wise static activation scale, App. A.1.2, the next layer's codes can be produced in this
+ * layer's epilogue and the bf16 activations never touch memory):
+ *   v = fl32(float(acc) * fl32(sx[m] * sw[n]));  v = max(v, 0) if relu;  q = clamp(rint(v / out_scale), -8, 7)
+ *   qy [M][N/8]: the codes packed like qx (so that qy is the next call's qx, with sx[m] = out_scale).
+ * Needs N % 8 == 0, out_scale > 0; otherwise as qil_linear_w4a4. */
+qil_status qil_linear_w4a4_requant(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw,
+                                   uint32_t* qy, float out_scale, int relu, int M, int N, int K,
+                                   void* workspace, size_t workspace_bytes, qil_stream_t stream);
+
 /* W8A8 integer GEMM (Table "CILRS performance", W8A8 row; Sec. 5.4): as qil_linear_w4a4 with one signed byte per
  * element: qx [M][K], qw [N][K] int8; acc exact in int32 (|acc| <= 2^14 K: K < 131072), K % 16 == 0; the same
  * workspace (qil_linear_w4a4_workspace_size). */

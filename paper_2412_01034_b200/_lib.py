@@ -30,6 +30,7 @@ SIGNATURES = {
     "qil_quantize_act_a4": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),
     "qil_linear_w4a4_workspace_size": (_sz, [_i, _i, _i]),
     "qil_linear_w4a4": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_linear_w4a4_requant": (_i, [_vp, _vp, _vp, _vp, _vp, C.c_float, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w8a8": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "qil_status_string": (C.c_char_p, [_i]),
     "qil_version": (_i, []),

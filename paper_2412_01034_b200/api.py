@@ -215,6 +215,20 @@ def linear_w4a4(qx, sx, qw, sw, want_acc: bool = False, out=None, workspace=None
     return (out, acc) if want_acc else out
 
 
+def linear_w4a4_requant(qx, sx, qw, sw, out_scale: float, relu: bool = False, workspace=None, stream=None):
+    """W4A4 GEMM whose epilogue quantises the output for the next layer: returns packed int4 codes [M][N/8]."""
+    _need_cuda(qx, sx, qw, sw, workspace)
+    M, K = qx.shape[0], qx.shape[1] * 8
+    N = qw.shape[0]
+    qy = torch.empty((M, max(N // 8, 1)), dtype=torch.int32, device=qx.device)
+    if workspace is None:
+        workspace = new_workspace(linear_w4a4_workspace_size(M, N, K), qx.device)
+    _check(_lib.load().qil_linear_w4a4_requant(_ptr(qx), _ptr(sx), _ptr(qw), _ptr(sw), _ptr(qy), C.c_float(out_scale),
+                                               int(bool(relu)), M, N, K, _ptr(workspace),
+                                               workspace.numel() * workspace.element_size(), _stream(stream)))
+    return qy
+
+
 def linear_w8a8(qx, sx, qw, sw, want_acc: bool = False, out=None, workspace=None, stream=None):
     """Integer GEMM of int8 operands (qx [M][K], qw [N][K]); returns y (bf16) or (y, acc int32)."""
     _need_cuda(qx, sx, qw, sw, out, workspace)

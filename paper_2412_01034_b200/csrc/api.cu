@@ -363,6 +363,20 @@ qil_status qil_linear_w4a4(const uint32_t* qx, const float* sx, const uint32_t* 
     return launch_w4a4(qx, sx, qw, sw, y, acc_out, M, N, K, 4, workspace, workspace_bytes, S(stream));
 }
 
+qil_status qil_linear_w4a4_requant(const uint32_t* qx, const float* sx, const uint32_t* qw, const float* sw, uint32_t* qy,
+                                   float out_scale, int relu, int M, int N, int K, void* workspace,
+                                   size_t workspace_bytes, qil_stream_t stream) {
+    if (!qx || !sx || !qw || !sw || !qy) return QIL_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || K >= 131072 || N % 8 != 0) return QIL_ERR_SHAPE;
+    if (!(out_scale > 0.0f)) return QIL_ERR_UNSUPPORTED;
+    if (!aligned16(qx) || !aligned16(sx) || !aligned16(qw) || !aligned16(sw) || !aligned16(qy) ||
+        (workspace && !aligned16(workspace)))
+        return QIL_ERR_ALIGN;
+    if (!workspace || workspace_bytes < w4a4_workspace(M, N, K)) return QIL_ERR_WORKSPACE;
+    return launch_w4a4(qx, sx, qw, sw, qy /*unused as y*/, nullptr, M, N, K, 4, workspace, workspace_bytes, S(stream), qy,
+                       out_scale, relu ? 1 : 0);
+}
+
 qil_status qil_linear_w8a8(const int8_t* qx, const float* sx, const int8_t* qw, const float* sw, void* y,
                            int32_t* acc_out, int M, int N, int K, void* workspace, size_t workspace_bytes,
                            qil_stream_t stream) {

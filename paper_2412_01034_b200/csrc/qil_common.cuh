@@ -94,7 +94,8 @@ void w4a16_tc_set_wait_limit(unsigned long long ns);  // 0 restores the default
 
 size_t w4a4_workspace(int M, int N, int K);
 qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const float* sw, void* y, int32_t* acc_out, int M,
-                       int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st);
+                       int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st, uint32_t* qy = nullptr,
+                       float out_scale = 1.f, int relu = 0);
 
 qil_status launch_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, cudaStream_t st);
 qil_status launch_probe_mma(bool i8, int iters, int commit_every, double* ops_out, int* status, cudaStream_t st);

@@ -99,7 +99,10 @@ template <int kBits>
 __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __restrict__ qx, const float* __restrict__ sx,
                                                              const uint32_t* __restrict__ qw, const float* __restrict__ sw,
                                                              __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out,
-                                                             int M, int N, int K, int* __restrict__ status) {
+                                                             int M, int N, int K, int* __restrict__ status,
+                                                             uint32_t* __restrict__ qy, float out_scale, int relu) {
+    // qy != null: instead of bf16 outputs the epilogue writes the next layer's int4 activations, quantised with the
+    // static scale out_scale from the fp32 product (optionally after ReLU), packed 8 per word (needs N % 8 == 0)
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* sa = smem;                                  // [kStages][kAStage]
     unsigned char* sb = smem + (size_t)kStages * kAStage;      // [kStages][kBStage]
@@ -232,7 +235,17 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
                     int a[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) a[j] = kBits == 4 ? ((int)d[8 * h + j] >> 8) : (int)d[8 * h + j];  // (4-bit: exact, the accumulator is a multiple of 256)
-                    if (vec) {
+                    if (qy) {
+                        uint32_t word = 0;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float v = __fmul_rn((float)a[j], __fmul_rn(sxm, sws[c0 + 8 * h + j]));
+                            if (relu) v = fmaxf(v, 0.f);
+                            const int q = (int)fminf(fmaxf(rintf(__fdiv_rn(v, out_scale)), -8.f), 7.f);
+                            word |= ((uint32_t)q & 0xFu) << (4 * j);
+                        }
+                        qy[(size_t)m * (N >> 3) + (nb >> 3)] = word;
+                    } else if (vec) {
                         uint32_t pk[4];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -298,7 +311,8 @@ size_t w4a4_workspace(int M, int N, int K) {
 
 // bits = 4: packed nibbles [M][K/8], [N][K/8]; bits = 8: signed bytes [M][K], [N][K]
 qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const float* sw, void* y, int32_t* acc_out, int M,
-                       int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st) {
+                       int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st, uint32_t* qy, float out_scale,
+                       int relu) {
     if (ws == nullptr || ws_bytes < 16) return QIL_ERR_WORKSPACE;
     const dim3 grid((M + kTileM - 1) / kTileM, (N + kTileN - 1) / kTileN);
     cudaError_t e;
@@ -306,12 +320,12 @@ qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const fl
         e = cudaFuncSetAttribute(w4a4_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e == cudaSuccess)
             w4a4_tc_kernel<8><<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const uint32_t*>(qx), sx, reinterpret_cast<const uint32_t*>(qw), sw,
-                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws));
+                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws), nullptr, 1.f, 0);
     } else {
         e = cudaFuncSetAttribute(w4a4_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e == cudaSuccess)
             w4a4_tc_kernel<4><<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const uint32_t*>(qx), sx, reinterpret_cast<const uint32_t*>(qw), sw,
-                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws));
+                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws), qy, out_scale, relu);
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();

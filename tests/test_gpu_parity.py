@@ -680,3 +680,20 @@ def test_ref_gemv_bf16(api):
     sink = torch.zeros(1, dtype=torch.int32, device="cuda")
     api.probe_hbm_read(buf, sink)
     assert int(sink.item()) & 0xFFFFFFFF == (sum(range(1 << 16))) & 0xFFFFFFFF
+
+
+@pytest.mark.parametrize("stage,batch,relu", [(2, 8, True), (3, 32, False), (1, 2, True)])
+def test_w4a4_requant_epilogue(api, stage, batch, relu):
+    """The W4A4 GEMM that writes the next layer's int4 activations (static scale) from its epilogue: codes bit-exact
+    against the oracle, and usable as the next call's packed operand."""
+    x, w = wl.conv_stage(stage, batch=batch)
+    qx_ref, sx_ref = np_oracle.quantize_sym4(wl.bf16_bits_to_f32(x))
+    qw_ref, sw_ref = np_oracle.quantize_sym4(w)
+    out_scale = 0.75
+    q_ref = c_oracle.linear_w4a4_requant(qx_ref, sx_ref, qw_ref, sw_ref, out_scale, relu)
+    assert q_ref.max() == 7 and (relu or q_ref.min() == -8)
+    qx, sx = api.quantize_act_a4(to_bf16_cuda(x))
+    qw, sw, _ = api.quantize_rtn_w4(cuda(w), w.shape[1], symmetric=True)
+    qy = api.linear_w4a4_requant(qx, sx, api.pack_w4(qw), sw.reshape(-1), out_scale, relu)
+    got = np_oracle.unpack_w4(qy.cpu().numpy().view(np.uint32), signed=True)
+    np.testing.assert_array_equal(got, q_ref)

@@ -581,7 +581,7 @@ def secondary_measurements(dev):
     del lin, xs
 
     # configs[3]: M sweep on the two FFN shapes, cold (6 weight copies in rotation = 144 MB of packed weights,
-    # larger than L2).  M <= 4 runs the tcgen05 decode kernel (STREAM128 units), M <= 16 the mma.sync skinny kernel
+    # larger than L2).  M <= 4 runs the tcgen05 decode kernel (STREAM128 units), M <= 8 the mma.sync skinny kernel
     # (TILE16), larger M the tcgen05 prefill kernel (canonical layout).
     sweep = []
     copies = 6
@@ -601,7 +601,7 @@ def secondary_measurements(dev):
             xm = torch.randn((Ms, K), device=dev, generator=g).to(torch.bfloat16)
             ym = torch.empty((Ms, N), dtype=torch.bfloat16, device=dev)
             ws = api.new_workspace(api.linear_w4a16_workspace_size(Ms, N, K, wl.GROUP_SIZE), dev)
-            for name in (("stream128", "tile16") if Ms <= 4 else ("tile16",) if Ms <= 16 else ("canonical",)):
+            for name in (("stream128", "tile16") if Ms <= 4 else ("tile16",) if Ms <= 8 else ("canonical",)):
                 st_ = {"i": 0}
 
                 def one():

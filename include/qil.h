@@ -121,7 +121,7 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  * into the matmul, accumulation is fp32, the result is rounded to bf16.
  *   x [M][K] bf16   qweight packed per `layout`   scales, zeros [N][K/group_size] fp16
  *   y [M][N] bf16
- * The kernel is chosen from the shape: on the canonical layout with M > 16,
+ * The kernel is chosen from the shape: on the canonical layout with M > 8,
  * K % 64 == 0 and group_size % 64 == 0 the tcgen05 prefill GEMM (weights
  * dequantised to bf16, one rounding per weight; K split over several CTAs where
  * that fills the GPU, partial tiles added in a fixed order); else the tensor-core skinny
@@ -173,7 +173,7 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
  * Arguments as qil_linear_w4a16, minus the workspace.  Two differences from
  * that call: QIL_LAYOUT_STREAM128 is not served (QIL_ERR_UNSUPPORTED: the list
  * kernel's workspace is larger than the array), and on the canonical layout
- * with M > 16 the result is the skinny kernel's (fp32 dequantisation), not the
+ * with M > 8 the result is the skinny kernel's (fp32 dequantisation), not the
  * prefill GEMM's (weights rounded to bf16): both are within the tolerance of
  * the linear, but their bits differ.  The array's address is looked up for the
  * device that is current at the call; `stream` must belong to that device.
@@ -253,7 +253,7 @@ qil_status qil_linear_w4a16_batch_host(const qil_linear_desc* descs /*host*/, in
  *   shared memory: K <= 24576) a streaming kernel runs, four activation rows per pass: it converts the
  *   activations to 16-bit block fixed point per 128 columns (error at most 2^-16 of the block maximum) and
  *   accumulates integer dot products exactly.  Other shapes (K % 16 == 0) use a general kernel.
- *   With M > 16, K % 64 == 0 and group_size % 64 == 0 the tcgen05 prefill GEMM of qil_linear_w4a16 runs on the
+ *   With M > 8, K % 64 == 0 and group_size % 64 == 0 the tcgen05 prefill GEMM of qil_linear_w4a16 runs on the
  *   8-bit codes (weights dequantised to bf16, one rounding per weight).
  *   workspace: qil_linear_w8a16_workspace_size() bytes (at least 256), zero-filled once; its first int is the
  *   status word (QIL_ERR_TIMEOUT if a bounded wait ran out), its second a counter the list kernel uses between

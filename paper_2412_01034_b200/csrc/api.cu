@@ -268,7 +268,7 @@ size_t qil_linear_w8a16_workspace_size(int M, int N, int K, int group_size) {
 // One linear: the streaming kernel in slabs of four activation rows where the shape allows it, the general kernel
 // otherwise.
 static qil_status w8a16_one(const qil_linear_desc& d, void* workspace, size_t workspace_bytes, cudaStream_t st) {
-    if (w4a16_prefill_supported(d.M, d.N, d.K, d.group_size, QIL_LAYOUT_CANONICAL)) {  // M > 16: the tensor-core GEMM
+    if (w4a16_prefill_supported(d.M, d.N, d.K, d.group_size, QIL_LAYOUT_CANONICAL)) {  // M > 8: the tensor-core GEMM
         const size_t off = w8a16_workspace();
         const bool have = workspace_bytes > off;
         return launch_w4a16_prefill(d.x, d.qweight, d.scales, d.zeros, d.y, d.M, d.N, d.K, d.group_size, 8,

@@ -501,7 +501,7 @@ PrefillPlan plan_prefill(int M, int N, int K) {
 }  // namespace
 
 bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout) {
-    return layout == QIL_LAYOUT_CANONICAL && M > 16 && N >= 1 && K % kStepK == 0 && G % kStepK == 0 && K % G == 0 &&
+    return layout == QIL_LAYOUT_CANONICAL && M > 8 && N >= 1 && K % kStepK == 0 && G % kStepK == 0 && K % G == 0 &&
            (long long)((N + kTileF - 1) / kTileF) * ((M + kMaxTN - 1) / kMaxTN) <= kCounterBytes / 4 && (M + kMaxTN - 1) / kMaxTN <= 65535;
 }
 

@@ -22,7 +22,7 @@ pytestmark = pytest.mark.gpu
 
 
 # (M, N, K, layout, uses the built-in scratch): split-K shapes on both layouts, one shape that needs no scratch, and one
-# canonical M > 16 shape, where the ordinary entry point runs the prefill GEMM (bf16-rounded weights) and this one the
+# canonical M > 8 shape, where the ordinary entry point runs the prefill GEMM (bf16-rounded weights) and this one the
 # skinny kernel, so that the two agree within the tolerance of the linear but not bit for bit.
 CASES = [(1, 4096, 4096, 1, True), (4, 512, 4096, 1, True), (2, 256, 4096, 0, True), (3, 11008, 1024, 1, False),
          (24, 512, 2048, 0, True)]
@@ -44,7 +44,7 @@ def test_static_ws_matches_workspace_entry_point_twice(M, N, K, layout, uses_scr
     packed = api.pack_w4(cuda(codes), layout)
     xd, sd, zd = to_bf16_cuda(x), cuda(scales), cuda(zeros)
     y_ws = api.linear_w4a16(xd, packed, sd, zd, N, G, layout)       # caller-allocated workspace
-    same_kernel = not (layout == api.LAYOUT_CANONICAL and M > 16)
+    same_kernel = not (layout == api.LAYOUT_CANONICAL and M > 8)
     stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     for call in range(2):
         y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")

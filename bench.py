@@ -466,6 +466,26 @@ def secondary_measurements(dev):
         t8_both = time_us(lambda: api.linear_w8a8(*api.quantize_act_a8(x), qw8, sw8.reshape(-1), out=y, workspace=ws), 50)
         conv8.append({"M": M, "K": K, "N": N, "gemm_us": t8, "gemm_tops": ops / t8 / 1e6, "quantise_plus_gemm_us": t8_both,
                       "frac_of_i8_probe": ops / t8 / 1e6 / i8_roof})
+    # the four GEMMs (independent operands) as one persistent launch
+    for bits_, key in ((4, "w4a4_conv_stages_one_launch"), (8, "w8a8_conv_stages_one_launch")):
+        ents, ops_all = [], 0.0
+        for stage in range(4):
+            M, K, N = wl.conv_gemm_shape(stage)
+            x = torch.relu(torch.randn((M, K), device=dev, generator=g)).to(torch.bfloat16)
+            w = torch.randn((N, K), device=dev, generator=g) * wl.SIGMA_CONV
+            if bits_ == 4:
+                qw_, sw_, _ = api.quantize_rtn_w4(w, K, symmetric=True)
+                qw_ = api.pack_w4(qw_)
+                qx_, sx_ = api.quantize_act_a4(x)
+            else:
+                qw_, sw_, _ = api.quantize_rtn_w8(w, K, symmetric=True)
+                qx_, sx_ = api.quantize_act_a8(x)
+            ents.append((qx_, sx_, qw_, sw_.reshape(-1), torch.empty((M, N), dtype=torch.bfloat16, device=dev), None, bits_))
+            ops_all += 2.0 * M * K * N
+        wsl = api.new_workspace(16, dev)
+        t_l = time_us(lambda: api.linear_int_batch(ents, workspace=wsl), 50)
+        out[key] = {"us": t_l, "tops": ops_all / t_l / 1e6, "frac_of_i8_probe": ops_all / t_l / 1e6 / i8_roof,
+                    "kernel": "igemm_list_kernel", "l2": "warm"}
     out["w4a4_conv_stages"] = conv
     out["w4a4_tops_total"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv) / sum(c["gemm_us"] for c in conv) / 1e6
     out["w4a4_tops_total_cold"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv) / sum(c["gemm_cold_us"] for c in conv) / 1e6

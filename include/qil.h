@@ -326,6 +326,23 @@ qil_status qil_linear_w8a8(const int8_t* qx, const float* sx, const int8_t* qw, 
                            int32_t* acc_out, int M, int N, int K, void* workspace, size_t workspace_bytes,
                            qil_stream_t stream);
 
+/* A list of independent integer GEMMs in one persistent launch (one CTA per SM walks output tiles of all entries;
+ * the conv stages of Sec. 5.1's driving policy are each shorter than the start-up of a kernel).  bits = 4: operands
+ * as for qil_linear_w4a4; bits = 8: as for qil_linear_w8a8.  No entry may read another entry's output.  At most 8
+ * entries and 1200 output tiles of 128 x 64 per call; larger lists are run entry by entry.  Descriptors are host
+ * memory, consumed before the call returns; workspace as for qil_linear_w4a4. */
+typedef struct {
+    const void* qx;          /* bits 4: packed [M][K/8] uint32; bits 8: int8 [M][K] */
+    const float* sx;         /* [M] */
+    const void* qw;          /* bits 4: packed [N][K/8]; bits 8: int8 [N][K] */
+    const float* sw;         /* [N] */
+    void* y;                 /* bf16 [M][N] */
+    int32_t* acc_out;        /* optional [M][N] */
+    int M, N, K, bits;
+} qil_igemm_desc;
+qil_status qil_linear_int_batch(const qil_igemm_desc* descs /*host*/, int count, void* workspace,
+                                size_t workspace_bytes, qil_stream_t stream);
+
 /* ------------------------------------------------------------------------
  * Helpers
  * ---------------------------------------------------------------------- */

@@ -32,6 +32,7 @@ SIGNATURES = {
     "qil_linear_w4a4": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w4a4_requant": (_i, [_vp, _vp, _vp, _vp, _vp, C.c_float, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w8a8": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_linear_int_batch": (_i, [_vp, _i, _vp, _sz, _vp]),
     "qil_status_string": (C.c_char_p, [_i]),
     "qil_version": (_i, []),
     "qil_device_status": (_i, [_vp, C.POINTER(C.c_int), _vp]),
@@ -47,6 +48,12 @@ class LinearDesc(C.Structure):
     """ctypes mirror of ``qil_linear_desc``."""
     _fields_ = [("x", _vp), ("qweight", _vp), ("scales", _vp), ("zeros", _vp), ("y", _vp),
                 ("M", _i), ("N", _i), ("K", _i), ("group_size", _i), ("layout", _i), ("flags", _i)]
+
+
+class IGemmDesc(C.Structure):
+    """ctypes mirror of ``qil_igemm_desc``."""
+    _fields_ = [("qx", _vp), ("sx", _vp), ("qw", _vp), ("sw", _vp), ("y", _vp), ("acc_out", _vp),
+                ("M", _i), ("N", _i), ("K", _i), ("bits", _i)]
 
 
 _lib = None

@@ -229,6 +229,25 @@ def linear_w4a4_requant(qx, sx, qw, sw, out_scale: float, relu: bool = False, wo
     return qy
 
 
+def linear_int_batch(entries, workspace=None, stream=None):
+    """A list of independent integer GEMMs in one launch.  entries: [(qx, sx, qw, sw, y, acc or None, bits)] with the
+    operands of linear_w4a4 (bits 4) or linear_w8a8 (bits 8); outputs are written into y (and acc)."""
+    descs = (_lib.IGemmDesc * len(entries))()
+    dev = None
+    for d, (qx, sx, qw, sw, y, acc, bits) in zip(descs, entries):
+        _need_cuda(qx, sx, qw, sw, y, acc)
+        dev = qx.device
+        d.qx, d.sx, d.qw, d.sw, d.y = qx.data_ptr(), sx.data_ptr(), qw.data_ptr(), sw.data_ptr(), y.data_ptr()
+        d.acc_out = None if acc is None else acc.data_ptr()
+        d.M, d.N = y.shape
+        d.K = qx.shape[1] * (8 if bits == 4 else 1)
+        d.bits = bits
+    if workspace is None:
+        workspace = new_workspace(16, dev)
+    _check(_lib.load().qil_linear_int_batch(descs, len(entries), _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
 def linear_w8a8(qx, sx, qw, sw, want_acc: bool = False, out=None, workspace=None, stream=None):
     """Integer GEMM of int8 operands (qx [M][K], qw [N][K]); returns y (bf16) or (y, acc int32)."""
     _need_cuda(qx, sx, qw, sw, out, workspace)

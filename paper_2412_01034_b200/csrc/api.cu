@@ -390,6 +390,31 @@ qil_status qil_linear_w8a8(const int8_t* qx, const float* sx, const int8_t* qw, 
     return launch_w4a4(qx, sx, qw, sw, y, acc_out, M, N, K, 8, workspace, workspace_bytes, S(stream));
 }
 
+qil_status qil_linear_int_batch(const qil_igemm_desc* descs, int count, void* workspace, size_t workspace_bytes,
+                                qil_stream_t stream) {
+    if (!descs) return QIL_ERR_NULL;
+    if (count <= 0) return QIL_ERR_SHAPE;
+    if (!workspace || workspace_bytes < 16) return QIL_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return QIL_ERR_ALIGN;
+    for (int i = 0; i < count; ++i) {
+        const qil_igemm_desc& d = descs[i];
+        if (!d.qx || !d.sx || !d.qw || !d.sw || !d.y) return QIL_ERR_NULL;
+        if (d.bits != 4 && d.bits != 8) return QIL_ERR_UNSUPPORTED;
+        if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.K % (d.bits == 4 ? 32 : 16) != 0 || d.K >= 131072) return QIL_ERR_SHAPE;
+        if (!aligned16(d.qx) || !aligned16(d.sx) || !aligned16(d.qw) || !aligned16(d.sw) || !aligned16(d.y) ||
+            (d.acc_out && !aligned16(d.acc_out)))
+            return QIL_ERR_ALIGN;
+    }
+    if (igemm_list_supported(descs, count)) return launch_igemm_list(descs, count, workspace, workspace_bytes, S(stream));
+    for (int i = 0; i < count; ++i) {
+        const qil_igemm_desc& d = descs[i];
+        const qil_status s = launch_w4a4(d.qx, d.sx, d.qw, d.sw, d.y, d.acc_out, d.M, d.N, d.K, d.bits, workspace,
+                                         workspace_bytes, S(stream));
+        if (s != QIL_OK) return s;
+    }
+    return QIL_OK;
+}
+
 qil_status qil_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, qil_stream_t stream) {
     if (!x || !w || !y) return QIL_ERR_NULL;
     if (N <= 0 || K <= 0 || K % 8 != 0) return QIL_ERR_SHAPE;

@@ -97,6 +97,9 @@ qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const fl
                        int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st, uint32_t* qy = nullptr,
                        float out_scale = 1.f, int relu = 0);
 
+bool igemm_list_supported(const qil_igemm_desc* d, int count);
+qil_status launch_igemm_list(const qil_igemm_desc* d, int count, void* ws, size_t ws_bytes, cudaStream_t st);
+
 qil_status launch_ref_gemv_bf16(const void* x, const void* w, void* y, int N, int K, cudaStream_t st);
 qil_status launch_probe_mma(bool i8, int iters, int commit_every, double* ops_out, int* status, cudaStream_t st);
 qil_status launch_probe_hbm_read(const void* buf, size_t bytes, unsigned int* sink, cudaStream_t st);

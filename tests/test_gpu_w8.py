@@ -270,3 +270,67 @@ def test_w8a8_conv_stages(api, stage, batch):
     y, acc = api.linear_w8a8(qx, sx, qw, sw.reshape(-1), want_acc=True)
     np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
     assert_rows_close(bf16_to_f64(y), y_ref)
+
+
+# ----------------------------------------------------------------------------
+# lists of integer GEMMs in one persistent launch
+# ----------------------------------------------------------------------------
+def test_int_gemm_list_conv_stages(api):
+    """The four conv GEMMs of config 4 at batch 32, as 4-bit and as 8-bit entries, all eight in one launch:
+    accumulators bit-exact, outputs within tolerance; a second launch reproduces the first."""
+    import torch
+    entries, refs = [], []
+    for stage in range(4):
+        x, w = wl.conv_stage(stage, batch=32)
+        xf = wl.bf16_bits_to_f32(x)
+        for bits in (4, 8):
+            if bits == 4:
+                qx_ref, sx_ref = np_oracle.quantize_sym4(xf)
+                qw_ref, sw_ref = np_oracle.quantize_sym4(w)
+                qx, qw = api.pack_w4(cuda(qx_ref)), api.pack_w4(cuda(qw_ref))
+            else:
+                qx_ref, sx_ref = np_oracle.quantize_sym8(xf)
+                qw_ref, sw_ref = np_oracle.quantize_sym8(w)
+                qx, qw = cuda(qx_ref), cuda(qw_ref)
+            acc_ref, y_ref = c_oracle.linear_w8a8(qx_ref, sx_ref, qw_ref, sw_ref)
+            M, N = acc_ref.shape
+            y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+            acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+            entries.append((qx, cuda(sx_ref.reshape(-1)), qw, cuda(sw_ref.reshape(-1)), y, acc, bits))
+            refs.append((acc_ref, y_ref))
+    first = None
+    for rep in range(2):
+        api.linear_int_batch(entries)
+        torch.cuda.synchronize()
+        got = [bits_of(e[4]) for e in entries]
+        if first is None:
+            first = got
+            for e, (acc_ref, y_ref) in zip(entries, refs):
+                np.testing.assert_array_equal(e[5].cpu().numpy().astype(np.int64), acc_ref)
+                assert_rows_close(bf16_to_f64(e[4]), y_ref)
+        else:
+            for a, b in zip(first, got):
+                np.testing.assert_array_equal(a, b)
+        for e in entries:
+            e[4].zero_()
+
+
+def test_int_gemm_list_ragged(api):
+    import torch
+    rng = np.random.default_rng(4)
+    entries, refs = [], []
+    for (M, N, K, bits) in [(1, 1, 32, 4), (17, 9, 96, 4), (130, 200, 160, 8), (300, 70, 48, 8), (64, 64, 1152, 4)]:
+        lo, hi = (-8, 8) if bits == 4 else (-128, 128)
+        qx = rng.integers(lo, hi, size=(M, K)).astype(np.int8)
+        qw = rng.integers(lo, hi, size=(N, K)).astype(np.int8)
+        sx = rng.random(M).astype(np.float32) + 0.1
+        sw = rng.random(N).astype(np.float32) + 0.1
+        refs.append(np_oracle.linear_w8a8(qx, sx, qw, sw))
+        dx, dw = (api.pack_w4(cuda(qx)), api.pack_w4(cuda(qw))) if bits == 4 else (cuda(qx), cuda(qw))
+        entries.append((dx, cuda(sx), dw, cuda(sw), torch.zeros((M, N), dtype=torch.bfloat16, device="cuda"),
+                        torch.zeros((M, N), dtype=torch.int32, device="cuda"), bits))
+    api.linear_int_batch(entries)
+    torch.cuda.synchronize()
+    for e, (acc_ref, y_ref) in zip(entries, refs):
+        np.testing.assert_array_equal(e[5].cpu().numpy().astype(np.int64), acc_ref)
+        assert_rows_close(bf16_to_f64(e[4]), y_ref)

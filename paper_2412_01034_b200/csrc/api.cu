@@ -160,7 +160,7 @@ size_t qil_linear_w4a16_workspace_size(int M, int N, int K, int group_size) {
     if (K % 128 != 0 || group_size % 128 != 0) return 0;
     size_t scratch = w4a16_skinny_workspace(M, N, K, group_size);
     if (w4a16_prefill_supported(M, N, K, group_size, QIL_LAYOUT_CANONICAL)) {
-        const size_t pf = w4a16_prefill_workspace(M, N, K);
+        const size_t pf = w4a16_prefill_workspace(M, N, K, group_size);
         if (pf > scratch) scratch = pf;
     }
     return w4a16_skinny_ws_offset() + scratch;  // serves every layout
@@ -261,7 +261,7 @@ static qil_status check_w8a16(const void* x, const void* qw, const void* sc, con
 size_t qil_linear_w8a16_workspace_size(int M, int N, int K, int group_size) {
     if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0) return 0;
     size_t scratch = 0;
-    if (w4a16_prefill_supported(M, N, K, group_size, QIL_LAYOUT_CANONICAL)) scratch = w4a16_prefill_workspace(M, N, K);
+    if (w4a16_prefill_supported(M, N, K, group_size, QIL_LAYOUT_CANONICAL)) scratch = w4a16_prefill_workspace(M, N, K, group_size);
     return w8a16_workspace() + scratch;
 }
 

@@ -80,7 +80,7 @@ qil_status launch_w4a16_skinny(const void* x, const uint32_t* qw, const void* sc
                                size_t ws_bytes, cudaStream_t st);
 
 bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout);
-size_t w4a16_prefill_workspace(int M, int N, int K);  // scratch of the split along K (0: none)
+size_t w4a16_prefill_workspace(int M, int N, int K, int G);  // tile counters + the fp32 parts of tiles that CTAs share
 qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scales, const void* zeros, void* y, int M, int N,
                                 int K, int G, int bits, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st);
 

@@ -2,25 +2,34 @@
 // App. A.4.2; M tokens, typically 280; 4-bit weights, and the 8-bit weights of the INT8 deployment point of
 // Sec. 5.4): a GEMM on tcgen05.mma kind::f16 (bf16 operands, fp32 accumulators in tensor memory).
 //
-// A CTA computes 256 output features x up to 144 tokens over a range of K.  The weights are the M side of the
-// MMAs (two accumulators of 128 features), the tokens the N side, so that every weight of the tile is dequantised
-// once for all its tokens.  Per step of 64 input features
-//   * one thread copies the 144 x 64 activation tile with one bulk tensor copy (128-byte swizzle; rows beyond M
-//     arrive as zeros),
-//   * another copies the packed 256 x 64 weight tile with one bulk tensor copy into a ring that runs eight steps
-//     ahead (the weights are the only operand that comes from HBM; loading them thread by thread, 16 or 32 bytes
-//     of a different row each, measured several times slower),
-//   * eight dequantising warps (thread = weight row) turn 64 codes of their row into bf16 - 128 + q by a byte
-//     permute, a multiply and a mask (exact), minus 128 + z (exact: integers below 256), times the group's scale
-//     rounded to bf16 (one rounding per weight) - and store them as the K-major operand in the 128-byte swizzle.
-//     The scales and zero points of two groups come with one 32-bit load each, four steps ahead: a 2-byte gather
-//     over 256 rows per step was the slowest thing in the loop,
-//   * one thread issues eight tcgen05.mma (128 x 144 x 16); tcgen05.commit recycles the stages (three).
-// The dequantising warps then read the accumulators (lane = feature) and write bf16 outputs, or, when K is split
-// over several CTAs to fill the GPU, fp32 partial tiles to the workspace; the last CTA of a tile to arrive (an
-// atomic counter, nobody waits) adds the partial tiles in split order, so the result does not depend on timing.
-// A stage of a ring is released only after the data read from it has been used (releasing it once the loads were
-// issued let the next copy overwrite words still in flight: seen as one warp's rows going wrong now and then).
+// A tile is 128 output features x up to 288 tokens.  The weights are the M side of the MMAs and live in TENSOR
+// MEMORY: the dequantising warps write the bf16 operand there with tcgen05.st (lane = feature, two bf16 per 32-bit
+// column), so that a dequantised weight never touches shared memory, needs no swizzle and no proxy fence, and the
+// MMAs read only the token tile from shared memory.  (With both operands in shared memory, 256 features x 144
+// tokens per CTA, the step time sat at what the shared-memory traffic of operand stores plus MMA reads allows,
+// whatever else was changed.)  Every weight of the tile is dequantised once for all its tokens.
+//
+// The launch is persistent: the (tile, step) pairs of the whole GEMM, a step being 64 input features, are numbered
+// tile by tile and dealt out to the CTAs in equal contiguous ranges, so that every SM has the same work whatever the
+// number of tiles (86 tiles of a 11008-wide projection on 148 SMs left 40 % of the GPU idle).  A CTA that holds only
+// part of a tile's steps writes its fp32 accumulators to the workspace; the last CTA of the tile to arrive (an
+// atomic counter, nobody waits) adds the parts in the order of the CTAs, so the result does not depend on timing.
+//
+// Per step
+//   * one thread copies the token tile with one or two bulk tensor copies (up to 144 tokens x 64 features each,
+//     128-byte swizzle; tokens beyond M arrive as zeros),
+//   * another copies the packed 128 x 64 weight tile with one bulk tensor copy into a ring that runs eight steps
+//     ahead (loading the weights thread by thread, 16 or 32 bytes of a different row each, measured several
+//     times slower),
+//   * eight dequantising warps (thread = weight row and half of the step) turn 32 codes into bf16 - 128 + q by a
+//     byte permute, a multiply and a mask (exact), minus 128 + z (exact: integers below 256), times the group's
+//     scale rounded to bf16 (one rounding per weight) - and store them to the operand ring in tensor memory (four
+//     stages of 32 columns).  The scales and zero points of two groups come with one 32-bit load each, a block of
+//     steps ahead: a 2-byte gather per step over all rows was the slowest thing in the loop,
+//   * one thread issues four or eight tcgen05.mma (128 x up to 144 x 16, A from tensor memory); tcgen05.commit
+//     recycles the stages.
+// The dequantising warps then read the accumulators (lane = feature) and write bf16 outputs or the fp32 part.
+// A stage of a ring is released only after the data read from it has been used.
 // Canonical layout only.  Every wait is bounded and polls; when one runs out QIL_ERR_TIMEOUT is recorded.
 #include <cuda.h>
 
@@ -32,15 +41,17 @@ namespace qil {
 
 namespace {
 
-constexpr int kTileF = 256, kHalfF = 128, kStepK = 64, kStages = 3, kBStages = 3, kMaxTN = 144;
-constexpr int kWRingBytes = 65536;                // ring of packed weight tiles (256 rows x 64 codes each)
-constexpr int kAHalf = kHalfF * kStepK * 2;       // one half of the weight operand tile (bf16): 8 KiB
-constexpr int kAStage = 2 * kAHalf;
-constexpr int kBStage = kMaxTN * kStepK * 2;      // activation tile: 9 KiB (a multiple of 1024)
-constexpr int kThreads = 352;                     // activation copy warp, MMA warp, 8 dequantising / read-out warps, weight copy warp
+constexpr int kTileF = 128, kStepK = 64, kAStages = 4, kBStages = 3, kMaxNN = 144, kMaxTT = 2 * kMaxNN;
+constexpr int kAccCols = kMaxTT;                  // accumulator columns (fp32, column = token)
+constexpr int kAStageCols = kStepK / 2;           // a step of the weight operand: 64 bf16 per lane = 32 columns
+constexpr int kBHalf = kMaxNN * kStepK * 2;       // up to 144 tokens x 64 bf16: 18 KiB (a multiple of 1024)
+constexpr int kBStage = 2 * kBHalf;
+constexpr int kWStages = 8;                       // ring of packed weight tiles (128 rows x 64 codes each)
+constexpr int kThreads = 352;                     // token copy warp, MMA warp, 8 dequantising / read-out warps, weight copy warp
 constexpr int kDqWarps = 8;
 constexpr int kMetaPre = 8;                       // steps by which a dequantising thread's scale / zero loads run ahead
 constexpr int kTmemCols = 512;
+static_assert(kAccCols + kAStages * kAStageCols <= kTmemCols, "tensor memory");
 constexpr int kCounterBytes = 16384;              // tile counters at the start of the scratch (same place as the skinny kernel's)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -50,13 +61,14 @@ struct PrefillParams {
     const __half* zeros;
     __nv_bfloat16* y;
     int M, N, K, G;
-    int g_shift;   // log2(G / 64) when that is a power of two, else -1
-    int pair_meta; // groups of 128 columns, an even number of them per row, K % 256 == 0: scales are loaded two groups at a time
-    int TN;        // tokens per tile (multiple of 16, <= 144)
-    int split;     // CTAs along K per tile
+    int g_shift;     // log2(G / 64) when that is a power of two, else -1
+    int pair_meta;   // groups of 128 columns, an even number of them per row, K % 256 == 0: scales are loaded two groups at a time
+    int NN, nh;      // tokens per MMA (multiple of 16, <= 144) and MMAs side by side (1 or 2): nh * NN tokens per tile
+    int mt;          // token tiles
+    int unit_steps;  // the ranges of the CTAs begin at multiples of this many steps
+    long long units; // unit_steps-sized pieces of the whole GEMM: tiles * (K / 64) / unit_steps
     int* status;
-    int* counters;
-    float* partials;
+    float* partials; // [2 * CTAs][nh * NN][128]
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -68,17 +80,6 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
 }
 __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -112,23 +113,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
                  : "memory");
-}
-// shared-memory operand descriptor, K-major, rows of 128 bytes in the 128-byte swizzle (tiles aligned to 1024 bytes)
-__device__ __forceinline__ uint64_t desc_swizzle128(uint32_t addr) {
-    uint64_t d = (uint64_t)((addr >> 4) & 0x3FFFu);
-    d |= (uint64_t)1 << 16;                        // (unused with a swizzle)
-    d |= (uint64_t)(1024u >> 4) << 32;             // 8 rows of 128 bytes
-    d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                        // 128-byte swizzle
-    return d;
-}
-// D[128 x N] (+)= A[128 x 16 bf16] * B[N x 16 bf16]^T, fp32 accumulate, operands in shared memory
-__device__ __forceinline__ void mma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
-        : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -169,50 +153,94 @@ __device__ __forceinline__ uint2 dequant4_w8(uint32_t w, float offf, __nv_bfloat
     return make_uint2(o[0], o[1]);
 }
 
+// D[128 x N] (+)= A[128 x 16 bf16] * B[N x 16 bf16]^T with A in tensor memory (lane = row, 8 columns of two bf16) and
+// B in shared memory.  The descriptor of B comes as its two 32-bit halves: the issuing thread keeps the high half and
+// the low half of every stage ready and adds small constants, because its own instruction stream - descriptors put
+// together from 64-bit shifts for every MMA, divisions for the ring positions - was what set the pace of the whole
+// pipeline before (a step took the same time with or without the MMAs' work, at any MMA width).
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 bd, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 16 consecutive 32-bit columns of this thread's lane of tensor memory
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&d)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]), "=r"(d[8]),
+          "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 16; ++j) asm volatile("" : "+r"(d[j]));
+}
+
+// The CTA's next run of steps inside one tile: steps [s0, s1) of tile `tile`.  g walks the CTA's range of numbered steps.
+struct Segment {
+    int tile, s0, s1;
+};
+__device__ __forceinline__ bool next_segment(long long& g, long long g_end, int S, Segment& sg) {
+    if (g >= g_end) return false;
+    sg.tile = (int)(g / S);
+    sg.s0 = (int)(g - (long long)sg.tile * S);
+    const long long n = min((long long)(S - sg.s0), g_end - g);
+    sg.s1 = sg.s0 + (int)n;
+    g += n;
+    return true;
+}
+// ranges of the CTAs in units: CTA c holds [units * c / C, units * (c + 1) / C)
+__device__ __forceinline__ long long range_begin(long long units, int C, int c) { return units * c / C; }
+__device__ __forceinline__ int cta_of_unit(long long units, int C, long long u) { return (int)(((u + 1) * C - 1) / units); }
+
 template <int kBits>
 __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid_constant__ CUtensorMap tmap_x,
                                                                    const __grid_constant__ CUtensorMap tmap_w,
                                                                    const PrefillParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    // (the swizzled activation tiles need 1024-byte alignment)
+    // (the swizzled token tiles need 1024-byte alignment)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char* sb = smem;                                  // [kStages][kBStage] activations
-    unsigned char* sa = smem + (size_t)kBStages * kBStage;     // [kStages][kAStage] weights
-    constexpr int kWStage = kTileF * kStepK * kBits / 8;       // packed weight tile: 8 KiB (4-bit), 16 KiB (8-bit)
-    constexpr int kWStages = kWRingBytes / kWStage;
-    unsigned char* sw = sa + (size_t)kStages * kAStage;        // [kWStages][256 rows][kStepK * kBits / 8 bytes]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sw + kWRingBytes);
-    const uint32_t full_a0 = smem_u32(bars), free0 = smem_u32(bars + kStages), done0 = smem_u32(bars + 2 * kStages);
-    const uint32_t full_b0 = smem_u32(bars + 2 * kStages + 1), free_b0 = smem_u32(bars + 2 * kStages + 1 + kBStages);
-    uint64_t* wbars = bars + 2 * kStages + 1 + 2 * kBStages;
+    unsigned char* sb = smem;                                  // [kBStages][kBStage] tokens
+    constexpr int kWStage = kTileF * kStepK * kBits / 8;       // packed weight tile: 4 KiB (4-bit), 8 KiB (8-bit)
+    unsigned char* sw = sb + (size_t)kBStages * kBStage;       // [kWStages][128 rows][kStepK * kBits / 8 bytes]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sw + (size_t)kWStages * kWStage);
+    const uint32_t full_a0 = smem_u32(bars), free_a0 = smem_u32(bars + kAStages);
+    const uint32_t full_b0 = smem_u32(bars + 2 * kAStages), free_b0 = smem_u32(bars + 2 * kAStages + kBStages);
+    uint64_t* wbars = bars + 2 * kAStages + 2 * kBStages;
     const uint32_t full_w0 = smem_u32(wbars), free_w0 = smem_u32(wbars + kWStages);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wbars + 2 * kWStages);
-    int* is_last = reinterpret_cast<int*>(tmem_slot + 1);
+    uint64_t* obars = wbars + 2 * kWStages;
+    const uint32_t done0 = smem_u32(obars), acc_free0 = smem_u32(obars + 1);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(obars + 2);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n0 = blockIdx.x * kTileF, m0 = blockIdx.y * p.TN;
-    const int steps_all = p.K / kStepK;
-    const int z = blockIdx.z;
-    // (with pair_meta the splits begin at multiples of 4 steps = two groups of 128 columns)
-    const int s_unit = p.pair_meta ? 4 : 1;
-    const int s_begin = (int)((long long)(steps_all / s_unit) * z / p.split) * s_unit,
-              s_end = (int)((long long)(steps_all / s_unit) * (z + 1) / p.split) * s_unit;
-    const int steps = s_end - s_begin;
+    const int S = p.K / kStepK;                   // steps per tile
+    const int C = (int)gridDim.x, cta = (int)blockIdx.x;
+    const long long g_begin = range_begin(p.units, C, cta) * p.unit_steps, g_end = range_begin(p.units, C, cta + 1) * p.unit_steps;
+    const int TT = p.NN * p.nh;
     const int ng = p.K / p.G;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kAStages; ++s) {
             mbar_init(full_a0 + 8 * s, kDqWarps);   // the dequantising warps
-            mbar_init(free0 + 8 * s, 1);     // the commit of the MMAs that read the stage
+            mbar_init(free_a0 + 8 * s, 1);          // the commit of the MMAs that read the stage
         }
         for (int s = 0; s < kBStages; ++s) {
-            mbar_init(full_b0 + 8 * s, 1);   // the copy (transaction bytes)
+            mbar_init(full_b0 + 8 * s, 1);   // the copies (transaction bytes)
             mbar_init(free_b0 + 8 * s, 1);   // the commit of the MMAs that read the stage
         }
-        mbar_init(done0, 1);
         for (int s = 0; s < kWStages; ++s) {
-            mbar_init(full_w0 + 8 * s, 1);   // the copy (transaction bytes)
+            mbar_init(full_w0 + 8 * s, 1);          // the copy (transaction bytes)
             mbar_init(free_w0 + 8 * s, kDqWarps);   // the dequantising warps have read the tile
         }
+        mbar_init(done0, 1);             // the commit after the last MMA of a segment
+        mbar_init(acc_free0, kDqWarps);  // the accumulators of a segment have been read
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -226,178 +254,205 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
     bool ok = true;
 
     if (warp == 0) {
-        // ---------------- activation copies ----------------
+        // ---------------- token copies ----------------
         if (lane == 0) {
-            int issued = 0;
-            for (int i = 0; i < steps; ++i, ++issued) {
-                const int s = i % kBStages, use = i / kBStages;
-                ok = mbar_wait(free_b0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
-                if (!ok) break;
-                mbar_expect_tx(full_b0 + 8 * s, (uint32_t)p.TN * kStepK * 2);
-                tma_load_2d(smem_u32(sb + (size_t)s * kBStage), &tmap_x, (s_begin + i) * kStepK, m0, full_b0 + 8 * s);
+            int it = 0;
+            Segment sg;
+            for (long long g = g_begin; ok && next_segment(g, g_end, S, sg);) {
+                const int m0 = (sg.tile % p.mt) * TT;
+                for (int i = sg.s0; i < sg.s1; ++i, ++it) {
+                    const int s = it % kBStages, use = it / kBStages;
+                    ok = mbar_wait(free_b0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
+                    if (!ok) break;
+                    mbar_expect_tx(full_b0 + 8 * s, (uint32_t)TT * kStepK * 2);
+                    for (int hb = 0; hb < p.nh; ++hb)
+                        tma_load_2d(smem_u32(sb + (size_t)s * kBStage) + (uint32_t)hb * p.NN * (kStepK * 2), &tmap_x, i * kStepK,
+                                    m0 + hb * p.NN, full_b0 + 8 * s);
+                }
             }
             // no copy may still be in flight when the CTA retires (this wait also holds after a time-out elsewhere)
-            for (int back = 0; back < kBStages && back < issued; ++back) {
-                const int i = issued - 1 - back;
+            for (int back = 0; back < kBStages && back < it; ++back) {
+                const int i = it - 1 - back;
                 (void)mbar_wait(full_b0 + 8 * (i % kBStages), (i / kBStages) & 1);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)p.TN >> 3) << 17) | (((uint32_t)kHalfF >> 4) << 24);
-            for (int i = 0; i < steps; ++i) {
-                const int s = i % kStages, use = i / kStages, bs = i % kBStages, buse = i / kBStages;
-                ok = mbar_wait(full_a0 + 8 * s, use & 1) && mbar_wait(full_b0 + 8 * bs, buse & 1);
-                if (!ok) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_addr = smem_u32(sa + (size_t)s * kAStage), b_addr = smem_u32(sb + (size_t)bs * kBStage);
-#pragma unroll
-                for (int k = 0; k < kStepK / 16; ++k) {  // K = 16 each: 32 bytes of a swizzled row of either operand
-                    const uint64_t bd = desc_swizzle128(b_addr + 32 * k);
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        mma_bf16_ss(tmem + 256 * h, desc_swizzle128(a_addr + h * kAHalf + 32 * k), bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)p.NN >> 3) << 17) | (((uint32_t)kTileF >> 4) << 24);
+            // descriptor of a token tile (K-major, 128-byte swizzle, 8 rows = 1024 bytes apart, version 1): its high half is
+            // a constant, its low half the address in 16-byte units
+            const uint32_t d_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            const uint32_t b_lo0 = ((smem_u32(sb) >> 4) & 0x3FFFu) | (1u << 16);
+            const uint32_t half_lo = ((uint32_t)p.NN * (kStepK * 2)) >> 4;   // the second MMA's tokens
+            const bool two = p.nh == 2;
+            uint32_t s = 0, aph = 0, bs = 0, bph = 0;
+            int seg = 0;
+            Segment sg;
+            for (long long g = g_begin; ok && next_segment(g, g_end, S, sg); ++seg) {
+                if (seg > 0) {
+                    ok = mbar_wait(acc_free0, (seg - 1) & 1);   // the accumulators of the segment before have been read
+                    if (!ok) break;
                 }
-                tc_commit(free0 + 8 * s);
-                tc_commit(free_b0 + 8 * bs);
+                uint32_t acc = 0u;                               // the first MMAs of a segment overwrite the accumulators
+#pragma unroll 1
+                for (int i = sg.s0; i < sg.s1; ++i) {
+                    ok = mbar_wait(full_a0 + 8 * s, aph) && mbar_wait(full_b0 + 8 * bs, bph);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_tmem = tmem + (uint32_t)kAccCols + s * kAStageCols;
+                    const uint32_t b_lo = b_lo0 + bs * (kBStage >> 4);
+#pragma unroll
+                    for (int k = 0; k < kStepK / 16; ++k) {  // K = 16 each: 8 columns of A, 32 bytes of a swizzled row of B
+                        mma_bf16_ts(tmem, a_tmem + 8 * k, b_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
+                        if (two) mma_bf16_ts(tmem + (uint32_t)p.NN, a_tmem + 8 * k, b_lo + half_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
+                    }
+                    acc = 1u;
+                    tc_commit(free_a0 + 8 * s);
+                    tc_commit(free_b0 + 8 * bs);
+                    if (++s == kAStages) { s = 0; aph ^= 1u; }
+                    if (++bs == kBStages) { bs = 0; bph ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(done0);   // every MMA of the segment is complete when this arrival happens
             }
-            // all MMAs of this thread are complete when this arrival happens (also needed before tensor memory is released)
-            tc_commit(done0);
-            if (!mbar_wait(done0, 0)) ok = false;
+            // all MMAs are complete before tensor memory is released
+            if (ok && seg > 0 && !mbar_wait(done0, (seg - 1) & 1)) ok = false;
         }
     } else if (warp == 2 + kDqWarps) {
         // ---------------- packed weight copies (rows beyond N arrive as zeros) ----------------
         if (lane == 0) {
-            int issued = 0;
-            for (int i = 0; i < steps; ++i, ++issued) {
-                const int s = i % kWStages, use = i / kWStages;
-                ok = mbar_wait(free_w0 + 8 * s, (use & 1) ^ 1);
-                if (!ok) break;
-                mbar_expect_tx(full_w0 + 8 * s, (uint32_t)kWStage);
-                tma_load_2d(smem_u32(sw + (size_t)s * kWStage), &tmap_w, (s_begin + i) * (kStepK * kBits / 8), n0, full_w0 + 8 * s);
+            int it = 0;
+            Segment sg;
+            for (long long g = g_begin; ok && next_segment(g, g_end, S, sg);) {
+                const int n0 = (sg.tile / p.mt) * kTileF;
+                for (int i = sg.s0; i < sg.s1; ++i, ++it) {
+                    const int s = it % kWStages, use = it / kWStages;
+                    ok = mbar_wait(free_w0 + 8 * s, (use & 1) ^ 1);
+                    if (!ok) break;
+                    mbar_expect_tx(full_w0 + 8 * s, (uint32_t)kWStage);
+                    tma_load_2d(smem_u32(sw + (size_t)s * kWStage), &tmap_w, i * (kStepK * kBits / 8), n0, full_w0 + 8 * s);
+                }
             }
-            for (int back = 0; back < kWStages && back < issued; ++back) {
-                const int i = issued - 1 - back;
+            for (int back = 0; back < kWStages && back < it; ++back) {
+                const int i = it - 1 - back;
                 (void)mbar_wait(full_w0 + 8 * (i % kWStages), (i / kWStages) & 1);
             }
         }
     } else {
-        // ---------------- dequantising warps: a thread owns half a step (32 codes) of weight row n0 + r ----------------
-        const int r = tid - 64;
-        const int h = r >> 7, rr = r & 127;
-        const bool w_row = n0 + r < p.N;
-        const size_t nrow = (size_t)(n0 + (w_row ? r : 0));
-        const __half* sr = p.scales + nrow * ng;
-        const __half* zr = p.zeros + nrow * ng;
-        // scale and zero point of the step's group, loaded kMetaPre steps ahead
-        uint32_t meta[kMetaPre];
-        auto fetch_meta = [&](int step) -> uint32_t {
-            const int g = p.g_shift >= 0 ? (step >> p.g_shift) : step * kStepK / p.G;  // steps per group: a power of two, usually
-            return w_row ? ((uint32_t)__half_as_ushort(__ldg(sr + g)) | ((uint32_t)__half_as_ushort(__ldg(zr + g)) << 16)) : 0u;
-        };
-#pragma unroll
-        for (int u = 0; u < kMetaPre; ++u) meta[u] = (u < steps && !p.pair_meta) ? fetch_meta(s_begin + u) : 0u;
-        // shared-memory addresses as 32-bit numbers, ring positions kept incrementally (this loop is issue bound)
-        constexpr int kRowW = kStepK * kBits / 8;                    // bytes of a row in the packed tile
-        const uint32_t w_row0 = smem_u32(sw) + (uint32_t)r * kRowW;
-        // weight operand: rows of 128 bytes (one step), 128-byte swizzle: 16-byte piece c of row rr sits at piece c ^ (rr % 8)
-        const uint32_t a_row0 = smem_u32(sa) + (uint32_t)h * kAHalf + (uint32_t)rr * 128;
-        const uint32_t a_xor = (uint32_t)(rr & 7), c_first = 0u;
+        // ---------------- dequantising warps: a thread owns half a step (32 codes) of weight row rr of the tile ----------------
+        // (a warp reaches the 32 lanes of tensor memory its number modulo 4 selects; two warps share a quarter and
+        //  split the step's columns)
+        const int q = warp & 3, hh = (warp - 2) >> 2;
+        const int rr = 32 * q + lane;
+        constexpr int kRowW = kStepK * kBits / 8;                     // bytes of a row in the packed tile
+        const uint32_t w_row0 = smem_u32(sw) + (uint32_t)rr * kRowW + (uint32_t)hh * (kRowW / 2);
+        const uint32_t a_lane = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(kAccCols + hh * (kAStageCols / 2));
         uint32_t s = 0, sph = 1;     // stage of the operand ring and the parity of "stage free" to wait for
         uint32_t ws_ = 0, wph = 0;   // stage of the packed ring and the parity of "tile landed"
         auto one_step = [&](uint32_t m) -> bool {
             if (!mbar_wait(full_w0 + 8 * ws_, wph)) return false;     // the packed tile has landed
-            uint32_t pk[kBits == 4 ? 8 : 16];
+            uint32_t pk[kBits == 4 ? 4 : 8];
 #pragma unroll
-            for (int q = 0; q < (kBits == 4 ? 2 : 4); ++q)
+            for (int c = 0; c < (kBits == 4 ? 1 : 2); ++c)
                 asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                             : "=r"(pk[4 * q]), "=r"(pk[4 * q + 1]), "=r"(pk[4 * q + 2]), "=r"(pk[4 * q + 3])
-                             : "r"(w_row0 + ws_ * kWStage + 16 * q));
-            if (!mbar_wait(free0 + 8 * s, sph)) return false;         // the MMAs that read this stage last are complete
-            const uint32_t a_st = a_row0 + s * kAStage;
+                             : "=r"(pk[4 * c]), "=r"(pk[4 * c + 1]), "=r"(pk[4 * c + 2]), "=r"(pk[4 * c + 3])
+                             : "r"(w_row0 + ws_ * kWStage + 16 * c));
             const float sf = __half2float(__ushort_as_half((unsigned short)(m & 0xFFFFu)));
             const float zf = __half2float(__ushort_as_half((unsigned short)(m >> 16)));
             const __nv_bfloat162 sc = __float2bfloat162_rn(sf);
+            uint32_t v[16];
             if constexpr (kBits == 4) {
                 const __nv_bfloat162 off = __float2bfloat162_rn(zf + 128.f);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint4 v = dequant8_w4(pk[c], off, sc);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a_st + (((c_first + c) ^ a_xor) << 4)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 d = dequant8_w4(pk[c], off, sc);
+                    v[4 * c] = d.x; v[4 * c + 1] = d.y; v[4 * c + 2] = d.z; v[4 * c + 3] = d.w;
                 }
             } else {
                 const float offf = 8388608.f + zf;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    const uint2 lo = dequant4_w8(pk[2 * c], offf, sc), hi = dequant4_w8(pk[2 * c + 1], offf, sc);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a_st + (((c_first + c) ^ a_xor) << 4)), "r"(lo.x), "r"(lo.y), "r"(hi.x), "r"(hi.y) : "memory");
+                    const uint2 d = dequant4_w8(pk[c], offf, sc);
+                    v[2 * c] = d.x; v[2 * c + 1] = d.y;
                 }
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read through the async proxy
+            if (!mbar_wait(free_a0 + 8 * s, sph)) return false;       // the MMAs that read this stage last are complete
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            tmem_st16(a_lane + s * kAStageCols, v);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
                 // (the packed tile is released only now: its words were still being consumed above)
                 mbar_arrive(free_w0 + 8 * ws_);
                 mbar_arrive(full_a0 + 8 * s);
             }
-            if (++s == kStages) { s = 0; sph ^= 1u; }
+            if (++s == kAStages) { s = 0; sph ^= 1u; }
             if (++ws_ == kWStages) { ws_ = 0; wph ^= 1u; }
             return true;
         };
-        int i = 0;
-        if (p.pair_meta) {
-            // One 32-bit load fetches the scales of two groups (4 steps), another their zero points, one block of
-            // steps ahead: a load per step and thread would be a 2-byte gather over 256 rows, and those gathers, not
-            // the arithmetic, then set the pace of the whole pipeline.
-            const uint32_t* s2 = reinterpret_cast<const uint32_t*>(sr);
-            const uint32_t* z2 = reinterpret_cast<const uint32_t*>(zr);
-            uint32_t ns = w_row ? __ldg(s2 + (s_begin >> 2)) : 0u, nz = w_row ? __ldg(z2 + (s_begin >> 2)) : 0u;
-            for (; ok && i < steps; i += 4) {
-                const uint32_t cs = ns, cz = nz;
-                if (i + 4 < steps) {
-                    ns = w_row ? __ldg(s2 + ((s_begin + i + 4) >> 2)) : 0u;
-                    nz = w_row ? __ldg(z2 + ((s_begin + i + 4) >> 2)) : 0u;
+        int seg = 0;
+        Segment sg;
+        for (long long g = g_begin, g_seg = g_begin; ok && next_segment(g, g_end, S, sg); ++seg, g_seg = g) {
+            const int n0 = (sg.tile / p.mt) * kTileF, m0 = (sg.tile % p.mt) * TT;
+            const bool w_row = n0 + rr < p.N;
+            const size_t nrow = (size_t)(n0 + (w_row ? rr : 0));
+            const __half* sr = p.scales + nrow * ng;
+            const __half* zr = p.zeros + nrow * ng;
+            const int s_begin = sg.s0, steps = sg.s1 - sg.s0;
+            int i = 0;
+            if (p.pair_meta) {
+                // One 32-bit load fetches the scales of two groups (4 steps), another their zero points, one block of
+                // steps ahead: a load per step and thread would be a 2-byte gather over all rows, and those gathers,
+                // not the arithmetic, then set the pace of the whole pipeline.  (Segments begin at multiples of 4 steps.)
+                const uint32_t* s2 = reinterpret_cast<const uint32_t*>(sr);
+                const uint32_t* z2 = reinterpret_cast<const uint32_t*>(zr);
+                uint32_t ns = w_row ? __ldg(s2 + (s_begin >> 2)) : 0u, nz = w_row ? __ldg(z2 + (s_begin >> 2)) : 0u;
+                for (; ok && i < steps; i += 4) {
+                    const uint32_t cs = ns, cz = nz;
+                    if (i + 4 < steps) {
+                        ns = w_row ? __ldg(s2 + ((s_begin + i + 4) >> 2)) : 0u;
+                        nz = w_row ? __ldg(z2 + ((s_begin + i + 4) >> 2)) : 0u;
+                    }
+                    const uint32_t m_lo = (cs & 0xFFFFu) | (cz << 16), m_hi = (cs >> 16) | (cz & 0xFFFF0000u);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (ok) ok = one_step(u < 2 ? m_lo : m_hi);
                 }
-                const uint32_t m_lo = (cs & 0xFFFFu) | (cz << 16), m_hi = (cs >> 16) | (cz & 0xFFFF0000u);
+            } else {
+                // scale and zero point of the step's group, loaded kMetaPre steps ahead
+                auto fetch_meta = [&](int step) -> uint32_t {
+                    const int gi = p.g_shift >= 0 ? (step >> p.g_shift) : step * kStepK / p.G;
+                    return w_row ? ((uint32_t)__half_as_ushort(__ldg(sr + gi)) | ((uint32_t)__half_as_ushort(__ldg(zr + gi)) << 16)) : 0u;
+                };
+                uint32_t meta[kMetaPre];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (ok) ok = one_step(u < 2 ? m_lo : m_hi);
+                for (int u = 0; u < kMetaPre; ++u) meta[u] = u < steps ? fetch_meta(s_begin + u) : 0u;
+                for (; ok && i + kMetaPre <= steps; i += kMetaPre) {
+#pragma unroll
+                    for (int u = 0; u < kMetaPre; ++u) {
+                        if (ok) ok = one_step(meta[u]);
+                        if (i + u + kMetaPre < steps) meta[u] = fetch_meta(s_begin + i + u + kMetaPre);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kMetaPre; ++u)   // the last, partial block of steps
+                    if (ok && i + u < steps) ok = one_step(meta[u]);
             }
-            i = steps;
-        }
-        for (; ok && i + kMetaPre <= steps; i += kMetaPre) {
-#pragma unroll
-            for (int u = 0; u < kMetaPre; ++u) {
-                if (ok) ok = one_step(meta[u]);
-                if (i + u + kMetaPre < steps) meta[u] = fetch_meta(s_begin + i + u + kMetaPre);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kMetaPre; ++u)   // the last, partial block of steps
-            if (ok && i + u < steps) ok = one_step(meta[u]);
-        // ---------------- read-out: lane = feature 32 q + lane of half h ----------------
-        if (ok) ok = mbar_wait(done0, 0);
-        if (ok) {
+            // ---------------- read-out: lane = feature; the two warps of a quarter take alternate blocks of 16 tokens ----------------
+            if (ok) ok = mbar_wait(done0, seg & 1);
+            if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int q = warp & 3;                       // the quarter of the tensor-memory lanes this warp may read
-            const int f = 128 * h + 32 * q + lane;        // (h from the thread's row: of every 8 warps the first 4 read half 0)
-            const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + 256u * (uint32_t)h;
-            const int n = n0 + f;
-            const int tile_id = blockIdx.x * gridDim.y + blockIdx.y;
-            float* part = p.split > 1 ? p.partials + ((size_t)(tile_id * p.split + z) * p.TN) * kTileF + f : nullptr;
-            const int c_begin = 0, c_end = p.TN;
+            const bool whole = sg.s0 == 0 && sg.s1 == S;               // the CTA holds every step of the tile
+            const int n = n0 + rr;
+            // the part of a tile a CTA begins its range with goes to slot 2 * cta, the part it ends with to slot 2 * cta + 1
+            float* part = whole ? nullptr : p.partials + ((size_t)(2 * cta + (g_seg == g_begin ? 0 : 1)) * TT) * kTileF + rr;
+            const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16);
 #pragma unroll 1
-            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+            for (int c0 = 16 * hh; c0 < TT; c0 += 32) {
                 uint32_t d[16];
-                asm volatile(
-                    "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                    : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]), "=r"(d[8]),
-                      "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
-                    : "r"(taddr + (uint32_t)c0));
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int j = 0; j < 16; ++j) asm volatile("" : "+r"(d[j]));
+                tmem_ld16(taddr + (uint32_t)c0, d);
                 if (part) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) __stcg(part + (size_t)(c0 + j) * kTileF, __uint_as_float(d[j]));
@@ -407,49 +462,52 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                         if (m0 + c0 + j < p.M) p.y[(size_t)(m0 + c0 + j) * p.N + n] = __float2bfloat16_rn(__uint_as_float(d[j]));
                 }
             }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_free0);
         }
     }
     if (!ok && p.status) atomicOr(p.status, (int)QIL_ERR_TIMEOUT);
-    if (p.split > 1) {
-        // the last CTA of the tile to arrive adds the partial tiles in split order
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            const int tile_id = blockIdx.x * gridDim.y + blockIdx.y;
-            const int prev = atomicAdd(&p.counters[tile_id], 1);
-            *is_last = (prev == p.split - 1);
-            if (*is_last) p.counters[tile_id] = 0;  // ready for the next call
-        }
-        __syncthreads();
-        if (*is_last && tid >= 64 && tid < 64 + kTileF) {
-            __threadfence();
-            const int f = tid - 64, n = n0 + f;
-            const int tile_id = blockIdx.x * gridDim.y + blockIdx.y;
-            const float* base = p.partials + ((size_t)tile_id * p.split * p.TN) * kTileF + f;
-            if (n < p.N) {
-                for (int t0 = 0; t0 < p.TN && m0 + t0 < p.M; t0 += 8) {  // 8 tokens x split loads in flight
-                    float acc[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-                    for (int sl = 0; sl < p.split; ++sl) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[j] += __ldcg(base + ((size_t)sl * p.TN + t0 + j) * kTileF);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        if (m0 + t0 + j < p.M) p.y[(size_t)(m0 + t0 + j) * p.N + n] = __float2bfloat16_rn(acc[j]);
-                }
-            }
-        }
-    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols));
 }
 
-constexpr size_t kSmemBytes = (size_t)kStages * kAStage + (size_t)kBStages * kBStage + kWRingBytes +
-                              (2 * kStages + 1 + 2 * kBStages + 2 * 12) * 8 + 16 + 1024;
+// Adds the parts of every tile that several CTAs share, in the order of the CTAs, and writes the bf16 outputs.
+// grid (tiles, blocks of 8 tokens); a warp = one token, a thread = 4 features.
+__global__ void __launch_bounds__(256) w4a16_prefill_reduce_kernel(const PrefillParams p, int C) {
+    const int tile = blockIdx.x, S = p.K / kStepK;
+    const long long su = S / p.unit_steps;                  // units per tile
+    const int c_first = cta_of_unit(p.units, C, (long long)tile * su), c_last = cta_of_unit(p.units, C, (long long)tile * su + su - 1);
+    if (c_first == c_last) return;                          // one CTA held the whole tile and wrote the outputs itself
+    const int TT = p.NN * p.nh;
+    const int n0 = (tile / p.mt) * kTileF, m0 = (tile % p.mt) * TT;
+    const int t = blockIdx.y * 8 + (threadIdx.x >> 5), f = 4 * (threadIdx.x & 31);
+    if (t >= TT || m0 + t >= p.M || n0 + f >= p.N) return;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int cc = c_first; cc <= c_last; ++cc) {
+        // the part a CTA begins its range with is in slot 2 * cta, the part it ends with in slot 2 * cta + 1
+        const int slot = 2 * cc + (range_begin(p.units, C, cc) * p.unit_steps >= (long long)tile * S ? 0 : 1);
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(p.partials + ((size_t)slot * TT + t) * kTileF + f));
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    __nv_bfloat16* out = p.y + (size_t)(m0 + t) * p.N + n0 + f;
+    if ((p.N & 3) == 0) {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        uint2 o;
+        o.x = *reinterpret_cast<const uint32_t*>(&lo);
+        o.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(out) = o;
+    } else {
+        const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+        for (int j = 0; j < 4 && n0 + f + j < p.N; ++j) out[j] = __float2bfloat16_rn(a4[j]);
+    }
+}
+
+constexpr size_t kSmemBytes = (size_t)kBStages * kBStage + (size_t)kWStages * (kTileF * kStepK) +
+                              (2 * kAStages + 2 * kBStages + 2 * kWStages + 2) * 8 + 16 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -474,27 +532,29 @@ EncodeFn encode_fn() {
 }
 
 struct PrefillPlan {
-    int chunks, TN, ftiles, split;
+    int mt, NN, nh, ftiles, ctas, unit_steps;
+    long long units;
 };
 
-PrefillPlan plan_prefill(int M, int N, int K) {
+// with_parts: the workspace can hold the parts of tiles that several CTAs share; without it every CTA gets whole tiles.
+PrefillPlan plan_prefill(int M, int N, int K, int G, bool with_parts) {
     PrefillPlan pl;
-    pl.chunks = (M + kMaxTN - 1) / kMaxTN;
-    const int per = (M + pl.chunks - 1) / pl.chunks;
-    pl.TN = (per + 15) / 16 * 16;
+    pl.mt = (M + kMaxTT - 1) / kMaxTT;
+    const int per = (M + pl.mt - 1) / pl.mt;
+    pl.nh = per > kMaxNN ? 2 : 1;
+    pl.NN = ((per + pl.nh - 1) / pl.nh + 15) / 16 * 16;
     pl.ftiles = (N + kTileF - 1) / kTileF;
-    // K is split where that fills the GPU.  Cost in steps: waves x (steps per CTA + the fixed cost of a CTA, about 12
-    // steps: launch, first loads, read-out) + the reduction of the partial tiles (about 10 steps), as measured.
-    const int tiles = pl.ftiles * pl.chunks, steps = K / kStepK, sms = num_sms();
-    int best = 1;
-    long best_cost = -1;
-    for (int s = 1; s <= 8; ++s) {
-        if (s > 1 && steps / s < 4) break;
-        const long waves = ((long)tiles * s + sms - 1) / sms;
-        const long cost = waves * ((steps + s - 1) / s + 12) + (s > 1 ? 10 : 0);
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
-    }
-    pl.split = best;
+    const int S = K / kStepK, sms = num_sms();
+    const long long tiles = (long long)pl.ftiles * pl.mt;
+    const bool pair = G == 128 && (K / G) % 2 == 0 && K % 256 == 0;
+    pl.unit_steps = with_parts ? (pair ? 4 : 1) : S;
+    pl.units = tiles * (S / pl.unit_steps);
+    // a CTA is worth launching for about eight steps; never more CTAs than SMs or units
+    long long c = with_parts ? tiles * S / 8 : tiles;
+    if (c > sms) c = sms;
+    if (c > pl.units) c = pl.units;
+    if (c < 1) c = 1;
+    pl.ctas = (int)c;
     return pl;
 }
 
@@ -502,33 +562,32 @@ PrefillPlan plan_prefill(int M, int N, int K) {
 
 bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout) {
     return layout == QIL_LAYOUT_CANONICAL && M > 8 && N >= 1 && K % kStepK == 0 && G % kStepK == 0 && K % G == 0 &&
-           (long long)((N + kTileF - 1) / kTileF) * ((M + kMaxTN - 1) / kMaxTN) <= kCounterBytes / 4 && (M + kMaxTN - 1) / kMaxTN <= 65535;
+           (long long)((N + kTileF - 1) / kTileF) * ((M + kMaxTT - 1) / kMaxTT) <= kCounterBytes / 4;
 }
 
-// Scratch the split along K needs (0 when K is not split): tile counters, then fp32 partial tiles.
-size_t w4a16_prefill_workspace(int M, int N, int K) {
-    const PrefillPlan pl = plan_prefill(M, N, K);
-    if (pl.split == 1) return 0;
-    return (size_t)kCounterBytes + (size_t)pl.ftiles * pl.chunks * pl.split * pl.TN * kTileF * sizeof(float);
+// Scratch for the parts of tiles that several CTAs share: tile counters, then two fp32 tiles per CTA.
+size_t w4a16_prefill_workspace(int M, int N, int K, int G) {
+    const PrefillPlan pl = plan_prefill(M, N, K, G, true);
+    return (size_t)kCounterBytes + (size_t)2 * pl.ctas * pl.nh * pl.NN * kTileF * sizeof(float);
 }
 
 // status (optional): receives QIL_ERR_TIMEOUT if a bounded device-side wait runs out.  scratch: as sized above; when it
-// is missing or too small K is not split.
+// is missing or too small every CTA computes whole tiles.
 qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scales, const void* zeros, void* y, int M, int N,
                                 int K, int G, int bits, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st) {
-    PrefillPlan pl = plan_prefill(M, N, K);
-    if (pl.split > 1 && (scratch == nullptr || scratch_bytes < w4a16_prefill_workspace(M, N, K))) pl.split = 1;
+    const bool with_parts = scratch != nullptr && scratch_bytes >= w4a16_prefill_workspace(M, N, K, G);
+    const PrefillPlan pl = plan_prefill(M, N, K, G, with_parts);
     const EncodeFn enc = encode_fn();
     if (!enc) return QIL_ERR_CUDA;
     CUtensorMap tmap;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kStepK, (cuuint32_t)pl.TN};
+    const cuuint32_t box[2] = {(cuuint32_t)kStepK, (cuuint32_t)pl.NN};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return QIL_ERR_CUDA;
-    // the packed weights as a byte matrix [N][K * bits / 8]: box = 64 codes x 256 rows, no swizzle
+    // the packed weights as a byte matrix [N][K * bits / 8]: box = 64 codes x 128 rows, no swizzle
     CUtensorMap tmap_w;
     const cuuint64_t wdims[2] = {(cuuint64_t)K * bits / 8, (cuuint64_t)N};
     const cuuint64_t wstrides[1] = {(cuuint64_t)K * bits / 8};
@@ -548,12 +607,12 @@ qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scale
     if ((spg & (spg - 1)) == 0)
         for (int sh = 0; sh < 31; ++sh)
             if ((1 << sh) == spg) p.g_shift = sh;
-    p.TN = pl.TN;
-    p.split = pl.split;
+    p.NN = pl.NN; p.nh = pl.nh; p.mt = pl.mt;
+    p.unit_steps = pl.unit_steps;
+    p.units = pl.units;
     p.status = status;
-    p.counters = reinterpret_cast<int*>(scratch);
-    p.partials = scratch ? reinterpret_cast<float*>(static_cast<char*>(scratch) + kCounterBytes) : nullptr;
-    const dim3 grid(pl.ftiles, pl.chunks, pl.split);
+    p.partials = with_parts ? reinterpret_cast<float*>(static_cast<char*>(scratch) + kCounterBytes) : nullptr;
+    const dim3 grid(pl.ctas);
     cudaError_t e;
     if (bits == 8) {
         e = cudaFuncSetAttribute(w4a16_prefill_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
@@ -565,6 +624,10 @@ qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scale
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return QIL_ERR_CUDA;
+    }
+    if (with_parts && pl.ctas > 1) {
+        const dim3 rgrid((unsigned)(pl.ftiles * pl.mt), (unsigned)((pl.nh * pl.NN + 7) / 8));
+        w4a16_prefill_reduce_kernel<<<rgrid, 256, 0, st>>>(p, pl.ctas);
     }
     return launch_status();
 }

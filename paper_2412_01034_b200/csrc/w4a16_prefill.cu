@@ -11,9 +11,14 @@
 //
 // The launch is persistent: the (tile, step) pairs of the whole GEMM, a step being 64 input features, are numbered
 // tile by tile and dealt out to the CTAs in equal contiguous ranges, so that every SM has the same work whatever the
-// number of tiles (86 tiles of a 11008-wide projection on 148 SMs left 40 % of the GPU idle).  A CTA that holds only
-// part of a tile's steps writes its fp32 accumulators to the workspace; the last CTA of the tile to arrive (an
-// atomic counter, nobody waits) adds the parts in the order of the CTAs, so the result does not depend on timing.
+// number of tiles (86 tiles of a 11008-wide projection on 148 SMs left 40 % of the GPU idle).  A tile that several
+// CTAs share is completed by the CTA that holds its first steps - the end of that CTA's range, so the last thing it
+// does: the others meet the tile at the beginning of their ranges, write their fp32 accumulators to their slot of the
+// workspace and count themselves in; the completing CTA adds the parts to its own accumulators in the order of the
+// CTAs (the result does not depend on timing) and writes the outputs.  Its wait for the count is bounded like every
+// other wait, and the launch is cooperative so that the CTAs it waits for are resident.
+// Where the ranges are short against a tile (four or more CTAs per tile) every CTA writes its parts instead and a
+// second, fully parallel kernel adds them: the completing CTA's serial additions cost more there.
 //
 // Per step
 //   * one thread copies the token tile with one or two bulk tensor copies (up to 144 tokens x 64 features each,
@@ -41,7 +46,7 @@ namespace qil {
 
 namespace {
 
-constexpr int kTileF = 128, kStepK = 64, kAStages = 4, kBStages = 3, kMaxNN = 144, kMaxTT = 2 * kMaxNN;
+constexpr int kTileF = 128, kStepK = 64, kStages = 4, kMaxNN = 144, kMaxTT = 2 * kMaxNN;
 constexpr int kAccCols = kMaxTT;                  // accumulator columns (fp32, column = token)
 constexpr int kAStageCols = kStepK / 2;           // a step of the weight operand: 64 bf16 per lane = 32 columns
 constexpr int kBHalf = kMaxNN * kStepK * 2;       // up to 144 tokens x 64 bf16: 18 KiB (a multiple of 1024)
@@ -51,7 +56,7 @@ constexpr int kThreads = 352;                     // token copy warp, MMA warp, 
 constexpr int kDqWarps = 8;
 constexpr int kMetaPre = 8;                       // steps by which a dequantising thread's scale / zero loads run ahead
 constexpr int kTmemCols = 512;
-static_assert(kAccCols + kAStages * kAStageCols <= kTmemCols, "tensor memory");
+static_assert(kAccCols + kStages * kAStageCols <= kTmemCols, "tensor memory");
 constexpr int kCounterBytes = 16384;              // tile counters at the start of the scratch (same place as the skinny kernel's)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -68,7 +73,9 @@ struct PrefillParams {
     int unit_steps;  // the ranges of the CTAs begin at multiples of this many steps
     long long units; // unit_steps-sized pieces of the whole GEMM: tiles * (K / 64) / unit_steps
     int* status;
-    float* partials; // [2 * CTAs][nh * NN][128]
+    int fix;         // 1: shared tiles are completed inside this kernel; 0: every part is written out and a second kernel adds them
+    int* counters;   // fix: per tile, parts written so far (zero between launches)
+    float* partials; // [2 * CTAs][nh * NN][128]: slot 2c holds the part CTA c begins its range with, slot 2c + 1 the part it ends with
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -208,17 +215,18 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // (the swizzled token tiles need 1024-byte alignment)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char* sb = smem;                                  // [kBStages][kBStage] tokens
+    unsigned char* sb = smem;                                  // [kStages][kBStage] tokens
     constexpr int kWStage = kTileF * kStepK * kBits / 8;       // packed weight tile: 4 KiB (4-bit), 8 KiB (8-bit)
-    unsigned char* sw = sb + (size_t)kBStages * kBStage;       // [kWStages][128 rows][kStepK * kBits / 8 bytes]
+    unsigned char* sw = sb + (size_t)kStages * kBStage;       // [kWStages][128 rows][kStepK * kBits / 8 bytes]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sw + (size_t)kWStages * kWStage);
-    const uint32_t full_a0 = smem_u32(bars), free_a0 = smem_u32(bars + kAStages);
-    const uint32_t full_b0 = smem_u32(bars + 2 * kAStages), free_b0 = smem_u32(bars + 2 * kAStages + kBStages);
-    uint64_t* wbars = bars + 2 * kAStages + 2 * kBStages;
+    // stage s of the weight operand (tensor memory) and of the token tiles (shared memory) travel together: one
+    // "free" barrier, one tcgen05.commit per step
+    const uint32_t full_a0 = smem_u32(bars), full_b0 = smem_u32(bars + kStages), free0 = smem_u32(bars + 2 * kStages);
+    uint64_t* wbars = bars + 3 * kStages;
     const uint32_t full_w0 = smem_u32(wbars), free_w0 = smem_u32(wbars + kWStages);
     uint64_t* obars = wbars + 2 * kWStages;
-    const uint32_t done0 = smem_u32(obars), acc_free0 = smem_u32(obars + 1);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(obars + 2);
+    const uint32_t done0 = smem_u32(obars), acc_free0 = smem_u32(obars + 1), part0 = smem_u32(obars + 2);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(obars + 3);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = p.K / kStepK;                   // steps per tile
     const int C = (int)gridDim.x, cta = (int)blockIdx.x;
@@ -227,13 +235,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
     const int ng = p.K / p.G;
 
     if (tid == 0) {
-        for (int s = 0; s < kAStages; ++s) {
-            mbar_init(full_a0 + 8 * s, kDqWarps);   // the dequantising warps
-            mbar_init(free_a0 + 8 * s, 1);          // the commit of the MMAs that read the stage
-        }
-        for (int s = 0; s < kBStages; ++s) {
-            mbar_init(full_b0 + 8 * s, 1);   // the copies (transaction bytes)
-            mbar_init(free_b0 + 8 * s, 1);   // the commit of the MMAs that read the stage
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_a0 + 8 * s, kDqWarps);   // the dequantising warps: weights stored, token tile seen to have landed
+            mbar_init(full_b0 + 8 * s, 1);          // the token copies (transaction bytes)
+            mbar_init(free0 + 8 * s, 1);            // the commit of the MMAs that read the stage
         }
         for (int s = 0; s < kWStages; ++s) {
             mbar_init(full_w0 + 8 * s, 1);          // the copy (transaction bytes)
@@ -241,6 +246,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
         }
         mbar_init(done0, 1);             // the commit after the last MMA of a segment
         mbar_init(acc_free0, kDqWarps);  // the accumulators of a segment have been read
+        mbar_init(part0, kDqWarps);      // the CTA's part of a shared tile has been written
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -261,8 +267,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
             for (long long g = g_begin; ok && next_segment(g, g_end, S, sg);) {
                 const int m0 = (sg.tile % p.mt) * TT;
                 for (int i = sg.s0; i < sg.s1; ++i, ++it) {
-                    const int s = it % kBStages, use = it / kBStages;
-                    ok = mbar_wait(free_b0 + 8 * s, (use & 1) ^ 1);  // the MMAs that read this stage last are complete
+                    const int s = it % kStages, use = it / kStages;
+                    ok = mbar_wait(free0 + 8 * s, (use & 1) ^ 1);    // the MMAs that read this stage last are complete
                     if (!ok) break;
                     mbar_expect_tx(full_b0 + 8 * s, (uint32_t)TT * kStepK * 2);
                     for (int hb = 0; hb < p.nh; ++hb)
@@ -271,9 +277,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                 }
             }
             // no copy may still be in flight when the CTA retires (this wait also holds after a time-out elsewhere)
-            for (int back = 0; back < kBStages && back < it; ++back) {
+            for (int back = 0; back < kStages && back < it; ++back) {
                 const int i = it - 1 - back;
-                (void)mbar_wait(full_b0 + 8 * (i % kBStages), (i / kBStages) & 1);
+                (void)mbar_wait(full_b0 + 8 * (i % kStages), (i / kStages) & 1);
             }
         }
     } else if (warp == 1) {
@@ -286,7 +292,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
             const uint32_t b_lo0 = ((smem_u32(sb) >> 4) & 0x3FFFu) | (1u << 16);
             const uint32_t half_lo = ((uint32_t)p.NN * (kStepK * 2)) >> 4;   // the second MMA's tokens
             const bool two = p.nh == 2;
-            uint32_t s = 0, aph = 0, bs = 0, bph = 0;
+            uint32_t s = 0, aph = 0;
             int seg = 0;
             Segment sg;
             for (long long g = g_begin; ok && next_segment(g, g_end, S, sg); ++seg) {
@@ -297,21 +303,20 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                 uint32_t acc = 0u;                               // the first MMAs of a segment overwrite the accumulators
 #pragma unroll 1
                 for (int i = sg.s0; i < sg.s1; ++i) {
-                    ok = mbar_wait(full_a0 + 8 * s, aph) && mbar_wait(full_b0 + 8 * bs, bph);
+                    // (the dequantising warps arrive once the step's token tile has landed as well: one wait here)
+                    ok = mbar_wait(full_a0 + 8 * s, aph);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_tmem = tmem + (uint32_t)kAccCols + s * kAStageCols;
-                    const uint32_t b_lo = b_lo0 + bs * (kBStage >> 4);
+                    const uint32_t b_lo = b_lo0 + s * (kBStage >> 4);
 #pragma unroll
                     for (int k = 0; k < kStepK / 16; ++k) {  // K = 16 each: 8 columns of A, 32 bytes of a swizzled row of B
                         mma_bf16_ts(tmem, a_tmem + 8 * k, b_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
                         if (two) mma_bf16_ts(tmem + (uint32_t)p.NN, a_tmem + 8 * k, b_lo + half_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
                     }
                     acc = 1u;
-                    tc_commit(free_a0 + 8 * s);
-                    tc_commit(free_b0 + 8 * bs);
-                    if (++s == kAStages) { s = 0; aph ^= 1u; }
-                    if (++bs == kBStages) { bs = 0; bph ^= 1u; }
+                    tc_commit(free0 + 8 * s);
+                    if (++s == kStages) { s = 0; aph ^= 1u; }
                 }
                 if (!ok) break;
                 tc_commit(done0);   // every MMA of the segment is complete when this arrival happens
@@ -377,18 +382,21 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                     v[2 * c] = d.x; v[2 * c + 1] = d.y;
                 }
             }
-            if (!mbar_wait(free_a0 + 8 * s, sph)) return false;       // the MMAs that read this stage last are complete
+            if (!mbar_wait(free0 + 8 * s, sph)) return false;         // the MMAs that read this stage last are complete
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             tmem_st16(a_lane + s * kAStageCols, v);
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            // the step's token tile has landed (parity of its ring = the complement of the one just waited for): the MMA
+            // thread, which acquires this warp's arrival below, then needs no wait of its own for it
+            if (!mbar_wait(full_b0 + 8 * s, sph ^ 1u)) return false;
             __syncwarp();
             if (lane == 0) {
                 // (the packed tile is released only now: its words were still being consumed above)
                 mbar_arrive(free_w0 + 8 * ws_);
                 mbar_arrive(full_a0 + 8 * s);
             }
-            if (++s == kAStages) { s = 0; sph ^= 1u; }
+            if (++s == kStages) { s = 0; sph ^= 1u; }
             if (++ws_ == kWStages) { ws_ = 0; wph ^= 1u; }
             return true;
         };
@@ -446,8 +454,34 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const bool whole = sg.s0 == 0 && sg.s1 == S;               // the CTA holds every step of the tile
             const int n = n0 + rr;
-            // the part of a tile a CTA begins its range with goes to slot 2 * cta, the part it ends with to slot 2 * cta + 1
-            float* part = whole ? nullptr : p.partials + ((size_t)(2 * cta + (g_seg == g_begin ? 0 : 1)) * TT) * kTileF + rr;
+            // A tile that several CTAs share: the CTA with the tile's first steps - for that CTA the last thing it does -
+            // adds the others' parts to its own accumulators, in the order of the CTAs, and writes the outputs.  The others
+            // meet the tile at the beginning of their ranges, write their part to their slot of the workspace and count
+            // themselves in; by the time the first CTA gets there they are long done (its wait is bounded all the same).
+            int c_first = cta, c_last = cta;
+            if (!whole) {
+                const long long su = S / p.unit_steps;                  // units per tile
+                c_first = cta_of_unit(p.units, C, (long long)sg.tile * su);
+                c_last = cta_of_unit(p.units, C, (long long)sg.tile * su + su - 1);
+            }
+            const bool fixer = p.fix && !whole && c_first == cta;
+            if (fixer) {
+                const int need = c_last - c_first;
+                const int* cnt = p.counters + sg.tile;
+                unsigned long long t0 = 0, t;
+                for (uint32_t spin = 0;; ++spin) {
+                    int have;
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(have) : "l"(cnt) : "memory");
+                    if (have >= need) break;
+                    if ((spin & 63u) == 0u) {
+                        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+                        if (spin == 0u) t0 = t;
+                        else if (t - t0 > kWaitLimitNs) { ok = false; break; }
+                    }
+                }
+                if (!ok) break;
+            }
+            float* part = (!whole && !fixer) ? p.partials + ((size_t)(2 * cta + (g_seg == g_begin ? 0 : 1)) * TT) * kTileF + rr : nullptr;
             const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16);
 #pragma unroll 1
             for (int c0 = 16 * hh; c0 < TT; c0 += 32) {
@@ -456,7 +490,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                 if (part) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) __stcg(part + (size_t)(c0 + j) * kTileF, __uint_as_float(d[j]));
-                } else if (n < p.N) {
+                } else if (n < p.N && m0 + c0 < p.M) {
+                    for (int cc = c_first + 1; cc <= c_last; ++cc) {
+                        const float* other = p.partials + ((size_t)(2 * cc) * TT + c0) * kTileF + rr;  // (their first part)
+                        float v[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = __ldcg(other + (size_t)j * kTileF);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) d[j] = __float_as_uint(__uint_as_float(d[j]) + v[j]);
+                    }
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (m0 + c0 + j < p.M) p.y[(size_t)(m0 + c0 + j) * p.N + n] = __float2bfloat16_rn(__uint_as_float(d[j]));
@@ -465,6 +507,20 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_free0);
+            if (part && p.fix) {
+                // (a CTA writes at most one part per launch here: the barrier is used once)
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(part0);
+                if (warp == 2) {
+                    ok = mbar_wait(part0, 0);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        __threadfence();
+                        atomicAdd(p.counters + sg.tile, 1);
+                    }
+                }
+            }
         }
     }
     if (!ok && p.status) atomicOr(p.status, (int)QIL_ERR_TIMEOUT);
@@ -472,6 +528,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols));
+    if (tid == 0 && g_end > g_begin && p.fix) {
+        // the counter of the shared tile this CTA completed (its last one) goes back to zero for the next launch
+        const int last_tile = (int)((g_end - 1) / S);
+        const long long su = S / p.unit_steps;
+        if (cta_of_unit(p.units, C, (long long)last_tile * su) == cta && cta_of_unit(p.units, C, (long long)last_tile * su + su - 1) != cta)
+            p.counters[last_tile] = 0;
+    }
 }
 
 // Adds the parts of every tile that several CTAs share, in the order of the CTAs, and writes the bf16 outputs.
@@ -506,8 +569,8 @@ __global__ void __launch_bounds__(256) w4a16_prefill_reduce_kernel(const Prefill
     }
 }
 
-constexpr size_t kSmemBytes = (size_t)kBStages * kBStage + (size_t)kWStages * (kTileF * kStepK) +
-                              (2 * kAStages + 2 * kBStages + 2 * kWStages + 2) * 8 + 16 + 1024;
+constexpr size_t kSmemBytes = (size_t)kStages * kBStage + (size_t)kWStages * (kTileF * kStepK) +
+                              (3 * kStages + 2 * kWStages + 3) * 8 + 16 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -611,21 +674,42 @@ qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scale
     p.unit_steps = pl.unit_steps;
     p.units = pl.units;
     p.status = status;
+    p.counters = with_parts ? reinterpret_cast<int*>(scratch) : nullptr;
+    // A tile shared by up to three CTAs is completed inside the kernel by the CTA that holds its first steps; when the
+    // ranges are short against a tile (more CTAs per tile) that CTA's serial additions cost more than a second, fully
+    // parallel kernel (measured on the 4096 x 4096 and 4096 x 11008 projections at 280 tokens).
+    const long long per_cta = pl.units / pl.ctas, per_tile = (long long)(K / kStepK) / pl.unit_steps;
+    p.fix = (with_parts && 2 * per_cta >= per_tile) ? 1 : 0;
     p.partials = with_parts ? reinterpret_cast<float*>(static_cast<char*>(scratch) + kCounterBytes) : nullptr;
-    const dim3 grid(pl.ctas);
+    // The CTAs of a shared tile wait for one another's parts: the launch is cooperative, so that all of them are resident
+    // (one CTA per SM by its shared memory, never more CTAs than SMs).
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)pl.ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.fix ? 1 : 0;
     cudaError_t e;
     if (bits == 8) {
         e = cudaFuncSetAttribute(w4a16_prefill_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e == cudaSuccess) w4a16_prefill_kernel<8><<<grid, kThreads, kSmemBytes, st>>>(tmap, tmap_w, p);
+        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, w4a16_prefill_kernel<8>, tmap, tmap_w, p);
     } else {
         e = cudaFuncSetAttribute(w4a16_prefill_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e == cudaSuccess) w4a16_prefill_kernel<4><<<grid, kThreads, kSmemBytes, st>>>(tmap, tmap_w, p);
+        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, w4a16_prefill_kernel<4>, tmap, tmap_w, p);
+    }
+    if (e == cudaErrorCooperativeLaunchTooLarge) {
+        (void)cudaGetLastError();
+        return QIL_ERR_UNSUPPORTED;
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return QIL_ERR_CUDA;
     }
-    if (with_parts && pl.ctas > 1) {
+    if (with_parts && !p.fix && pl.ctas > 1) {
         const dim3 rgrid((unsigned)(pl.ftiles * pl.mt), (unsigned)((pl.nh * pl.NN + 7) / 8));
         w4a16_prefill_reduce_kernel<<<rgrid, 256, 0, st>>>(p, pl.ctas);
     }

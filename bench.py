@@ -598,7 +598,22 @@ def secondary_measurements(dev):
         for (N, K, pk, s, z, yo, ws) in lin:
             api.linear_w4a16(xs[K], pk, s, z, N, wl.GROUP_SIZE, api.LAYOUT_CANONICAL, out=yo, workspace=ws)
     t_layer = time_us(layer, 10)
-    del lin, xs
+    del lin
+
+    # the same layer with q, k, v and gate, up stored as one linear each (4 launches instead of 7)
+    linf = []
+    for (_, N, K) in wl.LLAMA2_7B_LAYER_FUSED:
+        w = torch.randn((N, K), device=dev, generator=g) * wl.SIGMA_LLM
+        codes, s, z = api.quantize_rtn_w4(w, wl.GROUP_SIZE)
+        linf.append((N, K, api.pack_w4(codes), s, z, torch.empty((Mp, N), dtype=torch.bfloat16, device=dev),
+                     api.new_workspace(api.linear_w4a16_workspace_size(Mp, N, K, wl.GROUP_SIZE), dev)))
+        del w, codes
+
+    def layer_fused():
+        for (N, K, pk, s, z, yo, ws) in linf:
+            api.linear_w4a16(xs[K], pk, s, z, N, wl.GROUP_SIZE, api.LAYOUT_CANONICAL, out=yo, workspace=ws)
+    t_layer_fused = time_us(layer_fused, 10)
+    del linf, xs
 
     # configs[3]: M sweep on the two FFN shapes, cold (6 weight copies in rotation = 144 MB of packed weights,
     # larger than L2).  M <= 4 runs the tcgen05 decode kernel (STREAM128 units), M <= 8 the mma.sync skinny kernel
@@ -639,6 +654,8 @@ def secondary_measurements(dev):
     out["w4a16_m_sweep"] = sweep
     flops = sum(2.0 * Mp * N * K for (_, N, K) in wl.LLAMA2_7B_LAYER)
     out["w4a16_prefill_m280_layer"] = {"us": t_layer, "TFLOP/s": flops / t_layer / 1e6, "kernel": "w4a16_prefill_kernel (tcgen05 kind::f16)"}
+    out["w4a16_prefill_m280_layer_fused_qkv_gate_up"] = {"us": t_layer_fused, "TFLOP/s": flops / t_layer_fused / 1e6,
+                                                         "linears": [n for (n, _, _) in wl.LLAMA2_7B_LAYER_FUSED]}
     return out
 
 

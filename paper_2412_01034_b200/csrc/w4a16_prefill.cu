@@ -70,6 +70,7 @@ struct PrefillParams {
     int pair_meta;   // groups of 128 columns, an even number of them per row, K % 256 == 0: scales are loaded two groups at a time
     int NN, nh;      // tokens per MMA (multiple of 16, <= 144) and MMAs side by side (1 or 2): nh * NN tokens per tile
     int mt;          // token tiles
+    int nchain;      // accumulators per output that take the K slices in turn (nh == 1 only): 2 or 4, else 1
     int unit_steps;  // the ranges of the CTAs begin at multiples of this many steps
     long long units; // unit_steps-sized pieces of the whole GEMM: tiles * (K / 64) / unit_steps
     int* status;
@@ -292,6 +293,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
             const uint32_t b_lo0 = ((smem_u32(sb) >> 4) & 0x3FFFu) | (1u << 16);
             const uint32_t half_lo = ((uint32_t)p.NN * (kStepK * 2)) >> 4;   // the second MMA's tokens
             const bool two = p.nh == 2;
+            // MMAs into one accumulator follow one another at the latency of the tensor pipe, not at its throughput (about
+            // 200 cycles each here, whatever their width).  Two token halves are two independent chains; a tile of up to
+            // 144 tokens leaves room for more accumulators, which take the K slices in turn and are added at the read-out.
+            const uint32_t cmask = (uint32_t)p.nchain - 1u, cstride = p.nchain == 4 ? 64u : (uint32_t)kMaxNN;   // (columns 0, 64, 128, 192 or 0, 144)
             uint32_t s = 0, aph = 0;
             int seg = 0;
             Segment sg;
@@ -311,8 +316,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                     const uint32_t b_lo = b_lo0 + s * (kBStage >> 4);
 #pragma unroll
                     for (int k = 0; k < kStepK / 16; ++k) {  // K = 16 each: 8 columns of A, 32 bytes of a swizzled row of B
-                        mma_bf16_ts(tmem, a_tmem + 8 * k, b_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
-                        if (two) mma_bf16_ts(tmem + (uint32_t)p.NN, a_tmem + 8 * k, b_lo + half_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
+                        if (two) {
+                            mma_bf16_ts(tmem, a_tmem + 8 * k, b_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
+                            mma_bf16_ts(tmem + (uint32_t)p.NN, a_tmem + 8 * k, b_lo + half_lo + 2 * k, d_hi, idesc, k == 0 ? acc : 1u);
+                        } else {
+                            mma_bf16_ts(tmem + ((uint32_t)k & cmask) * cstride, a_tmem + 8 * k, b_lo + 2 * k, d_hi, idesc,
+                                        (uint32_t)k <= cmask ? acc : 1u);
+                        }
                     }
                     acc = 1u;
                     tc_commit(free0 + 8 * s);
@@ -487,6 +497,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
             for (int c0 = 16 * hh; c0 < TT; c0 += 32) {
                 uint32_t d[16];
                 tmem_ld16(taddr + (uint32_t)c0, d);
+                for (int ch = 1; ch < p.nchain; ++ch) {   // the other accumulators of these outputs
+                    uint32_t e[16];
+                    tmem_ld16(taddr + (uint32_t)(ch * (p.nchain == 4 ? 64 : kMaxNN) + c0), e);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) d[j] = __float_as_uint(__uint_as_float(d[j]) + __uint_as_float(e[j]));
+                }
                 if (part) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) __stcg(part + (size_t)(c0 + j) * kTileF, __uint_as_float(d[j]));
@@ -595,7 +611,7 @@ EncodeFn encode_fn() {
 }
 
 struct PrefillPlan {
-    int mt, NN, nh, ftiles, ctas, unit_steps;
+    int mt, NN, nh, nchain, ftiles, ctas, unit_steps;
     long long units;
 };
 
@@ -606,6 +622,7 @@ PrefillPlan plan_prefill(int M, int N, int K, int G, bool with_parts) {
     const int per = (M + pl.mt - 1) / pl.mt;
     pl.nh = per > kMaxNN ? 2 : 1;
     pl.NN = ((per + pl.nh - 1) / pl.nh + 15) / 16 * 16;
+    pl.nchain = pl.nh == 2 ? 1 : (pl.NN <= 64 ? 4 : 2);
     pl.ftiles = (N + kTileF - 1) / kTileF;
     const int S = K / kStepK, sms = num_sms();
     const long long tiles = (long long)pl.ftiles * pl.mt;
@@ -670,7 +687,7 @@ qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scale
     if ((spg & (spg - 1)) == 0)
         for (int sh = 0; sh < 31; ++sh)
             if ((1 << sh) == spg) p.g_shift = sh;
-    p.NN = pl.NN; p.nh = pl.nh; p.mt = pl.mt;
+    p.NN = pl.NN; p.nh = pl.nh; p.mt = pl.mt; p.nchain = pl.nchain;
     p.unit_steps = pl.unit_steps;
     p.units = pl.units;
     p.status = status;

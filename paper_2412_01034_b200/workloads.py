@@ -35,6 +35,12 @@ LLAMA2_7B_LAYER = (
     ("gate", FFN, HIDDEN), ("up", FFN, HIDDEN), ("down", HIDDEN, FFN),
 )
 
+# The same layer with the projections that read the same input stored as one linear each (q, k, v and gate, up:
+# group-wise quantisation is per output row, so stacking rows changes no code, scale or result)
+LLAMA2_7B_LAYER_FUSED = (
+    ("qkv", 3 * HIDDEN, HIDDEN), ("o", HIDDEN, HIDDEN), ("gate_up", 2 * FFN, HIDDEN), ("down", HIDDEN, FFN),
+)
+
 # (Cin = Cout, H, W) of the four 3x3 conv stages at batch 32, input 3x88x200
 CONV_STAGES = ((64, 22, 50), (128, 11, 25), (256, 6, 13), (512, 3, 7))
 CONV_BATCH = 32

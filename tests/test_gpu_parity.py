@@ -209,10 +209,14 @@ def test_w4a16_skinny_shapes(api, N, K, G, layout):
 
 @pytest.mark.parametrize("M,N,K,G", [
     (280, 512, 1024, 128), (130, 200, 256, 64), (65, 1000, 2176, 128), (129, 136, 128, 128), (300, 77, 192, 192),
+    # two tiles shared by eight CTAs each (all parts written, second kernel), tiles shared by two CTAs (completed in the
+    # kernel), three token tiles, tiles of up to 64 / 144 tokens (four / two accumulators per output)
+    (280, 256, 4096, 128), (280, 2048, 1024, 128), (600, 384, 1024, 128), (40, 640, 2048, 128), (100, 1280, 1024, 64),
 ])
 def test_w4a16_prefill_shapes(api, M, N, K, G):
     """The tcgen05 prefill GEMM (M > 8, canonical layout): ragged M and N, one to many K steps, groups of one or
-    several steps; run twice: the result must not depend on what the previous launch left behind."""
+    several steps, every way its persistent launch shares tiles between CTAs; run twice: the result must not depend
+    on what the previous launch left behind."""
     y1 = _w4a16_case(api, M, N, K, G, 0, seed=M + N + K)
     y2 = _w4a16_case(api, M, N, K, G, 0, seed=M + N + K)
     np.testing.assert_array_equal(bits_of(y1), bits_of(y2))
@@ -234,6 +238,30 @@ def test_cfg2_prefill_shapes(api, N, K):
     y_ref = c_oracle.linear_w4a16(x, *ref, G)
     # the row maximum over the sampled features lower-bounds the true row maximum: the check is stricter
     assert_rows_close(bf16_to_f64(y)[:, rows], y_ref, rel=CONTRACT_REL)
+
+
+def test_w4a16_prefill_workspace_is_reusable_across_shapes(api):
+    """One workspace serves prefill GEMMs of different shapes in turn (its tile counters return to zero after every
+    launch), and every repetition gives the same bits."""
+    shapes = [(280, 2048, 1024), (280, 256, 4096), (64, 1536, 512), (280, 2048, 1024), (280, 256, 4096)]
+    G = 128
+    size = max(api.linear_w4a16_workspace_size(M, N, K, G) for (M, N, K) in shapes)
+    ws = api.new_workspace(size)
+    seen = {}
+    for rep in range(2):
+        for (M, N, K) in shapes:
+            w = wl.normal_weights(310, N + K, N, K, 0.02)
+            x = wl.normal_activations_bf16(310, N + K + 1, M, K)
+            codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
+            y = api.linear_w4a16(to_bf16_cuda(x), api.pack_w4(cuda(codes)), cuda(scales), cuda(zeros), N, G, workspace=ws)
+            if (M, N, K) in seen:
+                np.testing.assert_array_equal(bits_of(y), seen[(M, N, K)])
+            else:
+                y_ref = c_oracle.linear_w4a16(x, codes, scales, zeros, G)
+                assert_rows_close(bf16_to_f64(y), y_ref, rel=CONTRACT_REL)
+                seen[(M, N, K)] = bits_of(y).copy()
+    import torch
+    assert int(ws[:4].view(torch.int32).cpu()[0]) == 0   # the status word: no wait ran out
 
 
 @pytest.mark.parametrize("N,K,G", [(24, 256, 32), (9, 40, 8), (17, 192, 64), (8, 320, 320)])

@@ -613,7 +613,13 @@ def secondary_measurements(dev):
         for (N, K, pk, s, z, yo, ws) in linf:
             api.linear_w4a16(xs[K], pk, s, z, N, wl.GROUP_SIZE, api.LAYOUT_CANONICAL, out=yo, workspace=ws)
     t_layer_fused = time_us(layer_fused, 10)
-    del linf, xs
+    # the gate_up linear alone, plain and with silu(gate) * up in its epilogue (the same rows read as interleaved pairs)
+    (Ng, Kg, pkg, sg, zg, yg, wsg) = linf[2]
+    ysw = torch.empty((Mp, Ng // 2), dtype=torch.bfloat16, device=dev)
+    wsw = api.new_workspace(api.linear_w4a16_swiglu_workspace_size(Mp, Ng, Kg, wl.GROUP_SIZE), dev)
+    t_gate_up = time_us(lambda: api.linear_w4a16(xs[Kg], pkg, sg, zg, Ng, wl.GROUP_SIZE, api.LAYOUT_CANONICAL, out=yg, workspace=wsg), 10)
+    t_gate_up_sw = time_us(lambda: api.linear_w4a16_swiglu(xs[Kg], pkg, sg, zg, Ng, wl.GROUP_SIZE, out=ysw, workspace=wsw), 10)
+    del linf, xs, ysw, wsw
 
     # configs[3]: M sweep on the two FFN shapes, cold (6 weight copies in rotation = 144 MB of packed weights,
     # larger than L2).  M <= 4 runs the tcgen05 decode kernel (STREAM128 units), M <= 8 the mma.sync skinny kernel
@@ -654,6 +660,8 @@ def secondary_measurements(dev):
     out["w4a16_m_sweep"] = sweep
     flops = sum(2.0 * Mp * N * K for (_, N, K) in wl.LLAMA2_7B_LAYER)
     out["w4a16_prefill_m280_layer"] = {"us": t_layer, "TFLOP/s": flops / t_layer / 1e6, "kernel": "w4a16_prefill_kernel (tcgen05 kind::f16)"}
+    out["w4a16_prefill_m280_gate_up_22016x4096"] = {"plain_us": t_gate_up, "swiglu_epilogue_us": t_gate_up_sw,
+                                                    "TFLOP/s": 2.0 * Mp * 2 * wl.FFN * wl.HIDDEN / t_gate_up_sw / 1e6}
     out["w4a16_prefill_m280_layer_fused_qkv_gate_up"] = {"us": t_layer_fused, "TFLOP/s": flops / t_layer_fused / 1e6,
                                                          "linears": [n for (n, _, _) in wl.LLAMA2_7B_LAYER_FUSED]}
     return out

@@ -123,8 +123,9 @@ qil_status qil_pack_stream128_w4(const uint8_t* codes, const void* scales, const
  *   y [M][N] bf16
  * The kernel is chosen from the shape: on the canonical layout with M > 8,
  * K % 64 == 0 and group_size % 64 == 0 the tcgen05 prefill GEMM (weights
- * dequantised to bf16, one rounding per weight; K split over several CTAs where
- * that fills the GPU, partial tiles added in a fixed order); else the tensor-core skinny
+ * dequantised to bf16, one rounding per weight; one persistent, cooperative
+ * launch whose CTAs take equal ranges of the GEMM's steps; tiles that several
+ * CTAs share are added up in a fixed order); else the tensor-core skinny
  * kernel (weights read once, any M handled in slabs of 64 rows) when
  * K % 128 == 0 and group_size % 128 == 0; a general kernel otherwise (any
  * K % 8 == 0, any group_size dividing K, canonical layout only).  With
@@ -157,6 +158,28 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
                             const void* zeros, void* y, int M, int N, int K, int group_size,
                             qil_layout layout, void* workspace, size_t workspace_bytes,
                             qil_stream_t stream);
+
+/* -------------------------------------------------------------------------
+ * qil_linear_w4a16_swiglu: the gate and up projections of a gated MLP (the
+ * Llama-2 backbone of the paper's OpenVLA deployment, App. A.4.2) as ONE
+ * weight-only linear with the activation fused into its epilogue:
+ *     y[m][i] = silu(x[m] . W_hat[2 i]) * (x[m] . W_hat[2 i + 1]),   silu(g) = g / (1 + exp(-g))
+ * Row 2 i of the N weight rows is gate row i, row 2 i + 1 is up row i
+ * (group-wise quantisation is per row, so interleaving rows changes no code,
+ * scale or zero point).  N must be even.
+ *   x [M][K] bf16   qweight, scales, zeros as for qil_linear_w4a16 (canonical layout)
+ *   y [M][N / 2] bf16
+ * On the shapes the prefill GEMM takes (M > 8, K % 64 == 0, group_size % 64
+ * == 0) gate and up products stay in fp32 until the result is rounded to bf16
+ * once; on all other shapes the linear is computed as by qil_linear_w4a16 into
+ * the workspace (bf16) and a second kernel applies the activation.
+ * workspace: qil_linear_w4a16_swiglu_workspace_size() bytes, zero-filled once.
+ * Errors: NULL, SHAPE (also odd N), ALIGN, WORKSPACE, UNSUPPORTED, CUDA.
+ * ---------------------------------------------------------------------- */
+size_t qil_linear_w4a16_swiglu_workspace_size(int M, int N, int K, int group_size);
+qil_status qil_linear_w4a16_swiglu(const void* x, const uint32_t* qweight, const void* scales,
+                                   const void* zeros, void* y, int M, int N, int K, int group_size,
+                                   void* workspace, size_t workspace_bytes, qil_stream_t stream);
 
 /* ------------------------------------------------------------------------
  * qil_linear_w4a16 for callers that must not allocate device memory.  (The paper

@@ -262,6 +262,21 @@ def linear_w4a16(x_bf16_bits, codes, scales, zeros, group_size: int) -> np.ndarr
     return np.matmul(x, w_hat.T)
 
 
+def silu(g: np.ndarray) -> np.ndarray:
+    """silu(g) = g / (1 + exp(-g)), fp64 (the activation of the Llama-2 gated MLP, the backbone of the paper's OpenVLA
+    deployment, App. A.4.2).  Written so that large |g| neither overflows nor loses the small side."""
+    g = np.asarray(g, dtype=np.float64)
+    e = np.exp(-np.abs(g))                       # in (0, 1]
+    return np.where(g >= 0, g / (1.0 + e), g * e / (1.0 + e))
+
+
+def linear_w4a16_swiglu(x_bf16_bits, codes, scales, zeros, group_size: int) -> np.ndarray:
+    """Gate and up projections with rows interleaved (row 2i = gate i, row 2i + 1 = up i) and the gated activation:
+    y[m][i] = silu(t[m][2i]) * t[m][2i + 1], t = the plain dequantise-then-matmul, fp64 throughout."""
+    t = linear_w4a16(x_bf16_bits, codes, scales, zeros, group_size)
+    return silu(t[:, 0::2]) * t[:, 1::2]
+
+
 def linear_w4a4(qx, sx, qw, sw):
     """acc[m][n] = sum_k qx[m][k]*qw[n][k] (int64); y = acc * sx[m] * sw[n] (fp64)."""
     a = np.asarray(qx).astype(np.int64)

@@ -182,6 +182,31 @@ def linear_w4a16(x, qweight, scales, zeros, N: int, group_size: int, layout: int
     return out
 
 
+def interleave_rows(gate, up):
+    """Rows 2i = gate[i], 2i + 1 = up[i] (codes, scales or zeros of the two projections of a gated MLP): the weight
+    layout `linear_w4a16_swiglu` expects.  A layout step done once, offline."""
+    assert gate.shape == up.shape
+    return torch.stack((gate, up), dim=1).reshape(2 * gate.shape[0], *gate.shape[1:]).contiguous()
+
+
+def linear_w4a16_swiglu_workspace_size(M: int, N: int, K: int, group_size: int) -> int:
+    return int(_lib.load().qil_linear_w4a16_swiglu_workspace_size(M, N, K, group_size))
+
+
+def linear_w4a16_swiglu(x, qweight, scales, zeros, N: int, group_size: int, out=None, workspace=None, stream=None):
+    """y[M][N/2] (bf16) = silu(x . dequant(W[0::2])^T) * (x . dequant(W[1::2])^T): gate and up rows interleaved in W."""
+    _need_cuda(x, qweight, scales, zeros, out, workspace)
+    M, K = x.shape
+    if out is None:
+        out = torch.empty((M, N // 2), dtype=torch.bfloat16, device=x.device)
+    if workspace is None:
+        workspace = new_workspace(linear_w4a16_swiglu_workspace_size(M, N, K, group_size), x.device)
+    _check(_lib.load().qil_linear_w4a16_swiglu(_ptr(x), _ptr(qweight), _ptr(scales), _ptr(zeros), _ptr(out), M, N, K,
+                                               int(group_size), _ptr(workspace),
+                                               workspace.numel() * workspace.element_size(), _stream(stream)))
+    return out
+
+
 def quantize_act_a4(x, static_scale: float | None = None, stream=None):
     """bf16 x [M][K] -> (packed int4 codes [M][K/8] int32, scales [M] fp32)."""
     _need_cuda(x)

@@ -197,6 +197,41 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
     return launch_w4a16_general(x, qweight, scales, zeros, y, M, N, K, group_size, S(stream));
 }
 
+// Bytes of the plain linear's workspace, rounded so that the bf16 scratch of the unfused path can follow it.
+static size_t swiglu_tmp_offset(int M, int N, int K, int group_size) {
+    return (qil_linear_w4a16_workspace_size(M, N, K, group_size) + 255) / 256 * 256;
+}
+
+size_t qil_linear_w4a16_swiglu_workspace_size(int M, int N, int K, int group_size) {
+    if (M <= 0 || N <= 0 || K <= 0 || group_size <= 0) return 0;
+    size_t bytes = swiglu_tmp_offset(M, N, K, group_size);
+    if (!w4a16_prefill_supported(M, N, K, group_size, QIL_LAYOUT_CANONICAL)) bytes += (size_t)M * N * 2;
+    return bytes;
+}
+
+qil_status qil_linear_w4a16_swiglu(const void* x, const uint32_t* qweight, const void* scales, const void* zeros, void* y,
+                                   int M, int N, int K, int group_size, void* workspace, size_t workspace_bytes,
+                                   qil_stream_t stream) {
+    const qil_status s = check_w4a16(x, qweight, scales, zeros, y, M, N, K, group_size, QIL_LAYOUT_CANONICAL);
+    if (s != QIL_OK) return s;
+    if (N % 2 != 0) return QIL_ERR_SHAPE;
+    if (workspace && !aligned16(workspace)) return QIL_ERR_ALIGN;
+    if (w4a16_prefill_supported(M, N, K, group_size, QIL_LAYOUT_CANONICAL)) {
+        const size_t off = w4a16_skinny_ws_offset();
+        const bool have = workspace != nullptr && workspace_bytes > off;
+        return launch_w4a16_prefill(x, qweight, scales, zeros, y, M, N, K, group_size, 4,
+                                    workspace_bytes >= sizeof(int) ? static_cast<int*>(workspace) : nullptr,
+                                    have ? static_cast<char*>(workspace) + off : nullptr, have ? workspace_bytes - off : 0,
+                                    S(stream), 1);
+    }
+    const size_t off = swiglu_tmp_offset(M, N, K, group_size);
+    if (!workspace || workspace_bytes < off + (size_t)M * N * 2) return QIL_ERR_WORKSPACE;
+    void* tmp = static_cast<char*>(workspace) + off;
+    const qil_status s2 = qil_linear_w4a16(x, qweight, scales, zeros, tmp, M, N, K, group_size, QIL_LAYOUT_CANONICAL, workspace, off, stream);
+    if (s2 != QIL_OK) return s2;
+    return launch_swiglu_rows(tmp, y, M, N, S(stream));
+}
+
 qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs, int count, void* workspace, size_t workspace_bytes,
                                   qil_stream_t stream) {
     if (!descs) return QIL_ERR_NULL;

@@ -73,6 +73,7 @@ struct PrefillParams {
     int nchain;      // accumulators per output that take the K slices in turn (nh == 1 only): 2 or 4, else 1
     int unit_steps;  // the ranges of the CTAs begin at multiples of this many steps
     long long units; // unit_steps-sized pieces of the whole GEMM: tiles * (K / 64) / unit_steps
+    int swiglu;      // rows 2i, 2i + 1 of the weights are gate i and up i: the output is silu(gate) * up, [M][N / 2]
     int* status;
     int fix;         // 1: shared tiles are completed inside this kernel; 0: every part is written out and a second kernel adds them
     int* counters;   // fix: per tile, parts written so far (zero between launches)
@@ -191,6 +192,9 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&d)[16]) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) asm volatile("" : "+r"(d[j]));
 }
+
+// silu(g) * u in fp32 (the gated MLP of the Llama-2 backbone; fused epilogue)
+__device__ __forceinline__ float swiglu(float g, float u) { return g / (1.f + __expf(-g)) * u; }
 
 // The CTA's next run of steps inside one tile: steps [s0, s1) of tile `tile`.  g walks the CTA's range of numbered steps.
 struct Segment {
@@ -506,7 +510,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                 if (part) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) __stcg(part + (size_t)(c0 + j) * kTileF, __uint_as_float(d[j]));
-                } else if (n < p.N && m0 + c0 < p.M) {
+                } else {
+                    const bool live = n < p.N && m0 + c0 < p.M;
+                    if (live)
                     for (int cc = c_first + 1; cc <= c_last; ++cc) {
                         const float* other = p.partials + ((size_t)(2 * cc) * TT + c0) * kTileF + rr;  // (their first part)
                         float v[16];
@@ -515,9 +521,19 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
 #pragma unroll
                         for (int j = 0; j < 16; ++j) d[j] = __float_as_uint(__uint_as_float(d[j]) + v[j]);
                     }
+                    if (p.swiglu) {
+                        // lane = feature: the even lane holds gate i, its neighbour up i (N is even, so both are live or neither)
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (m0 + c0 + j < p.M) p.y[(size_t)(m0 + c0 + j) * p.N + n] = __float2bfloat16_rn(__uint_as_float(d[j]));
+                        for (int j = 0; j < 16; ++j) {
+                            const float u = __uint_as_float(__shfl_xor_sync(0xFFFFFFFFu, d[j], 1));
+                            if (live && (lane & 1) == 0 && m0 + c0 + j < p.M)
+                                p.y[(size_t)(m0 + c0 + j) * (p.N >> 1) + (n >> 1)] = __float2bfloat16_rn(swiglu(__uint_as_float(d[j]), u));
+                        }
+                    } else if (live) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (m0 + c0 + j < p.M) p.y[(size_t)(m0 + c0 + j) * p.N + n] = __float2bfloat16_rn(__uint_as_float(d[j]));
+                    }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -571,6 +587,12 @@ __global__ void __launch_bounds__(256) w4a16_prefill_reduce_kernel(const Prefill
         const int slot = 2 * cc + (range_begin(p.units, C, cc) * p.unit_steps >= (long long)tile * S ? 0 : 1);
         const float4 v = __ldcg(reinterpret_cast<const float4*>(p.partials + ((size_t)slot * TT + t) * kTileF + f));
         acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    if (p.swiglu) {   // features f, f + 1 and f + 2, f + 3 are two (gate, up) pairs
+        __nv_bfloat16* out = p.y + (size_t)(m0 + t) * (p.N >> 1) + ((n0 + f) >> 1);
+        out[0] = __float2bfloat16_rn(swiglu(acc.x, acc.y));
+        if (n0 + f + 2 < p.N) out[1] = __float2bfloat16_rn(swiglu(acc.z, acc.w));
+        return;
     }
     __nv_bfloat16* out = p.y + (size_t)(m0 + t) * p.N + n0 + f;
     if ((p.N & 3) == 0) {
@@ -638,7 +660,22 @@ PrefillPlan plan_prefill(int M, int N, int K, int G, bool with_parts) {
     return pl;
 }
 
+__global__ void swiglu_rows_kernel(const __nv_bfloat16* __restrict__ t, __nv_bfloat16* __restrict__ y, int M, int N) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x, half = N >> 1;
+    if (i >= (long long)M * half) return;
+    const long long m = i / half, c = i - m * half;
+    const __nv_bfloat162 gu = *reinterpret_cast<const __nv_bfloat162*>(t + m * N + 2 * c);
+    y[i] = __float2bfloat16_rn(swiglu(__bfloat162float(gu.x), __bfloat162float(gu.y)));
+}
+
 }  // namespace
+
+qil_status launch_swiglu_rows(const void* t, void* y, int M, int N, cudaStream_t st) {
+    const long long total = (long long)M * (N >> 1);
+    swiglu_rows_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(t),
+                                                                        reinterpret_cast<__nv_bfloat16*>(y), M, N);
+    return launch_status();
+}
 
 bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout) {
     return layout == QIL_LAYOUT_CANONICAL && M > 8 && N >= 1 && K % kStepK == 0 && G % kStepK == 0 && K % G == 0 &&
@@ -654,7 +691,7 @@ size_t w4a16_prefill_workspace(int M, int N, int K, int G) {
 // status (optional): receives QIL_ERR_TIMEOUT if a bounded device-side wait runs out.  scratch: as sized above; when it
 // is missing or too small every CTA computes whole tiles.
 qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scales, const void* zeros, void* y, int M, int N,
-                                int K, int G, int bits, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+                                int K, int G, int bits, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st, int swiglu) {
     const bool with_parts = scratch != nullptr && scratch_bytes >= w4a16_prefill_workspace(M, N, K, G);
     const PrefillPlan pl = plan_prefill(M, N, K, G, with_parts);
     const EncodeFn enc = encode_fn();
@@ -691,6 +728,7 @@ qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scale
     p.unit_steps = pl.unit_steps;
     p.units = pl.units;
     p.status = status;
+    p.swiglu = swiglu;
     p.counters = with_parts ? reinterpret_cast<int*>(scratch) : nullptr;
     // A tile shared by up to three CTAs is completed inside the kernel by the CTA that holds its first steps; when the
     // ranges are short against a tile (more CTAs per tile) that CTA's serial additions cost more than a second, fully

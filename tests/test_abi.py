@@ -73,6 +73,19 @@ def test_linear_w4a16_validation(lib):
     assert lib.qil_linear_w4a16_workspace_size(0, 1, 1, 1) == 0
 
 
+def test_linear_w4a16_swiglu_validation(lib):
+    f = lib.qil_linear_w4a16_swiglu
+    assert f(None, A, A, A, A, 1, 16, 128, 128, None, 0, None) == 1
+    assert f(A, A, A, A, A, 0, 16, 128, 128, None, 0, None) == 2
+    assert f(A, A, A, A, A, 1, 15, 128, 128, None, 0, None) == 2    # gate / up rows come in pairs
+    assert f(A, A, A, A, A, 1, 16, 128, 48, None, 0, None) == 2     # K % group
+    assert f(A, U, A, A, A, 1, 16, 128, 128, None, 0, None) == 3
+    # the unfused shapes need the workspace (it holds the linear's bf16 output)
+    assert f(A, A, A, A, A, 1, 16, 128, 128, None, 0, None) == 5
+    assert lib.qil_linear_w4a16_swiglu_workspace_size(1, 16, 128, 128) >= lib.qil_linear_w4a16_workspace_size(1, 16, 128, 128) + 1 * 16 * 2
+    assert lib.qil_linear_w4a16_swiglu_workspace_size(0, 16, 128, 128) == 0
+
+
 def test_w4a4_and_act_validation(lib):
     assert lib.qil_quantize_act_a4(None, 1, 8, None, A, A, None) == 1
     assert lib.qil_quantize_act_a4(A, 1, 12, None, A, A, None) == 2

@@ -264,6 +264,36 @@ def test_w4a16_prefill_workspace_is_reusable_across_shapes(api):
     assert int(ws[:4].view(torch.int32).cpu()[0]) == 0   # the status word: no wait ran out
 
 
+@pytest.mark.parametrize("M,N,K,G", [
+    (280, 512, 1024, 128),   # the GEMM with the fused epilogue, tiles shared by two CTAs
+    (280, 256, 4096, 128),   # tiles shared by many CTAs: the epilogue runs in the kernel that adds the parts
+    (130, 154, 256, 64),     # ragged M and N (N / 2 odd)
+    (600, 384, 512, 128),    # three token tiles
+    (40, 640, 2048, 128),    # four accumulators per output
+    (4, 64, 256, 128), (280, 48, 200, 40),   # shapes the GEMM does not take: linear into the workspace, then the activation
+])
+def test_w4a16_swiglu(api, M, N, K, G):
+    """Gate and up rows interleaved, silu(gate) * up in the epilogue (the gated MLP of the Llama-2 backbone,
+    App. A.4.2) against the oracle.  Tolerance, per token row, from the linear's own contract REL (row-relative on gate
+    and on up): |d silu| <= 1.1 |d gate|, so |dy| <= REL (1.1 + 1) max|gate| max|up|, plus the output's bf16 rounding."""
+    w = wl.normal_weights(320, N + K, N, K, 0.05)
+    x = wl.normal_activations_bf16(320, N + K + 1, M, K)
+    codes, scales, zeros = np_oracle.quantize_rtn_w4_asym(w, G)
+    y = api.linear_w4a16_swiglu(to_bf16_cuda(x), api.pack_w4(cuda(codes)), cuda(scales), cuda(zeros), N, G)
+    assert tuple(y.shape) == (M, N // 2)
+    t = c_oracle.linear_w4a16(x, codes, scales, zeros, G)
+    y_ref = np_oracle.silu(t[:, 0::2]) * t[:, 1::2]
+    np.testing.assert_allclose(y_ref, np_oracle.linear_w4a16_swiglu(x, codes, scales, zeros, G), rtol=1e-9, atol=1e-12)
+    gmax, umax = np.abs(t[:, 0::2]).max(axis=1, keepdims=True), np.abs(t[:, 1::2]).max(axis=1, keepdims=True)
+    tol = (2.1 * CONTRACT_REL + 2.0 ** -8) * gmax * umax
+    got = bf16_to_f64(y)
+    assert np.all(np.isfinite(got))
+    assert np.all(np.abs(got - y_ref) <= tol + 1e-30), float((np.abs(got - y_ref) / tol).max())
+    # and the same bits on a second call
+    y2 = api.linear_w4a16_swiglu(to_bf16_cuda(x), api.pack_w4(cuda(codes)), cuda(scales), cuda(zeros), N, G)
+    np.testing.assert_array_equal(bits_of(y), bits_of(y2))
+
+
 @pytest.mark.parametrize("N,K,G", [(24, 256, 32), (9, 40, 8), (17, 192, 64), (8, 320, 320)])
 def test_w4a16_general_shapes(api, N, K, G):
     for M in (1, 6):

@@ -1,0 +1,84 @@
+"""Pins of the oracle's gated-MLP linear (`np_oracle.silu`, `np_oracle.linear_w4a16_swiglu`) against what the
+mathematics fixes: closed forms and identities of silu, a hand-computed case, and the reduction to two plain
+(already pinned) linears.  A dropped factor, a swapped gate / up, a wrong sign in the exponent or an off-by-one in the
+row interleave fails one of them.
+"""
+import math
+
+import numpy as np
+
+from oracle import np_oracle
+from paper_2412_01034_b200 import workloads as wl
+
+
+def test_silu_closed_forms():
+    s = np_oracle.silu
+    assert s(np.array([0.0]))[0] == 0.0
+    # silu(x) - silu(-x) = x  (sigmoid(x) + sigmoid(-x) = 1)
+    x = np.linspace(-30, 30, 241)
+    np.testing.assert_allclose(s(x) - s(-x), x, rtol=0, atol=1e-12)
+    # silu(ln 3) = ln 3 * 3/4, silu(-ln 3) = -ln 3 / 4
+    l3 = math.log(3.0)
+    np.testing.assert_allclose(s(np.array([l3, -l3])), [0.75 * l3, -0.25 * l3], rtol=1e-15)
+    # limits: x for large x, x e^x for very negative x; nothing overflows on the way (e^-800 flushing to 0 is meant)
+    with np.errstate(over="raise", invalid="raise", divide="raise"):
+        big = s(np.array([800.0, -800.0, 40.0]))
+    assert big[0] == 800.0 and big[1] == 0.0 and abs(big[2] - 40.0) < 1e-15
+    np.testing.assert_allclose(s(np.array([-20.0]))[0], -20.0 * math.exp(-20.0), rtol=1e-8)
+    # the minimum of silu is at the root of 1 + e^-x (1 + x) ... = 0: x = -1.2784645..., value -0.2784645...
+    grid = np.linspace(-3, 0, 300001)
+    v = s(grid)
+    i = int(np.argmin(v))
+    assert abs(grid[i] + 1.2784645427610738) < 2e-5 and abs(v[i] + 0.2784645427610738) < 1e-10
+
+
+def test_silu_derivative_matches_the_formula():
+    # d/dx silu = sigma (1 + x (1 - sigma)): a central difference of the oracle must agree
+    x = np.linspace(-6, 6, 49)
+    h = 1e-6
+    num = (np_oracle.silu(x + h) - np_oracle.silu(x - h)) / (2 * h)
+    sig = 1.0 / (1.0 + np.exp(-x))
+    np.testing.assert_allclose(num, sig * (1 + x * (1 - sig)), rtol=0, atol=1e-8)
+
+
+def test_swiglu_hand_case():
+    # one token, K = 8, one group; gate row (code - z) * s = [1, 1, 0, ...] * 0.5, up row = [2, 0, ...] * 0.25
+    G = 8
+    codes = np.array([[9, 9, 8, 8, 8, 8, 8, 8], [10, 8, 8, 8, 8, 8, 8, 8]], dtype=np.uint8)
+    scales = np.array([[0.5], [0.25]], dtype=np.float16)
+    zeros = np.array([[8.0], [8.0]], dtype=np.float16)
+    x = wl.f32_to_bf16_bits(np.array([[2.0, 1.0, 5.0, 0, 0, 0, 0, 0]], dtype=np.float32))
+    # gate = 0.5 * (2 + 1) = 1.5, up = 0.25 * 2 * 2 = 1.0
+    y = np_oracle.linear_w4a16_swiglu(x, codes, scales, zeros, G)
+    assert y.shape == (1, 1)
+    assert abs(y[0, 0] - 1.5 / (1.0 + math.exp(-1.5)) * 1.0) < 1e-15
+    # swapping the two rows swaps the roles: silu(1.0) * 1.5
+    y2 = np_oracle.linear_w4a16_swiglu(x, codes[::-1], scales[::-1], zeros[::-1], G)
+    assert abs(y2[0, 0] - 1.0 / (1.0 + math.exp(-1.0)) * 1.5) < 1e-15
+
+
+def test_swiglu_is_two_plain_linears_and_the_activation():
+    rng = wl.generator(77, 0)
+    N2, K, G, M = 24, 64, 32, 5
+    gate = rng.normal(0, 0.3, (N2, K)).astype(np.float32)
+    up = rng.normal(0, 0.3, (N2, K)).astype(np.float32)
+    x = wl.normal_activations_bf16(77, 1, M, K)
+    qg = np_oracle.quantize_rtn_w4_asym(gate, G)
+    qu = np_oracle.quantize_rtn_w4_asym(up, G)
+    inter = [np.stack((a, b), axis=1).reshape(2 * N2, -1) for a, b in zip(qg, qu)]
+    # interleaving rows before or after quantising is the same thing (the quantiser works row by row)
+    both = np.stack((gate, up), axis=1).reshape(2 * N2, K)
+    for a, b in zip(np_oracle.quantize_rtn_w4_asym(both, G), inter):
+        np.testing.assert_array_equal(a, b)
+    y = np_oracle.linear_w4a16_swiglu(x, *inter, G)
+    yg = np_oracle.linear_w4a16(x, *qg, G)
+    yu = np_oracle.linear_w4a16(x, *qu, G)
+    expect = yg / (1.0 + np.exp(-yg)) * yu
+    np.testing.assert_allclose(y, expect, rtol=1e-13, atol=1e-15)
+    # a zero up projection gives zero; a zero gate gives zero as well (silu(0) = 0)
+    z_up = [inter[0].copy(), inter[1], inter[2]]
+    z_up[0][1::2] = inter[2][1::2].astype(np.uint8).repeat(G, axis=1)   # code = zero point: dequantises to 0
+    assert np.all(np_oracle.linear_w4a16_swiglu(x, *z_up, G) == 0.0)
+    z_gate = [inter[0].copy(), inter[1], inter[2]]
+    z_gate[0][0::2] = inter[2][0::2].astype(np.uint8).repeat(G, axis=1)
+    assert np.all(np_oracle.linear_w4a16_swiglu(x, *z_gate, G) == 0.0)

@@ -660,6 +660,16 @@ def secondary_measurements(dev):
     out["w4a16_m_sweep"] = sweep
     flops = sum(2.0 * Mp * N * K for (_, N, K) in wl.LLAMA2_7B_LAYER)
     out["w4a16_prefill_m280_layer"] = {"us": t_layer, "TFLOP/s": flops / t_layer / 1e6, "kernel": "w4a16_prefill_kernel (tcgen05 kind::f16)"}
+    # the unmerged rank-32 adapter beside a 4096 x 4096 linear, at decode and at prefill length
+    lora = {}
+    for Ml in (1, Mp):
+        xl = torch.randn((Ml, wl.HIDDEN), device=dev, generator=g).to(torch.bfloat16)
+        al = (torch.randn((32, wl.HIDDEN), device=dev, generator=g) * 0.02).to(torch.bfloat16)
+        bl = (torch.randn((wl.HIDDEN, 32), device=dev, generator=g) * 0.02).to(torch.bfloat16)
+        yl = torch.zeros((Ml, wl.HIDDEN), dtype=torch.bfloat16, device=dev)
+        wsl = api.new_workspace(Ml * 32 * 4, dev)
+        lora[f"m{Ml}_us"] = time_us(lambda: api.lora_side_add(xl, al, bl, yl, 1.0, workspace=wsl), 20)
+    out["lora_side_rank32_4096x4096"] = lora
     out["w4a16_prefill_m280_gate_up_22016x4096"] = {"plain_us": t_gate_up, "swiglu_epilogue_us": t_gate_up_sw,
                                                     "TFLOP/s": 2.0 * Mp * 2 * wl.FFN * wl.HIDDEN / t_gate_up_sw / 1e6}
     out["w4a16_prefill_m280_layer_fused_qkv_gate_up"] = {"us": t_layer_fused, "TFLOP/s": flops / t_layer_fused / 1e6,

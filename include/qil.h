@@ -160,6 +160,23 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
                             qil_stream_t stream);
 
 /* -------------------------------------------------------------------------
+ * qil_lora_side_add: the low-rank side path of a quantised linear, for
+ * adapters that are kept beside the frozen 4-bit base instead of being merged
+ * (the paper fine-tunes OpenVLA with QLoRA adapters of rank 32, App. A.1.2):
+ *     y[m][n] = bf16( float(y[m][n]) + scale * sum_j (sum_k x[m][k] A[j][k]) B[n][j] )
+ *   x [M][K] bf16   A [rank][K] bf16   B [N][rank] bf16   y [M][N] bf16, in place
+ * fp32 accumulation; the inner product x . A^T is kept in fp32 in the
+ * workspace (qil_lora_side_workspace_size(M) bytes, no initialisation needed).
+ * Call it after the linear that produced y, on the same stream.
+ * rank <= 32 (larger: UNSUPPORTED); K even.
+ * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, CUDA.
+ * ---------------------------------------------------------------------- */
+size_t qil_lora_side_workspace_size(int M);
+qil_status qil_lora_side_add(const void* x, const void* a, const void* b, void* y, int M, int N, int K,
+                             int rank, float scale, void* workspace, size_t workspace_bytes,
+                             qil_stream_t stream);
+
+/* -------------------------------------------------------------------------
  * qil_linear_w4a16_swiglu: the gate and up projections of a gated MLP (the
  * Llama-2 backbone of the paper's OpenVLA deployment, App. A.4.2) as ONE
  * weight-only linear with the activation fused into its epilogue:

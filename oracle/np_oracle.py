@@ -262,6 +262,16 @@ def linear_w4a16(x_bf16_bits, codes, scales, zeros, group_size: int) -> np.ndarr
     return np.matmul(x, w_hat.T)
 
 
+def lora_side(x_bf16_bits, a_bf16_bits, b_bf16_bits, scale: float) -> np.ndarray:
+    """The term an unmerged low-rank adapter adds to a linear's output (the paper fine-tunes OpenVLA with QLoRA
+    adapters of rank 32 over the frozen quantised base, App. A.1.2): scale * (x . A^T) . B^T, fp64 throughout.
+    x [M][K], A [r][K], B [N][r], all given as bf16 bit patterns."""
+    x = bf16_to_f32(x_bf16_bits).astype(np.float64)
+    a = bf16_to_f32(a_bf16_bits).astype(np.float64)
+    b = bf16_to_f32(b_bf16_bits).astype(np.float64)
+    return float(scale) * np.matmul(np.matmul(x, a.T), b.T)
+
+
 def silu(g: np.ndarray) -> np.ndarray:
     """silu(g) = g / (1 + exp(-g)), fp64 (the activation of the Llama-2 gated MLP, the backbone of the paper's OpenVLA
     deployment, App. A.4.2).  Written so that large |g| neither overflows nor loses the small side."""

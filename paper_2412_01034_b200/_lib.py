@@ -17,6 +17,8 @@ SIGNATURES = {
     "qil_pack_stream128_w4": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "qil_linear_w4a16_workspace_size": (_sz, [_i, _i, _i, _i]),
     "qil_linear_w4a16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_lora_side_workspace_size": (_sz, [_i]),
+    "qil_lora_side_add": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, C.c_float, _vp, _sz, _vp]),
     "qil_linear_w4a16_swiglu_workspace_size": (_sz, [_i, _i, _i, _i]),
     "qil_linear_w4a16_swiglu": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w4a16_static_ws": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),

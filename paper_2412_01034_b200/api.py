@@ -182,6 +182,20 @@ def linear_w4a16(x, qweight, scales, zeros, N: int, group_size: int, layout: int
     return out
 
 
+def lora_side_add(x, a, b, y, scale: float = 1.0, workspace=None, stream=None):
+    """y[M][N] (bf16, in place) += scale * (x[M][K] . a[r][K]^T) . b[N][r]^T: an unmerged low-rank adapter, r <= 32."""
+    _need_cuda(x, a, b, y, workspace)
+    M, K = x.shape
+    r = a.shape[0]
+    N = b.shape[0]
+    assert a.shape == (r, K) and b.shape == (N, r) and y.shape == (M, N)
+    if workspace is None:
+        workspace = torch.empty(max(int(_lib.load().qil_lora_side_workspace_size(M)), 16), dtype=torch.uint8, device=x.device)
+    _check(_lib.load().qil_lora_side_add(_ptr(x), _ptr(a), _ptr(b), _ptr(y), M, N, K, r, float(scale), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)))
+    return y
+
+
 def interleave_rows(gate, up):
     """Rows 2i = gate[i], 2i + 1 = up[i] (codes, scales or zeros of the two projections of a gated MLP): the weight
     layout `linear_w4a16_swiglu` expects.  A layout step done once, offline."""

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libqil.so")
 SOURCES = ["api.cu", "quantize.cu", "w4a16_general.cu", "w4a16_skinny.cu", "w4a4.cu", "ref_gemv.cu",
-           "w4a16_static_ws.cu", "w4a16_tc.cu", "w4a16_prefill.cu", "w8a16.cu", "probe_mma.cu", "igemm_list.cu"]
+           "w4a16_static_ws.cu", "w4a16_tc.cu", "w4a16_prefill.cu", "w8a16.cu", "probe_mma.cu", "igemm_list.cu", "lora_side.cu"]
 
 
 def _nvcc() -> str:

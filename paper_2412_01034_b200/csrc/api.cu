@@ -232,6 +232,21 @@ qil_status qil_linear_w4a16_swiglu(const void* x, const uint32_t* qweight, const
     return launch_swiglu_rows(tmp, y, M, N, S(stream));
 }
 
+size_t qil_lora_side_workspace_size(int M) { return M > 0 ? lora_side_workspace(M) : 0; }
+
+qil_status qil_lora_side_add(const void* x, const void* a, const void* b, void* y, int M, int N, int K, int rank, float scale,
+                             void* workspace, size_t workspace_bytes, qil_stream_t stream) {
+    if (!x || !a || !b || !y) return QIL_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || rank <= 0 || K % 2 != 0) return QIL_ERR_SHAPE;
+    if (!lora_side_supported(M, N, K, rank)) return QIL_ERR_UNSUPPORTED;   // rank > 32
+    if (reinterpret_cast<uintptr_t>(x) % 4 || reinterpret_cast<uintptr_t>(a) % 4 || reinterpret_cast<uintptr_t>(b) % 2 ||
+        reinterpret_cast<uintptr_t>(y) % 2)
+        return QIL_ERR_ALIGN;
+    if (!workspace || workspace_bytes < lora_side_workspace(M)) return QIL_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) % 4) return QIL_ERR_ALIGN;
+    return launch_lora_side_add(x, a, b, y, M, N, K, rank, scale, workspace, S(stream));
+}
+
 qil_status qil_linear_w4a16_batch(const qil_linear_desc* descs, int count, void* workspace, size_t workspace_bytes,
                                   qil_stream_t stream) {
     if (!descs) return QIL_ERR_NULL;

@@ -83,6 +83,11 @@ bool w4a16_prefill_supported(int M, int N, int K, int G, qil_layout layout);
 size_t w4a16_prefill_workspace(int M, int N, int K, int G);  // tile counters + the fp32 parts of tiles that CTAs share
 qil_status launch_w4a16_prefill(const void* x, const void* qw, const void* scales, const void* zeros, void* y, int M, int N,
                                 int K, int G, int bits, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st, int swiglu = 0);
+// low-rank side path y += scale * (x . A^T) . B^T, rank <= 32 (lora_side.cu)
+size_t lora_side_workspace(int M);
+bool lora_side_supported(int M, int N, int K, int r);
+qil_status launch_lora_side_add(const void* x, const void* a, const void* b, void* y, int M, int N, int K, int r, float scale,
+                                void* ws, cudaStream_t st);
 // y[m][i] = silu(t[m][2 i]) * t[m][2 i + 1] for a linear's output t[M][N] (the shapes the GEMM above does not take)
 qil_status launch_swiglu_rows(const void* t, void* y, int M, int N, cudaStream_t st);
 

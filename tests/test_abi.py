@@ -86,6 +86,17 @@ def test_linear_w4a16_swiglu_validation(lib):
     assert lib.qil_linear_w4a16_swiglu_workspace_size(0, 16, 128, 128) == 0
 
 
+def test_lora_side_validation(lib):
+    f = lib.qil_lora_side_add
+    assert f(None, A, A, A, 1, 16, 128, 32, 1.0, A, 4096, None) == 1
+    assert f(A, A, A, A, 1, 16, 127, 32, 1.0, A, 4096, None) == 2    # K even
+    assert f(A, A, A, A, 1, 16, 128, 0, 1.0, A, 4096, None) == 2
+    assert f(A, A, A, A, 1, 16, 128, 33, 1.0, A, 4096, None) == 4    # rank above 32
+    assert f(A, A, A, A, 4, 16, 128, 32, 1.0, A, 16, None) == 5      # workspace too small
+    assert f(A, A, A, A, 4, 16, 128, 32, 1.0, None, 0, None) == 5
+    assert lib.qil_lora_side_workspace_size(4) == 4 * 32 * 4
+
+
 def test_w4a4_and_act_validation(lib):
     assert lib.qil_quantize_act_a4(None, 1, 8, None, A, A, None) == 1
     assert lib.qil_quantize_act_a4(A, 1, 12, None, A, A, None) == 2

@@ -294,6 +294,34 @@ def test_w4a16_swiglu(api, M, N, K, G):
     np.testing.assert_array_equal(bits_of(y), bits_of(y2))
 
 
+@pytest.mark.parametrize("M,N,K,r", [(1, 4096, 4096, 32), (7, 1000, 2176, 32), (280, 513, 1024, 16), (9, 64, 34, 5), (33, 2, 64, 1)])
+def test_lora_side_add(api, M, N, K, r):
+    """The unmerged low-rank adapter beside a quantised linear (QLoRA rank 32, App. A.1.2): y += scale (x A^T) B^T on
+    top of an existing bf16 y.  fp32 accumulation over K and over the rank, one bf16 rounding of the sum: the error is
+    bounded by the output's half ulp plus fp32 round-off of the two inner products."""
+    import torch
+    rng = wl.generator(330, N + K)
+    x = wl.normal_activations_bf16(330, 1, M, K)
+    a = wl.f32_to_bf16_bits(rng.normal(0, 0.05, (r, K)).astype(np.float32))
+    b = wl.f32_to_bf16_bits(rng.normal(0, 0.05, (N, r)).astype(np.float32))
+    y0 = wl.f32_to_bf16_bits(rng.normal(0, 1.0, (M, N)).astype(np.float32))
+    scale = 2.0
+    side = np_oracle.lora_side(x, a, b, scale)
+    want = np_oracle.bf16_to_f32(y0).astype(np.float64) + side
+    y = to_bf16_cuda(y0).clone()
+    api.lora_side_add(to_bf16_cuda(x), to_bf16_cuda(a), to_bf16_cuda(b), y, scale)
+    got = bf16_to_f64(y)
+    # |x A^T| terms: K products, fp32; the rank sum: r products
+    absside = scale * np.abs(np_oracle.bf16_to_f32(x).astype(np.float64)) @ np.abs(np_oracle.bf16_to_f32(a).astype(np.float64)).T \
+        @ np.abs(np_oracle.bf16_to_f32(b).astype(np.float64)).T
+    tol = 2.0 ** -8 * np.abs(want) + (K + r + 4) * 2.0 ** -24 * absside + 1e-30
+    assert np.all(np.abs(got - want) <= tol), float((np.abs(got - want) / tol).max())
+    # untouched when the scale is zero
+    y1 = to_bf16_cuda(y0).clone()
+    api.lora_side_add(to_bf16_cuda(x), to_bf16_cuda(a), to_bf16_cuda(b), y1, 0.0)
+    np.testing.assert_array_equal(bits_of(y1), bits_of(to_bf16_cuda(y0)))
+
+
 @pytest.mark.parametrize("N,K,G", [(24, 256, 32), (9, 40, 8), (17, 192, 64), (8, 320, 320)])
 def test_w4a16_general_shapes(api, N, K, G):
     for M in (1, 6):

@@ -82,3 +82,31 @@ def test_swiglu_is_two_plain_linears_and_the_activation():
     z_gate = [inter[0].copy(), inter[1], inter[2]]
     z_gate[0][0::2] = inter[2][0::2].astype(np.uint8).repeat(G, axis=1)
     assert np.all(np_oracle.linear_w4a16_swiglu(x, *z_gate, G) == 0.0)
+
+
+# ---- the low-rank side path (np_oracle.lora_side) ----
+def test_lora_side_hand_case_and_identities():
+    f = wl.f32_to_bf16_bits
+    # rank 1: A = [1, 2, 0, 0], B = [[3], [-1]], x = [[1, 1, 5, 7]]: x . A^T = 3, times B = [9, -3], times scale 0.5
+    x = f(np.array([[1.0, 1.0, 5.0, 7.0]], dtype=np.float32))
+    a = f(np.array([[1.0, 2.0, 0.0, 0.0]], dtype=np.float32))
+    b = f(np.array([[3.0], [-1.0]], dtype=np.float32))
+    np.testing.assert_array_equal(np_oracle.lora_side(x, a, b, 0.5), [[4.5, -1.5]])
+    # it is the dense linear with W = B A (exactly representable operands -> exact)
+    rng = wl.generator(78, 0)
+    M, K, r, N = 5, 16, 3, 7
+    xi = rng.integers(-4, 5, (M, K)).astype(np.float32)
+    ai = rng.integers(-3, 4, (r, K)).astype(np.float32)
+    bi = rng.integers(-3, 4, (N, r)).astype(np.float32)
+    got = np_oracle.lora_side(f(xi), f(ai), f(bi), 2.0)
+    np.testing.assert_array_equal(got, 2.0 * xi.astype(np.float64) @ (bi.astype(np.float64) @ ai.astype(np.float64)).T)
+    # linear in the scale, zero for a zero factor, and transposing the roles of A and B is a different thing
+    np.testing.assert_array_equal(np_oracle.lora_side(f(xi), f(ai), f(bi), -1.0), -0.5 * got)
+    assert np.all(np_oracle.lora_side(f(xi), f(0 * ai), f(bi), 1.0) == 0)
+    assert np.all(np_oracle.lora_side(f(xi), f(ai), f(0 * bi), 1.0) == 0)
+    # a rank-r identity embedding: A picks the first r inputs, B puts them on the first r outputs
+    a_id = np.zeros((r, K), dtype=np.float32); a_id[np.arange(r), np.arange(r)] = 1
+    b_id = np.zeros((N, r), dtype=np.float32); b_id[np.arange(r), np.arange(r)] = 1
+    out = np_oracle.lora_side(f(xi), f(a_id), f(b_id), 1.0)
+    np.testing.assert_array_equal(out[:, :r], xi[:, :r])
+    assert np.all(out[:, r:] == 0)

@@ -486,6 +486,23 @@ def secondary_measurements(dev):
         t_l = time_us(lambda: api.linear_int_batch(ents, workspace=wsl), 50)
         out[key] = {"us": t_l, "tops": ops_all / t_l / 1e6, "frac_of_i8_probe": ops_all / t_l / 1e6 / i8_roof,
                     "kernel": "igemm_list_kernel", "l2": "warm"}
+    # the same four layers read straight from int4 feature maps (no im2col matrix), bf16 output and int4 output
+    fm = []
+    for stage in range(4):
+        Cc, H, W = wl.CONV_STAGES[stage]
+        B = wl.CONV_BATCH
+        codes = torch.randint(-8, 8, (B * H * W, Cc), device=dev, generator=g, dtype=torch.int32).to(torch.int8)
+        qf = api.pack_w4(codes).reshape(B, H, W, Cc // 8)
+        w = torch.randn((Cc, 9 * Cc), device=dev, generator=g) * wl.SIGMA_CONV
+        qw_, sw_, _ = api.quantize_rtn_w4(w, 9 * Cc, symmetric=True)
+        pw_ = api.pack_w4(qw_)
+        wsc = api.new_workspace(api.linear_w4a4_workspace_size(B * H * W, Cc, 9 * Cc), dev)
+        t_bf = time_us(lambda: api.conv3x3_w4a4(qf, 0.25, pw_, sw_.reshape(-1), workspace=wsc), 50)
+        t_q = time_us(lambda: api.conv3x3_w4a4(qf, 0.25, pw_, sw_.reshape(-1), out_scale=0.5, relu=True, workspace=wsc), 50)
+        ops = 2.0 * B * H * W * 9 * Cc * Cc
+        fm.append({"C": Cc, "H": H, "W": W, "batch": B, "bf16_out_us": t_bf, "int4_out_us": t_q, "tops": ops / t_q / 1e6})
+    out["w4a4_conv3x3_from_feature_map"] = fm
+    out["w4a4_conv3x3_from_feature_map_tops_total"] = sum(2.0 * f["batch"] * f["H"] * f["W"] * 9 * f["C"] ** 2 for f in fm) / sum(f["int4_out_us"] for f in fm) / 1e6
     out["w4a4_conv_stages"] = conv
     out["w4a4_tops_total"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv) / sum(c["gemm_us"] for c in conv) / 1e6
     out["w4a4_tops_total_cold"] = sum(2.0 * c["M"] * c["K"] * c["N"] for c in conv) / sum(c["gemm_cold_us"] for c in conv) / 1e6

@@ -359,6 +359,23 @@ qil_status qil_linear_w4a4_requant(const uint32_t* qx, const float* sx, const ui
                                    uint32_t* qy, float out_scale, int relu, int M, int N, int K,
                                    void* workspace, size_t workspace_bytes, qil_stream_t stream);
 
+/* 3 x 3 convolution (stride 1, zero padding 1) of the W4A4 conv backbone (the CILRS-style encoder, Sec. 5.1,
+ * App. A.1.2) read straight from the int4 feature map, without a materialised im2col matrix: the GEMM's loader
+ * computes, for row (b, h, w) and column (3 kh + kw) C + c, the address of channel c of pixel (h + kh - 1, w + kw - 1)
+ * or takes zero outside the image.
+ *   qx [B][H][W][C/8]   the feature map, NHWC, signed 4-bit codes packed 8 per word along C; one static scale x_scale
+ *                       for the whole tensor (the paper's tensor-wise activation setting, App. A.1.2)
+ *   qw [Cout][9 C / 8]  filters, column (3 kh + kw) C + c, packed like qx; sw [Cout] fp32 per-filter scales
+ * Output, one of (the other pointer null):
+ *   y  [B][H][W][Cout] bf16 = float(acc) * (x_scale * sw[n]); acc_out: optional int32 copy of the accumulators;
+ *   qy [B][H][W][Cout/8]: the next layer's feature map, quantised in the epilogue as in qil_linear_w4a4_requant
+ *      (ReLU if relu, static scale out_scale; Cout % 8 == 0), so that a stack of conv layers never leaves 4 bits.
+ * Needs C % 32 == 0 and 9 C < 131072.  workspace: qil_linear_w4a4_workspace_size(B H W, Cout, 9 C) bytes.
+ * Errors: NULL (also both or neither output), SHAPE, ALIGN, UNSUPPORTED (out_scale <= 0), WORKSPACE, CUDA. */
+qil_status qil_conv3x3_w4a4(const uint32_t* qx, float x_scale, const uint32_t* qw, const float* sw, void* y,
+                            int32_t* acc_out, uint32_t* qy, float out_scale, int relu, int B, int H, int W,
+                            int C, int Cout, void* workspace, size_t workspace_bytes, qil_stream_t stream);
+
 /* W8A8 integer GEMM (Table "CILRS performance", W8A8 row; Sec. 5.4): as qil_linear_w4a4 with one signed byte per
  * element: qx [M][K], qw [N][K] int8; acc exact in int32 (|acc| <= 2^14 K: K < 131072), K % 16 == 0; the same
  * workspace (qil_linear_w4a4_workspace_size). */

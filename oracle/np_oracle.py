@@ -262,6 +262,33 @@ def linear_w4a16(x_bf16_bits, codes, scales, zeros, group_size: int) -> np.ndarr
     return np.matmul(x, w_hat.T)
 
 
+def conv3x3_w4a4(q_fmap, x_scale: float, qw, sw):
+    """3 x 3 convolution, stride 1, zero padding 1, on integer codes (the W4A4 conv layers of the CILRS-style encoder,
+    Sec. 5.1, App. A.1.2; one static activation scale for the tensor):
+        acc[b][h][w][n] = sum_{kh, kw, c} q[b][h + kh - 1][w + kw - 1][c] * qw[n][(3 kh + kw) C + c]   (0 outside the image)
+        y = acc * x_scale * sw[n]
+    q_fmap [B][H][W][C], qw [Cout][9 C] integers; returns (acc int64, y fp64), both [B][H][W][Cout].  Written tap by tap
+    from the definition (no im2col matrix)."""
+    q = np.asarray(q_fmap).astype(np.int64)
+    w = np.asarray(qw).astype(np.int64)
+    B, H, W, Cc = q.shape
+    Cout = w.shape[0]
+    assert w.shape[1] == 9 * Cc
+    acc = np.zeros((B, H, W, Cout), dtype=np.int64)
+    for kh in range(3):
+        for kw in range(3):
+            tap = w[:, (3 * kh + kw) * Cc:(3 * kh + kw + 1) * Cc]          # [Cout][C]
+            # output pixels (h, w) whose input pixel (h + kh - 1, w + kw - 1) lies inside the image
+            h0, h1 = max(0, 1 - kh), min(H, H + 1 - kh)
+            w0, w1 = max(0, 1 - kw), min(W, W + 1 - kw)
+            if h0 >= h1 or w0 >= w1:
+                continue
+            src = q[:, h0 + kh - 1:h1 + kh - 1, w0 + kw - 1:w1 + kw - 1, :]
+            acc[:, h0:h1, w0:w1, :] += np.matmul(src, tap.T)
+    y = acc.astype(np.float64) * float(x_scale) * np.asarray(sw, dtype=np.float64).reshape(1, 1, 1, -1)
+    return acc, y
+
+
 def lora_side(x_bf16_bits, a_bf16_bits, b_bf16_bits, scale: float) -> np.ndarray:
     """The term an unmerged low-rank adapter adds to a linear's output (the paper fine-tunes OpenVLA with QLoRA
     adapters of rank 32 over the frozen quantised base, App. A.1.2): scale * (x . A^T) . B^T, fp64 throughout.

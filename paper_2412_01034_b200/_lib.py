@@ -34,6 +34,7 @@ SIGNATURES = {
     "qil_quantize_act_a4": (_i, [_vp, _i, _i, C.POINTER(C.c_float), _vp, _vp, _vp]),
     "qil_linear_w4a4_workspace_size": (_sz, [_i, _i, _i]),
     "qil_linear_w4a4": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "qil_conv3x3_w4a4": (_i, [_vp, C.c_float, _vp, _vp, _vp, _vp, _vp, C.c_float, _i, _i, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w4a4_requant": (_i, [_vp, _vp, _vp, _vp, _vp, C.c_float, _i, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_w8a8": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "qil_linear_int_batch": (_i, [_vp, _i, _vp, _sz, _vp]),

@@ -268,6 +268,32 @@ def linear_w4a4_requant(qx, sx, qw, sw, out_scale: float, relu: bool = False, wo
     return qy
 
 
+def conv3x3_w4a4(qx, x_scale: float, qw, sw, out_scale: float | None = None, relu: bool = False, want_acc: bool = False,
+                 workspace=None, stream=None):
+    """3 x 3 convolution (stride 1, zero padding 1) on an int4 feature map qx [B][H][W][C/8] with filters qw
+    [Cout][9C/8] (column (3 kh + kw) C + c).  out_scale None: returns bf16 y [B][H][W][Cout] (and the int32
+    accumulators if want_acc); else the next layer's packed int4 feature map [B][H][W][Cout/8]."""
+    _need_cuda(qx, qw, sw, workspace)
+    B, H, W = qx.shape[0], qx.shape[1], qx.shape[2]
+    Cin, Cout = qx.shape[3] * 8, qw.shape[0]
+    assert qw.shape[1] * 8 == 9 * Cin
+    y = acc = qy = None
+    if out_scale is None:
+        y = torch.empty((B, H, W, Cout), dtype=torch.bfloat16, device=qx.device)
+        if want_acc:
+            acc = torch.empty((B, H, W, Cout), dtype=torch.int32, device=qx.device)
+    else:
+        qy = torch.empty((B, H, W, max(Cout // 8, 1)), dtype=torch.int32, device=qx.device)
+    if workspace is None:
+        workspace = new_workspace(linear_w4a4_workspace_size(B * H * W, Cout, 9 * Cin), qx.device)
+    _check(_lib.load().qil_conv3x3_w4a4(_ptr(qx), C.c_float(x_scale), _ptr(qw), _ptr(sw), _ptr(y), _ptr(acc), _ptr(qy),
+                                        C.c_float(out_scale if out_scale is not None else 1.0), int(bool(relu)), B, H, W, Cin,
+                                        Cout, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+    if out_scale is not None:
+        return qy
+    return (y, acc) if want_acc else y
+
+
 def linear_int_batch(entries, workspace=None, stream=None):
     """A list of independent integer GEMMs in one launch.  entries: [(qx, sx, qw, sw, y, acc or None, bits)] with the
     operands of linear_w4a4 (bits 4) or linear_w8a8 (bits 8); outputs are written into y (and acc)."""

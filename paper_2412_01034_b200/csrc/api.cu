@@ -427,6 +427,23 @@ qil_status qil_linear_w4a4_requant(const uint32_t* qx, const float* sx, const ui
                        out_scale, relu ? 1 : 0);
 }
 
+qil_status qil_conv3x3_w4a4(const uint32_t* qx, float x_scale, const uint32_t* qw, const float* sw, void* y, int32_t* acc_out,
+                            uint32_t* qy, float out_scale, int relu, int B, int H, int W, int C, int Cout, void* workspace,
+                            size_t workspace_bytes, qil_stream_t stream) {
+    if (!qx || !qw || !sw || (!y && !qy) || (y && qy)) return QIL_ERR_NULL;
+    if (B <= 0 || H <= 0 || W <= 0 || C <= 0 || Cout <= 0 || C % 32 != 0 || 9 * C >= 131072) return QIL_ERR_SHAPE;
+    if ((long long)B * H * W > 0x7FFFFFFFll) return QIL_ERR_SHAPE;
+    if (qy && (Cout % 8 != 0 || acc_out)) return QIL_ERR_SHAPE;
+    if (qy && !(out_scale > 0.0f)) return QIL_ERR_UNSUPPORTED;
+    if (!aligned16(qx) || !aligned16(qw) || !aligned16(sw) || (y && !aligned16(y)) || (qy && !aligned16(qy)) ||
+        (acc_out && !aligned16(acc_out)) || (workspace && !aligned16(workspace)))
+        return QIL_ERR_ALIGN;
+    const int M = B * H * W, K = 9 * C;
+    if (!workspace || workspace_bytes < w4a4_workspace(M, Cout, K)) return QIL_ERR_WORKSPACE;
+    return launch_w4a4(qx, nullptr, qw, sw, y ? y : static_cast<void*>(qy), acc_out, M, Cout, K, 4, workspace, workspace_bytes, S(stream),
+                       qy, qy ? out_scale : 1.f, relu ? 1 : 0, C, H, W, x_scale);
+}
+
 qil_status qil_linear_w8a8(const int8_t* qx, const float* sx, const int8_t* qw, const float* sw, void* y,
                            int32_t* acc_out, int M, int N, int K, void* workspace, size_t workspace_bytes,
                            qil_stream_t stream) {

@@ -102,7 +102,7 @@ void w4a16_tc_set_wait_limit(unsigned long long ns);  // 0 restores the default
 size_t w4a4_workspace(int M, int N, int K);
 qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const float* sw, void* y, int32_t* acc_out, int M,
                        int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st, uint32_t* qy = nullptr,
-                       float out_scale = 1.f, int relu = 0);
+                       float out_scale = 1.f, int relu = 0, int conv_C = 0, int conv_H = 0, int conv_W = 0, float x_scale = 1.f);
 
 bool igemm_list_supported(const qil_igemm_desc* d, int count);
 qil_status launch_igemm_list(const qil_igemm_desc* d, int count, void* ws, size_t ws_bytes, cudaStream_t st);

@@ -95,12 +95,21 @@ __device__ __forceinline__ void split32(const uint4& w, uint4& c0, uint4& c1) {
     c1 = make_uint4((w.z << 4) & m, w.z & m, (w.w << 4) & m, w.w & m);
 }
 
+// 3 x 3 convolution (stride 1, zero padding 1) read straight from the feature map, without a materialised im2col
+// matrix: row m of the GEMM is pixel (b, h, w), column (3 kh + kw) C + c is channel c of pixel (h + kh - 1,
+// w + kw - 1).  C = 0: a plain GEMM.  With a feature map every row has the tensor's static scale x_scale.
+struct ConvGeom {
+    int C, H, W;
+    float x_scale;
+};
+
 template <int kBits>
 __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __restrict__ qx, const float* __restrict__ sx,
                                                              const uint32_t* __restrict__ qw, const float* __restrict__ sw,
                                                              __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out,
                                                              int M, int N, int K, int* __restrict__ status,
-                                                             uint32_t* __restrict__ qy, float out_scale, int relu) {
+                                                             uint32_t* __restrict__ qy, float out_scale, int relu,
+                                                             const ConvGeom cg) {
     // qy != null: instead of bf16 outputs the epilogue writes the next layer's int4 activations, quantised with the
     // static scale out_scale from the fp32 product (optionally after ReLU), packed 8 per word (needs N % 8 == 0)
     extern __shared__ __align__(128) unsigned char smem[];
@@ -145,9 +154,36 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
         const uint32_t* xa = qx + (size_t)m0 * row_words + 4 * pq;
         const uint32_t* wb = qw + (size_t)n0 * row_words + 4 * pq;
         uint4 pa[kPre][4], pb[kPre][2];
+        // feature-map mode: the pixels of this thread's four rows
+        int px_h[4], px_w[4];
+        long long px_lin[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            px_h[j] = px_w[j] = 0;
+            px_lin[j] = -1;
+            if (cg.C > 0 && m0 + pr + 32 * j < M) {
+                const int m = m0 + pr + 32 * j;
+                px_w[j] = m % cg.W;
+                px_h[j] = (m / cg.W) % cg.H;
+                px_lin[j] = m;
+            }
+        }
         auto fetch = [&](uint4 (&da)[4], uint4 (&db)[2], int step) {  // packed words of one step (zeros beyond the matrix)
             const int w0 = step * (kStepBytes / 4);
             const bool in_k = w0 + 4 * pq < row_words;
+            if (cg.C > 0) {
+                // this thread's 16 bytes of the step lie inside one tap (C % 32 == 0)
+                constexpr int kPerWord = 32 / kBits;
+                const int k0 = (w0 + 4 * pq) * kPerWord, tap = k0 / cg.C, c0 = k0 - tap * cg.C;
+                const int dh = tap / 3 - 1, dw = tap - (tap / 3) * 3 - 1;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int hh = px_h[j] + dh, ww = px_w[j] + dw;
+                    const bool inside = in_k && px_lin[j] >= 0 && hh >= 0 && hh < cg.H && ww >= 0 && ww < cg.W;
+                    da[j] = inside ? __ldg(reinterpret_cast<const uint4*>(qx + ((px_lin[j] + dh * cg.W + dw) * cg.C + c0) / kPerWord))
+                                   : make_uint4(0, 0, 0, 0);
+                }
+            } else
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int row = pr + 32 * j;
@@ -213,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
         if (ok) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int m = m0 + r;
-            const float sxm = a_row ? sx[m] : 0.f;
+            const float sxm = a_row ? (cg.C > 0 ? cg.x_scale : sx[m]) : 0.f;
             const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
             const bool vec = (N % 8) == 0;  // rows of y are then 16-byte aligned pieces of 8 outputs
 #pragma unroll 1
@@ -312,7 +348,9 @@ size_t w4a4_workspace(int M, int N, int K) {
 // bits = 4: packed nibbles [M][K/8], [N][K/8]; bits = 8: signed bytes [M][K], [N][K]
 qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const float* sw, void* y, int32_t* acc_out, int M,
                        int N, int K, int bits, void* ws, size_t ws_bytes, cudaStream_t st, uint32_t* qy, float out_scale,
-                       int relu) {
+                       int relu, int conv_C, int conv_H, int conv_W, float x_scale) {
+    ConvGeom cg;
+    cg.C = conv_C; cg.H = conv_H; cg.W = conv_W; cg.x_scale = x_scale;
     if (ws == nullptr || ws_bytes < 16) return QIL_ERR_WORKSPACE;
     const dim3 grid((M + kTileM - 1) / kTileM, (N + kTileN - 1) / kTileN);
     cudaError_t e;
@@ -320,12 +358,12 @@ qil_status launch_w4a4(const void* qx, const float* sx, const void* qw, const fl
         e = cudaFuncSetAttribute(w4a4_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e == cudaSuccess)
             w4a4_tc_kernel<8><<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const uint32_t*>(qx), sx, reinterpret_cast<const uint32_t*>(qw), sw,
-                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws), nullptr, 1.f, 0);
+                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws), nullptr, 1.f, 0, cg);
     } else {
         e = cudaFuncSetAttribute(w4a4_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e == cudaSuccess)
             w4a4_tc_kernel<4><<<grid, kThreads, kSmemBytes, st>>>(reinterpret_cast<const uint32_t*>(qx), sx, reinterpret_cast<const uint32_t*>(qw), sw,
-                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws), qy, out_scale, relu);
+                                                                 reinterpret_cast<__nv_bfloat16*>(y), acc_out, M, N, K, reinterpret_cast<int*>(ws), qy, out_scale, relu, cg);
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();

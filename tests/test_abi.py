@@ -97,6 +97,19 @@ def test_lora_side_validation(lib):
     assert lib.qil_lora_side_workspace_size(4) == 4 * 32 * 4
 
 
+def test_conv3x3_validation(lib):
+    import ctypes as C
+    f = lib.qil_conv3x3_w4a4
+    one = C.c_float(1.0)
+    assert f(None, one, A, A, A, None, None, one, 0, 1, 4, 4, 32, 8, A, 16, None) == 1
+    assert f(A, one, A, A, None, None, None, one, 0, 1, 4, 4, 32, 8, A, 16, None) == 1      # no output
+    assert f(A, one, A, A, A, None, A, one, 0, 1, 4, 4, 32, 8, A, 16, None) == 1            # two outputs
+    assert f(A, one, A, A, A, None, None, one, 0, 1, 4, 4, 48, 8, A, 16, None) == 2         # C % 32
+    assert f(A, one, A, A, None, None, A, one, 0, 1, 4, 4, 32, 12, A, 16, None) == 2        # packed output needs Cout % 8
+    assert f(A, one, A, A, None, None, A, C.c_float(0.0), 0, 1, 4, 4, 32, 8, A, 16, None) == 4
+    assert f(A, one, A, A, A, None, None, one, 0, 1, 4, 4, 32, 8, None, 0, None) == 5
+
+
 def test_w4a4_and_act_validation(lib):
     assert lib.qil_quantize_act_a4(None, 1, 8, None, A, A, None) == 1
     assert lib.qil_quantize_act_a4(A, 1, 12, None, A, A, None) == 2

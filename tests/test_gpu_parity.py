@@ -738,6 +738,43 @@ def test_w4a4_conv_stages(api, stage, batch):
     np.testing.assert_array_equal(bits_of(y2), bits_of(y))
 
 
+@pytest.mark.parametrize("B,H,W,Cc,Cout", [
+    (2, 5, 7, 32, 24),        # ragged everything, a step spans four taps
+    (1, 1, 1, 64, 8),         # one pixel: only the centre tap is inside
+    (3, 22, 50, 64, 64),      # the first conv stage's geometry (a step spans two taps)
+    (2, 11, 25, 128, 128), (2, 3, 7, 512, 40),
+])
+def test_conv3x3_w4a4_from_the_feature_map(api, B, H, W, Cc, Cout):
+    """The 3 x 3 convolution read straight from the int4 feature map (no im2col matrix): accumulators bit-exact
+    against the oracle's tap-by-tap definition, bf16 outputs within the integer GEMM's tolerance, and the variant
+    whose epilogue writes the next layer's int4 feature map bit-exact against the oracle's requantiser."""
+    rng = np.random.default_rng(B * H * W + Cc + Cout)
+    q = rng.integers(-8, 8, size=(B, H, W, Cc)).astype(np.int8)
+    qw = rng.integers(-8, 8, size=(Cout, 9 * Cc)).astype(np.int8)
+    sw = (rng.random(Cout) * 0.05 + 0.01).astype(np.float32)
+    x_scale = 0.125
+    acc_ref, y_ref = np_oracle.conv3x3_w4a4(q, x_scale, qw, sw)
+    q_packed = api.pack_w4(cuda(q.reshape(B * H * W, Cc))).reshape(B, H, W, Cc // 8)
+    w_packed = api.pack_w4(cuda(qw))
+    y, acc = api.conv3x3_w4a4(q_packed, x_scale, w_packed, cuda(sw), want_acc=True)
+    np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert_rows_close(bf16_to_f64(y).reshape(B * H * W, Cout), y_ref.reshape(B * H * W, Cout))
+    if Cout % 8 == 0:
+        out_scale = float(np.abs(y_ref).max() / 7.0) or 1.0
+        for relu in (False, True):
+            cols = wl.im2col_3x3(q)    # (input generator: only feeds the oracle's requantiser its operand)
+            q_next_ref = np_oracle.linear_w4a4_requant(cols, np.full(B * H * W, x_scale, dtype=np.float32), qw, sw, out_scale, relu)
+            qy = api.conv3x3_w4a4(q_packed, x_scale, w_packed, cuda(sw), out_scale=out_scale, relu=relu)
+            got = np_oracle.unpack_w4(qy.cpu().numpy().view(np.uint32).reshape(B * H * W, Cout // 8), signed=True)
+            np.testing.assert_array_equal(got, q_next_ref)
+            # ... and it is a feature map the next layer can read
+            if Cout % 32 == 0:
+                qw2 = rng.integers(-8, 8, size=(8, 9 * Cout)).astype(np.int8)
+                acc2_ref, _ = np_oracle.conv3x3_w4a4(q_next_ref.reshape(B, H, W, Cout), out_scale, qw2, np.ones(8, dtype=np.float32))
+                _, acc2 = api.conv3x3_w4a4(qy, out_scale, api.pack_w4(cuda(qw2)), cuda(np.ones(8, dtype=np.float32)), want_acc=True)
+                np.testing.assert_array_equal(acc2.cpu().numpy().astype(np.int64), acc2_ref)
+
+
 @pytest.mark.parametrize("M,N,K", [(1, 1, 32), (17, 9, 96), (130, 200, 160), (64, 64, 1152)])
 def test_w4a4_ragged_shapes(api, M, N, K):
     rng = np.random.default_rng(M * N + K)

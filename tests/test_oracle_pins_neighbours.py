@@ -110,3 +110,55 @@ def test_lora_side_hand_case_and_identities():
     out = np_oracle.lora_side(f(xi), f(a_id), f(b_id), 1.0)
     np.testing.assert_array_equal(out[:, :r], xi[:, :r])
     assert np.all(out[:, r:] == 0)
+
+
+# ---- the 3 x 3 convolution on integer codes (np_oracle.conv3x3_w4a4) ----
+def test_conv3x3_hand_cases():
+    # one channel, one filter, 3 x 3 image 1..9, all-ones filter: the sum of each pixel's neighbourhood inside the image
+    q = np.arange(1, 10, dtype=np.int8).reshape(1, 3, 3, 1)
+    ones = np.ones((1, 9), dtype=np.int8)
+    acc, y = np_oracle.conv3x3_w4a4(q, 0.5, ones, np.array([2.0]))
+    np.testing.assert_array_equal(acc[0, :, :, 0], [[12, 21, 16], [27, 45, 33], [24, 39, 28]])
+    np.testing.assert_array_equal(y, acc.astype(np.float64))          # 0.5 * 2
+    # a delta filter at tap (kh, kw) shifts the image by (kh - 1, kw - 1), zeros coming in at the border
+    for kh in range(3):
+        for kw in range(3):
+            d = np.zeros((1, 9), dtype=np.int8)
+            d[0, 3 * kh + kw] = 1
+            a, _ = np_oracle.conv3x3_w4a4(q, 1.0, d, np.array([1.0]))
+            want = np.zeros((3, 3), dtype=np.int64)
+            for h in range(3):
+                for w in range(3):
+                    hh, ww = h + kh - 1, w + kw - 1
+                    if 0 <= hh < 3 and 0 <= ww < 3:
+                        want[h, w] = q[0, hh, ww, 0]
+            np.testing.assert_array_equal(a[0, :, :, 0], want)
+
+
+def test_conv3x3_is_im2col_then_the_integer_gemm_and_brute_force():
+    rng = np.random.default_rng(5)
+    B, H, W, Cc, Cout = 2, 4, 5, 8, 3
+    q = rng.integers(-8, 8, (B, H, W, Cc)).astype(np.int8)
+    w = rng.integers(-8, 8, (Cout, 9 * Cc)).astype(np.int8)
+    sw = rng.random(Cout) + 0.1
+    acc, y = np_oracle.conv3x3_w4a4(q, 0.25, w, sw)
+    # the input generator's im2col followed by the (pinned) integer GEMM
+    cols = wl.im2col_3x3(q)
+    acc2, y2 = np_oracle.linear_w4a4(cols, np.full(B * H * W, 0.25), w, sw)
+    np.testing.assert_array_equal(acc.reshape(B * H * W, Cout), acc2)
+    np.testing.assert_allclose(y.reshape(B * H * W, Cout), y2, rtol=1e-15)
+    # brute force, six nested loops
+    for b in range(B):
+        for h in range(H):
+            for x in range(W):
+                for n in range(Cout):
+                    t = 0
+                    for kh in range(3):
+                        for kw in range(3):
+                            hh, ww = h + kh - 1, x + kw - 1
+                            if 0 <= hh < H and 0 <= ww < W:
+                                t += int(np.dot(q[b, hh, ww].astype(np.int64), w[n, (3 * kh + kw) * Cc:(3 * kh + kw + 1) * Cc].astype(np.int64)))
+                    assert acc[b, h, x, n] == t
+    # one-pixel images: only the centre tap sees anything
+    a1, _ = np_oracle.conv3x3_w4a4(q[:, :1, :1], 1.0, w, sw)
+    np.testing.assert_array_equal(a1[:, 0, 0], q[:, 0, 0].astype(np.int64) @ w[:, 4 * Cc:5 * Cc].astype(np.int64).T)

@@ -193,8 +193,14 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&d)[16]) {
     for (int j = 0; j < 16; ++j) asm volatile("" : "+r"(d[j]));
 }
 
-// silu(g) * u in fp32 (the gated MLP of the Llama-2 backbone; fused epilogue)
-__device__ __forceinline__ float swiglu(float g, float u) { return g / (1.f + __expf(-g)) * u; }
+// silu(g) * u in fp32 (the gated MLP of the Llama-2 backbone; fused epilogue).  sigmoid(g) = (1 + tanh(g / 2)) / 2 with
+// the hardware tanh (one special-function instruction instead of an exponential and a reciprocal; its error, about
+// 2^-11 relative, is below the bf16 rounding of the result): the special-function unit set the pace of this epilogue.
+__device__ __forceinline__ float swiglu(float g, float u) {
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * g));
+    return fmaf(0.5f * g, t, 0.5f * g) * u;
+}
 
 // The CTA's next run of steps inside one tile: steps [s0, s1) of tile `tile`.  g walks the CTA's range of numbered steps.
 struct Segment {
@@ -522,12 +528,32 @@ __global__ void __launch_bounds__(kThreads, 1) w4a16_prefill_kernel(const __grid
                         for (int j = 0; j < 16; ++j) d[j] = __float_as_uint(__uint_as_float(d[j]) + v[j]);
                     }
                     if (p.swiglu) {
-                        // lane = feature: the even lane holds gate i, its neighbour up i (N is even, so both are live or neither)
+                        // lane = feature: the even lane holds gate i, its neighbour up i (N is even, so both are live or
+                        // neither).  The pair shares the work: of tokens j, j + 1 the even lane takes j (its own gate, the
+                        // neighbour's up), the odd lane j + 1 (the neighbour's gate, its own up): one exchange per two tokens,
+                        // no lane computes a value that is thrown away.
+                        const bool odd = (lane & 1) != 0;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float u = __uint_as_float(__shfl_xor_sync(0xFFFFFFFFu, d[j], 1));
-                            if (live && (lane & 1) == 0 && m0 + c0 + j < p.M)
-                                p.y[(size_t)(m0 + c0 + j) * (p.N >> 1) + (n >> 1)] = __float2bfloat16_rn(swiglu(__uint_as_float(d[j]), u));
+                        for (int j = 0; j < 16; j += 2) {
+                            const uint32_t mine = odd ? d[j + 1] : d[j];
+                            const uint32_t theirs = __shfl_xor_sync(0xFFFFFFFFu, odd ? d[j] : d[j + 1], 1);
+                            const float o = odd ? swiglu(__uint_as_float(theirs), __uint_as_float(mine))
+                                                : swiglu(__uint_as_float(mine), __uint_as_float(theirs));
+                            const int tk = m0 + c0 + j + (odd ? 1 : 0);
+                            if (live && tk < p.M) p.y[(size_t)tk * (p.N >> 1) + (n >> 1)] = __float2bfloat16_rn(o);
+                        }
+                    } else if ((p.N & 1) == 0) {
+                        // the same exchange: the even lane writes features n, n + 1 of token j as one 32-bit store, the odd
+                        // lane those of token j + 1 (half the store instructions; the read-out is bound by them)
+                        const bool odd = (lane & 1) != 0;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 2) {
+                            const uint32_t mine = odd ? d[j + 1] : d[j];
+                            const uint32_t theirs = __shfl_xor_sync(0xFFFFFFFFu, odd ? d[j] : d[j + 1], 1);
+                            const __nv_bfloat162 o = odd ? __floats2bfloat162_rn(__uint_as_float(theirs), __uint_as_float(mine))
+                                                         : __floats2bfloat162_rn(__uint_as_float(mine), __uint_as_float(theirs));
+                            const int tk = m0 + c0 + j + (odd ? 1 : 0);
+                            if (live && tk < p.M) *reinterpret_cast<__nv_bfloat162*>(p.y + (size_t)tk * p.N + (n & ~1)) = o;
                         }
                     } else if (live) {
 #pragma unroll

@@ -684,7 +684,7 @@ def secondary_measurements(dev):
         al = (torch.randn((32, wl.HIDDEN), device=dev, generator=g) * 0.02).to(torch.bfloat16)
         bl = (torch.randn((wl.HIDDEN, 32), device=dev, generator=g) * 0.02).to(torch.bfloat16)
         yl = torch.zeros((Ml, wl.HIDDEN), dtype=torch.bfloat16, device=dev)
-        wsl = api.new_workspace(Ml * 32 * 4, dev)
+        wsl = api.new_workspace(api.lora_side_workspace_size(Ml), dev)
         lora[f"m{Ml}_us"] = time_us(lambda: api.lora_side_add(xl, al, bl, yl, 1.0, workspace=wsl), 20)
     out["lora_side_rank32_4096x4096"] = lora
     out["w4a16_prefill_m280_gate_up_22016x4096"] = {"plain_us": t_gate_up, "swiglu_epilogue_us": t_gate_up_sw,

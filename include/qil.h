@@ -166,7 +166,8 @@ qil_status qil_linear_w4a16(const void* x, const uint32_t* qweight, const void* 
  *     y[m][n] = bf16( float(y[m][n]) + scale * sum_j (sum_k x[m][k] A[j][k]) B[n][j] )
  *   x [M][K] bf16   A [rank][K] bf16   B [N][rank] bf16   y [M][N] bf16, in place
  * fp32 accumulation; the inner product x . A^T is kept in fp32 in the
- * workspace (qil_lora_side_workspace_size(M) bytes, no initialisation needed).
+ * workspace, as up to 32 partial sums over slices of K that are added in a
+ * fixed order (qil_lora_side_workspace_size(M) bytes, no initialisation needed).
  * Call it after the linear that produced y, on the same stream.
  * rank <= 32 (larger: UNSUPPORTED); K even.
  * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, CUDA.

@@ -182,6 +182,10 @@ def linear_w4a16(x, qweight, scales, zeros, N: int, group_size: int, layout: int
     return out
 
 
+def lora_side_workspace_size(M: int) -> int:
+    return int(_lib.load().qil_lora_side_workspace_size(M))
+
+
 def lora_side_add(x, a, b, y, scale: float = 1.0, workspace=None, stream=None):
     """y[M][N] (bf16, in place) += scale * (x[M][K] . a[r][K]^T) . b[N][r]^T: an unmerged low-rank adapter, r <= 32."""
     _need_cuda(x, a, b, y, workspace)

@@ -294,6 +294,27 @@ def test_w4a16_swiglu(api, M, N, K, G):
     np.testing.assert_array_equal(bits_of(y), bits_of(y2))
 
 
+def test_cfg2_gate_up_swiglu_full_size(api):
+    """The fused gate_up projection of config 2 at full size (22016 x 4096, 280 tokens), the oracle on 192 sampled
+    (gate, up) pairs; same tolerance as test_w4a16_swiglu."""
+    M, K, G = wl.PREFILL_M, wl.HIDDEN, wl.GROUP_SIZE
+    N = 2 * wl.FFN
+    w = wl.normal_weights(2, 9001, N, K, 0.02, outlier_prob=0.001)
+    x = wl.normal_activations_bf16(2, 9002, M, K)
+    got = api.quantize_rtn_w4(cuda(w), G)
+    pairs = np.sort(np.random.default_rng(11).choice(N // 2, 192, replace=False))
+    rows = np.stack((2 * pairs, 2 * pairs + 1), axis=1).reshape(-1)
+    ref = np_oracle.quantize_rtn_w4_asym(w[rows], G)
+    np.testing.assert_array_equal(got[0].cpu().numpy()[rows], ref[0])
+    y = api.linear_w4a16_swiglu(to_bf16_cuda(x), api.pack_w4(got[0]), got[1], got[2], N, G)
+    t = c_oracle.linear_w4a16(x, *ref, G)
+    y_ref = np_oracle.silu(t[:, 0::2]) * t[:, 1::2]
+    gmax, umax = np.abs(t[:, 0::2]).max(axis=1, keepdims=True), np.abs(t[:, 1::2]).max(axis=1, keepdims=True)
+    tol = (2.1 * CONTRACT_REL + 2.0 ** -8) * gmax * umax   # (sampled maxima lower-bound the row's: the check is stricter)
+    err = np.abs(bf16_to_f64(y)[:, pairs] - y_ref)
+    assert np.all(err <= tol), float((err / tol).max())
+
+
 @pytest.mark.parametrize("M,N,K,r", [(1, 4096, 4096, 32), (7, 1000, 2176, 32), (280, 513, 1024, 16), (9, 64, 34, 5), (33, 2, 64, 1)])
 def test_lora_side_add(api, M, N, K, r):
     """The unmerged low-rank adapter beside a quantised linear (QLoRA rank 32, App. A.1.2): y += scale (x A^T) B^T on
@@ -743,6 +764,7 @@ def test_w4a4_conv_stages(api, stage, batch):
     (1, 1, 1, 64, 8),         # one pixel: only the centre tap is inside
     (3, 22, 50, 64, 64),      # the first conv stage's geometry (a step spans two taps)
     (2, 11, 25, 128, 128), (2, 3, 7, 512, 40),
+    (32, 22, 50, 64, 64), (32, 3, 7, 512, 512),   # the first and the last conv stage at the benchmark's batch
 ])
 def test_conv3x3_w4a4_from_the_feature_map(api, B, H, W, Cc, Cout):
     """The 3 x 3 convolution read straight from the int4 feature map (no im2col matrix): accumulators bit-exact

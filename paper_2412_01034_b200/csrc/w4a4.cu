@@ -88,6 +88,18 @@ __device__ __forceinline__ void mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 
+// rint(f / s) with the IEEE division of the specification, without paying for a division per element: the product
+// with the reciprocal is within a few ulp of the quotient, so unless it lies that close to a rounding boundary
+// (k + 0.5) it rounds to the same integer; the rare close calls (and anything not finite) take the true division.
+// (The division primitive also leaves its fast path for a zero numerator, which is every other element after a ReLU:
+// an epilogue of 64 divisions per thread then cost 10 us a launch.)
+__device__ __forceinline__ float rint_div(float f, float s, float inv_s) {
+    const float r = f * inv_s;
+    const float dist = fabsf(fabsf(r - rintf(r)) - 0.5f);  // distance of r from the nearest k + 0.5
+    if (dist > 1e-4f * fmaxf(fabsf(r), 1.0f) && fabsf(r) < 1e6f) return rintf(r);
+    return rintf(__fdiv_rn(f, s));
+}
+
 // 32 packed codes (one uint4) -> 32 signed bytes (x16) = two 16-byte K chunks
 __device__ __forceinline__ void split32(const uint4& w, uint4& c0, uint4& c1) {
     constexpr uint32_t m = 0xF0F0F0F0u;
@@ -252,6 +264,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
             const float sxm = a_row ? (cg.C > 0 ? cg.x_scale : sx[m]) : 0.f;
             const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
             const bool vec = (N % 8) == 0;  // rows of y are then 16-byte aligned pieces of 8 outputs
+            const float inv_out = __frcp_rn(out_scale);
 #pragma unroll 1
             for (int c0 = 0; c0 < kTileN; c0 += 16) {
                 uint32_t d[16];
@@ -277,7 +290,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_tc_kernel(const uint32_t* __
                         for (int j = 0; j < 8; ++j) {
                             float v = __fmul_rn((float)a[j], __fmul_rn(sxm, sws[c0 + 8 * h + j]));
                             if (relu) v = fmaxf(v, 0.f);
-                            const int q = (int)fminf(fmaxf(rintf(__fdiv_rn(v, out_scale)), -8.f), 7.f);
+                            const int q = (int)fminf(fmaxf(rint_div(v, out_scale, inv_out), -8.f), 7.f);
                             word |= ((uint32_t)q & 0xFu) << (4 * j);
                         }
                         qy[(size_t)m * (N >> 3) + (nb >> 3)] = word;
